@@ -1,0 +1,721 @@
+/*
+ * Sali-Cache pre-attention filter + mixed-precision K/V store: CPU ORACLE.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the plain, slow statement of what the
+ * hot path computes.  It shares no code, table or constant generator with the
+ * CUDA library; only tests, the smoke check and the benchmark's CPU-baseline leg
+ * may call it.  Scores are computed in double; the decision rule and the
+ * quantisers use single IEEE-754 binary32 operations in a fixed order
+ * (compile with -ffp-contract=off, no fast-math).
+ *
+ * Every function names the passage of the paper it follows.  Where the paper
+ * is silent the reading taken is stated next to the code.
+ *
+ * Parity pins: every function here is pinned by tests/test_oracle_*.py against
+ * closed forms, brute force or library routines.  The paper's aggregate numbers
+ * (2.20x compression, 26.7 % reuse, per-frame latency) are "parity unpinned":
+ * they need the authors' videos, thresholds and model.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define EXPORT __attribute__((visibility("default")))
+
+static int clampi(int v, int lo, int hi) { return v < lo ? lo : (v > hi ? hi : v); }
+
+EXPORT int oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ------------------------------------------------------------------------- */
+/* Gray level.  The paper does not say how colour becomes intensity; reading:  */
+/* integer luma g = (77 R + 150 G + 29 B + 128) >> 8 so that the edge branch   */
+/* is exact integer work.                                                      */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_gray(const uint8_t* rgb, int h, int w, uint8_t* g) {
+    for (int i = 0; i < h * w; ++i) {
+        int R = rgb[3 * i], G = rgb[3 * i + 1], B = rgb[3 * i + 2];
+        g[i] = (uint8_t)((77 * R + 150 * G + 29 * B + 128) >> 8);
+    }
+}
+
+/* Anyres base image: exact 2x2 integer box mean (a+b+c+d+2)>>2 per channel.   */
+/* (The paper only mentions dynamic-resolution encoding, Sec. II-A.)           */
+EXPORT void oracle_box_down2(const uint8_t* rgb, int h, int w, uint8_t* out) {
+    int h2 = h / 2, w2 = w / 2;
+    for (int y = 0; y < h2; ++y)
+        for (int x = 0; x < w2; ++x)
+            for (int c = 0; c < 3; ++c) {
+                int s = rgb[((2 * y) * w + 2 * x) * 3 + c] + rgb[((2 * y) * w + 2 * x + 1) * 3 + c] +
+                        rgb[((2 * y + 1) * w + 2 * x) * 3 + c] + rgb[((2 * y + 1) * w + 2 * x + 1) * 3 + c];
+                out[(y * w2 + x) * 3 + c] = (uint8_t)((s + 2) >> 2);
+            }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Pyramid, scale 0.5 (Sec. IV-B "pyramid scale of 0.5 and 3 pyramid levels"). */
+/* Reading: 5x5 binomial smoothing [1 4 6 4 1]/16, sample at (2y, 2x), clamp.  */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_pyr_down(const double* src, int h, int w, double* dst) {
+    static const double k[5] = {1.0 / 16, 4.0 / 16, 6.0 / 16, 4.0 / 16, 1.0 / 16};
+    int h2 = h / 2, w2 = w / 2;
+    for (int y = 0; y < h2; ++y)
+        for (int x = 0; x < w2; ++x) {
+            double acc = 0.0;
+            for (int a = -2; a <= 2; ++a)
+                for (int b = -2; b <= 2; ++b)
+                    acc += k[a + 2] * k[b + 2] *
+                           src[clampi(2 * y + a, 0, h - 1) * w + clampi(2 * x + b, 0, w - 1)];
+            dst[y * w2 + x] = acc;
+        }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Polynomial expansion (Farneback's method, named in Sec. IV-B).              */
+/* f(x+d) ~ r1 + r2 dx + r3 dy + r4 dx^2 + r5 dy^2 + r6 dx dy, fitted by       */
+/* least squares with separable Gaussian weights g(dx) g(dy) on a              */
+/* (2n+1)^2 neighbourhood.  Because g is even the normal equations decouple:   */
+/*   r2 = m10/mu2, r3 = m01/mu2, r6 = m11/mu2^2,                               */
+/*   r4 = (m20 - mu2 m00)/(mu4 - mu2^2), r5 = (m02 - mu2 m00)/(mu4 - mu2^2),   */
+/* with m_pq = sum g(dx) g(dy) dx^p dy^q f(x+d).  Output planes: r2 r3 r4 r5 r6*/
+/* Reading (paper silent): n = 2, sigma = 1.2, clamp-to-edge.                  */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_poly_exp(const double* f, int h, int w, int n, double sigma, double* r) {
+    double g[33];
+    double Z = 0.0, mu2 = 0.0, mu4 = 0.0;
+    for (int k = -n; k <= n; ++k) { g[k + n] = exp(-(double)(k * k) / (2.0 * sigma * sigma)); Z += g[k + n]; }
+    for (int k = -n; k <= n; ++k) {
+        g[k + n] /= Z;
+        mu2 += g[k + n] * k * k;
+        mu4 += g[k + n] * k * k * (double)(k * k);
+    }
+    double den = mu4 - mu2 * mu2;
+    size_t P = (size_t)h * w;
+    for (int y = 0; y < h; ++y)
+        for (int x = 0; x < w; ++x) {
+            double m00 = 0, m10 = 0, m01 = 0, m20 = 0, m02 = 0, m11 = 0;
+            for (int dy = -n; dy <= n; ++dy)
+                for (int dx = -n; dx <= n; ++dx) {
+                    double v = g[dy + n] * g[dx + n] * f[clampi(y + dy, 0, h - 1) * w + clampi(x + dx, 0, w - 1)];
+                    m00 += v;
+                    m10 += v * dx;
+                    m01 += v * dy;
+                    m20 += v * dx * dx;
+                    m02 += v * dy * dy;
+                    m11 += v * dx * dy;
+                }
+            size_t i = (size_t)y * w + x;
+            r[0 * P + i] = m10 / mu2;
+            r[1 * P + i] = m01 / mu2;
+            r[2 * P + i] = (m20 - mu2 * m00) / den;
+            r[3 * P + i] = (m02 - mu2 * m00) / den;
+            r[4 * P + i] = m11 / (mu2 * mu2);
+        }
+}
+
+/* Bilinear sample of one plane at a clamped continuous position. */
+static double bilin(const double* p, int h, int w, double y, double x) {
+    if (x < 0) x = 0;
+    if (x > w - 1) x = w - 1;
+    if (y < 0) y = 0;
+    if (y > h - 1) y = h - 1;
+    int x0 = (int)floor(x), y0 = (int)floor(y);
+    int x1 = x0 + 1 < w ? x0 + 1 : w - 1, y1 = y0 + 1 < h ? y0 + 1 : h - 1;
+    double fx = x - x0, fy = y - y0;
+    double top = p[y0 * w + x0] * (1.0 - fx) + p[y0 * w + x1] * fx;
+    double bot = p[y1 * w + x0] * (1.0 - fx) + p[y1 * w + x1] * fx;
+    return top * (1.0 - fy) + bot * fy;
+}
+
+/* ------------------------------------------------------------------------- */
+/* One displacement update at one pyramid level (Farneback's estimate with an  */
+/* a-priori displacement).  Convention: I_cur(x + d) ~ I_prev(x); d = (u, v),  */
+/* u along x.  c1, c2: expansion planes of the previous and current frame.     */
+/*   xt   = clamp(x + d~)                                                      */
+/*   A    = (A1(x) + A2(xt))/2,      A = [[r4, r6/2],[r6/2, r5]]               */
+/*   db   = -(b2(xt) - b1(x))/2 + A d~,   b = (r2, r3)                          */
+/*   G    = A^T A,  hv = A^T db; both summed over the in-image part of the     */
+/*   win x win box centred on x (uniform weights);                             */
+/*   d    = adj(G) hv / (det G + eps)                                          */
+/* Reading (paper silent): bilinear fetch, box window 15, eps = 1e-3.          */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_flow_iter(const double* c1, const double* c2, int h, int w, const double* d_in,
+                             int win, double eps, double* d_out) {
+    size_t P = (size_t)h * w;
+    double* t = (double*)malloc(5 * P * sizeof(double));
+    for (int y = 0; y < h; ++y)
+        for (int x = 0; x < w; ++x) {
+            size_t i = (size_t)y * w + x;
+            double du = d_in[i], dv = d_in[P + i];
+            double xt = x + du, yt = y + dv;
+            double b2x = bilin(c2 + 0 * P, h, w, yt, xt), b2y = bilin(c2 + 1 * P, h, w, yt, xt);
+            double a2xx = bilin(c2 + 2 * P, h, w, yt, xt), a2yy = bilin(c2 + 3 * P, h, w, yt, xt);
+            double a2xy = 0.5 * bilin(c2 + 4 * P, h, w, yt, xt);
+            double axx = 0.5 * (c1[2 * P + i] + a2xx);
+            double ayy = 0.5 * (c1[3 * P + i] + a2yy);
+            double axy = 0.5 * (0.5 * c1[4 * P + i] + a2xy);
+            double dbx = -0.5 * (b2x - c1[0 * P + i]) + (axx * du + axy * dv);
+            double dby = -0.5 * (b2y - c1[1 * P + i]) + (axy * du + ayy * dv);
+            t[0 * P + i] = axx * axx + axy * axy;       /* g11 */
+            t[1 * P + i] = axx * axy + axy * ayy;       /* g12 */
+            t[2 * P + i] = axy * axy + ayy * ayy;       /* g22 */
+            t[3 * P + i] = axx * dbx + axy * dby;       /* h1  */
+            t[4 * P + i] = axy * dbx + ayy * dby;       /* h2  */
+        }
+    int rad = win / 2;
+    for (int y = 0; y < h; ++y)
+        for (int x = 0; x < w; ++x) {
+            double s[5] = {0, 0, 0, 0, 0};
+            for (int yy = y - rad; yy <= y + rad; ++yy) {
+                if (yy < 0 || yy >= h) continue;
+                for (int xx = x - rad; xx <= x + rad; ++xx) {
+                    if (xx < 0 || xx >= w) continue;
+                    size_t j = (size_t)yy * w + xx;
+                    for (int c = 0; c < 5; ++c) s[c] += t[c * P + j];
+                }
+            }
+            double det = s[0] * s[2] - s[1] * s[1] + eps;
+            size_t i = (size_t)y * w + x;
+            d_out[i] = (s[2] * s[3] - s[1] * s[4]) / det;
+            d_out[P + i] = (s[0] * s[4] - s[1] * s[3]) / det;
+        }
+    free(t);
+}
+
+/* Coarse-to-fine transfer: d_fine(y,x) = 2 * bilinear(d_coarse) sampled at    */
+/* ((x+1/2)/2 - 1/2, (y+1/2)/2 - 1/2), clamped (pixel-centre alignment).       */
+EXPORT void oracle_flow_upsample(const double* dc, int hc, int wc, double* df, int hf, int wf) {
+    size_t Pc = (size_t)hc * wc, Pf = (size_t)hf * wf;
+    for (int y = 0; y < hf; ++y)
+        for (int x = 0; x < wf; ++x) {
+            double xs = (x + 0.5) / 2.0 - 0.5, ys = (y + 0.5) / 2.0 - 0.5;
+            df[(size_t)y * wf + x] = 2.0 * bilin(dc, hc, wc, ys, xs);
+            df[Pf + (size_t)y * wf + x] = 2.0 * bilin(dc + Pc, hc, wc, ys, xs);
+        }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Dense flow between two RGB frames (Sec. III-A; Farneback, scale 0.5,        */
+/* `levels` pyramid levels, Sec. IV-B).  Coarse to fine, `iters` updates per   */
+/* level, zero prior at the coarsest level.  flow = [2][h][w] (u then v).      */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_flow(const uint8_t* prev, const uint8_t* cur, int h, int w, int levels, int poly_n,
+                        double poly_sigma, int win, int iters, double eps, double* flow) {
+    const uint8_t* fr[2] = {prev, cur};
+    double* pyr[2][8];
+    double* coef[2][8];
+    int hs[8], ws[8];
+    for (int l = 0; l < levels; ++l) { hs[l] = h >> l; ws[l] = w >> l; }
+    for (int f = 0; f < 2; ++f) {
+        uint8_t* g = (uint8_t*)malloc((size_t)h * w);
+        oracle_gray(fr[f], h, w, g);
+        pyr[f][0] = (double*)malloc((size_t)h * w * sizeof(double));
+        for (int i = 0; i < h * w; ++i) pyr[f][0][i] = (double)g[i];
+        free(g);
+        for (int l = 1; l < levels; ++l) {
+            pyr[f][l] = (double*)malloc((size_t)hs[l] * ws[l] * sizeof(double));
+            oracle_pyr_down(pyr[f][l - 1], hs[l - 1], ws[l - 1], pyr[f][l]);
+        }
+        for (int l = 0; l < levels; ++l) {
+            coef[f][l] = (double*)malloc((size_t)5 * hs[l] * ws[l] * sizeof(double));
+            oracle_poly_exp(pyr[f][l], hs[l], ws[l], poly_n / 2, poly_sigma, coef[f][l]);
+        }
+    }
+    double* d = NULL;
+    for (int l = levels - 1; l >= 0; --l) {
+        size_t P = (size_t)hs[l] * ws[l];
+        double* dl = (double*)calloc(2 * P, sizeof(double));
+        if (d) {
+            oracle_flow_upsample(d, hs[l + 1], ws[l + 1], dl, hs[l], ws[l]);
+            free(d);
+        }
+        double* tmp = (double*)malloc(2 * P * sizeof(double));
+        for (int it = 0; it < iters; ++it) {
+            oracle_flow_iter(coef[0][l], coef[1][l], hs[l], ws[l], dl, win, eps, tmp);
+            memcpy(dl, tmp, 2 * P * sizeof(double));
+        }
+        free(tmp);
+        d = dl;
+    }
+    memcpy(flow, d, (size_t)2 * h * w * sizeof(double));
+    free(d);
+    for (int f = 0; f < 2; ++f)
+        for (int l = 0; l < levels; ++l) { free(pyr[f][l]); free(coef[f][l]); }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Patch temporal score (Eq. 5).  Reading: F in Eq. 5 is the displacement      */
+/* field (the text, Alg. 1 and Sec. IV-B all say optical flow); the L2 norm    */
+/* over the patch is normalised by its area, so dP is an RMS in pixels:        */
+/*   dP_i = sqrt( (1/|P_i|) sum_{P_i} (u^2 + v^2) ).                            */
+/* Patches row-major on the (h/patch) x (w/patch) grid.                        */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_delta_p(const double* flow, int h, int w, int patch, double* dP) {
+    int gh = h / patch, gw = w / patch;
+    size_t P = (size_t)h * w;
+    for (int py = 0; py < gh; ++py)
+        for (int px = 0; px < gw; ++px) {
+            double acc = 0.0;
+            for (int y = py * patch; y < (py + 1) * patch; ++y)
+                for (int x = px * patch; x < (px + 1) * patch; ++x) {
+                    double u = flow[(size_t)y * w + x], v = flow[P + (size_t)y * w + x];
+                    acc += u * u + v * v;
+                }
+            dP[py * gw + px] = sqrt(acc / (double)(patch * patch));
+        }
+}
+
+/* Frame pairs -> dP, B pairs in parallel over host threads.  dP: [B][n_patches]. */
+EXPORT void oracle_flow_score_batch(const uint8_t* prev, const uint8_t* cur, int B, int h, int w, int patch,
+                                    int levels, int poly_n, double poly_sigma, int win, int iters, double eps,
+                                    double* dP, double* flow_or_null) {
+    size_t fb = (size_t)h * w * 3;
+    int np = (h / patch) * (w / patch);
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        double* fl = flow_or_null ? flow_or_null + (size_t)b * 2 * h * w : (double*)malloc((size_t)2 * h * w * sizeof(double));
+        oracle_flow(prev + b * fb, cur + b * fb, h, w, levels, poly_n, poly_sigma, win, iters, eps, fl);
+        oracle_delta_p(fl, h, w, patch, dP + (size_t)b * np);
+        if (!flow_or_null) free(fl);
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Edge map E (Canny, Sec. III-B / IV-B), all integer.  Reading of the steps   */
+/* the paper leaves open:                                                      */
+/*  (i)  blur  Bl = (sum k(a) k(b) g + 128) >> 8, k = [1 4 6 4 1], clamp;      */
+/*  (ii) Sobel 3x3 on Bl, clamp;  (iii) m = gx^2 + gy^2;                       */
+/*  (iv) non-maximum suppression along the gradient sector: |gy|/|gx| <=       */
+/*       13573/32768 (tan 22.5 deg) -> x; the transposed test -> y; else the   */
+/*       diagonal picked by the sign of gx*gy.  Keep when m > m(n-) and        */
+/*       m >= m(n+), n- the neighbour that comes first in (y, x) order;        */
+/*       neighbours outside the image count as 0;                              */
+/*  (v)  strong: m >= hi^2, weak: m >= lo^2;                                   */
+/*  (vi) hysteresis: kept strong pixels, plus kept weak pixels 8-connected     */
+/*       through kept weak/strong pixels to a strong one (flood fill).         */
+/* cls_or_null receives 0 / 1 (kept weak) / 2 (kept strong) before hysteresis. */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_canny(const uint8_t* g, int h, int w, int lo, int hi, uint8_t* E, uint8_t* cls_or_null) {
+    static const int k[5] = {1, 4, 6, 4, 1};
+    size_t P = (size_t)h * w;
+    int* Bl = (int*)malloc(P * sizeof(int));
+    int* gx = (int*)malloc(P * sizeof(int));
+    int* gy = (int*)malloc(P * sizeof(int));
+    int* m = (int*)malloc(P * sizeof(int));
+    uint8_t* cls = (uint8_t*)calloc(P, 1);
+    for (int y = 0; y < h; ++y)
+        for (int x = 0; x < w; ++x) {
+            int acc = 0;
+            for (int a = -2; a <= 2; ++a)
+                for (int b = -2; b <= 2; ++b)
+                    acc += k[a + 2] * k[b + 2] * g[clampi(y + a, 0, h - 1) * w + clampi(x + b, 0, w - 1)];
+            Bl[y * w + x] = (acc + 128) >> 8;
+        }
+#define BL(yy, xx) Bl[clampi((yy), 0, h - 1) * w + clampi((xx), 0, w - 1)]
+    for (int y = 0; y < h; ++y)
+        for (int x = 0; x < w; ++x) {
+            int sx = (BL(y - 1, x + 1) + 2 * BL(y, x + 1) + BL(y + 1, x + 1)) -
+                     (BL(y - 1, x - 1) + 2 * BL(y, x - 1) + BL(y + 1, x - 1));
+            int sy = (BL(y + 1, x - 1) + 2 * BL(y + 1, x) + BL(y + 1, x + 1)) -
+                     (BL(y - 1, x - 1) + 2 * BL(y - 1, x) + BL(y - 1, x + 1));
+            gx[y * w + x] = sx;
+            gy[y * w + x] = sy;
+            m[y * w + x] = sx * sx + sy * sy;
+        }
+#undef BL
+#define M(yy, xx) (((yy) < 0 || (yy) >= h || (xx) < 0 || (xx) >= w) ? 0 : m[(yy) * w + (xx)])
+    for (int y = 0; y < h; ++y)
+        for (int x = 0; x < w; ++x) {
+            int sx = gx[y * w + x], sy = gy[y * w + x], mm = m[y * w + x];
+            long ax = labs((long)sx), ay = labs((long)sy);
+            int mneg, mpos;
+            if (32768 * ay <= 13573 * ax) { mneg = M(y, x - 1); mpos = M(y, x + 1); }
+            else if (32768 * ax <= 13573 * ay) { mneg = M(y - 1, x); mpos = M(y + 1, x); }
+            else if ((sx > 0) == (sy > 0)) { mneg = M(y - 1, x - 1); mpos = M(y + 1, x + 1); }
+            else { mneg = M(y - 1, x + 1); mpos = M(y + 1, x - 1); }
+            int keep = (mm > mneg) && (mm >= mpos);
+            if (keep && mm >= hi * hi) cls[y * w + x] = 2;
+            else if (keep && mm >= lo * lo) cls[y * w + x] = 1;
+        }
+#undef M
+    memset(E, 0, P);
+    int* stack = (int*)malloc(P * sizeof(int));
+    size_t top = 0;
+    for (size_t i = 0; i < P; ++i)
+        if (cls[i] == 2) { E[i] = 1; stack[top++] = (int)i; }
+    while (top) {
+        int i = stack[--top];
+        int y = i / w, x = i % w;
+        for (int dy = -1; dy <= 1; ++dy)
+            for (int dx = -1; dx <= 1; ++dx) {
+                int yy = y + dy, xx = x + dx;
+                if (yy < 0 || yy >= h || xx < 0 || xx >= w) continue;
+                int j = yy * w + xx;
+                if (cls[j] && !E[j]) { E[j] = 1; stack[top++] = j; }
+            }
+    }
+    if (cls_or_null) memcpy(cls_or_null, cls, P);
+    free(stack); free(cls); free(m); free(gy); free(gx); free(Bl);
+}
+
+/* ------------------------------------------------------------------------- */
+/* sRGB (8-bit) -> CIE L*a*b*, D65.  IEC 61966-2-1 transfer curve, sRGB        */
+/* primaries, white (0.95047, 1, 1.08883).  lab = [3] per pixel.               */
+/* ------------------------------------------------------------------------- */
+static double srgb_to_linear(int c) {
+    double v = c / 255.0;
+    return v <= 0.04045 ? v / 12.92 : pow((v + 0.055) / 1.055, 2.4);
+}
+static double lab_f(double t) {
+    const double d = 6.0 / 29.0;
+    return t > d * d * d ? cbrt(t) : t / (3.0 * d * d) + 4.0 / 29.0;
+}
+EXPORT void oracle_rgb_to_lab(const uint8_t* rgb, int n, double* lab) {
+    for (int i = 0; i < n; ++i) {
+        double r = srgb_to_linear(rgb[3 * i]), g = srgb_to_linear(rgb[3 * i + 1]), b = srgb_to_linear(rgb[3 * i + 2]);
+        double X = 0.4124564 * r + 0.3575761 * g + 0.1804375 * b;
+        double Y = 0.2126729 * r + 0.7151522 * g + 0.0721750 * b;
+        double Zv = 0.0193339 * r + 0.1191920 * g + 0.9503041 * b;
+        double fx = lab_f(X / 0.95047), fy = lab_f(Y / 1.0), fz = lab_f(Zv / 1.08883);
+        lab[3 * i] = 116.0 * fy - 16.0;
+        lab[3 * i + 1] = 500.0 * (fx - fy);
+        lab[3 * i + 2] = 200.0 * (fy - fz);
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Colour branch C (Sec. III-B "color variance analysis in the LAB color       */
+/* space", Sec. IV-B "adaptive thresholding based on the local color           */
+/* variance").  Reading: V = sum over L, a, b of the population variance in    */
+/* the (2r+1)^2 clamp-to-edge window; C = min(1, sqrt(V)/sigma_ref).           */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_color_contrast(const uint8_t* rgb, int h, int w, int radius, double sigma_ref, double* C) {
+    size_t P = (size_t)h * w;
+    double* lab = (double*)malloc(3 * P * sizeof(double));
+    oracle_rgb_to_lab(rgb, (int)P, lab);
+    int n = (2 * radius + 1) * (2 * radius + 1);
+    for (int y = 0; y < h; ++y)
+        for (int x = 0; x < w; ++x) {
+            double V = 0.0;
+            for (int c = 0; c < 3; ++c) {
+                double mean = 0.0;
+                for (int dy = -radius; dy <= radius; ++dy)
+                    for (int dx = -radius; dx <= radius; ++dx)
+                        mean += lab[3 * ((size_t)clampi(y + dy, 0, h - 1) * w + clampi(x + dx, 0, w - 1)) + c];
+                mean /= n;
+                double var = 0.0;
+                for (int dy = -radius; dy <= radius; ++dy)
+                    for (int dx = -radius; dx <= radius; ++dx) {
+                        double dv = lab[3 * ((size_t)clampi(y + dy, 0, h - 1) * w + clampi(x + dx, 0, w - 1)) + c] - mean;
+                        var += dv * dv;
+                    }
+                V += var / n;
+            }
+            double c01 = sqrt(V) / sigma_ref;
+            C[(size_t)y * w + x] = c01 < 1.0 ? c01 : 1.0;
+        }
+    free(lab);
+}
+
+/* ------------------------------------------------------------------------- */
+/* Saliency map S in [0,1] and patch score s_i (Eq. 7):                        */
+/*   S = clamp(w_edge E + w_color C, 0, 1),  s_i = mean over patch i of S.      */
+/* S_or_null receives the per-pixel map.                                       */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_saliency(const uint8_t* rgb, int h, int w, int patch, int lo, int hi, int radius,
+                            double sigma_ref, double w_edge, double w_color, double* s, double* S_or_null) {
+    size_t P = (size_t)h * w;
+    uint8_t* g = (uint8_t*)malloc(P);
+    uint8_t* E = (uint8_t*)malloc(P);
+    double* C = (double*)malloc(P * sizeof(double));
+    oracle_gray(rgb, h, w, g);
+    oracle_canny(g, h, w, lo, hi, E, NULL);
+    oracle_color_contrast(rgb, h, w, radius, sigma_ref, C);
+    int gh = h / patch, gw = w / patch;
+    for (size_t i = 0; i < P; ++i) {
+        double v = w_edge * E[i] + w_color * C[i];
+        C[i] = v < 0.0 ? 0.0 : (v > 1.0 ? 1.0 : v);
+    }
+    for (int py = 0; py < gh; ++py)
+        for (int px = 0; px < gw; ++px) {
+            double acc = 0.0;
+            for (int y = py * patch; y < (py + 1) * patch; ++y)
+                for (int x = px * patch; x < (px + 1) * patch; ++x) acc += C[(size_t)y * w + x];
+            s[py * gw + px] = acc / (double)(patch * patch);
+        }
+    if (S_or_null) memcpy(S_or_null, C, P * sizeof(double));
+    free(C); free(E); free(g);
+}
+
+EXPORT void oracle_saliency_batch(const uint8_t* frames, int B, int h, int w, int patch, int lo, int hi, int radius,
+                                  double sigma_ref, double w_edge, double w_color, double* s) {
+    size_t fb = (size_t)h * w * 3;
+    int np = (h / patch) * (w / patch);
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b)
+        oracle_saliency(frames + b * fb, h, w, patch, lo, hi, radius, sigma_ref, w_edge, w_color,
+                        s + (size_t)b * np, NULL);
+}
+
+/* ------------------------------------------------------------------------- */
+/* Decision rule for one frame (Eq. 6, Eq. 8, Alg. 1).  Scores are binary32.   */
+/*   static_i = dP_i < tau_t (strict, Eq. 6);  R = count / N_tok (binary32);   */
+/*   has_prev && R > theta_R  -> frame redundant: every token REUSE (Alg. 1    */
+/*   lines 6-8), saliency not consulted;                                       */
+/*   else, per token: patch_reuse && has_prev && static_i -> REUSE (reading:   */
+/*   Fig. 3 counts skipped *patches*), else Eq. 8 as printed.                  */
+/* Codes: 0 REUSE, 1 PRUNE, 2 INT4, 3 INT8, 4 FP16.  idx = [3][n_tok] lists    */
+/* (FP16, INT8, INT4) of ascending token ids; counts[5] by code.               */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_select(const float* dP, const float* s, int n_tok, int has_prev, int patch_reuse, float tau_t,
+                          float theta_R, float tau_high, float tau_med, float tau_low, uint8_t* decision,
+                          int32_t* idx, int32_t* counts, uint8_t* frame_redundant, float* R_out) {
+    int n_static = 0;
+    if (has_prev)
+        for (int i = 0; i < n_tok; ++i) n_static += (dP[i] < tau_t);
+    float R = has_prev ? (float)n_static / (float)n_tok : 0.0f;
+    int redundant = has_prev && (R > theta_R);
+    for (int c = 0; c < 5; ++c) counts[c] = 0;
+    int n16 = 0, n8 = 0, n4 = 0;
+    for (int i = 0; i < n_tok; ++i) {
+        uint8_t d;
+        if (redundant) d = 0;
+        else if (patch_reuse && has_prev && dP[i] < tau_t) d = 0;
+        else if (s[i] > tau_high) d = 4;
+        else if (s[i] > tau_med) d = 3;
+        else if (s[i] > tau_low) d = 2;
+        else d = 1;
+        decision[i] = d;
+        counts[d]++;
+        if (d == 4) idx[0 * n_tok + n16++] = i;
+        else if (d == 3) idx[1 * n_tok + n8++] = i;
+        else if (d == 2) idx[2 * n_tok + n4++] = i;
+    }
+    for (int i = n16; i < n_tok; ++i) idx[0 * n_tok + i] = -1;
+    for (int i = n8; i < n_tok; ++i) idx[1 * n_tok + i] = -1;
+    for (int i = n4; i < n_tok; ++i) idx[2 * n_tok + i] = -1;
+    *frame_redundant = (uint8_t)redundant;
+    if (R_out) *R_out = R;
+}
+
+/* ------------------------------------------------------------------------- */
+/* binary16 <-> binary32, written out on the bits (round to nearest even).     */
+/* ------------------------------------------------------------------------- */
+EXPORT float oracle_half_to_float(uint16_t hbits) {
+    int sign = (hbits >> 15) & 1, e = (hbits >> 10) & 31, mant = hbits & 1023;
+    float v;
+    if (e == 0) v = ldexpf((float)mant, -24);
+    else if (e == 31) v = mant ? NAN : INFINITY;
+    else v = ldexpf((float)(mant | 1024), e - 25);
+    return sign ? -v : v;
+}
+
+EXPORT uint16_t oracle_float_to_half(float f) {
+    uint32_t x;
+    memcpy(&x, &f, 4);
+    uint16_t sign = (uint16_t)((x >> 16) & 0x8000u);
+    uint32_t a = x & 0x7fffffffu;
+    if (a > 0x7f800000u) return (uint16_t)(sign | 0x7e00u);      /* NaN */
+    if (a >= 0x477ff000u) return (uint16_t)(sign | 0x7c00u);     /* >= 65520 rounds to inf */
+    if (a <= 0x33000000u) return sign;                           /* <= 2^-25 rounds to 0 */
+    int e = (int)(a >> 23) - 127;
+    uint32_t mant = (a & 0x7fffffu) | 0x800000u;                 /* 24-bit significand */
+    int shift = e >= -14 ? 13 : 13 + (-14 - e);                  /* bits dropped */
+    uint32_t kept = mant >> shift;
+    uint32_t rem = mant & ((1u << shift) - 1u), half = 1u << (shift - 1);
+    if (rem > half || (rem == half && (kept & 1u))) kept++;
+    uint32_t out;
+    if (e >= -14) out = ((uint32_t)(e + 14) << 10) + kept;        /* kept carries the implicit 1 (1<<10) */
+    else out = kept;                                             /* subnormal; a carry lands on 2^-14 */
+    return (uint16_t)(sign | out);
+}
+
+/* ------------------------------------------------------------------------- */
+/* Quantisers (Sec. IV-B: symmetric min-max INT8, asymmetric INT4), one group  */
+/* of G consecutive fp16 elements.  Reading of what the paper leaves open:     */
+/* scale and zero are stored as fp16 and quantisation uses the STORED scale;   */
+/* q = rint(x * (1/s)) with a multiply (not a divide, not an FMA), rint =      */
+/* round half to even; a zero range takes s = 1.                               */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_quant_int8_group(const uint16_t* x, int G, int8_t* q, uint16_t* scale16) {
+    float amax = 0.0f;
+    for (int i = 0; i < G; ++i) {
+        float v = fabsf(oracle_half_to_float(x[i]));
+        if (v > amax) amax = v;
+    }
+    uint16_t s16 = oracle_float_to_half(amax / 127.0f);
+    if ((s16 & 0x7fffu) == 0) s16 = 0x3c00u;
+    float s = oracle_half_to_float(s16);
+    float inv = 1.0f / s;
+    for (int i = 0; i < G; ++i) {
+        volatile float p = oracle_half_to_float(x[i]) * inv;
+        float r = rintf(p);
+        if (r > 127.0f) r = 127.0f;
+        if (r < -127.0f) r = -127.0f;
+        q[i] = (int8_t)r;
+    }
+    *scale16 = s16;
+}
+
+EXPORT void oracle_dequant_int8_group(const int8_t* q, int G, uint16_t scale16, uint16_t* xh) {
+    float s = oracle_half_to_float(scale16);
+    for (int i = 0; i < G; ++i) {
+        volatile float p = (float)q[i] * s;
+        xh[i] = oracle_float_to_half(p);
+    }
+}
+
+/* INT4 asymmetric: s = fp16((max - min)/15), zero point = the group minimum    */
+/* kept as fp16; q = clamp(rint((x - z) * (1/s)), 0, 15); element 2j in the    */
+/* low nibble of byte j, 2j+1 in the high nibble.                              */
+EXPORT void oracle_quant_int4_group(const uint16_t* x, int G, uint8_t* packed, uint16_t* scale16, uint16_t* zero16) {
+    float mn = INFINITY, mx = -INFINITY;
+    uint16_t mn16 = 0;
+    for (int i = 0; i < G; ++i) {
+        float v = oracle_half_to_float(x[i]);
+        if (v < mn) { mn = v; mn16 = x[i]; }
+        if (v > mx) mx = v;
+    }
+    if (mn == 0.0f) mn16 = 0; /* -0 and +0 compare equal: store +0 */
+    volatile float range = mx - mn;
+    uint16_t s16 = oracle_float_to_half(range / 15.0f);
+    if ((s16 & 0x7fffu) == 0) s16 = 0x3c00u;
+    float s = oracle_half_to_float(s16);
+    float inv = 1.0f / s;
+    float z = oracle_half_to_float(mn16);
+    for (int i = 0; i < G; i += 2) {
+        uint8_t qq[2];
+        for (int j = 0; j < 2; ++j) {
+            volatile float dlt = oracle_half_to_float(x[i + j]) - z;
+            volatile float p = dlt * inv;
+            float r = rintf(p);
+            if (r > 15.0f) r = 15.0f;
+            if (r < 0.0f) r = 0.0f;
+            qq[j] = (uint8_t)r;
+        }
+        packed[i / 2] = (uint8_t)(qq[0] | (qq[1] << 4));
+    }
+    *scale16 = s16;
+    *zero16 = mn16;
+}
+
+EXPORT void oracle_dequant_int4_group(const uint8_t* packed, int G, uint16_t scale16, uint16_t zero16, uint16_t* xh) {
+    float s = oracle_half_to_float(scale16), z = oracle_half_to_float(zero16);
+    for (int i = 0; i < G; ++i) {
+        int q = (i & 1) ? (packed[i / 2] >> 4) : (packed[i / 2] & 15);
+        volatile float p = (float)q * s;
+        volatile float r = p + z;
+        xh[i] = oracle_float_to_half(r);
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Mixed-precision store of one frame's K/V (Alg. 1 line 16).                  */
+/* K, V: fp16 bits [L][n_tok][HD].  Pools (per tier, shared by all frames):    */
+/*   fp16_pool  u16 [L][2][cap16][HD]                                          */
+/*   int8_codes i8  [L][2][cap8][HD],   int8_scale u16 [L][2][cap8][HD/G]      */
+/*   int4_codes u8  [L][2][cap4][HD/2], int4_sz    u16 [L][2][cap4][HD/G][2]   */
+/* The j-th token of a tier list goes to row (off + j) mod cap of that tier    */
+/* (ring != 0) or row off + j (ring == 0; rows past cap are dropped and the    */
+/* return value is -1).  Index 0 of the second axis is K, 1 is V.              */
+/* ------------------------------------------------------------------------- */
+static int64_t pool_row(int64_t off, int64_t j, int64_t cap, int ring) {
+    int64_t r = off + j;
+    if (ring) return cap > 0 ? r % cap : -1;
+    return r < cap ? r : -1;
+}
+
+EXPORT int oracle_pack_frame(const uint16_t* K, const uint16_t* V, int L, int n_tok, int HD, int G,
+                             const int32_t* idx, const int32_t* counts, const int64_t* off, int ring,
+                             uint16_t* fp16_pool, int64_t cap16, int8_t* int8_codes, uint16_t* int8_scale,
+                             int64_t cap8, uint8_t* int4_codes, uint16_t* int4_sz, int64_t cap4) {
+    int status = 0;
+    int ng = HD / G;
+    int n16 = counts[4], n8 = counts[3], n4 = counts[2];
+#pragma omp parallel for schedule(static) reduction(min : status)
+    for (int l = 0; l < L; ++l)
+        for (int kv = 0; kv < 2; ++kv) {
+            const uint16_t* src = (kv ? V : K) + (size_t)l * n_tok * HD;
+            size_t plane = (size_t)l * 2 + kv;
+            for (int j = 0; j < n16; ++j) {
+                int64_t r = pool_row(off[0], j, cap16, ring);
+                if (r < 0) { status = -1; continue; }
+                memcpy(fp16_pool + (plane * cap16 + r) * HD, src + (size_t)idx[0 * n_tok + j] * HD, (size_t)HD * 2);
+            }
+            for (int j = 0; j < n8; ++j) {
+                int64_t r = pool_row(off[1], j, cap8, ring);
+                if (r < 0) { status = -1; continue; }
+                const uint16_t* row = src + (size_t)idx[1 * n_tok + j] * HD;
+                for (int g = 0; g < ng; ++g)
+                    oracle_quant_int8_group(row + g * G, G, int8_codes + (plane * cap8 + r) * HD + g * G,
+                                            int8_scale + (plane * cap8 + r) * ng + g);
+            }
+            for (int j = 0; j < n4; ++j) {
+                int64_t r = pool_row(off[2], j, cap4, ring);
+                if (r < 0) { status = -1; continue; }
+                const uint16_t* row = src + (size_t)idx[2 * n_tok + j] * HD;
+                for (int g = 0; g < ng; ++g)
+                    oracle_quant_int4_group(row + g * G, G, int4_codes + (plane * cap4 + r) * (HD / 2) + g * (G / 2),
+                                            int4_sz + ((plane * cap4 + r) * ng + g) * 2,
+                                            int4_sz + ((plane * cap4 + r) * ng + g) * 2 + 1);
+            }
+        }
+    return status;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Just-in-time dequantisation of one frame (Sec. III-C) into dense fp16       */
+/* K^, V^ [L][n_tok][HD].  FP16 rows are bit copies.  PRUNE rows are zeroed    */
+/* when zero_fill_pruned; REUSE rows are left untouched (the caller resolves   */
+/* them through the source-frame table).                                       */
+/* ------------------------------------------------------------------------- */
+EXPORT int oracle_unpack_frame(int L, int n_tok, int HD, int G, const int32_t* idx, const int32_t* counts,
+                               const uint8_t* decision, const int64_t* off, int ring, const uint16_t* fp16_pool,
+                               int64_t cap16, const int8_t* int8_codes, const uint16_t* int8_scale, int64_t cap8,
+                               const uint8_t* int4_codes, const uint16_t* int4_sz, int64_t cap4,
+                               int zero_fill_pruned, uint16_t* K_out, uint16_t* V_out) {
+    int status = 0;
+    int ng = HD / G;
+    int n16 = counts[4], n8 = counts[3], n4 = counts[2];
+#pragma omp parallel for schedule(static) reduction(min : status)
+    for (int l = 0; l < L; ++l)
+        for (int kv = 0; kv < 2; ++kv) {
+            uint16_t* dst = (kv ? V_out : K_out) + (size_t)l * n_tok * HD;
+            size_t plane = (size_t)l * 2 + kv;
+            for (int j = 0; j < n16; ++j) {
+                int64_t r = pool_row(off[0], j, cap16, ring);
+                if (r < 0) { status = -1; continue; }
+                memcpy(dst + (size_t)idx[0 * n_tok + j] * HD, fp16_pool + (plane * cap16 + r) * HD, (size_t)HD * 2);
+            }
+            for (int j = 0; j < n8; ++j) {
+                int64_t r = pool_row(off[1], j, cap8, ring);
+                if (r < 0) { status = -1; continue; }
+                uint16_t* row = dst + (size_t)idx[1 * n_tok + j] * HD;
+                for (int g = 0; g < ng; ++g)
+                    oracle_dequant_int8_group(int8_codes + (plane * cap8 + r) * HD + g * G, G,
+                                              int8_scale[(plane * cap8 + r) * ng + g], row + g * G);
+            }
+            for (int j = 0; j < n4; ++j) {
+                int64_t r = pool_row(off[2], j, cap4, ring);
+                if (r < 0) { status = -1; continue; }
+                uint16_t* row = dst + (size_t)idx[2 * n_tok + j] * HD;
+                for (int g = 0; g < ng; ++g)
+                    oracle_dequant_int4_group(int4_codes + (plane * cap4 + r) * (HD / 2) + g * (G / 2), G,
+                                              int4_sz[((plane * cap4 + r) * ng + g) * 2],
+                                              int4_sz[((plane * cap4 + r) * ng + g) * 2 + 1], row + g * G);
+            }
+            if (zero_fill_pruned)
+                for (int i = 0; i < n_tok; ++i)
+                    if (decision[i] == 1) memset(dst + (size_t)i * HD, 0, (size_t)HD * 2);
+        }
+    return status;
+}
