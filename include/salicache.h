@@ -1,0 +1,190 @@
+/*
+ * salicache.h -- C ABI of the B200 (sm_100a) Sali-Cache pre-attention filter and
+ * mixed-precision K/V store.
+ *
+ * The hot path every video frame takes before its visual tokens reach attention
+ * (paper Sec. III, Alg. 1):
+ *     flow_score  ->  saliency  ->  select  ->  pack_kv        (+ unpack_kv)
+ *
+ * Conventions
+ *   - Pointers named d_* are DEVICE pointers owned by the caller; h_* are HOST
+ *     pointers.  The library never frees or reallocates caller memory.
+ *   - A context owns only its scratch memory, sized at salicache_create.  No hot
+ *     call allocates.
+ *   - Every hot call is asynchronous on `cuda_stream` (a cudaStream_t passed as
+ *     void*; NULL = the default stream) and does not synchronise the host.
+ *   - Return value: 0 on success, a negative SALICACHE_E_* code otherwise.  No
+ *     exceptions, no abort, no device trap.  Conditions only the device can see
+ *     (pool overflow, hysteresis iteration cap) are recorded in a device status
+ *     word and returned by salicache_poll_status.
+ *   - Frames are uint8 HWC (R,G,B), 16-byte aligned, W a multiple of 16.
+ *   - K/V are IEEE binary16, finite; NaN/Inf inputs give unspecified codes.
+ *   - One context is used by one host thread at a time; contexts are independent.
+ */
+#ifndef SALICACHE_H
+#define SALICACHE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define SALICACHE_API __attribute__((visibility("default")))
+#else
+#define SALICACHE_API
+#endif
+
+#define SALICACHE_OK            0
+#define SALICACHE_E_NULL       -1   /* a required pointer is NULL                          */
+#define SALICACHE_E_SHAPE      -2   /* sizes inconsistent with the context                 */
+#define SALICACHE_E_ALIGN      -3   /* a pointer is not 16-byte aligned                    */
+#define SALICACHE_E_PARAM      -4   /* unsupported parameter value                         */
+#define SALICACHE_E_CUDA       -5   /* a CUDA runtime call failed                          */
+#define SALICACHE_E_CAPACITY   -6   /* a tier pool is too small (rows dropped, ring == 0)  */
+#define SALICACHE_E_NOCONVERGE -7   /* edge hysteresis hit hyst_max_iters                  */
+#define SALICACHE_E_NOMEM      -8   /* scratch allocation failed at create                 */
+
+/* Decision code per token (Fig. 3 categories; Eq. 8 tiers). */
+#define SALICACHE_REUSE 0   /* "skipped": K/V of the previous frame's token is reused       */
+#define SALICACHE_PRUNE 1
+#define SALICACHE_INT4  2
+#define SALICACHE_INT8  3
+#define SALICACHE_FP16  4
+
+typedef struct salicache_ctx salicache_ctx;
+
+/* Parameters.  The paper fixes: Farneback flow with pyramid scale 0.5 and 3 levels,
+ * Canny + LAB colour variance, Eq. 5-8, symmetric INT8 and asymmetric INT4 (Sec. IV-B).
+ * It prints no value for any threshold (Alg. 1 input); the other fields are the
+ * readings this library takes where the paper is silent. */
+typedef struct salicache_params {
+    int32_t H, W;            /* frame size; multiples of `patch`, W % 16 == 0 (336 or 672)          */
+    int32_t patch;           /* 14 (Sec. II-A)                                                       */
+    int32_t n_images;        /* 1, or 5 = anyres: 336x336 base (2x2 box mean of the frame) followed  */
+                             /* by the 2x2 grid of 336x336 tiles; H = W = 672 then                   */
+    int32_t max_batch;       /* largest B accepted by any call                                       */
+    int32_t chunk_frames;    /* frames per internal pass of flow/saliency (scratch size); 0 = 16     */
+    /* temporal branch */
+    int32_t pyr_levels;      /* 3 (only value supported)                                             */
+    int32_t poly_n;          /* 5 (only value supported)                                             */
+    double  poly_sigma;      /* 1.2                                                                  */
+    int32_t win;             /* 15 (only value supported)                                            */
+    int32_t iters;           /* updates per level, 3                                                 */
+    double  eps_det;         /* regulariser added to det G, 1e-3                                     */
+    /* spatial branch */
+    int32_t canny_lo, canny_hi;   /* 50, 150 on the Sobel magnitude                                  */
+    int32_t var_radius;      /* 3 (7x7 window; only value supported)                                 */
+    double  sigma_ref;       /* 16.0: C = min(1, sqrt(V)/sigma_ref)                                  */
+    double  w_edge, w_color; /* 0.5, 0.5                                                             */
+    int32_t hyst_max_iters;  /* 4096                                                                 */
+    /* decisions (Alg. 1 input) */
+    float   tau_t, theta_R, tau_high, tau_med, tau_low;
+    int32_t patch_reuse;     /* 1: static patches of a non-redundant frame are REUSE (Fig. 3)        */
+    /* K/V shape and quantiser */
+    int32_t L, heads, head_dim;   /* layers, heads, head size; heads*head_dim = row length HD        */
+    int32_t group;           /* elements per quantisation group: 128 (only value supported)          */
+} salicache_params;
+
+/* Fills *p with the defaults listed above for a 336x336, L=32, 32x128 configuration. */
+SALICACHE_API int salicache_default_params(salicache_params* p);
+
+/* Allocates a context and its scratch on the current CUDA device.  Errors: E_NULL, E_PARAM
+ * (unsupported value), E_SHAPE (sizes not multiples), E_NOMEM, E_CUDA. */
+SALICACHE_API int salicache_create(salicache_ctx** out, const salicache_params* p);
+SALICACHE_API int salicache_destroy(salicache_ctx* ctx);
+SALICACHE_API const char* salicache_strerror(int status);
+
+/* Tokens per frame: n_images * (336/patch)^2 for anyres, else (H/patch)*(W/patch). */
+SALICACHE_API int salicache_tokens_per_frame(const salicache_ctx* ctx);
+
+/*
+ * Temporal score (Sec. III-A, Eq. 5; Farneback flow, Sec. IV-B).
+ * For b in [0,B): dense flow from d_prev[b] to d_cur[b] (frames of H*W*3 bytes, consecutive),
+ * reduced to d_deltaP[b][i] = RMS flow magnitude (pixels) over patch i, i in token order.
+ * d_cur == d_prev + H*W*3 (a video: pair b is frames b, b+1) is recognised and each frame is
+ * expanded once.  d_flow_or_null, if given, receives the level-0 flow as double [B][2][H][W]
+ * (u along x, then v); anyres contexts write only the full-resolution field.
+ * Device arithmetic: double.  Errors: E_NULL, E_SHAPE (B < 0 or > max_batch), E_ALIGN, E_CUDA.
+ */
+SALICACHE_API int salicache_flow_score(salicache_ctx* ctx, const uint8_t* d_prev, const uint8_t* d_cur, int B,
+                         float* d_deltaP, double* d_flow_or_null, void* cuda_stream);
+
+/*
+ * Spatial score (Sec. III-B, Eq. 7): Canny edge map E and LAB local colour variance C give
+ * S = clamp(w_edge E + w_color C, 0, 1); d_s[b][i] = mean of S over patch i.
+ * d_frames: B frames.  Edge hysteresis runs to its fixed point on the device; if it needs more
+ * than hyst_max_iters sweeps the status word records E_NOCONVERGE (see salicache_poll_status).
+ */
+SALICACHE_API int salicache_saliency(salicache_ctx* ctx, const uint8_t* d_frames, int B, float* d_s, void* cuda_stream);
+
+/*
+ * Decisions (Eq. 6, Eq. 8, Alg. 1) for B frames, one row of d_deltaP / d_s per frame.
+ * d_deltaP may be NULL (no frame has a predecessor).  If first_has_no_prev != 0, frame 0 is the
+ * first frame of the video: its d_deltaP row is ignored and it is never REUSE (Alg. 1 line 4).
+ * Outputs (all device):
+ *   d_decision        u8  [B][N_tok]     SALICACHE_* code per token
+ *   d_idx             i32 [B][3][N_tok]  ascending token ids kept as FP16 / INT8 / INT4; -1 padded
+ *   d_counts          i32 [B][5]         tokens per code (indexed by code)
+ *   d_frame_redundant u8  [B]            1 when R_frame > theta_R (whole frame points at t-1)
+ *   d_row_offset      i64 [B][3]         first pool row of the frame in the FP16 / INT8 / INT4 pool
+ *   d_fill            i64 [3]            running rows written per pool; read, used as the offset of
+ *                                        frame 0 and advanced by the batch totals (zero it once)
+ * pack_kv / unpack_kv consume these from device memory: no host round trip is needed.
+ */
+SALICACHE_API int salicache_select(salicache_ctx* ctx, const float* d_deltaP, const float* d_s, int B, int first_has_no_prev,
+                     uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts, uint8_t* d_frame_redundant,
+                     int64_t* d_row_offset, int64_t* d_fill, void* cuda_stream);
+
+/* Per-tier pools of the mixed-precision store (device memory, caller-owned).  Axis 2 of the
+ * second dimension: 0 = K, 1 = V.  ng = HD / group.
+ *   fp16_pool   f16 [L][2][cap_fp16][HD]
+ *   int8_codes  i8  [L][2][cap_int8][HD]      int8_scale f16 [L][2][cap_int8][ng]
+ *   int4_codes  u8  [L][2][cap_int4][HD/2]    int4_sz    f16 [L][2][cap_int4][ng][2]  (scale, zero)
+ * The j-th token of a frame's tier list lives in row (row_offset + j) % cap when ring != 0
+ * (oldest rows are overwritten: oldest-first eviction; one call must not store more than cap
+ * rows in a pool, or rows of the same call overwrite each other in unspecified order), else in
+ * row row_offset + j, and rows at or past cap are dropped with E_CAPACITY in the status word. */
+typedef struct salicache_pools {
+    void* fp16_pool;
+    void* int8_codes;
+    void* int8_scale;
+    void* int4_codes;
+    void* int4_sz;
+    int64_t cap_fp16, cap_int8, cap_int4;
+    int32_t ring;
+} salicache_pools;
+
+/*
+ * Mixed-precision store (Alg. 1 line 16; quantisers of Sec. IV-B).  d_K, d_V: f16
+ * [B][L][N_tok][HD] with `frame_stride` elements between frames (L*N_tok*HD when dense).
+ * FP16 rows are copied; INT8: s = fp16(max|x|/127), q = rint(x * (1/s)); INT4: s =
+ * fp16((max-min)/15), zero = min (fp16), q = rint((x - zero) * (1/s)), element 2j in the low
+ * nibble; s == 0 -> 1.  All binary32, round-to-nearest-even, no fused multiply-add.
+ * PRUNE and REUSE tokens move no bytes.  Errors: E_NULL, E_SHAPE, E_ALIGN, E_CUDA; deferred
+ * E_CAPACITY.
+ */
+SALICACHE_API int salicache_pack_kv(salicache_ctx* ctx, const void* d_K, const void* d_V, int64_t frame_stride,
+                      const int32_t* d_idx, const int32_t* d_counts, const int64_t* d_row_offset, int B,
+                      const salicache_pools* pools, void* cuda_stream);
+
+/*
+ * Just-in-time dequantisation (Sec. III-C) into dense f16 d_K_out, d_V_out [B][L][N_tok][HD].
+ * INT8: fp16(q*s); INT4: fp16(q*s + zero) (multiply, then add); FP16 rows are bit copies;
+ * PRUNE rows are zeroed when zero_fill_pruned != 0, otherwise untouched; REUSE rows are left
+ * untouched (the caller resolves them through its source-frame table).
+ */
+SALICACHE_API int salicache_unpack_kv(salicache_ctx* ctx, const salicache_pools* pools, const int32_t* d_idx,
+                        const int32_t* d_counts, const uint8_t* d_decision, const int64_t* d_row_offset, int B,
+                        int zero_fill_pruned, void* d_K_out, void* d_V_out, int64_t frame_stride,
+                        void* cuda_stream);
+
+/* Synchronises `cuda_stream`, returns the deferred device status (0, E_CAPACITY or
+ * E_NOCONVERGE; E_CUDA if the stream reports an error) and clears it. */
+SALICACHE_API int salicache_poll_status(salicache_ctx* ctx, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SALICACHE_H */

@@ -1,0 +1,319 @@
+// Spatial branch (Sec. III-B, Eq. 7): integer Canny edge map, LAB local colour variance,
+// S = clamp(w_edge E + w_color C, 0, 1), per-patch mean.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace {
+
+__device__ __forceinline__ int clampi(int v, int lo, int hi) { return v < lo ? lo : (v > hi ? hi : v); }
+
+__device__ __forceinline__ int gray_at(const uint8_t* __restrict__ fr, int w, int y, int x) {
+    const uint8_t* p = fr + ((size_t)y * w + x) * 3;
+    return (77 * p[0] + 150 * p[1] + 29 * p[2] + 128) >> 8;
+}
+
+// ---- anyres base image: 2x2 integer box mean (a+b+c+d+2)>>2 per channel.
+__global__ void k_box_down2(const uint8_t* __restrict__ src, int H, int W, int n_frames, uint8_t* __restrict__ dst) {
+    int h2 = H / 2, w2 = W / 2;
+    long long gid = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (gid >= (long long)h2 * w2 * n_frames) return;
+    int f = (int)(gid / (h2 * w2)), r = (int)(gid % (h2 * w2));
+    int y = r / w2, x = r % w2;
+    const uint8_t* s = src + (size_t)f * H * W * 3;
+    const uint8_t* a = s + ((size_t)(2 * y) * W + 2 * x) * 3;
+    const uint8_t* b = a + (size_t)W * 3;
+    uint8_t* o = dst + ((size_t)f * h2 * w2 + r) * 3;
+#pragma unroll
+    for (int c = 0; c < 3; ++c) o[c] = (uint8_t)((a[c] + a[3 + c] + b[c] + b[3 + c] + 2) >> 2);
+}
+
+// ---- Canny up to the double threshold.  Tile 32x32, halo 4 (blur 2 + Sobel 1 + NMS 1).
+// Writes two bit planes (bit i of word wx = pixel 32*wx + i): kept = NMS-kept with m >= lo^2,
+// strong = kept with m >= hi^2.
+constexpr int CT = 32;
+constexpr int CG = CT + 8;   // gray tile
+constexpr int CB = CT + 4;   // blur tile
+constexpr int CM = CT + 2;   // magnitude tile
+
+__global__ void __launch_bounds__(256)
+k_canny_classify(const uint8_t* __restrict__ frames, size_t frame_bytes, int h, int w, int words, int lo2, int hi2,
+                 uint32_t* __restrict__ bits_kept, uint32_t* __restrict__ bits_strong) {
+    __shared__ uint8_t sg[CG][CG];
+    __shared__ uint8_t sb[CB][CB];
+    __shared__ int smag[CM][CM];
+    const int f = blockIdx.z, x0 = blockIdx.x * CT, y0 = blockIdx.y * CT;
+    const uint8_t* fr = frames + (size_t)f * frame_bytes;
+    for (int i = threadIdx.x; i < CG * CG; i += blockDim.x) {
+        int ry = i / CG, rx = i % CG;
+        sg[ry][rx] = (uint8_t)gray_at(fr, w, clampi(y0 - 4 + ry, 0, h - 1), clampi(x0 - 4 + rx, 0, w - 1));
+    }
+    __syncthreads();
+    // blur at the clamped position, so that the Sobel taps read Bl(clamp(y), clamp(x))
+    for (int i = threadIdx.x; i < CB * CB; i += blockDim.x) {
+        int ry = i / CB, rx = i % CB;
+        int yc = clampi(y0 - 2 + ry, 0, h - 1), xc = clampi(x0 - 2 + rx, 0, w - 1);
+        int gy0 = yc - (y0 - 4), gx0 = xc - (x0 - 4);
+        const int k[5] = {1, 4, 6, 4, 1};
+        int acc = 0;
+#pragma unroll
+        for (int a = -2; a <= 2; ++a) {
+            int ra = 0;
+#pragma unroll
+            for (int b = -2; b <= 2; ++b) ra += k[b + 2] * sg[gy0 + a][gx0 + b];
+            acc += k[a + 2] * ra;
+        }
+        sb[ry][rx] = (uint8_t)((acc + 128) >> 8);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < CM * CM; i += blockDim.x) {
+        int ry = i / CM, rx = i % CM;
+        int y = y0 - 1 + ry, x = x0 - 1 + rx;
+        int m = 0;
+        if (y >= 0 && y < h && x >= 0 && x < w) {
+            int by = ry + 1, bx = rx + 1;   // position in the blur tile
+            int gx = (sb[by - 1][bx + 1] + 2 * sb[by][bx + 1] + sb[by + 1][bx + 1]) -
+                     (sb[by - 1][bx - 1] + 2 * sb[by][bx - 1] + sb[by + 1][bx - 1]);
+            int gy = (sb[by + 1][bx - 1] + 2 * sb[by + 1][bx] + sb[by + 1][bx + 1]) -
+                     (sb[by - 1][bx - 1] + 2 * sb[by - 1][bx] + sb[by - 1][bx + 1]);
+            m = gx * gx + gy * gy;
+        }
+        smag[ry][rx] = m;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < CT * CT; i += blockDim.x) {
+        int oy = i / CT, ox = i % CT;     // a warp covers one row of the tile
+        int y = y0 + oy, x = x0 + ox;
+        int cls = 0;
+        if (y < h && x < w) {
+            int by = oy + 2, bx = ox + 2;
+            int gx = (sb[by - 1][bx + 1] + 2 * sb[by][bx + 1] + sb[by + 1][bx + 1]) -
+                     (sb[by - 1][bx - 1] + 2 * sb[by][bx - 1] + sb[by + 1][bx - 1]);
+            int gy = (sb[by + 1][bx - 1] + 2 * sb[by + 1][bx] + sb[by + 1][bx + 1]) -
+                     (sb[by - 1][bx - 1] + 2 * sb[by - 1][bx] + sb[by - 1][bx + 1]);
+            int my = oy + 1, mx = ox + 1;
+            int mm = smag[my][mx];
+            int ax = abs(gx), ay = abs(gy);
+            int mneg, mpos;
+            if (32768 * ay <= 13573 * ax) { mneg = smag[my][mx - 1]; mpos = smag[my][mx + 1]; }
+            else if (32768 * ax <= 13573 * ay) { mneg = smag[my - 1][mx]; mpos = smag[my + 1][mx]; }
+            else if ((gx > 0) == (gy > 0)) { mneg = smag[my - 1][mx - 1]; mpos = smag[my + 1][mx + 1]; }
+            else { mneg = smag[my - 1][mx + 1]; mpos = smag[my + 1][mx - 1]; }
+            bool keep = (mm > mneg) && (mm >= mpos);
+            if (keep && mm >= hi2) cls = 2;
+            else if (keep && mm >= lo2) cls = 1;
+        }
+        uint32_t kept = __ballot_sync(0xffffffffu, cls > 0);
+        uint32_t strong = __ballot_sync(0xffffffffu, cls == 2);
+        if ((threadIdx.x & 31) == 0 && y < h) {
+            size_t o = ((size_t)f * h + y) * words + blockIdx.x;
+            bits_kept[o] = kept;
+            bits_strong[o] = strong;
+        }
+    }
+}
+
+// ---- hysteresis to the fixed point: one CTA per frame, both bit planes in shared memory.
+// E starts as the strong plane and grows through 8-neighbours restricted to the kept plane.
+// Every word is owned by one thread (updates are monotone, so stale neighbour reads only delay).
+__global__ void __launch_bounds__(1024)
+k_hysteresis(const uint32_t* __restrict__ bits_kept, uint32_t* __restrict__ bits_edge, int h, int words, int max_iters,
+             int* __restrict__ status) {
+    extern __shared__ uint32_t sh[];
+    uint32_t* K = sh;                      // [h][words]
+    uint32_t* E = sh + (size_t)h * words;  // [h][words]
+    const int f = blockIdx.x, n = h * words;
+    const uint32_t* gk = bits_kept + (size_t)f * n;
+    uint32_t* ge = bits_edge + (size_t)f * n;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) { K[i] = gk[i]; E[i] = ge[i]; }
+    __syncthreads();
+    int it = 0;
+    for (;;) {
+        int changed = 0;
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            uint32_t k = K[i], e = E[i];
+            if (k == e) continue;
+            int y = i / words, wx = i % words;
+            uint32_t acc = 0;
+#pragma unroll
+            for (int dy = -1; dy <= 1; ++dy) {
+                int yy = y + dy;
+                if (yy < 0 || yy >= h) continue;
+                const uint32_t* row = E + yy * words;
+                uint32_t v = row[wx];
+                uint32_t l = wx > 0 ? row[wx - 1] : 0u;
+                uint32_t r = wx + 1 < words ? row[wx + 1] : 0u;
+                acc |= v | (v << 1) | (v >> 1) | (l >> 31) | (r << 31);
+            }
+            uint32_t ne = (e | acc) & k;
+            for (;;) {   // run along the row inside the word
+                uint32_t g = (ne | (ne << 1) | (ne >> 1)) & k;
+                if (g == ne) break;
+                ne = g;
+            }
+            if (ne != e) { E[i] = ne; changed = 1; }
+        }
+        if (!__syncthreads_or(changed)) break;
+        if (++it >= max_iters) {
+            if (threadIdx.x == 0) atomicMin(status, SALICACHE_E_NOCONVERGE);
+            break;
+        }
+    }
+    for (int i = threadIdx.x; i < n; i += blockDim.x) ge[i] = E[i];
+}
+
+// ---- sRGB -> CIE L*a*b* (D65) in double; cube root = float seed + one Newton step in double.
+__device__ __forceinline__ double lab_f(double t) {
+    const double d = 6.0 / 29.0;
+    if (t > d * d * d) {
+        double y = (double)cbrtf((float)t);          // relative error ~1e-7; one Newton step squares it
+        return y - (y * y * y - t) / (3.0 * y * y);
+    }
+    return t / (3.0 * d * d) + 4.0 / 29.0;
+}
+__device__ __forceinline__ void rgb_to_lab(const double* __restrict__ lut, int R, int G, int B, double& L, double& a,
+                                           double& b) {
+    double r = lut[R], g = lut[G], bl = lut[B];
+    double X = 0.4124564 * r + 0.3575761 * g + 0.1804375 * bl;
+    double Y = 0.2126729 * r + 0.7151522 * g + 0.0721750 * bl;
+    double Z = 0.0193339 * r + 0.1191920 * g + 0.9503041 * bl;
+    double fx = lab_f(X / 0.95047), fy = lab_f(Y), fz = lab_f(Z / 1.08883);
+    L = 116.0 * fy - 16.0;
+    a = 500.0 * (fx - fy);
+    b = 200.0 * (fy - fz);
+}
+
+// ---- colour branch + blend + patch mean.  One CTA per 2x2 patches (28x28 pixels), halo 3.
+// Variances are taken about the LAB value of the tile's first pixel (variance is shift invariant),
+// which keeps flat regions exactly zero and small contrasts accurate.
+constexpr int ST = 28;
+constexpr int SR = 3;
+constexpr int SE = ST + 2 * SR;   // 34
+
+__global__ void __launch_bounds__(256)
+k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom g, int patch,
+              const double* __restrict__ lut, const uint32_t* __restrict__ bits_edge, int words, double inv_sigma,
+              double w_edge, double w_color, float* __restrict__ s_out) {
+    extern __shared__ double cs[];
+    double (*lab)[SE][SE + 1] = reinterpret_cast<double (*)[SE][SE + 1]>(cs);                    // [3]
+    double (*hs)[SE][ST] = reinterpret_cast<double (*)[SE][ST]>(cs + 3 * SE * (SE + 1));          // [6]
+    __shared__ double psum[8][4];
+    const int f = blockIdx.z, x0 = blockIdx.x * ST, y0 = blockIdx.y * ST;
+    const int h = g.H, w = g.W;
+    const uint8_t* fr = frames + (size_t)f * frame_bytes;
+    double L0, a0, b0;
+    {
+        const uint8_t* p = fr + ((size_t)y0 * w + x0) * 3;
+        rgb_to_lab(lut, p[0], p[1], p[2], L0, a0, b0);
+    }
+    for (int i = threadIdx.x; i < SE * SE; i += blockDim.x) {
+        int ry = i / SE, rx = i % SE;
+        const uint8_t* p = fr + ((size_t)clampi(y0 - SR + ry, 0, h - 1) * w + clampi(x0 - SR + rx, 0, w - 1)) * 3;
+        double L, a, b;
+        rgb_to_lab(lut, p[0], p[1], p[2], L, a, b);
+        lab[0][ry][rx] = L - L0;
+        lab[1][ry][rx] = a - a0;
+        lab[2][ry][rx] = b - b0;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 3 * SE * ST; i += blockDim.x) {
+        int c = i / (SE * ST), r = i % (SE * ST);
+        int ry = r / ST, ox = r % ST;
+        double s1 = 0.0, s2 = 0.0;
+#pragma unroll
+        for (int k = 0; k < 2 * SR + 1; ++k) {
+            double v = lab[c][ry][ox + k];
+            s1 += v;
+            s2 += v * v;
+        }
+        hs[c][ry][ox] = s1;
+        hs[3 + c][ry][ox] = s2;
+    }
+    __syncthreads();
+    const double inv_n = 1.0 / (double)((2 * SR + 1) * (2 * SR + 1));
+    double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;   // the four patches of the tile
+    for (int i = threadIdx.x; i < ST * ST; i += blockDim.x) {
+        int oy = i / ST, ox = i % ST;
+        double V = 0.0;
+#pragma unroll
+        for (int c = 0; c < 3; ++c) {
+            double s1 = 0.0, s2 = 0.0;
+#pragma unroll
+            for (int k = 0; k < 2 * SR + 1; ++k) {
+                s1 += hs[c][oy + k][ox];
+                s2 += hs[3 + c][oy + k][ox];
+            }
+            double mean = s1 * inv_n;
+            V += s2 * inv_n - mean * mean;
+        }
+        double C = sqrt(fmax(V, 0.0)) * inv_sigma;
+        C = fmin(C, 1.0);
+        int y = y0 + oy, x = x0 + ox;
+        uint32_t e = (bits_edge[((size_t)f * h + y) * words + (x >> 5)] >> (x & 31)) & 1u;
+        double S = w_edge * (double)e + w_color * C;
+        S = fmin(fmax(S, 0.0), 1.0);
+        bool lower = oy >= patch, right = ox >= patch;
+        acc0 += (!lower && !right) ? S : 0.0;
+        acc1 += (!lower && right) ? S : 0.0;
+        acc2 += (lower && !right) ? S : 0.0;
+        acc3 += (lower && right) ? S : 0.0;
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+        acc0 += __shfl_xor_sync(0xffffffffu, acc0, o);
+        acc1 += __shfl_xor_sync(0xffffffffu, acc1, o);
+        acc2 += __shfl_xor_sync(0xffffffffu, acc2, o);
+        acc3 += __shfl_xor_sync(0xffffffffu, acc3, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        double* ps = psum[threadIdx.x >> 5];
+        ps[0] = acc0; ps[1] = acc1; ps[2] = acc2; ps[3] = acc3;
+    }
+    __syncthreads();
+    if (threadIdx.x < 4) {
+        double tot = 0.0;
+        for (int wp = 0; wp < 8; ++wp) tot += psum[wp][threadIdx.x];      // fixed order: deterministic
+        int py = blockIdx.y * 2 + threadIdx.x / 2, px = blockIdx.x * 2 + threadIdx.x % 2;
+        s_out[(size_t)f * g.n_tok + patch_token(g, py, px)] = (float)(tot / (double)(patch * patch));
+    }
+}
+
+inline unsigned blocks_for(long long n, int threads) { return (unsigned)((n + threads - 1) / threads); }
+
+}  // namespace
+
+static size_t color_smem() { return (size_t)(3 * SE * (SE + 1) + 6 * SE * ST) * sizeof(double); }
+
+int sc_saliency_init(int max_h, int max_words) {
+    SC_CHECK(cudaFuncSetAttribute(k_color_patch, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)color_smem()));
+    size_t smem = (size_t)2 * max_h * max_words * sizeof(uint32_t);
+    if (smem > 227 * 1024) return SALICACHE_E_SHAPE;
+    SC_CHECK(cudaFuncSetAttribute(k_hysteresis, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    return SALICACHE_OK;
+}
+
+int sc_box_down2(const uint8_t* d_src, int H, int W, int B, uint8_t* d_dst, cudaStream_t st) {
+    k_box_down2<<<blocks_for((long long)(H / 2) * (W / 2) * B, 256), 256, 0, st>>>(d_src, H, W, B, d_dst);
+    SC_CHECK(cudaGetLastError());
+    return SALICACHE_OK;
+}
+
+int sc_saliency(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_frames, size_t frame_bytes, int B, float* d_s,
+                cudaStream_t st) {
+    const salicache_params& p = c->p;
+    const int words = (g.W + 31) / 32;
+    for (int b0 = 0; b0 < B; b0 += c->chunk) {
+        int nb = B - b0 < c->chunk ? B - b0 : c->chunk;
+        const uint8_t* fr = d_frames + (size_t)b0 * frame_bytes;
+        dim3 gc((g.W + CT - 1) / CT, (g.H + CT - 1) / CT, nb);
+        k_canny_classify<<<gc, 256, 0, st>>>(fr, frame_bytes, g.H, g.W, words, p.canny_lo * p.canny_lo,
+                                             p.canny_hi * p.canny_hi, c->bits_kept, c->bits_edge);
+        size_t smem = (size_t)2 * g.H * words * sizeof(uint32_t);
+        k_hysteresis<<<nb, 1024, smem, st>>>(c->bits_kept, c->bits_edge, g.H, words, p.hyst_max_iters, c->d_status);
+        dim3 gs(g.W / ST, g.H / ST, nb);
+        k_color_patch<<<gs, 256, color_smem(), st>>>(fr, frame_bytes, g, p.patch, c->lut, c->bits_edge, words, 1.0 / p.sigma_ref,
+                                          p.w_edge, p.w_color, d_s + (size_t)b0 * g.n_tok);
+    }
+    SC_CHECK(cudaGetLastError());
+    return SALICACHE_OK;
+}

@@ -1,0 +1,120 @@
+// Decision rule (Eq. 6, Eq. 8, Alg. 1): per frame, the redundancy ratio, one code per token and the
+// stable per-tier index lists; then the pool row offsets of the batch.
+#include "common.cuh"
+
+namespace {
+
+constexpr int SEL_THREADS = 256;
+
+__global__ void __launch_bounds__(SEL_THREADS)
+k_select(const float* __restrict__ dP, const float* __restrict__ s, int n_tok, int first_has_no_prev, int patch_reuse,
+         float tau_t, float theta_R, float tau_high, float tau_med, float tau_low, uint8_t* __restrict__ decision,
+         int32_t* __restrict__ idx, int32_t* __restrict__ counts, uint8_t* __restrict__ frame_redundant) {
+    __shared__ int s_red[SEL_THREADS / 32];
+    __shared__ int s_static;
+    __shared__ int s_warp[3][SEL_THREADS / 32];
+    __shared__ int s_base[3];
+    __shared__ int s_cnt[5];
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const bool has_prev = dP != nullptr && !(first_has_no_prev && b == 0);
+    const float* dp = has_prev ? dP + (size_t)b * n_tok : nullptr;
+    const float* sb = s + (size_t)b * n_tok;
+    // Eq. 6: R = (1/N) sum [dP_i < tau_t]
+    int n_static = 0;
+    if (has_prev)
+        for (int i = tid; i < n_tok; i += SEL_THREADS) n_static += (dp[i] < tau_t) ? 1 : 0;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) n_static += __shfl_xor_sync(0xffffffffu, n_static, o);
+    if (lane == 0) s_red[wid] = n_static;
+    if (tid < 3) s_base[tid] = 0;
+    if (tid < 5) s_cnt[tid] = 0;
+    __syncthreads();
+    if (tid == 0) {
+        int t = 0;
+        for (int k = 0; k < SEL_THREADS / 32; ++k) t += s_red[k];
+        s_static = t;
+    }
+    __syncthreads();
+    const float R = has_prev ? __fdiv_rn((float)s_static, (float)n_tok) : 0.0f;
+    const bool redundant = has_prev && (R > theta_R);
+    int my_cnt[5] = {0, 0, 0, 0, 0};
+    for (int base = 0; base < n_tok; base += SEL_THREADS) {
+        int i = base + tid;
+        int d = -1;
+        if (i < n_tok) {
+            if (redundant) d = SALICACHE_REUSE;
+            else if (patch_reuse && has_prev && dp[i] < tau_t) d = SALICACHE_REUSE;
+            else {
+                float sv = sb[i];
+                d = sv > tau_high ? SALICACHE_FP16 : (sv > tau_med ? SALICACHE_INT8 : (sv > tau_low ? SALICACHE_INT4 : SALICACHE_PRUNE));
+            }
+            decision[(size_t)b * n_tok + i] = (uint8_t)d;
+        }
+        unsigned m[3];
+        m[0] = __ballot_sync(0xffffffffu, d == SALICACHE_FP16);
+        m[1] = __ballot_sync(0xffffffffu, d == SALICACHE_INT8);
+        m[2] = __ballot_sync(0xffffffffu, d == SALICACHE_INT4);
+        if (lane == 0) {
+#pragma unroll
+            for (int t = 0; t < 3; ++t) s_warp[t][wid] = __popc(m[t]);
+        }
+        __syncthreads();
+        int tier = d == SALICACHE_FP16 ? 0 : (d == SALICACHE_INT8 ? 1 : (d == SALICACHE_INT4 ? 2 : -1));
+        if (tier >= 0) {
+            int pos = s_base[tier];
+            for (int k = 0; k < wid; ++k) pos += s_warp[tier][k];
+            pos += __popc(m[tier] & ((1u << lane) - 1u));
+            idx[((size_t)b * 3 + tier) * n_tok + pos] = i;
+        }
+        if (d >= 0) my_cnt[d]++;
+        __syncthreads();
+        if (tid < 3) {
+            int t = 0;
+            for (int k = 0; k < SEL_THREADS / 32; ++k) t += s_warp[tid][k];
+            s_base[tid] += t;
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int c = 0; c < 5; ++c) {
+        int v = my_cnt[c];
+#pragma unroll
+        for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0 && v) atomicAdd(&s_cnt[c], v);
+    }
+    __syncthreads();
+    if (tid < 5) counts[(size_t)b * 5 + tid] = s_cnt[tid];
+    if (tid == 0) frame_redundant[b] = redundant ? 1 : 0;
+    // pad the lists with -1
+    for (int t = 0; t < 3; ++t)
+        for (int i = s_base[t] + tid; i < n_tok; i += SEL_THREADS) idx[((size_t)b * 3 + t) * n_tok + i] = -1;
+}
+
+// Pool row offsets: exclusive scan over the frames of the batch, continuing from the running fill.
+__global__ void k_row_offsets(const int32_t* __restrict__ counts, int B, int64_t* __restrict__ row_offset,
+                              int64_t* __restrict__ fill) {
+    int t = threadIdx.x;
+    if (t >= 3) return;
+    const int code = t == 0 ? SALICACHE_FP16 : (t == 1 ? SALICACHE_INT8 : SALICACHE_INT4);
+    int64_t acc = fill[t];
+    for (int b = 0; b < B; ++b) {
+        row_offset[(size_t)b * 3 + t] = acc;
+        acc += counts[(size_t)b * 5 + code];
+    }
+    fill[t] = acc;
+}
+
+}  // namespace
+
+int sc_select(salicache_ctx* c, const float* d_deltaP, const float* d_s, int B, int first_has_no_prev,
+              uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts, uint8_t* d_frame_redundant,
+              int64_t* d_row_offset, int64_t* d_fill, cudaStream_t st) {
+    const salicache_params& p = c->p;
+    if (B == 0) return SALICACHE_OK;
+    k_select<<<B, SEL_THREADS, 0, st>>>(d_deltaP, d_s, c->n_tok, first_has_no_prev, p.patch_reuse, p.tau_t, p.theta_R,
+                                        p.tau_high, p.tau_med, p.tau_low, d_decision, d_idx, d_counts,
+                                        d_frame_redundant);
+    k_row_offsets<<<1, 32, 0, st>>>(d_counts, B, d_row_offset, d_fill);
+    SC_CHECK(cudaGetLastError());
+    return SALICACHE_OK;
+}
