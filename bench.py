@@ -1,0 +1,436 @@
+#!/usr/bin/env python
+"""Benchmark of the Sali-Cache hot path on B200: frames/s through flow + saliency + select + KV-pack.
+
+One step = the whole hot path over all frames of the workload (default: workload 3, 300 frames of
+336x336, K/V 32 layers x 32 heads x 128, int4 background).  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 3] [--impl ours|reference]
+
+N > 1 (torchrun): every rank runs the same workload on its own GPU (independent video streams, no
+collective on the data path); the value is the aggregate over ranks, timed as the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+RING = 8            # K/V frame slabs resident on the device (slot = frame % RING); 8 x 302 MB >> L2
+PAPER_CONTEXT = {"compression_ratio": 2.20, "time_per_frame_s": 0.068, "baseline_time_per_frame_s": 0.055,
+                 "hardware": "1x RTX 3090 24 GB, LLaVA-1.6 Mistral-7B, fp16 (paper Tables I and III)"}
+# DRAM bytes of the pack kernel per algorithmic byte, from the ncu capture summarised in
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over the algorithmic bytes of the same launch).
+NCU_TRAFFIC_RATIO = None
+
+
+def _peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.mktemp(suffix=".csv")
+        self.idx = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.idx)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 9:
+                    continue
+                try:
+                    sm.append(float(p[1]))
+                    mx.append(float(p[2]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, p[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out = {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                   "samples": len(sm)}
+        return out
+
+
+def algorithmic_bytes(counts: np.ndarray, L: int, HD: int, G: int = 128):
+    """Bytes the store must move for frames with the per-code counts [T][5]: every stored row is read once
+    as fp16 and written once in its tier's format (codes + scale/zero); PRUNE and REUSE move nothing."""
+    c = np.asarray(counts, np.int64).reshape(-1, 5)
+    ng = HD // G
+    n4, n8, n16 = c[:, 2].sum(), c[:, 3].sum(), c[:, 4].sum()
+    read = 2 * L * (n4 + n8 + n16) * HD * 2
+    write = 2 * L * (n16 * HD * 2 + n8 * (HD + 2 * ng) + n4 * (HD // 2 + 4 * ng))
+    return int(read), int(write)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2602_14236_b200 import binding as sc
+    from paper_2602_14236_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    wl = synth.WORKLOADS[args.workload]
+    T = wl.T if args.frames <= 0 else min(args.frames, wl.T)
+    L, HD, n_tok = wl.L, wl.HD, wl.n_tok
+    th = synth.thresholds(wl.background)
+    params = sc.salicache_default_params(H=wl.H, W=wl.W, n_images=wl.n_images, max_batch=max(T, RING),
+                                         chunk_frames=args.chunk, L=L, heads=wl.heads, head_dim=wl.head_dim, **th)
+    ctx = sc.Context(params)
+    frames_np = synth.frames(wl.index, T=T)
+    frames = torch.from_numpy(frames_np).to(dev)
+    ring = min(RING, T)
+    Kring = torch.empty((ring, L, n_tok, HD), dtype=torch.float16, device=dev)
+    Vring = torch.empty_like(Kring)
+    for slot in range(ring):
+        k, v = synth.kv_torch(wl.index, slot, dev, L=L, n_tok=n_tok)
+        Kring[slot].copy_(k)
+        Vring[slot].copy_(v)
+    del k, v
+    frame_stride = L * n_tok * HD
+
+    dP = torch.zeros((T, n_tok), dtype=torch.float32, device=dev)
+    s = torch.zeros((T, n_tok), dtype=torch.float32, device=dev)
+    dec = torch.zeros((T, n_tok), dtype=torch.uint8, device=dev)
+    idx = torch.zeros((T, 3, n_tok), dtype=torch.int32, device=dev)
+    counts = torch.zeros((T, 5), dtype=torch.int32, device=dev)
+    red = torch.zeros((T,), dtype=torch.uint8, device=dev)
+    off = torch.zeros((T, 3), dtype=torch.int64, device=dev)
+    fill = torch.zeros((3,), dtype=torch.int64, device=dev)
+
+    def filter_stage():
+        fill.zero_()
+        if T > 1:
+            sc.salicache_flow_score(ctx, frames[:-1], frames[1:], T - 1, dP[1:])
+        sc.salicache_saliency(ctx, frames, T, s)
+        sc.salicache_select(ctx, dP, s, T, True, dec, idx, counts, red, off, fill)
+
+    # sizing pass (untimed): the decisions fix the pool capacities
+    filter_stage()
+    torch.cuda.synchronize()
+    counts_h = counts.cpu().numpy()
+    tot = counts_h[:, [4, 3, 2]].sum(axis=0)
+    pools = sc.PoolSet(L, HD, int(tot[0]) + 1, int(tot[1]) + 1, int(tot[2]) + 1, ring=False, device=dev)
+    rd, wr = algorithmic_bytes(counts_h, L, HD)
+
+    n_chunks = (T + ring - 1) // ring
+    ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(n_chunks)] for _ in range(args.steps)]
+    ev_f = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+
+    def step(k: int):
+        timed_events = k >= 0
+        if timed_events:
+            ev_f[k][0].record()
+        filter_stage()
+        if timed_events:
+            ev_f[k][1].record()
+        for c in range(n_chunks):
+            b0 = c * ring
+            nb = min(ring, T - b0)
+            if timed_events:
+                ev[k][c][0].record()
+            sc.salicache_pack_kv(ctx, Kring, Vring, frame_stride, idx[b0:], counts[b0:], off[b0:], nb, pools.c)
+            if timed_events:
+                ev[k][c][1].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    for _ in range(args.warmup):
+        step(-1)
+    torch.cuda.synchronize()
+    assert sc.salicache_poll_status(ctx) == 0, "device status after warm-up"
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = ctx.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    pack_ms, filt_ms = 0.0, 0.0
+    barrier()
+    torch.cuda.synchronize()
+    e0.record()
+    for k in range(args.steps):
+        step(k)
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    for k in range(args.steps):
+        pack_ms += sum(a.elapsed_time(b) for a, b in ev[k])
+        filt_ms += ev_f[k][0].elapsed_time(ev_f[k][1])
+    total_ms = e0.elapsed_time(e1)
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else {}
+    status = sc.salicache_poll_status(ctx)
+    assert status == 0, f"device status {status}"
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+
+    ms_per_step = total_ms / args.steps
+    fps = world * T * args.steps / (total_ms / 1e3)
+    peak, peak_src = _peaks()
+    pack_launches = n_chunks * args.steps
+    pack_s = pack_ms / 1e3
+    achieved = (rd + wr) * args.steps / pack_s / 1e9 if pack_s > 0 else 0.0
+    roofline = {"kernel": "k_pack", "bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                "frac": round(achieved / peak, 4), "peak_source": peak_src,
+                "traffic": (None if NCU_TRAFFIC_RATIO is None else int(NCU_TRAFFIC_RATIO * (rd + wr) / n_chunks)),
+                "algorithmic_bytes_per_launch": int((rd + wr) / n_chunks), "launches_per_step": n_chunks,
+                "avg_launch_ms": round(pack_ms / pack_launches, 4),
+                "pack_ms_per_step": round(pack_ms / args.steps, 3), "filter_ms_per_step": round(filt_ms / args.steps, 3),
+                "pipeline_frac_of_peak": round((rd + wr) / (ms_per_step / 1e3) / 1e9 / peak, 4)}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- end to end: host buffers in, decisions out; copies inside the timed region (single rank)
+    cpu = None
+    if not args.no_cpu and world == 1:
+        cpu = cpu_baseline(args, wl, T, frames_np, Kring, Vring, th)
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(args, sc, ctx, wl, T, frames_np, Kring, Vring, pools, dev,
+                      (dP, s, dec, idx, counts, red, off, fill), world)
+
+    raw = 2 * L * T * n_tok * HD * 2
+    stored = wr + T * (n_tok + 52) + 4 * int(tot.sum())     # payload + decisions, tables, index lists
+    line = {
+        "metric": "frames/s through flow+saliency+select+KV-pack at LLaVA-1.6-7B shape", "value": round(fps, 2),
+        "unit": "frames/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": round(ms_per_step, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f16->i8/i4 (store), f64 (scores)", "data": "synthetic",
+        "config": {"workload": f"configs[{wl.index - 1}]: {wl.description}", "frames": T, "tokens_per_frame": n_tok,
+                   "layers": L, "heads": wl.heads, "head_dim": wl.head_dim, "background": wl.background,
+                   "kv_ring_slabs": ring, "l2_policy": "inputs larger than L2 (K/V ring of %.1f GB)" % (2 * Kring.numel() * 2 / 1e9),
+                   "parallelism": "independent video stream per GPU"},
+        "tokens_per_s": round(fps * n_tok, 1),
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
+        "clocks": clocks,
+        "compression_ratio": round(raw / stored, 4),
+        "tier_counts": {"reuse": int(counts_h[:, 0].sum()), "prune": int(counts_h[:, 1].sum()),
+                        "int4": int(counts_h[:, 2].sum()), "int8": int(counts_h[:, 3].sum()),
+                        "fp16": int(counts_h[:, 4].sum()), "frames_redundant": int(red.sum().item())},
+        "paper_context": PAPER_CONTEXT,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, sc, ctx, wl, T, frames_np, Kring, Vring, pools, dev, bufs, world):
+    """Frames and K/V start in pinned host memory; each step copies them to the device (K/V through the two
+    halves of the device ring, copy of one half overlapping the pack of the other) and reads the decisions back."""
+    import torch
+    dP, s, dec, idx, counts, red, off, fill = bufs
+    L, HD, n_tok = wl.L, wl.HD, wl.n_tok
+    ring = Kring.shape[0]
+    half = max(ring // 2, 1)
+    frame_stride = L * n_tok * HD
+    h_frames = torch.from_numpy(frames_np).pin_memory()
+    hK = Kring.cpu().pin_memory()
+    hV = Vring.cpu().pin_memory()
+    d_frames = torch.empty_like(h_frames, device=dev)
+    h_counts = torch.empty((T, 5), dtype=torch.int32).pin_memory()
+    h_dec = torch.empty((T, n_tok), dtype=torch.uint8).pin_memory()
+    h_red = torch.empty((T,), dtype=torch.uint8).pin_memory()
+    copy_stream = torch.cuda.Stream(device=dev)
+    main = torch.cuda.current_stream()
+    n_half = (T + half - 1) // half
+    copied = [torch.cuda.Event() for _ in range(2)]
+    packed = [torch.cuda.Event() for _ in range(2)]
+
+    def step():
+        d_frames.copy_(h_frames, non_blocking=True)
+        fill.zero_()
+        if T > 1:
+            sc.salicache_flow_score(ctx, d_frames[:-1], d_frames[1:], T - 1, dP[1:])
+        sc.salicache_saliency(ctx, d_frames, T, s)
+        sc.salicache_select(ctx, dP, s, T, True, dec, idx, counts, red, off, fill)
+        h_counts.copy_(counts, non_blocking=True)
+        h_dec.copy_(dec, non_blocking=True)
+        h_red.copy_(red, non_blocking=True)
+        for c in range(n_half):
+            b0 = c * half
+            nb = min(half, T - b0)
+            side = c % 2
+            slot0 = side * half
+            with torch.cuda.stream(copy_stream):
+                if c >= 2:
+                    copy_stream.wait_event(packed[side])
+                for j in range(nb):
+                    src = (b0 + j) % ring
+                    Kring[slot0 + j].copy_(hK[src], non_blocking=True)
+                    Vring[slot0 + j].copy_(hV[src], non_blocking=True)
+                copied[side].record(copy_stream)
+            main.wait_event(copied[side])
+            sc.salicache_pack_kv(ctx, Kring[slot0:], Vring[slot0:], frame_stride, idx[b0:], counts[b0:], off[b0:], nb,
+                                 pools.c)
+            packed[side].record(main)
+        main.synchronize()
+
+    steps = max(1, min(args.steps, args.e2e_steps))
+    step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    h2d = h_frames.numel() + 2 * T * frame_stride * 2
+    d2h = h_counts.numel() * 4 + h_dec.numel() + h_red.numel()
+    return {"value": round(world * T / (ms / 1e3), 2), "unit": "frames/s", "h2d_bytes_per_step": int(h2d),
+            "d2h_bytes_per_step": int(d2h), "ms_per_step": round(ms, 2), "steps": steps,
+            "note": "every frame's fp16 K/V crosses PCIe (%.1f GB per step); single rank" % (h2d / 1e9)}
+
+
+def _oracle_sample(wl, T, frames_np, Kring_h, Vring_h, th, sample):
+    """The oracle, as it stands, on the sampled frames: flow (t-1 -> t), saliency, decisions, store."""
+    import oracle
+    p = oracle.Params(**th)
+    prev = np.stack([frames_np[max(t - 1, 0)] for t in sample])
+    cur = np.stack([frames_np[t] for t in sample])
+    t0 = time.perf_counter()
+    dP = oracle.flow_score(prev, cur, p).astype(np.float32)
+    s = oracle.saliency(cur, p).astype(np.float32)
+    caps = len(sample) * wl.n_tok
+    pools = oracle.Pools(wl.L, wl.HD, 128, caps, caps, caps)
+    off = np.zeros(3, np.int64)
+    stored = 0
+    for i, t in enumerate(sample):
+        d, idx, counts, r, _ = oracle.select(dP[i], s[i], t > 0, p)
+        slot = t % Kring_h.shape[0]
+        oracle.pack_frame(Kring_h[slot], Vring_h[slot], idx, counts, off, pools)
+        off += counts[[4, 3, 2]]
+        stored += int(counts[[4, 3, 2]].sum())
+    return time.perf_counter() - t0, stored
+
+
+def cpu_baseline(args, wl, T, frames_np, Kring, Vring, th):
+    import oracle
+    n = min(args.cpu_sample, T)
+    sample = sorted(set(int(round(x)) for x in np.linspace(0, T - 1, n)))
+    Kh = Kring.cpu().numpy().view(np.uint16)
+    Vh = Vring.cpu().numpy().view(np.uint16)
+    secs, stored = _oracle_sample(wl, T, frames_np, Kh, Vh, th, sample)
+    return {"value": round(len(sample) / secs, 4), "unit": "frames/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{len(sample)} evenly spaced frames {sample} of the {T}-frame workload "
+                      f"({stored} stored token rows x {2 * wl.L} planes), {secs:.1f} s",
+            "seconds": round(secs, 2)}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2602_14236_b200 import synth
+    wl = synth.WORKLOADS[args.workload]
+    T = wl.T if args.frames <= 0 else min(args.frames, wl.T)
+    th = synth.thresholds(wl.background)
+    frames_np = synth.frames(wl.index, T=T)
+    ring = min(RING, T)
+    KV = [synth.kv_numpy(wl.index, 0)]      # one frame slab serves every sampled frame (values are i.i.d.)
+    Kh = np.stack([k for k, _ in KV]).view(np.uint16)
+    Vh = np.stack([v for _, v in KV]).view(np.uint16)
+    n = min(args.ref_sample, T)
+    sample = sorted(set(int(round(x)) for x in np.linspace(0, T - 1, n)))
+    times = []
+    for k in range(args.warmup + args.steps):
+        secs, stored = _oracle_sample(wl, T, frames_np, Kh, Vh, th, sample)
+        if k >= args.warmup:
+            times.append(secs)
+    secs = float(np.mean(times))
+    fps = len(sample) / secs
+    desc = f"{len(sample)} evenly spaced frames {sample} of the {T}-frame workload per step ({stored} stored rows x {2 * wl.L} planes)"
+    line = {"impl": "reference", "metric": "frames/s through flow+saliency+select+KV-pack at LLaVA-1.6-7B shape",
+            "value": round(fps, 4), "unit": "frames/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(secs * 1e3, 1), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f16->i8/i4 (store), f64 (scores)", "data": "synthetic",
+            "config": {"workload": f"configs[{wl.index - 1}]: {wl.description}", "frames": T,
+                       "tokens_per_frame": wl.n_tok, "layers": wl.L, "background": wl.background},
+            "cpu_baseline": {"value": round(fps, 4), "unit": "frames/s", "cores": oracle.num_threads(),
+                             "kind": "oracle", "sample": desc},
+            "e2e": {"value": round(fps, 4), "unit": "frames/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=3)
+    ap.add_argument("--frames", type=int, default=0, help="use only the first N frames of the workload (profiling)")
+    ap.add_argument("--chunk", type=int, default=16, help="frames per internal pass of flow/saliency")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--cpu-sample", type=int, default=6)
+    ap.add_argument("--ref-sample", type=int, default=4)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -99,6 +99,9 @@ SALICACHE_API const char* salicache_strerror(int status);
 /* Tokens per frame: n_images * (336/patch)^2 for anyres, else (H/patch)*(W/patch). */
 SALICACHE_API int salicache_tokens_per_frame(const salicache_ctx* ctx);
 
+/* Number of CUDA kernels this context has launched since it was created (host-side count). */
+SALICACHE_API int64_t salicache_launch_count(const salicache_ctx* ctx);
+
 /*
  * Temporal score (Sec. III-A, Eq. 5; Farneback flow, Sec. IV-B).
  * For b in [0,B): dense flow from d_prev[b] to d_cur[b] (frames of H*W*3 bytes, consecutive),

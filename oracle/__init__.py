@@ -73,9 +73,9 @@ class Params:
     w_color: float = 0.5
     tau_t: float = 0.5
     theta_R: float = 0.90
-    tau_high: float = 0.20
-    tau_med: float = 0.10
-    tau_low: float = 0.05
+    tau_high: float = 0.40
+    tau_med: float = 0.36
+    tau_low: float = 0.25
     patch_reuse: int = 1
 
 

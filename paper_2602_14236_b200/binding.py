@@ -47,7 +47,7 @@ class Pools(C.Structure):
 
 EXPORTS = [
     "salicache_default_params", "salicache_create", "salicache_destroy", "salicache_strerror",
-    "salicache_tokens_per_frame", "salicache_flow_score", "salicache_saliency", "salicache_select",
+    "salicache_tokens_per_frame", "salicache_launch_count", "salicache_flow_score", "salicache_saliency", "salicache_select",
     "salicache_pack_kv", "salicache_unpack_kv", "salicache_poll_status",
 ]
 
@@ -71,6 +71,8 @@ def lib():
         _lib.salicache_destroy.argtypes = [C.c_void_p]
         _lib.salicache_tokens_per_frame.argtypes = [C.c_void_p]
         _lib.salicache_default_params.argtypes = [C.POINTER(Params)]
+        _lib.salicache_launch_count.argtypes = [C.c_void_p]
+        _lib.salicache_launch_count.restype = C.c_int64
         vp, i32, i64 = C.c_void_p, C.c_int, C.c_int64
         _lib.salicache_flow_score.argtypes = [vp, vp, vp, i32, vp, vp, vp]
         _lib.salicache_saliency.argtypes = [vp, vp, i32, vp, vp]
@@ -126,6 +128,9 @@ class Context:
             self.close()
         except Exception:
             pass
+
+    def launch_count(self) -> int:
+        return int(lib().salicache_launch_count(self._h))
 
     @property
     def handle(self):

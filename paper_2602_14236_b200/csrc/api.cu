@@ -39,7 +39,7 @@ int salicache_default_params(salicache_params* p) {
     p->pyr_levels = 3; p->poly_n = 5; p->poly_sigma = 1.2; p->win = 15; p->iters = 3; p->eps_det = 1e-3;
     p->canny_lo = 50; p->canny_hi = 150; p->var_radius = 3; p->sigma_ref = 16.0; p->w_edge = 0.5; p->w_color = 0.5;
     p->hyst_max_iters = 4096;
-    p->tau_t = 0.5f; p->theta_R = 0.90f; p->tau_high = 0.20f; p->tau_med = 0.10f; p->tau_low = 0.05f;
+    p->tau_t = 0.5f; p->theta_R = 0.90f; p->tau_high = 0.40f; p->tau_med = 0.36f; p->tau_low = 0.25f;
     p->patch_reuse = 1;
     p->L = 32; p->heads = 32; p->head_dim = 128; p->group = 128;
     return SALICACHE_OK;
@@ -150,6 +150,8 @@ int salicache_destroy(salicache_ctx* c) {
 
 int salicache_tokens_per_frame(const salicache_ctx* c) { return c ? c->n_tok : SALICACHE_E_NULL; }
 
+int64_t salicache_launch_count(const salicache_ctx* c) { return c ? (int64_t)c->launches : (int64_t)SALICACHE_E_NULL; }
+
 int salicache_flow_score(salicache_ctx* c, const uint8_t* d_prev, const uint8_t* d_cur, int B, float* d_deltaP,
                          double* d_flow_or_null, void* cuda_stream) {
     if (!c || !d_prev || !d_cur || !d_deltaP) return SALICACHE_E_NULL;
@@ -167,6 +169,7 @@ int salicache_flow_score(salicache_ctx* c, const uint8_t* d_prev, const uint8_t*
     uint8_t* base = c->base_frames;
     if (sequence) {
         rc = sc_box_down2(d_prev, c->p.H, c->p.W, B + 1, base, st);
+        c->launches++;
         if (rc != SALICACHE_OK) return rc;
         return sc_flow_score(c, c->plane[1], base, base + fbb, fbb, B, true, d_deltaP, nullptr, st);
     }
@@ -176,6 +179,7 @@ int salicache_flow_score(salicache_ctx* c, const uint8_t* d_prev, const uint8_t*
         if (nb > B - b0) nb = B - b0;
         rc = sc_box_down2(d_prev + (size_t)b0 * fb, c->p.H, c->p.W, nb, base, st);
         if (rc == SALICACHE_OK) rc = sc_box_down2(d_cur + (size_t)b0 * fb, c->p.H, c->p.W, nb, base + (size_t)nb * fbb, st);
+        c->launches += 2;
         if (rc == SALICACHE_OK)
             rc = sc_flow_score(c, c->plane[1], base, base + (size_t)nb * fbb, fbb, nb, false,
                                d_deltaP + (size_t)b0 * c->n_tok, nullptr, st);
@@ -195,6 +199,7 @@ int salicache_saliency(salicache_ctx* c, const uint8_t* d_frames, int B, float* 
     int rc = sc_saliency(c, c->plane[0], d_frames, fb, B, d_s, st);
     if (rc != SALICACHE_OK || c->n_planes == 1) return rc;
     rc = sc_box_down2(d_frames, c->p.H, c->p.W, B, c->base_frames, st);
+    c->launches++;
     if (rc != SALICACHE_OK) return rc;
     return sc_saliency(c, c->plane[1], c->base_frames, fb / 4, B, d_s, st);
 }

@@ -48,6 +48,7 @@ struct salicache_ctx {
     int64_t* row_prefix;       // [max_batch+1] stored rows before each frame of the batch
     int* d_status;             // deferred status word
     int sm_count;
+    long long launches;        // kernels launched through this context so far
 };
 
 // flow.cu

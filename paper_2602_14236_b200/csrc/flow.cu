@@ -286,7 +286,9 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
             int n = sequence ? nf : nb;
             float* dst = c->pyr[0] + (size_t)part * nb * P0;
             k_gray<<<blocks_for((long long)(P0 / 16) * n, T), T, 0, st>>>(src, frame_bytes, (int)P0, n, dst);
+            c->launches++;
         }
+        c->launches += 6;   // two pyramid levels, three expansions
         for (int l = 1; l < 3; ++l)
             k_pyr_down<<<blocks_for((long long)hs[l] * ws[l] * nf, T), T, 0, st>>>(c->pyr[l - 1], hs[l - 1], ws[l - 1], nf,
                                                                                    c->pyr[l]);
@@ -304,6 +306,7 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
                 k_flow_upsample<<<blocks_for((long long)Pl * nb, T), T, 0, st>>>(cur, hs[l + 1], ws[l + 1], nxt, hs[l],
                                                                                  ws[l], nb, 2 * P0, 2 * P0);
                 double* t = cur; cur = nxt; nxt = t;
+                c->launches++;
             }
             dim3 grid((ws[l] + FT - 1) / FT, (hs[l] + FT - 1) / FT, nb);
             for (int it = 0; it < p.iters; ++it) {
@@ -313,6 +316,7 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
                 if (l == 0 && it == p.iters - 1 && d_flow_or_null) { out = d_flow_or_null + (size_t)b0 * 2 * P0; }
                 k_flow_iter<<<grid, FLOW_THREADS, sc_flow_iter_smem(), st>>>(c1, c2, cstride, hs[l], ws[l], cur, out,
                                                                              ostride, zero_prior, p.eps_det);
+                c->launches++;
                 if (out == nxt) { double* t = cur; cur = nxt; nxt = t; }
                 else cur = out;
             }
@@ -321,7 +325,7 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
         const double* fin = cur;
         k_delta_p<<<blocks_for((long long)np * nb * 32, T), T, 0, st>>>(fin, 2 * P0, g, p.patch, nb,
                                                                         d_deltaP + (size_t)b0 * g.n_tok);
-        if (cur != c->flow_a && cur != c->flow_b) { /* final field went to the caller's buffer */ }
+        c->launches++;
     }
     SC_CHECK(cudaGetLastError());
     return SALICACHE_OK;

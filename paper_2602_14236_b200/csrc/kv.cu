@@ -321,6 +321,7 @@ int sc_pack(salicache_ctx* c, const void* d_K, const void* d_V, int64_t frame_st
     k_pack<<<grid, KV_THREADS, (size_t)(B + 1) * sizeof(int), st>>>((const __half*)d_K, (const __half*)d_V, g, d_idx,
                                                                     d_counts, (const long long*)d_row_offset,
                                                                     make_pools(pools), c->d_status);
+    c->launches++;
     SC_CHECK(cudaGetLastError());
     return SALICACHE_OK;
 }
@@ -334,9 +335,11 @@ int sc_unpack(salicache_ctx* c, const salicache_pools* pools, const int32_t* d_i
     k_unpack<<<grid, KV_THREADS, (size_t)(B + 1) * sizeof(int), st>>>((__half*)d_K_out, (__half*)d_V_out, g, d_idx,
                                                                       d_counts, (const long long*)d_row_offset,
                                                                       make_pools(pools), c->d_status);
+    c->launches++;
     if (zero_fill_pruned) {
         dim3 gz(2 * g.L, B);
         k_zero_pruned<<<gz, KV_THREADS, 0, st>>>((__half*)d_K_out, (__half*)d_V_out, g, d_decision);
+        c->launches++;
     }
     SC_CHECK(cudaGetLastError());
     return SALICACHE_OK;

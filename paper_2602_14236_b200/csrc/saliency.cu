@@ -313,6 +313,7 @@ int sc_saliency(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_frames, s
         dim3 gs(g.W / ST, g.H / ST, nb);
         k_color_patch<<<gs, 256, color_smem(), st>>>(fr, frame_bytes, g, p.patch, c->lut, c->bits_edge, words, 1.0 / p.sigma_ref,
                                           p.w_edge, p.w_color, d_s + (size_t)b0 * g.n_tok);
+        c->launches += 3;
     }
     SC_CHECK(cudaGetLastError());
     return SALICACHE_OK;

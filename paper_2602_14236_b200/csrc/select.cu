@@ -115,6 +115,7 @@ int sc_select(salicache_ctx* c, const float* d_deltaP, const float* d_s, int B, 
                                         p.tau_high, p.tau_med, p.tau_low, d_decision, d_idx, d_counts,
                                         d_frame_redundant);
     k_row_offsets<<<1, 32, 0, st>>>(d_counts, B, d_row_offset, d_fill);
+    c->launches += 2;
     SC_CHECK(cudaGetLastError());
     return SALICACHE_OK;
 }

@@ -36,6 +36,7 @@ def test_params_struct_matches_the_header_defaults():
     assert (p.canny_lo, p.canny_hi, p.var_radius, p.hyst_max_iters) == (50, 150, 3, 4096)
     assert (p.L, p.heads, p.head_dim, p.group, p.patch_reuse) == (32, 32, 128, 128, 1)
     assert abs(p.tau_t - 0.5) < 1e-7 and abs(p.theta_R - 0.9) < 1e-7
+    assert (round(p.tau_high, 4), round(p.tau_med, 4), round(p.tau_low, 4)) == (0.40, 0.36, 0.25)
     assert binding.lib().salicache_strerror(binding.E_CAPACITY).decode().startswith("tier pool")
 
 

@@ -139,7 +139,7 @@ def test_pipeline_decisions_match_oracle_up_to_near_threshold_tokens(wl1_frames,
 
 def test_select_without_temporal_scores_and_empty_batch():
     ctx = _ctx()
-    s = np.random.default_rng(0).uniform(0, 0.4, (3, 576)).astype(np.float32)
+    s = np.random.default_rng(0).uniform(0, 0.6, (3, 576)).astype(np.float32)
     out = gu.gpu_select(ctx, None, s, first_has_no_prev=False)
     dec, idx, counts, red, off = gu.oracle_select_all(None, s, gu.oracle_params(ctx.params))
     assert np.array_equal(out["decision"].cpu().numpy(), dec) and np.array_equal(out["idx"].cpu().numpy(), idx)
@@ -155,7 +155,7 @@ def _pack_case(background, L=2, T=3, n_tok=576, ring=False, caps=None, seed=0, f
     import torch
     ctx = _ctx(L=L, **synth.thresholds(background))
     rng = np.random.default_rng(seed)
-    s = rng.uniform(0.0, 0.4, (T, n_tok)).astype(np.float32)
+    s = rng.uniform(0.0, 0.6, (T, n_tok)).astype(np.float32)
     dP = rng.uniform(0.0, 1.2, (T, n_tok)).astype(np.float32)
     if T > 2:
         dP[2] = 0.0                                    # a fully redundant frame stores nothing
@@ -262,7 +262,7 @@ def test_pack_special_values():
     K[0, 0, 7, ::2] = 65504.0
     K[0, 0, 7, 1::2] = -65504.0
     V = K[:, :, ::-1].copy()
-    for tier_s in (0.15, 0.07):            # all tokens INT8, then all INT4
+    for tier_s in (0.38, 0.30):            # all tokens INT8, then all INT4
         s = np.full((1, n_tok), tier_s, np.float32)
         dec, idx, counts, red, off = gu.oracle_select_all(None, s, gu.oracle_params(ctx.params))
         ref = oracle.Pools(L, 4096, 128, 1, 576, 576)

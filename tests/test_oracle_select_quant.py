@@ -35,7 +35,7 @@ def test_select_brute_force_with_values_on_the_thresholds(has_prev, patch_reuse)
     p = oracle.Params(patch_reuse=patch_reuse)
     rng = np.random.default_rng(5)
     n = 576
-    s = rng.uniform(0, 0.3, n).astype(np.float32)
+    s = rng.uniform(0, 0.6, n).astype(np.float32)
     dP = rng.uniform(0, 1.0, n).astype(np.float32)
     s[:6] = [p.tau_high, p.tau_med, p.tau_low, np.nextafter(np.float32(p.tau_high), np.float32(1)),
              np.nextafter(np.float32(p.tau_med), np.float32(1)), np.nextafter(np.float32(p.tau_low), np.float32(1))]
@@ -198,7 +198,7 @@ def _frame_case(L=2, n_tok=24, HD=256, G=128, seed=1):
     rng = np.random.default_rng(seed)
     K = rng.standard_normal((L, n_tok, HD)).astype(np.float16).view(np.uint16)
     V = rng.standard_normal((L, n_tok, HD)).astype(np.float16).view(np.uint16)
-    s = rng.uniform(0, 0.3, n_tok).astype(np.float32)
+    s = rng.uniform(0, 0.6, n_tok).astype(np.float32)
     dP = rng.uniform(0, 1, n_tok).astype(np.float32)
     dec, idx, counts, _, _ = oracle.select(dP, s, True, oracle.Params())
     return K, V, dec, idx, counts
