@@ -122,12 +122,12 @@ def run_ours(args):
     T = wl.T if args.frames <= 0 else min(args.frames, wl.T)
     L, HD, n_tok = wl.L, wl.HD, wl.n_tok
     th = synth.thresholds(wl.background)
-    params = sc.salicache_default_params(H=wl.H, W=wl.W, n_images=wl.n_images, max_batch=max(T, RING),
+    params = sc.salicache_default_params(H=wl.H, W=wl.W, n_images=wl.n_images, max_batch=max(T, args.ring),
                                          chunk_frames=args.chunk, L=L, heads=wl.heads, head_dim=wl.head_dim, **th)
     ctx = sc.Context(params)
     frames_np = synth.frames(wl.index, T=T)
     frames = torch.from_numpy(frames_np).to(dev)
-    ring = min(RING, T)
+    ring = min(args.ring, T)
     Kring = torch.empty((ring, L, n_tok, HD), dtype=torch.float16, device=dev)
     Vring = torch.empty_like(Kring)
     for slot in range(ring):
@@ -384,7 +384,7 @@ def run_reference(args):
     T = wl.T if args.frames <= 0 else min(args.frames, wl.T)
     th = synth.thresholds(wl.background)
     frames_np = synth.frames(wl.index, T=T)
-    ring = min(RING, T)
+    ring = min(args.ring, T)
     KV = [synth.kv_numpy(wl.index, 0)]      # one frame slab serves every sampled frame (values are i.i.d.)
     Kh = np.stack([k for k, _ in KV]).view(np.uint16)
     Vh = np.stack([v for _, v in KV]).view(np.uint16)
@@ -420,6 +420,7 @@ def main():
     ap.add_argument("--workload", type=int, default=3)
     ap.add_argument("--frames", type=int, default=0, help="use only the first N frames of the workload (profiling)")
     ap.add_argument("--chunk", type=int, default=16, help="frames per internal pass of flow/saliency")
+    ap.add_argument("--ring", type=int, default=RING, help="K/V frame slabs resident on the device")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=1)

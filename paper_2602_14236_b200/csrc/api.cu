@@ -8,6 +8,7 @@
 int sc_flow_init();
 int sc_saliency_init(int max_h, int max_words);
 int sc_kv_max_batch();
+bool sc_kv_supported_hd(int HD);
 
 namespace {
 
@@ -69,7 +70,7 @@ int salicache_create(salicache_ctx** out, const salicache_params* p) {
         (p->n_images != 1 && p->n_images != 5) || p->L < 1 || p->heads < 1 || p->head_dim < 1)
         return SALICACHE_E_PARAM;
     const int HD = p->heads * p->head_dim;
-    if (HD % 256 != 0 || HD > 4096) return SALICACHE_E_PARAM;
+    if (!sc_kv_supported_hd(HD)) return SALICACHE_E_PARAM;
     if (p->H <= 0 || p->W <= 0 || p->H % 56 != 0 || p->W % 112 != 0) return SALICACHE_E_SHAPE;   // 28-px tiles, 4 | H>>2, 16 | W
     if (p->n_images == 5 && (p->H != 672 || p->W != 672)) return SALICACHE_E_SHAPE;
     if (p->max_batch < 1 || p->max_batch > sc_kv_max_batch()) return SALICACHE_E_SHAPE;

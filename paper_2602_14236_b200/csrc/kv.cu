@@ -1,6 +1,7 @@
 // Mixed-precision K/V store (Alg. 1 line 16; quantisers of Sec. IV-B) and its just-in-time
-// dequantisation (Sec. III-C).  HBM-bound: one warp moves one 8 KiB token row (HD = 4096 fp16) with
-// 16-byte loads, one quantisation group (128 elements) per half warp, packed stores.
+// dequantisation (Sec. III-C).  HBM-bound.  One warp moves one token row (HD fp16, 8 KiB at HD = 4096):
+// all 16-byte loads of the row are issued before any arithmetic, one quantisation group (128 elements)
+// is reduced per half warp, each lane then owns one group's scale, and codes leave as packed stores.
 #include <cuda_fp16.h>
 
 #include "common.cuh"
@@ -23,7 +24,7 @@ struct PoolPtrs {
     uint8_t* int8_scale;
     uint8_t* int4_codes;
     uint8_t* int4_sz;
-    long long cap[3];
+    long long cap0, cap1, cap2;
     int ring;
 };
 
@@ -32,6 +33,16 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                  : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint2 ld_stream(const uint2* p) {
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint32_t ld_stream(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
     return v;
 }
 __device__ __forceinline__ void st_stream(uint4* p, uint4 v) {
@@ -47,9 +58,21 @@ __device__ __forceinline__ void st_stream(uint32_t* p, uint32_t v) {
 __device__ __forceinline__ __half2 as_h2(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
 __device__ __forceinline__ uint32_t as_u32(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
 
+// d = (c << 16) | (sat_s8(a) << 8) | sat_s8(b)   (saturation to [-128, 127])
+__device__ __forceinline__ uint32_t pack_s8(int a, int b, uint32_t c) {
+    uint32_t d;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+// d = (c << 8) | (sat_u4(a) << 4) | sat_u4(b)    (saturation to [0, 15])
+__device__ __forceinline__ uint32_t pack_u4(int a, int b, uint32_t c) {
+    uint32_t d;
+    asm("cvt.pack.sat.u4.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
 // Rows stored before each frame of the batch, built by every CTA in shared memory from the counts.
 __device__ __forceinline__ void build_prefix(const int32_t* __restrict__ counts, int B, int* pre) {
-    // pre[b] = sum_{b' < b} (n16 + n8 + n4); B <= MAX_PREFIX
     __shared__ int wsum[KV_WARPS];
     int carry = 0;
     for (int base = 0; base < B; base += KV_THREADS) {
@@ -76,16 +99,18 @@ __device__ __forceinline__ void build_prefix(const int32_t* __restrict__ counts,
     __syncthreads();
 }
 
-// Work unit u -> (frame b, plane = layer*2 + kv, position j in the frame's stored-row list).
+// Work unit u -> (frame b, plane = layer*2 + kv, tier, token, pool row).  Units of one frame are ordered
+// plane-major, position-minor, so neighbouring warps read neighbouring token rows and write neighbouring
+// pool rows.
 struct Unit {
-    int b, plane, tier, j, tok;
+    int b, plane, tier, tok;
     long long row;   // pool row, or -1 when dropped
+    long long cap;
 };
 
 __device__ __forceinline__ Unit decode_unit(long long u, const int* pre, int B, int planes,
                                             const int32_t* __restrict__ counts, const int32_t* __restrict__ idx,
-                                            const long long* __restrict__ row_offset, int n_tok, const long long* cap,
-                                            int ring) {
+                                            const long long* __restrict__ row_offset, int n_tok, const PoolPtrs& pp) {
     Unit r;
     int q = (int)(u / planes);          // lies in [pre[b], pre[b+1]) of exactly one frame
     int lo = 0, hi = B;                 // largest b with pre[b] <= q
@@ -99,21 +124,21 @@ __device__ __forceinline__ Unit decode_unit(long long u, const int* pre, int B, 
     r.plane = (int)(local / stored);
     int j = (int)(local % stored);
     int n16 = counts[lo * 5 + SALICACHE_FP16], n8 = counts[lo * 5 + SALICACHE_INT8];
-    if (j < n16) r.tier = 0;
-    else if (j < n16 + n8) { r.tier = 1; j -= n16; }
-    else { r.tier = 2; j -= n16 + n8; }
-    r.j = j;
+    if (j < n16) { r.tier = 0; r.cap = pp.cap0; }
+    else if (j < n16 + n8) { r.tier = 1; j -= n16; r.cap = pp.cap1; }
+    else { r.tier = 2; j -= n16 + n8; r.cap = pp.cap2; }
     r.tok = idx[((size_t)lo * 3 + r.tier) * n_tok + j];
     long long row = row_offset[(size_t)lo * 3 + r.tier] + j;
-    long long cp = cap[r.tier];
-    if (ring) row = cp > 0 ? row % cp : -1;
-    else if (row >= cp) row = -1;
+    if (pp.ring) row = r.cap > 0 ? row % r.cap : -1;
+    else if (row >= r.cap) row = -1;
     r.row = row;
     return r;
 }
 
 // ---- pack ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(KV_THREADS)
+// ITERS = HD / 256: 16-byte loads per lane per row; groups per row = 2 * ITERS (<= 32, one per lane).
+template <int ITERS>
+__global__ void __launch_bounds__(KV_THREADS, 2)
 k_pack(const __half* __restrict__ K, const __half* __restrict__ V, KvGeom g, const int32_t* __restrict__ idx,
        const int32_t* __restrict__ counts, const long long* __restrict__ row_offset, PoolPtrs pp,
        int* __restrict__ status) {
@@ -122,100 +147,106 @@ k_pack(const __half* __restrict__ K, const __half* __restrict__ V, KvGeom g, con
     const int planes = 2 * g.L;
     const long long n_units = (long long)pre[g.B] * planes;
     const int lane = threadIdx.x & 31;
-    const int half_id = lane >> 4;
+    const int src_lane = (lane & 1) << 4;                  // a lane of the half warp that reduced my group
     const long long warp0 = (long long)blockIdx.x * KV_WARPS + (threadIdx.x >> 5);
     const long long wstride = (long long)gridDim.x * KV_WARPS;
-    const int vec_per_row = g.HD / 8;             // uint4 per row (512)
-    const int iters = vec_per_row / 32;           // 16
     for (long long u = warp0; u < n_units; u += wstride) {
-        Unit un = decode_unit(u, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp.cap, pp.ring);
+        Unit un = decode_unit(u, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp);
         if (un.row < 0) {
             if (lane == 0) atomicMin(status, SALICACHE_E_CAPACITY);
             continue;
         }
         const int layer = un.plane >> 1, kv = un.plane & 1;
         const __half* src_h = (kv ? V : K) + (size_t)un.b * g.frame_stride + ((size_t)layer * g.n_tok + un.tok) * g.HD;
-        const uint4* src = reinterpret_cast<const uint4*>(src_h);
-        const size_t prow = (size_t)un.plane * pp.cap[un.tier] + un.row;
+        const uint4* src = reinterpret_cast<const uint4*>(src_h) + lane;
+        uint4 v[ITERS];
+#pragma unroll
+        for (int i = 0; i < ITERS; ++i) v[i] = ld_stream(src + i * 32);
+        const size_t prow = (size_t)un.plane * un.cap + un.row;
         if (un.tier == 0) {
-            uint4* dst = reinterpret_cast<uint4*>(pp.fp16_pool + prow * (size_t)g.HD * 2);
-#pragma unroll 8
-            for (int i = 0; i < iters; ++i) st_stream(dst + i * 32 + lane, ld_stream(src + i * 32 + lane));
+            uint4* dst = reinterpret_cast<uint4*>(pp.fp16_pool + prow * (size_t)g.HD * 2) + lane;
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) st_stream(dst + i * 32, v[i]);
         } else if (un.tier == 1) {
-            uint2* dst = reinterpret_cast<uint2*>(pp.int8_codes + prow * (size_t)g.HD);
-            uint32_t my_scale = 0;
-#pragma unroll 8
-            for (int i = 0; i < iters; ++i) {
-                uint4 v = ld_stream(src + i * 32 + lane);
-                __half2 h0 = as_h2(v.x), h1 = as_h2(v.y), h2 = as_h2(v.z), h3 = as_h2(v.w);
-                __half2 m = __hmax2(__hmax2(__habs2(h0), __habs2(h1)), __hmax2(__habs2(h2), __habs2(h3)));
+            // INT8 symmetric: s = fp16(max|x| / 127), q = rint(x * (1/s)) clamped to [-127, 127]
+            uint32_t mine = 0;
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) {
+                __half2 m = __hmax2(__hmax2(__habs2(as_h2(v[i].x)), __habs2(as_h2(v[i].y))),
+                                    __hmax2(__habs2(as_h2(v[i].z)), __habs2(as_h2(v[i].w))));
 #pragma unroll
                 for (int o = 8; o; o >>= 1) m = __hmax2(m, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(m), o)));
-                float amax = fmaxf(__low2float(m), __high2float(m));
-                __half s16 = __float2half_rn(__fdiv_rn(amax, 127.0f));
-                if (__half_as_ushort(s16) == 0) s16 = __ushort_as_half(0x3c00);
-                float inv = __fdiv_rn(1.0f, __half2float(s16));
-                float2 f0 = __half22float2(h0), f1 = __half22float2(h1), f2 = __half22float2(h2), f3 = __half22float2(h3);
+                uint32_t sv = __shfl_sync(0xffffffffu, as_u32(m), src_lane);
+                if ((lane >> 1) == i) mine = sv;             // lane l owns group l = 2i + (l & 1)
+            }
+            float amax = fmaxf(__low2float(as_h2(mine)), __high2float(as_h2(mine)));
+            __half s16 = __float2half_rn(__fdiv_rn(amax, 127.0f));
+            if ((__half_as_ushort(s16) & 0x7fff) == 0) s16 = __ushort_as_half(0x3c00);
+            const float my_inv = __fdiv_rn(1.0f, __half2float(s16));
+            if (lane < g.ng) reinterpret_cast<uint16_t*>(pp.int8_scale + prow * (size_t)g.ng * 2)[lane] = __half_as_ushort(s16);
+            uint2* dst = reinterpret_cast<uint2*>(pp.int8_codes + prow * (size_t)g.HD) + lane;
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) {
+                const float inv = __shfl_sync(0xffffffffu, my_inv, 2 * i + (lane >> 4));
+                float2 f0 = __half22float2(as_h2(v[i].x)), f1 = __half22float2(as_h2(v[i].y));
+                float2 f2 = __half22float2(as_h2(v[i].z)), f3 = __half22float2(as_h2(v[i].w));
                 int q0 = __float2int_rn(__fmul_rn(f0.x, inv)), q1 = __float2int_rn(__fmul_rn(f0.y, inv));
                 int q2 = __float2int_rn(__fmul_rn(f1.x, inv)), q3 = __float2int_rn(__fmul_rn(f1.y, inv));
                 int q4 = __float2int_rn(__fmul_rn(f2.x, inv)), q5 = __float2int_rn(__fmul_rn(f2.y, inv));
                 int q6 = __float2int_rn(__fmul_rn(f3.x, inv)), q7 = __float2int_rn(__fmul_rn(f3.y, inv));
-                q0 = max(-127, min(127, q0)); q1 = max(-127, min(127, q1));
-                q2 = max(-127, min(127, q2)); q3 = max(-127, min(127, q3));
-                q4 = max(-127, min(127, q4)); q5 = max(-127, min(127, q5));
-                q6 = max(-127, min(127, q6)); q7 = max(-127, min(127, q7));
                 uint2 o;
-                o.x = (q0 & 255) | ((q1 & 255) << 8) | ((q2 & 255) << 16) | ((uint32_t)(q3 & 255) << 24);
-                o.y = (q4 & 255) | ((q5 & 255) << 8) | ((q6 & 255) << 16) | ((uint32_t)(q7 & 255) << 24);
-                st_stream(dst + i * 32 + lane, o);
-                // group 2i + half_id: lane (2i + h) collects it for one coalesced scale store
-                uint32_t sv = __shfl_sync(0xffffffffu, (uint32_t)__half_as_ushort(s16), (lane & 1) << 4);
-                if ((lane >> 1) == i) my_scale = sv;
+                o.x = __vmaxs4(pack_s8(q1, q0, pack_s8(q3, q2, 0)), 0x81818181u);
+                o.y = __vmaxs4(pack_s8(q5, q4, pack_s8(q7, q6, 0)), 0x81818181u);
+                st_stream(dst + i * 32, o);
             }
-            reinterpret_cast<uint16_t*>(pp.int8_scale + prow * (size_t)g.ng * 2)[lane] = (uint16_t)my_scale;
         } else {
-            uint32_t* dst = reinterpret_cast<uint32_t*>(pp.int4_codes + prow * (size_t)(g.HD / 2));
-            uint32_t my_sz = 0;
-#pragma unroll 8
-            for (int i = 0; i < iters; ++i) {
-                uint4 v = ld_stream(src + i * 32 + lane);
-                __half2 h0 = as_h2(v.x), h1 = as_h2(v.y), h2 = as_h2(v.z), h3 = as_h2(v.w);
-                __half2 mx = __hmax2(__hmax2(h0, h1), __hmax2(h2, h3));
-                __half2 mn = __hmin2(__hmin2(h0, h1), __hmin2(h2, h3));
+            // INT4 asymmetric: zero = min, s = fp16((max - min) / 15), q = rint((x - zero) * (1/s)) in [0, 15].
+            // One half2 carries (max, -min) so a single max-reduction serves both.
+            uint32_t mine = 0;
 #pragma unroll
-                for (int o = 8; o; o >>= 1) {
-                    mx = __hmax2(mx, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(mx), o)));
-                    mn = __hmin2(mn, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(mn), o)));
-                }
-                float fmx = fmaxf(__low2float(mx), __high2float(mx));
-                float fmn = fminf(__low2float(mn), __high2float(mn));
-                __half z16 = __float2half_rn(fmn);                      // exact: fmn is an fp16 value
-                if (fmn == 0.0f) z16 = __ushort_as_half(0);             // a zero minimum is stored as +0
-                __half s16 = __float2half_rn(__fdiv_rn(__fsub_rn(fmx, fmn), 15.0f));
-                if ((__half_as_ushort(s16) & 0x7fff) == 0) s16 = __ushort_as_half(0x3c00);
-                float inv = __fdiv_rn(1.0f, __half2float(s16));
-                float z = __half2float(z16);
-                float2 f0 = __half22float2(h0), f1 = __half22float2(h1), f2 = __half22float2(h2), f3 = __half22float2(h3);
-                float e[8] = {f0.x, f0.y, f1.x, f1.y, f2.x, f2.y, f3.x, f3.y};
-                uint32_t o = 0;
+            for (int i = 0; i < ITERS; ++i) {
+                __half2 a = as_h2(v[i].x), b = as_h2(v[i].y), c = as_h2(v[i].z), d = as_h2(v[i].w);
+                __half2 mx = __hmax2(__hmax2(a, b), __hmax2(c, d));
+                __half2 nmn = __hneg2(__hmin2(__hmin2(a, b), __hmin2(c, d)));
+                __half2 m = __hmax2(as_h2(__byte_perm(as_u32(mx), as_u32(nmn), 0x5410)),
+                                    as_h2(__byte_perm(as_u32(mx), as_u32(nmn), 0x7632)));   // (max, -min)
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    float r = rintf(__fmul_rn(__fsub_rn(e[k], z), inv));
-                    r = fminf(fmaxf(r, 0.0f), 15.0f);
-                    o |= (uint32_t)(int)r << (4 * k);
-                }
-                st_stream(dst + i * 32 + lane, o);
-                uint32_t pair = (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(z16) << 16);
-                uint32_t sv = __shfl_sync(0xffffffffu, pair, (lane & 1) << 4);
-                if ((lane >> 1) == i) my_sz = sv;
+                for (int o = 8; o; o >>= 1) m = __hmax2(m, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(m), o)));
+                uint32_t sv = __shfl_sync(0xffffffffu, as_u32(m), src_lane);
+                if ((lane >> 1) == i) mine = sv;
             }
-            reinterpret_cast<uint32_t*>(pp.int4_sz + prow * (size_t)g.ng * 4)[lane] = my_sz;
+            const float fmx = __low2float(as_h2(mine));
+            float fmn = -__high2float(as_h2(mine));
+            __half z16 = __float2half_rn(fmn);                       // exact: fmn is an fp16 value
+            if (fmn == 0.0f) z16 = __ushort_as_half(0);              // a zero minimum is stored as +0
+            __half s16 = __float2half_rn(__fdiv_rn(__fsub_rn(fmx, fmn), 15.0f));
+            if ((__half_as_ushort(s16) & 0x7fff) == 0) s16 = __ushort_as_half(0x3c00);
+            const float my_inv = __fdiv_rn(1.0f, __half2float(s16));
+            const float my_z = __half2float(z16);
+            if (lane < g.ng)
+                reinterpret_cast<uint32_t*>(pp.int4_sz + prow * (size_t)g.ng * 4)[lane] =
+                    (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(z16) << 16);
+            uint32_t* dst = reinterpret_cast<uint32_t*>(pp.int4_codes + prow * (size_t)(g.HD / 2)) + lane;
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) {
+                const int owner = 2 * i + (lane >> 4);
+                const float inv = __shfl_sync(0xffffffffu, my_inv, owner);
+                const float z = __shfl_sync(0xffffffffu, my_z, owner);
+                float2 f0 = __half22float2(as_h2(v[i].x)), f1 = __half22float2(as_h2(v[i].y));
+                float2 f2 = __half22float2(as_h2(v[i].z)), f3 = __half22float2(as_h2(v[i].w));
+                int q0 = __float2int_rn(__fmul_rn(__fsub_rn(f0.x, z), inv)), q1 = __float2int_rn(__fmul_rn(__fsub_rn(f0.y, z), inv));
+                int q2 = __float2int_rn(__fmul_rn(__fsub_rn(f1.x, z), inv)), q3 = __float2int_rn(__fmul_rn(__fsub_rn(f1.y, z), inv));
+                int q4 = __float2int_rn(__fmul_rn(__fsub_rn(f2.x, z), inv)), q5 = __float2int_rn(__fmul_rn(__fsub_rn(f2.y, z), inv));
+                int q6 = __float2int_rn(__fmul_rn(__fsub_rn(f3.x, z), inv)), q7 = __float2int_rn(__fmul_rn(__fsub_rn(f3.y, z), inv));
+                st_stream(dst + i * 32, pack_u4(q1, q0, pack_u4(q3, q2, pack_u4(q5, q4, pack_u4(q7, q6, 0)))));
+            }
         }
     }
 }
 
 // ---- unpack -------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(KV_THREADS)
+template <int ITERS>
+__global__ void __launch_bounds__(KV_THREADS, 2)
 k_unpack(__half* __restrict__ K, __half* __restrict__ V, KvGeom g, const int32_t* __restrict__ idx,
          const int32_t* __restrict__ counts, const long long* __restrict__ row_offset, PoolPtrs pp,
          int* __restrict__ status) {
@@ -226,56 +257,65 @@ k_unpack(__half* __restrict__ K, __half* __restrict__ V, KvGeom g, const int32_t
     const int lane = threadIdx.x & 31;
     const long long warp0 = (long long)blockIdx.x * KV_WARPS + (threadIdx.x >> 5);
     const long long wstride = (long long)gridDim.x * KV_WARPS;
-    const int iters = g.HD / 8 / 32;
     for (long long u = warp0; u < n_units; u += wstride) {
-        Unit un = decode_unit(u, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp.cap, pp.ring);
+        Unit un = decode_unit(u, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp);
         if (un.row < 0) {
             if (lane == 0) atomicMin(status, SALICACHE_E_CAPACITY);
             continue;
         }
         const int layer = un.plane >> 1, kv = un.plane & 1;
         __half* dst_h = (kv ? V : K) + (size_t)un.b * g.frame_stride + ((size_t)layer * g.n_tok + un.tok) * g.HD;
-        uint4* dst = reinterpret_cast<uint4*>(dst_h);
-        const size_t prow = (size_t)un.plane * pp.cap[un.tier] + un.row;
+        uint4* dst = reinterpret_cast<uint4*>(dst_h) + lane;
+        const size_t prow = (size_t)un.plane * un.cap + un.row;
         if (un.tier == 0) {
-            const uint4* src = reinterpret_cast<const uint4*>(pp.fp16_pool + prow * (size_t)g.HD * 2);
-#pragma unroll 8
-            for (int i = 0; i < iters; ++i) st_stream(dst + i * 32 + lane, ld_stream(src + i * 32 + lane));
+            const uint4* src = reinterpret_cast<const uint4*>(pp.fp16_pool + prow * (size_t)g.HD * 2) + lane;
+            uint4 v[ITERS];
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) v[i] = ld_stream(src + i * 32);
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) st_stream(dst + i * 32, v[i]);
         } else if (un.tier == 1) {
-            const uint2* src = reinterpret_cast<const uint2*>(pp.int8_codes + prow * (size_t)g.HD);
-            uint32_t my_scale = reinterpret_cast<const uint16_t*>(pp.int8_scale + prow * (size_t)g.ng * 2)[lane];
-#pragma unroll 8
-            for (int i = 0; i < iters; ++i) {
-                uint2 c = __ldg(src + i * 32 + lane);
-                float s = __half2float(__ushort_as_half((uint16_t)__shfl_sync(0xffffffffu, my_scale, 2 * i + (lane >> 4))));
-                uint32_t w[2] = {c.x, c.y};
+            const uint2* src = reinterpret_cast<const uint2*>(pp.int8_codes + prow * (size_t)g.HD) + lane;
+            uint2 c[ITERS];
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) c[i] = ld_stream(src + i * 32);
+            uint32_t my_scale = 0;
+            if (lane < g.ng) my_scale = reinterpret_cast<const uint16_t*>(pp.int8_scale + prow * (size_t)g.ng * 2)[lane];
+            const float my_s = __half2float(__ushort_as_half((uint16_t)my_scale));
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) {
+                const float s = __shfl_sync(0xffffffffu, my_s, 2 * i + (lane >> 4));
+                const uint32_t w[2] = {c[i].x, c[i].y};
                 uint32_t o[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     int qa = (int)(int8_t)((w[k >> 1] >> (16 * (k & 1))) & 255);
                     int qb = (int)(int8_t)((w[k >> 1] >> (16 * (k & 1) + 8)) & 255);
-                    __half2 h = __floats2half2_rn(__fmul_rn((float)qa, s), __fmul_rn((float)qb, s));
-                    o[k] = as_u32(h);
+                    o[k] = as_u32(__floats2half2_rn(__fmul_rn((float)qa, s), __fmul_rn((float)qb, s)));
                 }
-                st_stream(dst + i * 32 + lane, make_uint4(o[0], o[1], o[2], o[3]));
+                st_stream(dst + i * 32, make_uint4(o[0], o[1], o[2], o[3]));
             }
         } else {
-            const uint32_t* src = reinterpret_cast<const uint32_t*>(pp.int4_codes + prow * (size_t)(g.HD / 2));
-            uint32_t my_sz = reinterpret_cast<const uint32_t*>(pp.int4_sz + prow * (size_t)g.ng * 4)[lane];
-#pragma unroll 8
-            for (int i = 0; i < iters; ++i) {
-                uint32_t c = __ldg(src + i * 32 + lane);
-                uint32_t pair = __shfl_sync(0xffffffffu, my_sz, 2 * i + (lane >> 4));
-                float s = __half2float(__ushort_as_half((uint16_t)(pair & 0xffff)));
-                float z = __half2float(__ushort_as_half((uint16_t)(pair >> 16)));
+            const uint32_t* src = reinterpret_cast<const uint32_t*>(pp.int4_codes + prow * (size_t)(g.HD / 2)) + lane;
+            uint32_t c[ITERS];
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) c[i] = ld_stream(src + i * 32);
+            uint32_t my_sz = 0;
+            if (lane < g.ng) my_sz = reinterpret_cast<const uint32_t*>(pp.int4_sz + prow * (size_t)g.ng * 4)[lane];
+            const float my_s = __half2float(__ushort_as_half((uint16_t)(my_sz & 0xffff)));
+            const float my_z = __half2float(__ushort_as_half((uint16_t)(my_sz >> 16)));
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) {
+                const int owner = 2 * i + (lane >> 4);
+                const float s = __shfl_sync(0xffffffffu, my_s, owner);
+                const float z = __shfl_sync(0xffffffffu, my_z, owner);
                 uint32_t o[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    float qa = (float)((c >> (8 * k)) & 15), qb = (float)((c >> (8 * k + 4)) & 15);
-                    __half2 h = __floats2half2_rn(__fadd_rn(__fmul_rn(qa, s), z), __fadd_rn(__fmul_rn(qb, s), z));
-                    o[k] = as_u32(h);
+                    float qa = (float)((c[i] >> (8 * k)) & 15), qb = (float)((c[i] >> (8 * k + 4)) & 15);
+                    o[k] = as_u32(__floats2half2_rn(__fadd_rn(__fmul_rn(qa, s), z), __fadd_rn(__fmul_rn(qb, s), z)));
                 }
-                st_stream(dst + i * 32 + lane, make_uint4(o[0], o[1], o[2], o[3]));
+                st_stream(dst + i * 32, make_uint4(o[0], o[1], o[2], o[3]));
             }
         }
     }
@@ -302,25 +342,50 @@ PoolPtrs make_pools(const salicache_pools* p) {
     pp.int8_scale = (uint8_t*)p->int8_scale;
     pp.int4_codes = (uint8_t*)p->int4_codes;
     pp.int4_sz = (uint8_t*)p->int4_sz;
-    pp.cap[0] = p->cap_fp16;
-    pp.cap[1] = p->cap_int8;
-    pp.cap[2] = p->cap_int4;
+    pp.cap0 = p->cap_fp16;
+    pp.cap1 = p->cap_int8;
+    pp.cap2 = p->cap_int4;
     pp.ring = p->ring;
     return pp;
+}
+
+template <int ITERS>
+void launch_pack(int grid, size_t smem, cudaStream_t st, const __half* K, const __half* V, const KvGeom& g,
+                 const int32_t* idx, const int32_t* counts, const long long* off, const PoolPtrs& pp, int* status) {
+    k_pack<ITERS><<<grid, KV_THREADS, smem, st>>>(K, V, g, idx, counts, off, pp, status);
+}
+template <int ITERS>
+void launch_unpack(int grid, size_t smem, cudaStream_t st, __half* K, __half* V, const KvGeom& g, const int32_t* idx,
+                   const int32_t* counts, const long long* off, const PoolPtrs& pp, int* status) {
+    k_unpack<ITERS><<<grid, KV_THREADS, smem, st>>>(K, V, g, idx, counts, off, pp, status);
 }
 
 }  // namespace
 
 int sc_kv_max_batch() { return MAX_PREFIX; }
 
+// Row lengths the kernels are instantiated for (HD = 256 * ITERS).
+bool sc_kv_supported_hd(int HD) { return HD == 4096 || HD == 2048 || HD == 1024 || HD == 512 || HD == 256; }
+
 int sc_pack(salicache_ctx* c, const void* d_K, const void* d_V, int64_t frame_stride, const int32_t* d_idx,
             const int32_t* d_counts, const int64_t* d_row_offset, int B, const salicache_pools* pools, cudaStream_t st) {
     if (B == 0) return SALICACHE_OK;
-    KvGeom g{c->p.L, c->n_tok, c->p.heads * c->p.head_dim, c->p.heads * c->p.head_dim / 128, frame_stride, B};
-    int grid = c->sm_count * 4;
-    k_pack<<<grid, KV_THREADS, (size_t)(B + 1) * sizeof(int), st>>>((const __half*)d_K, (const __half*)d_V, g, d_idx,
-                                                                    d_counts, (const long long*)d_row_offset,
-                                                                    make_pools(pools), c->d_status);
+    const int HD = c->p.heads * c->p.head_dim;
+    KvGeom g{c->p.L, c->n_tok, HD, HD / 128, frame_stride, B};
+    const int grid = c->sm_count * 2;
+    const size_t smem = (size_t)(B + 1) * sizeof(int);
+    const __half* K = (const __half*)d_K;
+    const __half* V = (const __half*)d_V;
+    const long long* off = (const long long*)d_row_offset;
+    PoolPtrs pp = make_pools(pools);
+    switch (HD / 256) {
+        case 16: launch_pack<16>(grid, smem, st, K, V, g, d_idx, d_counts, off, pp, c->d_status); break;
+        case 8: launch_pack<8>(grid, smem, st, K, V, g, d_idx, d_counts, off, pp, c->d_status); break;
+        case 4: launch_pack<4>(grid, smem, st, K, V, g, d_idx, d_counts, off, pp, c->d_status); break;
+        case 2: launch_pack<2>(grid, smem, st, K, V, g, d_idx, d_counts, off, pp, c->d_status); break;
+        case 1: launch_pack<1>(grid, smem, st, K, V, g, d_idx, d_counts, off, pp, c->d_status); break;
+        default: return SALICACHE_E_PARAM;
+    }
     c->launches++;
     SC_CHECK(cudaGetLastError());
     return SALICACHE_OK;
@@ -330,15 +395,26 @@ int sc_unpack(salicache_ctx* c, const salicache_pools* pools, const int32_t* d_i
               const uint8_t* d_decision, const int64_t* d_row_offset, int B, int zero_fill_pruned, void* d_K_out,
               void* d_V_out, int64_t frame_stride, cudaStream_t st) {
     if (B == 0) return SALICACHE_OK;
-    KvGeom g{c->p.L, c->n_tok, c->p.heads * c->p.head_dim, c->p.heads * c->p.head_dim / 128, frame_stride, B};
-    int grid = c->sm_count * 4;
-    k_unpack<<<grid, KV_THREADS, (size_t)(B + 1) * sizeof(int), st>>>((__half*)d_K_out, (__half*)d_V_out, g, d_idx,
-                                                                      d_counts, (const long long*)d_row_offset,
-                                                                      make_pools(pools), c->d_status);
+    const int HD = c->p.heads * c->p.head_dim;
+    KvGeom g{c->p.L, c->n_tok, HD, HD / 128, frame_stride, B};
+    const int grid = c->sm_count * 2;
+    const size_t smem = (size_t)(B + 1) * sizeof(int);
+    __half* K = (__half*)d_K_out;
+    __half* V = (__half*)d_V_out;
+    const long long* off = (const long long*)d_row_offset;
+    PoolPtrs pp = make_pools(pools);
+    switch (HD / 256) {
+        case 16: launch_unpack<16>(grid, smem, st, K, V, g, d_idx, d_counts, off, pp, c->d_status); break;
+        case 8: launch_unpack<8>(grid, smem, st, K, V, g, d_idx, d_counts, off, pp, c->d_status); break;
+        case 4: launch_unpack<4>(grid, smem, st, K, V, g, d_idx, d_counts, off, pp, c->d_status); break;
+        case 2: launch_unpack<2>(grid, smem, st, K, V, g, d_idx, d_counts, off, pp, c->d_status); break;
+        case 1: launch_unpack<1>(grid, smem, st, K, V, g, d_idx, d_counts, off, pp, c->d_status); break;
+        default: return SALICACHE_E_PARAM;
+    }
     c->launches++;
     if (zero_fill_pruned) {
         dim3 gz(2 * g.L, B);
-        k_zero_pruned<<<gz, KV_THREADS, 0, st>>>((__half*)d_K_out, (__half*)d_V_out, g, d_decision);
+        k_zero_pruned<<<gz, KV_THREADS, 0, st>>>(K, V, g, d_decision);
         c->launches++;
     }
     SC_CHECK(cudaGetLastError());
