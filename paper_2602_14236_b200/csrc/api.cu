@@ -19,6 +19,8 @@ void free_scratch(salicache_ctx* c) {
         if (c->pyr[l]) cudaFree(c->pyr[l]);
         if (c->coef[l]) cudaFree(c->coef[l]);
     }
+    if (c->gh_a) cudaFree(c->gh_a);
+    if (c->gh_b) cudaFree(c->gh_b);
     if (c->flow_a) cudaFree(c->flow_a);
     if (c->flow_b) cudaFree(c->flow_b);
     if (c->bits_kept) cudaFree(c->bits_kept);
@@ -71,7 +73,7 @@ int salicache_create(salicache_ctx** out, const salicache_params* p) {
         return SALICACHE_E_PARAM;
     const int HD = p->heads * p->head_dim;
     if (!sc_kv_supported_hd(HD)) return SALICACHE_E_PARAM;
-    if (p->H <= 0 || p->W <= 0 || p->H % 56 != 0 || p->W % 112 != 0) return SALICACHE_E_SHAPE;   // 28-px tiles, 4 | H>>2, 16 | W
+    if (p->H <= 0 || p->W <= 0 || p->H % 112 != 0 || p->W % 112 != 0) return SALICACHE_E_SHAPE;  // 28-px tiles at 1/4 scale, 16 | W
     if (p->n_images == 5 && (p->H != 672 || p->W != 672)) return SALICACHE_E_SHAPE;
     if (p->max_batch < 1 || p->max_batch > sc_kv_max_batch()) return SALICACHE_E_SHAPE;
     salicache_ctx* c = new (std::nothrow) salicache_ctx();
@@ -105,8 +107,10 @@ int salicache_create(salicache_ctx** out, const salicache_params* p) {
     for (int l = 0; l < 3 && ok; ++l) {
         size_t Pl = P0 >> (2 * l);
         ok = ok && cudaMalloc(&c->pyr[l], slots * Pl * sizeof(float)) == cudaSuccess;
-        ok = ok && cudaMalloc(&c->coef[l], slots * 5 * Pl * sizeof(double)) == cudaSuccess;
+        ok = ok && cudaMalloc(&c->coef[l], slots * 5 * Pl * sizeof(float)) == cudaSuccess;
     }
+    ok = ok && cudaMalloc(&c->gh_a, (size_t)c->chunk * 5 * P0 * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->gh_b, (size_t)c->chunk * 5 * P0 * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->flow_a, (size_t)c->chunk * 2 * P0 * sizeof(double)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->flow_b, (size_t)c->chunk * 2 * P0 * sizeof(double)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->bits_kept, (size_t)c->chunk * p->H * words * sizeof(uint32_t)) == cudaSuccess;

@@ -36,8 +36,10 @@ struct salicache_ctx {
     PlaneGeom plane[2];
     // flow scratch (sized for the largest plane)
     float* pyr[3];             // [chunk+1][h_l*w_l]
-    double* coef[3];           // [chunk+1][5][h_l*w_l]
-    double* flow_a;            // [chunk][2][H*W]
+    float* coef[3];            // [2*chunk][5][h_l*w_l] expansion planes
+    float* gh_a;               // [chunk][5][H*W] normal-equation terms, ping
+    float* gh_b;               //                                         pong
+    double* flow_a;            // [chunk][2][H*W] displacement carried between levels
     double* flow_b;
     // saliency scratch
     uint32_t* bits_kept;       // [chunk][H][Ww]  NMS-kept weak or strong pixels
