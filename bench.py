@@ -103,6 +103,22 @@ def algorithmic_bytes(counts: np.ndarray, L: int, HD: int, G: int = 128):
     return int(read), int(write)
 
 
+def max_over_ranks(ms: float, device=None) -> float:
+    """Step time of the job = the slowest rank's device time (all-reduce MAX; identity on one rank)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_fps(frames_per_rank: int, steps: int, world: int, total_ms: float) -> float:
+    """Whole-job frames/s: every rank runs its own stream of `frames_per_rank` frames per step."""
+    return world * frames_per_rank * steps / (total_ms / 1e3)
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -212,13 +228,10 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else {}
     status = sc.salicache_poll_status(ctx)
     assert status == 0, f"device status {status}"
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dev)
 
     ms_per_step = total_ms / args.steps
-    fps = world * T * args.steps / (total_ms / 1e3)
+    fps = aggregate_fps(T, args.steps, world, total_ms)
     peak, peak_src = _peaks()
     pack_launches = n_chunks * args.steps
     pack_s = pack_ms / 1e3
