@@ -288,7 +288,9 @@ int sc_saliency_init(int max_h, int max_words) {
     SC_CHECK(cudaFuncSetAttribute(k_color_patch, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)color_smem()));
     size_t smem = (size_t)2 * max_h * max_words * sizeof(uint32_t);
     if (smem > 227 * 1024) return SALICACHE_E_SHAPE;
-    SC_CHECK(cudaFuncSetAttribute(k_hysteresis, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    // always the full opt-in limit: the attribute belongs to the function, not to a context, so a
+    // later context with smaller frames must not lower it under an earlier context with larger ones
+    SC_CHECK(cudaFuncSetAttribute(k_hysteresis, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     return SALICACHE_OK;
 }
 
