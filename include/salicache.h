@@ -183,6 +183,43 @@ SALICACHE_API int salicache_unpack_kv(salicache_ctx* ctx, const salicache_pools*
                         int zero_fill_pruned, void* d_K_out, void* d_V_out, int64_t frame_stride,
                         void* cuda_stream);
 
+/*
+ * The spatial score without any allocation.  (The paper has no counterpart: this entry point
+ * exists for the way the library is embedded, not for the method.)
+ *
+ * For callers that cannot allocate device memory while they run -- a serving process whose memory
+ * pool already owns the whole GPU, a plug-in that may not grow the process, code under an
+ * allocator lock -- and therefore cannot create a context.  It computes exactly what
+ * salicache_saliency computes (same kernels, same bits), but keeps the edge bit planes, the sRGB
+ * table and the status word in one fixed array inside the library's device image
+ * (about 233 KB, held by every GPU that loads the library until the process exits).  It calls no
+ * cudaMalloc / cudaFree and no allocating library routine.
+ *
+ *   p           HOST pointer; the fields read are H, W, patch, n_images, canny_lo, canny_hi,
+ *               var_radius, sigma_ref, w_edge, w_color, hyst_max_iters.  n_images must be 1 and
+ *               H, W at most SALICACHE_NOALLOC_MAX_SIDE (multiples of 112 as for a context).
+ *   d_frames    DEVICE, u8 [B][H][W][3], 16-byte aligned, caller-owned
+ *   B           0 .. SALICACHE_NOALLOC_MAX_FRAMES; larger batches are rejected with E_SHAPE and
+ *               nothing is launched (split them into several calls on the same stream)
+ *   d_s         DEVICE, f32 [B][(H/patch)*(W/patch)], caller-owned, written
+ *   d_status_or_null  DEVICE int32 the caller zeroed: receives SALICACHE_E_NOCONVERGE if edge
+ *               hysteresis hits hyst_max_iters.  With NULL the condition is recorded in the
+ *               library's own word, which this call clears first and nobody reads.
+ *
+ * The first call on each device resolves the array's device address, sets two kernel attributes
+ * and copies the 2 KB sRGB table with a blocking copy; make that call once per device with that
+ * device current before capturing a stream or entering a latency-critical section.  Later calls
+ * are asynchronous on `cuda_stream`.
+ * All calls on one device share the array and it keeps the previous call's contents (each call
+ * overwrites what it reads, and clears the status word).  Two calls that overlap on the GPU --
+ * different streams, or different host threads without ordering -- race on it: serialise them.
+ * Errors: E_NULL, E_PARAM, E_SHAPE, E_ALIGN, E_CUDA, as for salicache_saliency.
+ */
+#define SALICACHE_NOALLOC_MAX_FRAMES 8
+#define SALICACHE_NOALLOC_MAX_SIDE   336
+SALICACHE_API int salicache_saliency_noalloc(const salicache_params* p, const uint8_t* d_frames, int B, float* d_s,
+                                             int32_t* d_status_or_null, void* cuda_stream);
+
 /* Synchronises `cuda_stream`, returns the deferred device status (0, E_CAPACITY or
  * E_NOCONVERGE; E_CUDA if the stream reports an error) and clears it. */
 SALICACHE_API int salicache_poll_status(salicache_ctx* ctx, void* cuda_stream);

@@ -48,7 +48,7 @@ class Pools(C.Structure):
 EXPORTS = [
     "salicache_default_params", "salicache_create", "salicache_destroy", "salicache_strerror",
     "salicache_tokens_per_frame", "salicache_launch_count", "salicache_flow_score", "salicache_saliency", "salicache_select",
-    "salicache_pack_kv", "salicache_unpack_kv", "salicache_poll_status",
+    "salicache_pack_kv", "salicache_unpack_kv", "salicache_poll_status", "salicache_saliency_noalloc",
 ]
 
 _lib = None
@@ -80,6 +80,7 @@ def lib():
         _lib.salicache_pack_kv.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, C.POINTER(Pools), vp]
         _lib.salicache_unpack_kv.argtypes = [vp, C.POINTER(Pools), vp, vp, vp, vp, i32, i32, vp, vp, i64, vp]
         _lib.salicache_poll_status.argtypes = [vp, vp]
+        _lib.salicache_saliency_noalloc.argtypes = [C.POINTER(Params), vp, i32, vp, vp, vp]
     return _lib
 
 
@@ -144,6 +145,17 @@ def salicache_flow_score(ctx: Context, d_prev, d_cur, B: int, d_deltaP, d_flow=N
 
 def salicache_saliency(ctx: Context, d_frames, B: int, d_s, stream=None):
     _check(lib().salicache_saliency(ctx.handle, _ptr(d_frames), B, _ptr(d_s), _stream(stream)), "salicache_saliency")
+
+
+def salicache_saliency_noalloc(params: Params, d_frames, B: int, d_s, d_status=None, stream=None):
+    """Spatial score for hosts that cannot allocate device memory (no context needed): at most
+    NOALLOC_MAX_FRAMES frames of at most NOALLOC_MAX_SIDE pixels a side per call.  Calls on one
+    device share a fixed scratch array inside the library, so they must not overlap on the GPU."""
+    _check(lib().salicache_saliency_noalloc(C.byref(params), _ptr(d_frames), B, _ptr(d_s), _ptr(d_status),
+                                            _stream(stream)), "salicache_saliency_noalloc")
+
+
+NOALLOC_MAX_FRAMES, NOALLOC_MAX_SIDE = 8, 336
 
 
 def salicache_select(ctx: Context, d_deltaP, d_s, B: int, first_has_no_prev: bool, d_decision, d_idx, d_counts,

@@ -9,7 +9,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 LIB = os.path.join(_PKG, "libsalicache.so")
-SOURCES = ["api.cu", "flow.cu", "saliency.cu", "select.cu", "kv.cu"]
+SOURCES = ["api.cu", "flow.cu", "saliency.cu", "select.cu", "kv.cu", "noalloc.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--fmad=true",
          "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-I", os.path.join(_ROOT, "include"), "-I", CSRC]
 
@@ -42,7 +42,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if p.returncode:
             raise RuntimeError("nvcc failed: " + " ".join(cmd))
     tmp = LIB + f".tmp{os.getpid()}"
-    subprocess.check_call([nvcc, "-shared", "-o", tmp] + objs + ["-lcudart"])
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp] + objs + ["-lcudart"])
     os.replace(tmp, LIB)
     return LIB
 
