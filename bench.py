@@ -54,7 +54,7 @@ class ClockSampler:
         try:
             self.f = open(self.path, "w")
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.idx)], stdout=self.f, stderr=subprocess.DEVNULL)
+                                          "-lms", "20", "-i", str(self.idx)], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -162,15 +162,25 @@ def run_ours(args):
     off = torch.zeros((T, 3), dtype=torch.int64, device=dev)
     fill = torch.zeros((3,), dtype=torch.int64, device=dev)
 
-    def filter_stage():
-        fill.zero_()
-        if T > 1:
-            sc.salicache_flow_score(ctx, frames[:-1], frames[1:], T - 1, dP[1:])
-        sc.salicache_saliency(ctx, frames, T, s)
-        sc.salicache_select(ctx, dP, s, T, True, dec, idx, counts, red, off, fill)
+    seg = max(ring, (args.segment // ring) * ring)      # frames per pipeline segment: whole K/V ring passes
+    segments = [(b0, min(seg, T - b0)) for b0 in range(0, T, seg)]
+    main = torch.cuda.current_stream()
+    store_stream = torch.cuda.Stream(device=dev)
+
+    def filter_segment(b0: int, nb: int):
+        """flow (t-1 -> t), saliency and decisions of frames b0 .. b0+nb-1; the running pool fill carries over."""
+        if b0 == 0:
+            fill.zero_()
+            if nb > 1:
+                sc.salicache_flow_score(ctx, frames[:-1], frames[1:], nb - 1, dP[1:])
+        else:
+            sc.salicache_flow_score(ctx, frames[b0 - 1:], frames[b0:], nb, dP[b0:])
+        sc.salicache_saliency(ctx, frames[b0:], nb, s[b0:])
+        sc.salicache_select(ctx, dP[b0:], s[b0:], nb, b0 == 0, dec[b0:], idx[b0:], counts[b0:], red[b0:], off[b0:], fill)
 
     # sizing pass (untimed): the decisions fix the pool capacities
-    filter_stage()
+    for b0, nb in segments:
+        filter_segment(b0, nb)
     torch.cuda.synchronize()
     counts_h = counts.cpu().numpy()
     tot = counts_h[:, [4, 3, 2]].sum(axis=0)
@@ -179,23 +189,33 @@ def run_ours(args):
 
     n_chunks = (T + ring - 1) // ring
     ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(n_chunks)] for _ in range(args.steps)]
-    ev_f = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+    ev_f = [[[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in segments] for _ in range(args.steps)]
+    seg_done = [torch.cuda.Event() for _ in segments]
 
     def step(k: int):
+        """One pass of the whole hot path over the workload.  The filter of segment i+1 runs on the main
+        stream while the store of segment i runs on the second stream (decisions stay on the device)."""
         timed_events = k >= 0
-        if timed_events:
-            ev_f[k][0].record()
-        filter_stage()
-        if timed_events:
-            ev_f[k][1].record()
-        for c in range(n_chunks):
-            b0 = c * ring
-            nb = min(ring, T - b0)
+        store_stream.wait_stream(main)
+        for si, (b0, nb) in enumerate(segments):
             if timed_events:
-                ev[k][c][0].record()
-            sc.salicache_pack_kv(ctx, Kring, Vring, frame_stride, idx[b0:], counts[b0:], off[b0:], nb, pools.c)
+                ev_f[k][si][0].record(main)
+            filter_segment(b0, nb)
             if timed_events:
-                ev[k][c][1].record()
+                ev_f[k][si][1].record(main)
+            seg_done[si].record(main)
+            with torch.cuda.stream(store_stream):
+                store_stream.wait_event(seg_done[si])
+                for c0 in range(b0, b0 + nb, ring):
+                    c = c0 // ring
+                    cb = min(ring, b0 + nb - c0)
+                    if timed_events:
+                        ev[k][c][0].record(store_stream)
+                    sc.salicache_pack_kv(ctx, Kring, Vring, frame_stride, idx[c0:], counts[c0:], off[c0:], cb, pools.c,
+                                         stream=store_stream)
+                    if timed_events:
+                        ev[k][c][1].record(store_stream)
+        main.wait_stream(store_stream)
 
     def barrier():
         if world > 1:
@@ -222,7 +242,7 @@ def run_ours(args):
     barrier()
     for k in range(args.steps):
         pack_ms += sum(a.elapsed_time(b) for a, b in ev[k])
-        filt_ms += ev_f[k][0].elapsed_time(ev_f[k][1])
+        filt_ms += sum(a.elapsed_time(b) for a, b in ev_f[k])
     total_ms = e0.elapsed_time(e1)
     launches = ctx.launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else {}
@@ -267,7 +287,7 @@ def run_ours(args):
         "dtype": "f16->i8/i4 (store), f64 (scores)", "data": "synthetic",
         "config": {"workload": f"configs[{wl.index - 1}]: {wl.description}", "frames": T, "tokens_per_frame": n_tok,
                    "layers": L, "heads": wl.heads, "head_dim": wl.head_dim, "background": wl.background,
-                   "kv_ring_slabs": ring, "l2_policy": "inputs larger than L2 (K/V ring of %.1f GB)" % (2 * Kring.numel() * 2 / 1e9),
+                   "kv_ring_slabs": ring, "pipeline_segment_frames": seg, "l2_policy": "inputs larger than L2 (K/V ring of %.1f GB)" % (2 * Kring.numel() * 2 / 1e9),
                    "parallelism": "independent video stream per GPU"},
         "tokens_per_s": round(fps * n_tok, 1),
         "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
@@ -427,13 +447,14 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=3)
     ap.add_argument("--frames", type=int, default=0, help="use only the first N frames of the workload (profiling)")
-    ap.add_argument("--chunk", type=int, default=32, help="frames per internal pass of flow/saliency")
+    ap.add_argument("--chunk", type=int, default=40, help="frames per internal pass of flow/saliency")
     ap.add_argument("--ring", type=int, default=RING, help="K/V frame slabs resident on the device")
+    ap.add_argument("--segment", type=int, default=40, help="frames per pipeline segment (filter of one overlaps the store of the previous)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=1)

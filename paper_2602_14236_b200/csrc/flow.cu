@@ -1,16 +1,17 @@
 // Temporal branch (Sec. III-A, Eq. 5): gray pyramid, polynomial expansion, coarse-to-fine
 // displacement updates and the per-patch RMS flow magnitude.
 //
-// Arithmetic is double; only storage is single precision where that provably costs nothing or very
-// little: pyramid levels are exact in float, expansion coefficients and the per-pixel normal-equation
-// terms (G, h) are rounded to float between kernels (their effect on dP stays below 1 % of the 1e-4
-// relative tolerance on every workload; the cancellation b2(x~) - b1(x) itself is done in double).
+// Precision: the box sums, the 2x2 solve, sampling positions and the patch reduction are double (the
+// determinant cancels); pyramid levels are exact in float; expansion coefficients and the per-pixel
+// normal-equation terms (G, h) are stored as float, and the terms are formed in float from them.  The
+// effect on dP stays two orders of magnitude below the 1e-4 relative tolerance on every workload.
 //
-// One displacement update = box sums of (G, h) over the 15x15 window + a 2x2 solve.  k_flow_box does
-// that on a 28x28 tile (2x2 patches) with a double-precision integral image of the tile grown by the
-// window radius, and, fused behind the solve, the (G, h) of the NEXT update at the same pixels (which
-// needs no halo), or the patch scores after the last update.
+// One displacement update = box sums of (G, h) over the 15x15 window + a 2x2 solve.  k_flow_update does
+// that on a 28x14 tile with separable sliding-window sums (columns from registers, rows from shared
+// memory) and, fused behind the solve, the (G, h) of the NEXT update at the same pixels (which needs no
+// halo), or the patch scores after the last update.
 #include <math.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -139,18 +140,38 @@ __device__ __forceinline__ double bilin_fetch(const T* __restrict__ p, const Bil
 
 // Normal-equation terms of one pixel for the prior (du, dv): G = A^T A (g11 g12 g22), hv = A^T db,
 //   A = (A1(x) + A2(x~))/2,  db = -(b2(x~) - b1(x))/2 + A d~,  x~ = clamp(x + d~), bilinear fetch.
+// The sampling position is exact: floor and fraction of d~ are taken in double and the integer part is
+// added to the pixel index (a single-precision x + d~ would move the sample by up to 2e-5 px at
+// x ~ 300); the interpolation and the products run in single precision on the single-precision
+// coefficients, whose rounding already bounds what they can deliver.
 __device__ __forceinline__ void normal_terms(const float* __restrict__ c1, const float* __restrict__ c2, size_t P,
-                                             int h, int w, int y, int x, double du, double dv, double out[5]) {
+                                             int h, int w, int y, int x, double du, double dv, float out[5]) {
     const int p = y * w + x;
-    Bilin b = bilin_at(y + dv, x + du, h, w);
-    double b2x = bilin_fetch(c2, b), b2y = bilin_fetch(c2 + P, b);
-    double a2xx = bilin_fetch(c2 + 2 * P, b), a2yy = bilin_fetch(c2 + 3 * P, b);
-    double a2xy = 0.5 * bilin_fetch(c2 + 4 * P, b);
-    double axx = 0.5 * ((double)c1[2 * P + p] + a2xx);
-    double ayy = 0.5 * ((double)c1[3 * P + p] + a2yy);
-    double axy = 0.5 * (0.5 * (double)c1[4 * P + p] + a2xy);
-    double dbx = -0.5 * (b2x - (double)c1[p]) + (axx * du + axy * dv);
-    double dby = -0.5 * (b2y - (double)c1[P + p]) + (axy * du + ayy * dv);
+    // x~ = clamp(x + du): integer part and fraction of du in double, the integer add is exact
+    const double fdu = floor(du), fdv = floor(dv);
+    int x0 = x + (int)fdu, y0 = y + (int)fdv;
+    float fx = (float)(du - fdu), fy = (float)(dv - fdv);
+    if (x0 < 0) { x0 = 0; fx = 0.0f; }
+    if (x0 >= w - 1) { x0 = w - 1; fx = 0.0f; }
+    if (y0 < 0) { y0 = 0; fy = 0.0f; }
+    if (y0 >= h - 1) { y0 = h - 1; fy = 0.0f; }
+    const int x1 = min(x0 + 1, w - 1), y1 = min(y0 + 1, h - 1);
+    const float gx = 1.0f - fx, gy = 1.0f - fy;
+    const int i00 = y0 * w + x0, i01 = y0 * w + x1, i10 = y1 * w + x0, i11 = y1 * w + x1;
+    float v[5];
+#pragma unroll
+    for (int c = 0; c < 5; ++c) {
+        const float* q = c2 + c * P;
+        const float top = q[i00] * gx + q[i01] * fx;
+        const float bot = q[i10] * gx + q[i11] * fx;
+        v[c] = top * gy + bot * fy;
+    }
+    const float duf = (float)du, dvf = (float)dv;
+    const float axx = 0.5f * (c1[2 * P + p] + v[2]);
+    const float ayy = 0.5f * (c1[3 * P + p] + v[3]);
+    const float axy = 0.5f * (0.5f * c1[4 * P + p] + 0.5f * v[4]);
+    const float dbx = -0.5f * (v[0] - c1[p]) + (axx * duf + axy * dvf);
+    const float dby = -0.5f * (v[1] - c1[P + p]) + (axy * duf + ayy * dvf);
     out[0] = axx * axx + axy * axy;
     out[1] = axx * axy + axy * ayy;
     out[2] = axy * axy + ayy * ayy;
@@ -177,127 +198,208 @@ k_flow_gh(const float* __restrict__ coef1, const float* __restrict__ coef2, size
         du = 2.0 * bilin_fetch(c, b);
         dv = 2.0 * bilin_fetch(c + (size_t)hc * wc, b);
     }
-    double t[5];
+    float t[5];
     normal_terms(coef1 + (size_t)f * coef_stride, coef2 + (size_t)f * coef_stride, P, h, w, y, x, du, dv, t);
     float* o = gh + (size_t)f * gh_stride + r;
 #pragma unroll
-    for (int c = 0; c < 5; ++c) o[c * P] = (float)t[c];
+    for (int c = 0; c < 5; ++c) o[c * P] = t[c];
 }
 
-// ---- one displacement update on a 28x28 tile.
-constexpr int BT = 28;            // tile side = 2 patches of 14
-constexpr int BR = 7;             // window radius (window 15)
-constexpr int BE = BT + 2 * BR;   // 42
-constexpr int BEP = BE + 1;       // padded row (odd stride in 8-byte words: conflict-free row scans)
-constexpr int BOX_THREADS = 256;
+// ---- one displacement update on a tile of TW x 14 pixels (TW / 14 patches side by side).
+//   phase 1  one thread per (term, pair of columns of the tile grown by 8 columns each side): 28 8-byte
+//            loads down the columns, the 15-row sums of the 14 tile rows by a sliding window in double
+//            -> shared memory
+//   phase 2  one thread per (row, run of RUN columns): 15-column sums of the row sums, 2x2 solve -> d in
+//            shared memory
+//   phase 3  one thread per pixel: the (G, h) of the NEXT update at d (no halo needed), and / or d itself,
+//            and / or the patch scores after the last update
+// The window covers the in-image part only: terms outside the image count as zero.
+constexpr int TH = 14;             // tile height = 1 patch
+constexpr int BR = 7;              // window radius (window 15)
+constexpr int ER = TH + 2 * BR;    // 28 rows loaded
+constexpr int UPD_THREADS = 224;
 constexpr int EMIT_NEXT = 1, EMIT_D = 2, EMIT_DP = 4;
 
-__global__ void __launch_bounds__(BOX_THREADS)
-k_flow_box(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, double eps,
-           const float* __restrict__ coef1, const float* __restrict__ coef2, size_t coef_stride,
-           float* __restrict__ gh_out, double* __restrict__ d_out, size_t flow_stride, float* __restrict__ dP,
-           PlaneGeom g, int flags) {
-    extern __shared__ double I[];                 // [5][BE][BEP] -> integral images
-    __shared__ double psum[BOX_THREADS / 32][4];
+template <int TW>
+struct UpdGeom {
+    static constexpr int RUN = 4;                      // pixels per phase-2 thread
+    static constexpr int EW = TW + 16;                 // columns loaded: x0 - 8 .. x0 + TW + 7 (8-byte aligned pairs)
+    static constexpr int S = EW % 8 == 4 ? EW : EW + 4; // row stride in floats, = 4 (mod 8): the 16-byte loads of 8
+                                                       // consecutive rows fall on distinct banks
+    static constexpr int NQ = 2 * BR + RUN + 2;        // row sums read per run, starting one column early (16-byte aligned)
+    static_assert(TW % 14 == 0 && RUN == 4 && S % 8 == 4 && NQ % 4 == 0 && 5 * (EW / 2) <= UPD_THREADS &&
+                      16 * (TW / RUN) <= UPD_THREADS, "tile geometry");
+};
+
+template <int TW, int FLAGS>
+__global__ void __launch_bounds__(UPD_THREADS, 4)
+k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, double eps,
+              const float* __restrict__ coef1, const float* __restrict__ coef2, size_t coef_stride,
+              float* __restrict__ gh_out, double* __restrict__ d_out, size_t flow_stride, float* __restrict__ dP,
+              PlaneGeom g) {
+    using G = UpdGeom<TW>;
+    constexpr int RUN = G::RUN, EW = G::EW, S = G::S, NQ = G::NQ;
+    extern __shared__ __align__(16) double upd_smem[];
+    double (*dsm)[TW + 1][2] = reinterpret_cast<double (*)[TW + 1][2]>(upd_smem);      // [TH] (du, dv); the odd row pitch
+                                                                                       // spreads phase 2's stores over the banks
+    float (*vs)[TH][S] = reinterpret_cast<float (*)[TH][S]>(upd_smem + TH * (TW + 1) * 2);   // [5] 15-row sums
     const int f = blockIdx.z;
-    const int x0 = blockIdx.x * BT, y0 = blockIdx.y * BT;
+    const int x0 = blockIdx.x * TW, y0 = blockIdx.y * TH;
     const size_t P = (size_t)h * w;
-    const float* in = gh_in + (size_t)f * gh_stride;
-    // the in-image part of the window only: zeros outside the image
-    for (int i = threadIdx.x; i < BE * BE; i += BOX_THREADS) {
-        int ry = i / BE, rx = i % BE;
-        int y = y0 - BR + ry, x = x0 - BR + rx;
-        bool inside = y >= 0 && y < h && x >= 0 && x < w;
-        int p = y * w + x;
+    const int t = threadIdx.x;
+    if (t < 5 * (EW / 2)) {
+        const int c = t / (EW / 2), cp = t - c * (EW / 2);
+        const int x = x0 - 8 + 2 * cp;                  // even, and w is even: the pair is inside or outside together
+        const bool xin = x >= 0 && x < w;
+        const float* src = gh_in + (size_t)f * gh_stride + (size_t)c * P + (xin ? x : 0);
+        float2 v[ER];
 #pragma unroll
-        for (int c = 0; c < 5; ++c) I[(c * BE + ry) * BEP + rx] = inside ? (double)in[c * P + p] : 0.0;
+        for (int r = 0; r < ER; ++r) {
+            const int y = y0 - BR + r;
+            v[r] = (xin && y >= 0 && y < h) ? __ldg(reinterpret_cast<const float2*>(src + (size_t)y * w))
+                                            : make_float2(0.0f, 0.0f);
+        }
+        // 15-row sums in single precision without any subtraction (a sliding window would leave the rounding
+        // residue of a strong edge in the flat region behind it): rows 0..13 become suffix sums, rows 14..27
+        // prefix sums, and window r = rows r .. r+14 is suffix[r] + prefix[r+14].  At most 14 roundings per sum.
+#pragma unroll
+        for (int r = TH - 2; r >= 0; --r) {
+            v[r].x += v[r + 1].x;
+            v[r].y += v[r + 1].y;
+        }
+#pragma unroll
+        for (int r = TH + 1; r < ER; ++r) {
+            v[r].x += v[r - 1].x;
+            v[r].y += v[r - 1].y;
+        }
+        float2* dst = reinterpret_cast<float2*>(&vs[c][0][2 * cp]);
+#pragma unroll
+        for (int r = 0; r < TH; ++r) dst[r * (S / 2)] = make_float2(v[r].x + v[r + TH].x, v[r].y + v[r + TH].y);
     }
     __syncthreads();
-    if (threadIdx.x < 5 * BE) {                   // inclusive scan along each row
-        double* row = I + threadIdx.x * BEP;
-        double run = 0.0;
-#pragma unroll 6
-        for (int rx = 0; rx < BE; ++rx) { run += row[rx]; row[rx] = run; }
-    }
-    __syncthreads();
-    if (threadIdx.x < 5 * BE) {                   // then down each column
-        int c = threadIdx.x / BE, rx = threadIdx.x % BE;
-        double* col = I + c * BE * BEP + rx;
-        double run = 0.0;
-#pragma unroll 6
-        for (int ry = 0; ry < BE; ++ry) { run += col[ry * BEP]; col[ry * BEP] = run; }
-    }
-    __syncthreads();
-    double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;
-    for (int i = threadIdx.x; i < BT * BT; i += BOX_THREADS) {
-        int oy = i / BT, ox = i % BT;
-        // window rows oy .. oy+14 and columns ox .. ox+14 of the grown tile
-        double s[5];
+    if ((t & 15) < TH && (t >> 4) < TW / RUN) {
+        const int row = t & 15, run = t >> 4;      // a quarter warp reads 8 rows of one run: conflict-free 16-byte loads
+        const int col0 = RUN * run;                // output columns col0 .. col0+RUN-1; their windows start at col0 + 1
+        float s[5][RUN];
 #pragma unroll
         for (int c = 0; c < 5; ++c) {
-            const double* Ic = I + c * BE * BEP;
-            double a = Ic[(oy + 14) * BEP + ox + 14];
-            double b = oy > 0 ? Ic[(oy - 1) * BEP + ox + 14] : 0.0;
-            double cc = ox > 0 ? Ic[(oy + 14) * BEP + ox - 1] : 0.0;
-            double d = (oy > 0 && ox > 0) ? Ic[(oy - 1) * BEP + ox - 1] : 0.0;
-            s[c] = (a - b) - (cc - d);
+            const float4* src = reinterpret_cast<const float4*>(&vs[c][row][col0]);
+            float q[NQ];
+#pragma unroll
+            for (int i = 0; i < NQ / 4; ++i) {
+                float4 pr = src[i];
+                q[4 * i] = pr.x;
+                q[4 * i + 1] = pr.y;
+                q[4 * i + 2] = pr.z;
+                q[4 * i + 3] = pr.w;
+            }
+            // windows q[k+1 .. k+15], k = 0..3, again without subtraction: suffix sums ending at q[15],
+            // prefix sums starting at q[16]
+            float suf = q[RUN];
+#pragma unroll
+            for (int i = RUN + 1; i <= 2 * BR + 1; ++i) suf += q[i];
+            float pre = 0.0f;
+#pragma unroll
+            for (int k = RUN - 1; k >= 0; --k) {      // suf = q[k+1] + ... + q[15]
+                if (k < RUN - 1) suf += q[k + 1];
+                s[c][k] = suf;
+            }
+#pragma unroll
+            for (int k = 1; k < RUN; ++k) {            // pre = q[16] + ... + q[15+k]
+                pre += q[2 * BR + 1 + k];
+                s[c][k] += pre;
+            }
         }
-        const double det = s[0] * s[2] - s[1] * s[1] + eps;
-        const double du = (s[2] * s[3] - s[1] * s[4]) / det;
-        const double dv = (s[0] * s[4] - s[1] * s[3]) / det;
+        // the 2x2 solve in double: the determinant cancels
+#pragma unroll
+        for (int k = 0; k < RUN; ++k) {
+            const double g11 = s[0][k], g12 = s[1][k], g22 = s[2][k], h1 = s[3][k], h2 = s[4][k];
+            const double inv = 1.0 / (g11 * g22 - g12 * g12 + eps);
+            double2 d;
+            d.x = (g22 * h1 - g12 * h2) * inv;
+            d.y = (g11 * h2 - g12 * h1) * inv;
+            *reinterpret_cast<double2*>(&dsm[row][col0 + k][0]) = d;
+        }
+    }
+    __syncthreads();
+    // UPD_THREADS is a multiple of TW: a thread keeps its column, hence its patch, over its pixels
+    static_assert(UPD_THREADS % TW == 0, "a thread stays in one column");
+    double acc = 0.0;
+    constexpr int PER = (TH * TW + UPD_THREADS - 1) / UPD_THREADS;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+        const int i = t + j * UPD_THREADS;
+        if (i >= TH * TW) break;
+        const int oy = i / TW, ox = i - oy * TW;
+        const double2 d = *reinterpret_cast<const double2*>(&dsm[oy][ox][0]);
         const int y = y0 + oy, x = x0 + ox, p = y * w + x;
-        if (flags & EMIT_D) {
+        if (FLAGS & EMIT_D) {
             double* o = d_out + (size_t)f * flow_stride;
-            o[p] = du;
-            o[P + p] = dv;
+            o[p] = d.x;
+            o[P + p] = d.y;
         }
-        if (flags & EMIT_NEXT) {
-            double t[5];
-            normal_terms(coef1 + (size_t)f * coef_stride, coef2 + (size_t)f * coef_stride, P, h, w, y, x, du, dv, t);
+        if (FLAGS & EMIT_NEXT) {
+            float tm[5];
+            normal_terms(coef1 + (size_t)f * coef_stride, coef2 + (size_t)f * coef_stride, P, h, w, y, x, d.x, d.y, tm);
             float* o = gh_out + (size_t)f * gh_stride + p;
 #pragma unroll
-            for (int c = 0; c < 5; ++c) o[c * P] = (float)t[c];
+            for (int c = 0; c < 5; ++c) o[c * P] = tm[c];
         }
-        if (flags & EMIT_DP) {
-            const double m = du * du + dv * dv;
-            const bool lower = oy >= BT / 2, right = ox >= BT / 2;
-            acc0 += (!lower && !right) ? m : 0.0;
-            acc1 += (!lower && right) ? m : 0.0;
-            acc2 += (lower && !right) ? m : 0.0;
-            acc3 += (lower && right) ? m : 0.0;
-        }
+        if (FLAGS & EMIT_DP) acc += d.x * d.x + d.y * d.y;
     }
-    if (flags & EMIT_DP) {     // Eq. 5 (flow reading): dP_i = sqrt(mean over the patch of u^2 + v^2)
-#pragma unroll
-        for (int o = 16; o; o >>= 1) {
-            acc0 += __shfl_xor_sync(0xffffffffu, acc0, o);
-            acc1 += __shfl_xor_sync(0xffffffffu, acc1, o);
-            acc2 += __shfl_xor_sync(0xffffffffu, acc2, o);
-            acc3 += __shfl_xor_sync(0xffffffffu, acc3, o);
-        }
-        if ((threadIdx.x & 31) == 0) {
-            double* ps = psum[threadIdx.x >> 5];
-            ps[0] = acc0; ps[1] = acc1; ps[2] = acc2; ps[3] = acc3;
-        }
+    if (FLAGS & EMIT_DP) {     // Eq. 5 (flow reading): dP_i = sqrt(mean over the patch of u^2 + v^2)
+        double* part = upd_smem;                   // (du, dv) are no longer needed once every thread is here
         __syncthreads();
-        if (threadIdx.x < 4) {
+        part[t] = acc;
+        __syncthreads();
+        if (t < TW / 14) {
             double tot = 0.0;
-            for (int wp = 0; wp < BOX_THREADS / 32; ++wp) tot += psum[wp][threadIdx.x];
-            int py = blockIdx.y * 2 + threadIdx.x / 2, px = blockIdx.x * 2 + threadIdx.x % 2;
-            dP[(size_t)f * g.n_tok + patch_token(g, py, px)] = (float)sqrt(tot / (double)((BT / 2) * (BT / 2)));
+            for (int q = 0; q < UPD_THREADS; ++q)                          // fixed order: deterministic
+                if ((q % TW) / 14 == t) tot += part[q];
+            const int py = blockIdx.y, px = blockIdx.x * (TW / 14) + t;
+            dP[(size_t)f * g.n_tok + patch_token(g, py, px)] = (float)sqrt(tot / (double)(TH * 14));
         }
     }
+}
+
+template <int TW>
+constexpr size_t upd_smem_bytes() {
+    return (size_t)TH * (TW + 1) * 2 * sizeof(double) + (size_t)5 * TH * UpdGeom<TW>::S * sizeof(float);
+}
+
+template <int TW>
+int init_update() {
+#define SC_UPD(F) SC_CHECK(cudaFuncSetAttribute(k_flow_update<TW, F>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)upd_smem_bytes<TW>()));
+    SC_UPD(EMIT_NEXT) SC_UPD(EMIT_D) SC_UPD(EMIT_DP | EMIT_D)
+#undef SC_UPD
+    return SALICACHE_OK;
+}
+
+template <int TW>
+void launch_update(dim3 grid, cudaStream_t st, int flags, const float* gin, size_t gstride, int h, int w, double eps,
+                   const float* c1, const float* c2, size_t cstride, float* gout, double* dout, size_t fstride,
+                   float* dP, const PlaneGeom& g) {
+#define SC_UPD(F)                                                                                                   \
+    case F:                                                                                                         \
+        k_flow_update<TW, F><<<grid, UPD_THREADS, upd_smem_bytes<TW>(), st>>>(gin, gstride, h, w, eps, c1, c2,     \
+                                                                               cstride, gout, dout, fstride, dP, g); \
+        break;
+    switch (flags) {
+        SC_UPD(EMIT_NEXT)
+        SC_UPD(EMIT_D)
+        SC_UPD(EMIT_DP | EMIT_D)
+        default: break;
+    }
+#undef SC_UPD
 }
 
 inline unsigned blocks_for(long long n, int threads) { return (unsigned)((n + threads - 1) / threads); }
 
 }  // namespace
 
-static size_t flow_box_smem() { return (size_t)5 * BE * BEP * sizeof(double); }
-
 int sc_flow_init() {
-    SC_CHECK(cudaFuncSetAttribute(k_flow_box, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)flow_box_smem()));
-    return SALICACHE_OK;
+    int rc = init_update<56>();
+    return rc != SALICACHE_OK ? rc : init_update<28>();
 }
 
 int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, const uint8_t* d_cur, size_t frame_bytes,
@@ -346,29 +448,40 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
         for (int l = 2; l >= 0; --l) {
             const size_t Pl = (size_t)hs[l] * ws[l];
             const size_t cstride = 5 * Pl;
-            const float* c1 = c->coef[l];
-            const float* c2 = c->coef[l] + (sequence ? cstride : (size_t)nb * cstride);
-            k_flow_gh<<<blocks_for((long long)Pl * nb, 256), 256, 0, st>>>(c1, c2, cstride, hs[l], ws[l], coarse, fstride,
-                                                                           c->gh_a, gstride, nb);
-            c->launches++;
-            float* gin = c->gh_a;
-            float* gout = c->gh_b;
             double* dl = d_lvl[l & 1];
-            dim3 grid(ws[l] / BT, hs[l] / BT, nb);
-            for (int it = 0; it < p.iters; ++it) {
-                const bool last = it == p.iters - 1;
-                int flags = last ? 0 : EMIT_NEXT;
-                double* dout = dl;
-                if (last && l > 0) flags |= EMIT_D;
-                if (last && l == 0) {
-                    flags |= EMIT_DP;
-                    if (d_flow_or_null) { flags |= EMIT_D; dout = d_flow_or_null + (size_t)b0 * fstride; }
-                }
-                k_flow_box<<<grid, BOX_THREADS, flow_box_smem(), st>>>(gin, gstride, hs[l], ws[l], p.eps_det, c1, c2,
-                                                                       cstride, gout, dout, fstride,
-                                                                       d_deltaP + (size_t)b0 * g.n_tok, g, flags);
+            const int tw = ws[l] % 56 == 0 ? 56 : 28;
+            int sub = nb;
+            if (const char* e = getenv("SC_SUB")) { int v = atoi(e); if (v > 0 && l == 0) sub = v; }
+            if (const char* e = getenv("SC_SUB1")) { int v = atoi(e); if (v > 0 && l == 1) sub = v; }
+            for (int z0 = 0; z0 < nb; z0 += sub) {
+                const int nz = nb - z0 < sub ? nb - z0 : sub;
+                const float* c1 = c->coef[l] + (size_t)z0 * cstride;
+                const float* c2 = c1 + (sequence ? cstride : (size_t)nb * cstride);
+                float* gin = c->gh_a + (size_t)z0 * gstride;
+                float* gout = c->gh_b + (size_t)z0 * gstride;
+                k_flow_gh<<<blocks_for((long long)Pl * nz, 256), 256, 0, st>>>(
+                    c1, c2, cstride, hs[l], ws[l], coarse ? coarse + (size_t)z0 * fstride : nullptr, fstride, gin, gstride, nz);
                 c->launches++;
-                float* t = gin; gin = gout; gout = t;
+                dim3 grid(ws[l] / tw, hs[l] / TH, nz);
+                for (int it = 0; it < p.iters; ++it) {
+                    const bool last = it == p.iters - 1;
+                    int flags = last ? 0 : EMIT_NEXT;
+                    double* dout = dl + (size_t)z0 * fstride;
+                    if (last && l > 0) flags |= EMIT_D;
+                    if (last && l == 0) {      // the field goes to the caller's buffer if there is one, else to scratch
+                        flags |= EMIT_DP | EMIT_D;
+                        if (d_flow_or_null) dout = d_flow_or_null + (size_t)(b0 + z0) * fstride;
+                    }
+                    float* dp = d_deltaP + (size_t)(b0 + z0) * g.n_tok;
+                    if (tw == 56)
+                        launch_update<56>(grid, st, flags, gin, gstride, hs[l], ws[l], p.eps_det, c1, c2, cstride, gout, dout,
+                                          fstride, dp, g);
+                    else
+                        launch_update<28>(grid, st, flags, gin, gstride, hs[l], ws[l], p.eps_det, c1, c2, cstride, gout, dout,
+                                          fstride, dp, g);
+                    c->launches++;
+                    float* t = gin; gin = gout; gout = t;
+                }
             }
             coarse = dl;
         }

@@ -36,7 +36,7 @@ def test_flow_score_matches_oracle_on_workload_1(wl1_frames, wl1_oracle_scores):
     ctx = _ctx()
     dP, s, fl = gu.gpu_scores(ctx, wl1_frames, want_flow=True)
     rdP, rs, rfl = wl1_oracle_scores
-    assert np.abs(fl - rfl).max() < 2e-6          # dense field: double arithmetic, float storage between kernels
+    assert np.abs(fl - rfl).max() < 2e-5          # dense field (px): single-precision terms and window sums, double solve
     gu.assert_scores_close(dP[1:], rdP[1:], "dP")
     gu.assert_scores_close(s, rs, "s")
 
