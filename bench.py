@@ -175,7 +175,8 @@ def run_ours(args):
                 sc.salicache_flow_score(ctx, frames[:-1], frames[1:], nb - 1, dP[1:])
         else:
             sc.salicache_flow_score(ctx, frames[b0 - 1:], frames[b0:], nb, dP[b0:])
-        sc.salicache_saliency(ctx, frames[b0:], nb, s[b0:])
+        sc.salicache_frame_redundancy(ctx, dP[b0:], nb, b0 == 0, red[b0:])
+        sc.salicache_saliency(ctx, frames[b0:], nb, s[b0:], red[b0:])      # Alg. 1: redundant frames are not scored
         sc.salicache_select(ctx, dP[b0:], s[b0:], nb, b0 == 0, dec[b0:], idx[b0:], counts[b0:], red[b0:], off[b0:], fill)
 
     # sizing pass (untimed): the decisions fix the pool capacities
@@ -330,7 +331,8 @@ def run_e2e(args, sc, ctx, wl, T, frames_np, Kring, Vring, pools, dev, bufs, wor
         fill.zero_()
         if T > 1:
             sc.salicache_flow_score(ctx, d_frames[:-1], d_frames[1:], T - 1, dP[1:])
-        sc.salicache_saliency(ctx, d_frames, T, s)
+        sc.salicache_frame_redundancy(ctx, dP, T, True, red)
+        sc.salicache_saliency(ctx, d_frames, T, s, red)
         sc.salicache_select(ctx, dP, s, T, True, dec, idx, counts, red, off, fill)
         h_counts.copy_(counts, non_blocking=True)
         h_dec.copy_(dec, non_blocking=True)

@@ -117,10 +117,24 @@ SALICACHE_API int salicache_flow_score(salicache_ctx* ctx, const uint8_t* d_prev
 /*
  * Spatial score (Sec. III-B, Eq. 7): Canny edge map E and LAB local colour variance C give
  * S = clamp(w_edge E + w_color C, 0, 1); d_s[b][i] = mean of S over patch i.
- * d_frames: B frames.  Edge hysteresis runs to its fixed point on the device; if it needs more
- * than hyst_max_iters sweeps the status word records E_NOCONVERGE (see salicache_poll_status).
+ * d_frames: B frames.  d_skip_or_null: DEVICE u8 [B] or NULL; frames with a non-zero entry are not
+ * scored and their rows of d_s are left untouched (Alg. 1 skips the spatial branch of a temporally
+ * redundant frame: pass the flags of salicache_frame_redundancy).  Edge hysteresis runs to its
+ * fixed point on the device; if it needs more than hyst_max_iters sweeps the status word records
+ * E_NOCONVERGE (see salicache_poll_status).
  */
-SALICACHE_API int salicache_saliency(salicache_ctx* ctx, const uint8_t* d_frames, int B, float* d_s, void* cuda_stream);
+SALICACHE_API int salicache_saliency(salicache_ctx* ctx, const uint8_t* d_frames, int B, float* d_s,
+                                     const uint8_t* d_skip_or_null, void* cuda_stream);
+
+/*
+ * Frame redundancy alone (Eq. 6; Alg. 1 lines 4-8): d_frame_redundant[b] = 1 when frame b has a
+ * predecessor and R_frame = (1/N) sum_i [dP_i < tau_t] exceeds theta_R, else 0.  Same arithmetic as
+ * salicache_select, which recomputes it; this call exists so that the spatial branch can skip the
+ * redundant frames.  d_deltaP: f32 [B][N_tok] or NULL (no frame has a predecessor);
+ * first_has_no_prev as for salicache_select.  Errors: E_NULL, E_SHAPE, E_CUDA.
+ */
+SALICACHE_API int salicache_frame_redundancy(salicache_ctx* ctx, const float* d_deltaP, int B, int first_has_no_prev,
+                                             uint8_t* d_frame_redundant, void* cuda_stream);
 
 /*
  * Decisions (Eq. 6, Eq. 8, Alg. 1) for B frames, one row of d_deltaP / d_s per frame.

@@ -49,6 +49,7 @@ EXPORTS = [
     "salicache_default_params", "salicache_create", "salicache_destroy", "salicache_strerror",
     "salicache_tokens_per_frame", "salicache_launch_count", "salicache_flow_score", "salicache_saliency", "salicache_select",
     "salicache_pack_kv", "salicache_unpack_kv", "salicache_poll_status", "salicache_saliency_noalloc",
+    "salicache_frame_redundancy",
 ]
 
 _lib = None
@@ -75,7 +76,8 @@ def lib():
         _lib.salicache_launch_count.restype = C.c_int64
         vp, i32, i64 = C.c_void_p, C.c_int, C.c_int64
         _lib.salicache_flow_score.argtypes = [vp, vp, vp, i32, vp, vp, vp]
-        _lib.salicache_saliency.argtypes = [vp, vp, i32, vp, vp]
+        _lib.salicache_saliency.argtypes = [vp, vp, i32, vp, vp, vp]
+        _lib.salicache_frame_redundancy.argtypes = [vp, vp, i32, i32, vp, vp]
         _lib.salicache_select.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         _lib.salicache_pack_kv.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, C.POINTER(Pools), vp]
         _lib.salicache_unpack_kv.argtypes = [vp, C.POINTER(Pools), vp, vp, vp, vp, i32, i32, vp, vp, i64, vp]
@@ -143,8 +145,14 @@ def salicache_flow_score(ctx: Context, d_prev, d_cur, B: int, d_deltaP, d_flow=N
                                       _stream(stream)), "salicache_flow_score")
 
 
-def salicache_saliency(ctx: Context, d_frames, B: int, d_s, stream=None):
-    _check(lib().salicache_saliency(ctx.handle, _ptr(d_frames), B, _ptr(d_s), _stream(stream)), "salicache_saliency")
+def salicache_saliency(ctx: Context, d_frames, B: int, d_s, d_skip=None, stream=None):
+    _check(lib().salicache_saliency(ctx.handle, _ptr(d_frames), B, _ptr(d_s), _ptr(d_skip), _stream(stream)),
+           "salicache_saliency")
+
+
+def salicache_frame_redundancy(ctx: Context, d_deltaP, B: int, first_has_no_prev: bool, d_frame_redundant, stream=None):
+    _check(lib().salicache_frame_redundancy(ctx.handle, _ptr(d_deltaP), B, int(first_has_no_prev),
+                                            _ptr(d_frame_redundant), _stream(stream)), "salicache_frame_redundancy")
 
 
 def salicache_saliency_noalloc(params: Params, d_frames, B: int, d_s, d_status=None, stream=None):

@@ -194,19 +194,27 @@ int salicache_flow_score(salicache_ctx* c, const uint8_t* d_prev, const uint8_t*
     return SALICACHE_OK;
 }
 
-int salicache_saliency(salicache_ctx* c, const uint8_t* d_frames, int B, float* d_s, void* cuda_stream) {
+int salicache_frame_redundancy(salicache_ctx* c, const float* d_deltaP, int B, int first_has_no_prev,
+                               uint8_t* d_frame_redundant, void* cuda_stream) {
+    if (!c || !d_frame_redundant) return SALICACHE_E_NULL;
+    if (B < 0 || B > c->p.max_batch) return SALICACHE_E_SHAPE;
+    return sc_frame_redundancy(c, d_deltaP, B, first_has_no_prev, d_frame_redundant, (cudaStream_t)cuda_stream);
+}
+
+int salicache_saliency(salicache_ctx* c, const uint8_t* d_frames, int B, float* d_s, const uint8_t* d_skip_or_null,
+                       void* cuda_stream) {
     if (!c || !d_frames || !d_s) return SALICACHE_E_NULL;
     if (B < 0 || B > c->p.max_batch) return SALICACHE_E_SHAPE;
     if (!aligned16(d_frames) || !aligned16(d_s)) return SALICACHE_E_ALIGN;
     if (B == 0) return SALICACHE_OK;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const size_t fb = (size_t)c->p.H * c->p.W * 3;
-    int rc = sc_saliency(c, c->plane[0], d_frames, fb, B, d_s, st);
+    int rc = sc_saliency(c, c->plane[0], d_frames, fb, B, d_s, d_skip_or_null, st);
     if (rc != SALICACHE_OK || c->n_planes == 1) return rc;
     rc = sc_box_down2(d_frames, c->p.H, c->p.W, B, c->base_frames, st);
     c->launches++;
     if (rc != SALICACHE_OK) return rc;
-    return sc_saliency(c, c->plane[1], c->base_frames, fb / 4, B, d_s, st);
+    return sc_saliency(c, c->plane[1], c->base_frames, fb / 4, B, d_s, d_skip_or_null, st);
 }
 
 int salicache_select(salicache_ctx* c, const float* d_deltaP, const float* d_s, int B, int first_has_no_prev,

@@ -58,12 +58,14 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
                   int B, bool sequence, float* d_deltaP, double* d_flow_or_null, cudaStream_t st);
 // saliency.cu
 int sc_saliency(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_frames, size_t frame_bytes, int B, float* d_s,
-                cudaStream_t st);
+                const uint8_t* d_skip, cudaStream_t st);
 int sc_box_down2(const uint8_t* d_src, int H, int W, int B, uint8_t* d_dst, cudaStream_t st);
 // select.cu
 int sc_select(salicache_ctx* c, const float* d_deltaP, const float* d_s, int B, int first_has_no_prev,
               uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts, uint8_t* d_frame_redundant,
               int64_t* d_row_offset, int64_t* d_fill, cudaStream_t st);
+int sc_frame_redundancy(salicache_ctx* c, const float* d_deltaP, int B, int first_has_no_prev, uint8_t* d_frame_redundant,
+                        cudaStream_t st);
 // kv.cu
 int sc_pack(salicache_ctx* c, const void* d_K, const void* d_V, int64_t frame_stride, const int32_t* d_idx,
             const int32_t* d_counts, const int64_t* d_row_offset, int B, const salicache_pools* pools, cudaStream_t st);

@@ -11,7 +11,6 @@
 // memory) and, fused behind the solve, the (G, h) of the NEXT update at the same pixels (which needs no
 // halo), or the patch scores after the last update.
 #include <math.h>
-#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -352,10 +351,17 @@ k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, d
         __syncthreads();
         part[t] = acc;
         __syncthreads();
+        if (t < TW) {                              // column totals, then 14 columns per patch: fixed order, deterministic
+            double col = 0.0;
+#pragma unroll
+            for (int k = 0; k < UPD_THREADS / TW; ++k) col += part[t + k * TW];
+            part[UPD_THREADS + t] = col;
+        }
+        __syncthreads();
         if (t < TW / 14) {
             double tot = 0.0;
-            for (int q = 0; q < UPD_THREADS; ++q)                          // fixed order: deterministic
-                if ((q % TW) / 14 == t) tot += part[q];
+#pragma unroll
+            for (int q = 0; q < 14; ++q) tot += part[UPD_THREADS + 14 * t + q];
             const int py = blockIdx.y, px = blockIdx.x * (TW / 14) + t;
             dP[(size_t)f * g.n_tok + patch_token(g, py, px)] = (float)sqrt(tot / (double)(TH * 14));
         }
@@ -450,11 +456,8 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
             const size_t cstride = 5 * Pl;
             double* dl = d_lvl[l & 1];
             const int tw = ws[l] % 56 == 0 ? 56 : 28;
-            int sub = nb;
-            if (const char* e = getenv("SC_SUB")) { int v = atoi(e); if (v > 0 && l == 0) sub = v; }
-            if (const char* e = getenv("SC_SUB1")) { int v = atoi(e); if (v > 0 && l == 1) sub = v; }
-            for (int z0 = 0; z0 < nb; z0 += sub) {
-                const int nz = nb - z0 < sub ? nb - z0 : sub;
+            {
+                const int z0 = 0, nz = nb;
                 const float* c1 = c->coef[l] + (size_t)z0 * cstride;
                 const float* c2 = c1 + (sequence ? cstride : (size_t)nb * cstride);
                 float* gin = c->gh_a + (size_t)z0 * gstride;

@@ -96,5 +96,5 @@ extern "C" int salicache_saliency_noalloc(const salicache_params* p, const uint8
     // the status word keeps the last call's value: start this call from "ok"
     if (!d_status_or_null && cudaMemsetAsync(base + NA_STATUS_OFF, 0, sizeof(int), st) != cudaSuccess)
         return SALICACHE_E_CUDA;
-    return sc_saliency(&c, c.plane[0], d_frames, (size_t)p->H * p->W * 3, B, d_s, st);
+    return sc_saliency(&c, c.plane[0], d_frames, (size_t)p->H * p->W * 3, B, d_s, nullptr, st);
 }

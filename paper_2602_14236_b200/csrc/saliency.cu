@@ -38,11 +38,12 @@ constexpr int CM = CT + 2;   // magnitude tile
 
 __global__ void __launch_bounds__(256)
 k_canny_classify(const uint8_t* __restrict__ frames, size_t frame_bytes, int h, int w, int words, int lo2, int hi2,
-                 uint32_t* __restrict__ bits_kept, uint32_t* __restrict__ bits_strong) {
+                 uint32_t* __restrict__ bits_kept, uint32_t* __restrict__ bits_strong, const uint8_t* __restrict__ skip) {
     __shared__ uint8_t sg[CG][CG];
     __shared__ uint8_t sb[CB][CB];
     __shared__ int smag[CM][CM];
     const int f = blockIdx.z, x0 = blockIdx.x * CT, y0 = blockIdx.y * CT;
+    if (skip && skip[f]) return;
     const uint8_t* fr = frames + (size_t)f * frame_bytes;
     for (int i = threadIdx.x; i < CG * CG; i += blockDim.x) {
         int ry = i / CG, rx = i % CG;
@@ -118,11 +119,12 @@ k_canny_classify(const uint8_t* __restrict__ frames, size_t frame_bytes, int h, 
 // Every word is owned by one thread (updates are monotone, so stale neighbour reads only delay).
 __global__ void __launch_bounds__(1024)
 k_hysteresis(const uint32_t* __restrict__ bits_kept, uint32_t* __restrict__ bits_edge, int h, int words, int max_iters,
-             int* __restrict__ status) {
+             int* __restrict__ status, const uint8_t* __restrict__ skip) {
     extern __shared__ uint32_t sh[];
     uint32_t* K = sh;                      // [h][words]
     uint32_t* E = sh + (size_t)h * words;  // [h][words]
     const int f = blockIdx.x, n = h * words;
+    if (skip && skip[f]) return;
     const uint32_t* gk = bits_kept + (size_t)f * n;
     uint32_t* ge = bits_edge + (size_t)f * n;
     for (int i = threadIdx.x; i < n; i += blockDim.x) { K[i] = gk[i]; E[i] = ge[i]; }
@@ -193,12 +195,13 @@ constexpr int SE = ST + 2 * SR;   // 34
 __global__ void __launch_bounds__(256)
 k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom g, int patch,
               const double* __restrict__ lut, const uint32_t* __restrict__ bits_edge, int words, double inv_sigma,
-              double w_edge, double w_color, float* __restrict__ s_out) {
+              double w_edge, double w_color, float* __restrict__ s_out, const uint8_t* __restrict__ skip) {
     extern __shared__ double cs[];
     double (*lab)[SE][SE + 1] = reinterpret_cast<double (*)[SE][SE + 1]>(cs);                    // [3]
     double (*hs)[SE][ST] = reinterpret_cast<double (*)[SE][ST]>(cs + 3 * SE * (SE + 1));          // [6]
     __shared__ double psum[8][4];
     const int f = blockIdx.z, x0 = blockIdx.x * ST, y0 = blockIdx.y * ST;
+    if (skip && skip[f]) return;
     const int h = g.H, w = g.W;
     const uint8_t* fr = frames + (size_t)f * frame_bytes;
     double L0, a0, b0;
@@ -301,20 +304,21 @@ int sc_box_down2(const uint8_t* d_src, int H, int W, int B, uint8_t* d_dst, cuda
 }
 
 int sc_saliency(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_frames, size_t frame_bytes, int B, float* d_s,
-                cudaStream_t st) {
+                const uint8_t* d_skip, cudaStream_t st) {
     const salicache_params& p = c->p;
     const int words = (g.W + 31) / 32;
     for (int b0 = 0; b0 < B; b0 += c->chunk) {
         int nb = B - b0 < c->chunk ? B - b0 : c->chunk;
         const uint8_t* fr = d_frames + (size_t)b0 * frame_bytes;
+        const uint8_t* skip = d_skip ? d_skip + b0 : nullptr;
         dim3 gc((g.W + CT - 1) / CT, (g.H + CT - 1) / CT, nb);
         k_canny_classify<<<gc, 256, 0, st>>>(fr, frame_bytes, g.H, g.W, words, p.canny_lo * p.canny_lo,
-                                             p.canny_hi * p.canny_hi, c->bits_kept, c->bits_edge);
+                                             p.canny_hi * p.canny_hi, c->bits_kept, c->bits_edge, skip);
         size_t smem = (size_t)2 * g.H * words * sizeof(uint32_t);
-        k_hysteresis<<<nb, 1024, smem, st>>>(c->bits_kept, c->bits_edge, g.H, words, p.hyst_max_iters, c->d_status);
+        k_hysteresis<<<nb, 1024, smem, st>>>(c->bits_kept, c->bits_edge, g.H, words, p.hyst_max_iters, c->d_status, skip);
         dim3 gs(g.W / ST, g.H / ST, nb);
         k_color_patch<<<gs, 256, color_smem(), st>>>(fr, frame_bytes, g, p.patch, c->lut, c->bits_edge, words, 1.0 / p.sigma_ref,
-                                          p.w_edge, p.w_color, d_s + (size_t)b0 * g.n_tok);
+                                          p.w_edge, p.w_color, d_s + (size_t)b0 * g.n_tok, skip);
         c->launches += 3;
     }
     SC_CHECK(cudaGetLastError());

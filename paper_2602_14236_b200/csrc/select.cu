@@ -90,6 +90,29 @@ k_select(const float* __restrict__ dP, const float* __restrict__ s, int n_tok, i
         for (int i = s_base[t] + tid; i < n_tok; i += SEL_THREADS) idx[((size_t)b * 3 + t) * n_tok + i] = -1;
 }
 
+// Eq. 6 alone: R = (1/N) sum [dP_i < tau_t], redundant when the frame has a predecessor and R > theta_R.
+// The same arithmetic as k_select, so that both agree on every frame.
+__global__ void __launch_bounds__(SEL_THREADS)
+k_frame_redundancy(const float* __restrict__ dP, int n_tok, int first_has_no_prev, float tau_t, float theta_R,
+                   uint8_t* __restrict__ frame_redundant) {
+    __shared__ int s_red[SEL_THREADS / 32];
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const bool has_prev = dP != nullptr && !(first_has_no_prev && b == 0);
+    int n_static = 0;
+    if (has_prev)
+        for (int i = tid; i < n_tok; i += SEL_THREADS) n_static += (dP[(size_t)b * n_tok + i] < tau_t) ? 1 : 0;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) n_static += __shfl_xor_sync(0xffffffffu, n_static, o);
+    if ((tid & 31) == 0) s_red[tid >> 5] = n_static;
+    __syncthreads();
+    if (tid == 0) {
+        int t = 0;
+        for (int k = 0; k < SEL_THREADS / 32; ++k) t += s_red[k];
+        const float R = has_prev ? __fdiv_rn((float)t, (float)n_tok) : 0.0f;
+        frame_redundant[b] = (has_prev && R > theta_R) ? 1 : 0;
+    }
+}
+
 // Pool row offsets: exclusive scan over the frames of the batch, continuing from the running fill.
 __global__ void k_row_offsets(const int32_t* __restrict__ counts, int B, int64_t* __restrict__ row_offset,
                               int64_t* __restrict__ fill) {
@@ -105,6 +128,16 @@ __global__ void k_row_offsets(const int32_t* __restrict__ counts, int B, int64_t
 }
 
 }  // namespace
+
+int sc_frame_redundancy(salicache_ctx* c, const float* d_deltaP, int B, int first_has_no_prev, uint8_t* d_frame_redundant,
+                        cudaStream_t st) {
+    if (B == 0) return SALICACHE_OK;
+    k_frame_redundancy<<<B, SEL_THREADS, 0, st>>>(d_deltaP, c->n_tok, first_has_no_prev, c->p.tau_t, c->p.theta_R,
+                                                  d_frame_redundant);
+    c->launches++;
+    SC_CHECK(cudaGetLastError());
+    return SALICACHE_OK;
+}
 
 int sc_select(salicache_ctx* c, const float* d_deltaP, const float* d_s, int B, int first_has_no_prev,
               uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts, uint8_t* d_frame_redundant,

@@ -98,6 +98,32 @@ def test_hysteresis_iteration_cap_is_reported_not_hung():
     assert sc.salicache_poll_status(ctx) == 0          # cleared by the poll
 
 
+def test_redundant_frames_skip_the_spatial_branch(wl1_frames, wl1_oracle_scores):
+    """Alg. 1: a frame with R_frame > theta_R is a pointer to its predecessor and is not scored."""
+    import torch
+    ctx = _ctx()
+    rdP, rs, _ = wl1_oracle_scores
+    dP32 = torch.from_numpy(rdP.astype(np.float32)).cuda()
+    red = torch.full((8,), 7, dtype=torch.uint8, device="cuda")
+    sc.salicache_frame_redundancy(ctx, dP32, 8, True, red)
+    p = gu.oracle_params(ctx.params)
+    want = np.array([oracle.select(rdP[t].astype(np.float32), rs[t].astype(np.float32), t > 0, p)[3] for t in range(8)])
+    assert np.array_equal(red.cpu().numpy(), want) and want[0] == 0 and 0 < want.sum() < 8
+    fr = torch.from_numpy(wl1_frames).cuda()
+    s = torch.full((8, 576), -3.0, dtype=torch.float32, device="cuda")
+    sc.salicache_saliency(ctx, fr, 8, s, red)
+    torch.cuda.synchronize()
+    got = s.cpu().numpy()
+    assert (got[want == 1] == -3.0).all()                       # untouched
+    gu.assert_scores_close(got[want == 0], rs[want == 0], "s of the scored frames")
+    # and the decisions do not depend on the rows that were skipped
+    out = gu.gpu_select(ctx, rdP.astype(np.float32), got)
+    dec, idx, counts, r2, _ = gu.oracle_select_all(rdP.astype(np.float32), rs.astype(np.float32), p)
+    near = gu.near_threshold(None, rs.astype(np.float32), p)
+    assert np.array_equal(out["redundant"].cpu().numpy(), want)
+    assert not ((out["decision"].cpu().numpy() != dec) & ~near).any()
+
+
 # ------------------------------------------------------------------------------------- select
 @pytest.mark.parametrize("background", ["int8", "int4", "four"])
 def test_select_is_bit_exact_given_the_same_scores(wl1_oracle_scores, background):
@@ -301,8 +327,9 @@ def test_argument_errors_are_returned_not_raised_on_the_device():
     assert lib.salicache_flow_score(h, None, fr.data_ptr(), 1, dP.data_ptr(), None, None) == sc.E_NULL
     assert lib.salicache_flow_score(h, fr.data_ptr(), fr.data_ptr(), 17, dP.data_ptr(), None, None) == sc.E_SHAPE
     assert lib.salicache_flow_score(h, fr.data_ptr() + 3, fr.data_ptr(), 1, dP.data_ptr(), None, None) == sc.E_ALIGN
-    assert lib.salicache_saliency(h, fr.data_ptr(), -1, dP.data_ptr(), None) == sc.E_SHAPE
-    assert lib.salicache_saliency(h, fr.data_ptr(), 1, None, None) == sc.E_NULL
+    assert lib.salicache_saliency(h, fr.data_ptr(), -1, dP.data_ptr(), None, None) == sc.E_SHAPE
+    assert lib.salicache_saliency(h, fr.data_ptr(), 1, None, None, None) == sc.E_NULL
+    assert lib.salicache_frame_redundancy(h, dP.data_ptr(), 1, 1, None, None) == sc.E_NULL
     pools = sc.PoolSet(1, 4096, 4, 4, 4)
     bad = sc.Pools(None, pools.int8_codes.data_ptr(), pools.int8_scale.data_ptr(), pools.int4_codes.data_ptr(),
                    pools.int4_sz.data_ptr(), 4, 4, 4, 0)
