@@ -165,7 +165,8 @@ def run_ours(args):
     seg = max(ring, (args.segment // ring) * ring)      # frames per pipeline segment: whole K/V ring passes
     segments = [(b0, min(seg, T - b0)) for b0 in range(0, T, seg)]
     main = torch.cuda.current_stream()
-    store_stream = torch.cuda.Stream(device=dev)
+    # one stream by default: the store keeps every SM's registers busy, so a second stream only time-slices
+    store_stream = torch.cuda.Stream(device=dev) if args.overlap else main
 
     def filter_segment(b0: int, nb: int):
         """flow (t-1 -> t), saliency and decisions of frames b0 .. b0+nb-1; the running pool fill carries over."""
@@ -197,16 +198,19 @@ def run_ours(args):
         """One pass of the whole hot path over the workload.  The filter of segment i+1 runs on the main
         stream while the store of segment i runs on the second stream (decisions stay on the device)."""
         timed_events = k >= 0
-        store_stream.wait_stream(main)
+        if args.overlap:
+            store_stream.wait_stream(main)
         for si, (b0, nb) in enumerate(segments):
             if timed_events:
                 ev_f[k][si][0].record(main)
             filter_segment(b0, nb)
             if timed_events:
                 ev_f[k][si][1].record(main)
-            seg_done[si].record(main)
+            if args.overlap:
+                seg_done[si].record(main)
             with torch.cuda.stream(store_stream):
-                store_stream.wait_event(seg_done[si])
+                if args.overlap:
+                    store_stream.wait_event(seg_done[si])
                 for c0 in range(b0, b0 + nb, ring):
                     c = c0 // ring
                     cb = min(ring, b0 + nb - c0)
@@ -216,7 +220,8 @@ def run_ours(args):
                                          stream=store_stream)
                     if timed_events:
                         ev[k][c][1].record(store_stream)
-        main.wait_stream(store_stream)
+        if args.overlap:
+            main.wait_stream(store_stream)
 
     def barrier():
         if world > 1:
@@ -454,9 +459,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=3)
     ap.add_argument("--frames", type=int, default=0, help="use only the first N frames of the workload (profiling)")
-    ap.add_argument("--chunk", type=int, default=40, help="frames per internal pass of flow/saliency")
+    ap.add_argument("--chunk", type=int, default=104, help="frames per internal pass of flow/saliency")
     ap.add_argument("--ring", type=int, default=RING, help="K/V frame slabs resident on the device")
-    ap.add_argument("--segment", type=int, default=40, help="frames per pipeline segment (filter of one overlaps the store of the previous)")
+    ap.add_argument("--segment", type=int, default=104, help="frames per pipeline segment (filter of one overlaps the store of the previous)")
+    ap.add_argument("--overlap", action="store_true", help="store of segment i on a second stream beside the filter of segment i+1")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=1)

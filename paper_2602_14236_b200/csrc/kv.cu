@@ -71,6 +71,24 @@ __device__ __forceinline__ uint32_t pack_u4(int a, int b, uint32_t c) {
     return d;
 }
 
+// Both halves of a word minus z, in binary32: the mixed-precision subtract converts the binary16 operand
+// exactly and rounds once, so it equals convert-then-subtract.
+__device__ __forceinline__ float2 sub_h2_f32(uint32_t w, float z) {
+    float2 r;
+    asm("{ .reg .b16 lo, hi; mov.b32 {lo, hi}, %2; sub.rn.f32.f16 %0, lo, %3; sub.rn.f32.f16 %1, hi, %3; }"
+        : "=f"(r.x), "=f"(r.y)
+        : "r"(w), "f"(z));
+    return r;
+}
+// rint(d * inv) clamped to at most 15: multiply and round to nearest even as separate operations.
+__device__ __forceinline__ int quant4(float d, float inv) { return __float2int_rn(fminf(__fmul_rn(d, inv), 15.0f)); }
+// Bytes (q0 q1 q2 q3), (q4 q5 q6 q7), each 0..15 -> nibbles q0 | q1 << 4 | ... | q7 << 28.
+__device__ __forceinline__ uint32_t nibbles(uint32_t lo, uint32_t hi) {
+    lo |= lo >> 4;
+    hi |= hi >> 4;
+    return __byte_perm(lo, hi, 0x6420);
+}
+
 // Rows stored before each frame of the batch, built by every CTA in shared memory from the counts.
 __device__ __forceinline__ void build_prefix(const int32_t* __restrict__ counts, int B, int* pre) {
     __shared__ int wsum[KV_WARPS];
@@ -232,13 +250,11 @@ k_pack(const __half* __restrict__ K, const __half* __restrict__ V, KvGeom g, con
                 const int owner = 2 * i + (lane >> 4);
                 const float inv = __shfl_sync(0xffffffffu, my_inv, owner);
                 const float z = __shfl_sync(0xffffffffu, my_z, owner);
-                float2 f0 = __half22float2(as_h2(v[i].x)), f1 = __half22float2(as_h2(v[i].y));
-                float2 f2 = __half22float2(as_h2(v[i].z)), f3 = __half22float2(as_h2(v[i].w));
-                int q0 = __float2int_rn(__fmul_rn(__fsub_rn(f0.x, z), inv)), q1 = __float2int_rn(__fmul_rn(__fsub_rn(f0.y, z), inv));
-                int q2 = __float2int_rn(__fmul_rn(__fsub_rn(f1.x, z), inv)), q3 = __float2int_rn(__fmul_rn(__fsub_rn(f1.y, z), inv));
-                int q4 = __float2int_rn(__fmul_rn(__fsub_rn(f2.x, z), inv)), q5 = __float2int_rn(__fmul_rn(__fsub_rn(f2.y, z), inv));
-                int q6 = __float2int_rn(__fmul_rn(__fsub_rn(f3.x, z), inv)), q7 = __float2int_rn(__fmul_rn(__fsub_rn(f3.y, z), inv));
-                st_stream(dst + i * 32, pack_u4(q1, q0, pack_u4(q3, q2, pack_u4(q5, q4, pack_u4(q7, q6, 0)))));
+                const float2 f0 = sub_h2_f32(v[i].x, z), f1 = sub_h2_f32(v[i].y, z), f2 = sub_h2_f32(v[i].z, z), f3 = sub_h2_f32(v[i].w, z);
+                // x >= zero, so the product is >= 0; the upper clamp matters only for tiny ranges whose scale rounded down
+                int q0 = quant4(f0.x, inv), q1 = quant4(f0.y, inv), q2 = quant4(f1.x, inv), q3 = quant4(f1.y, inv);
+                int q4 = quant4(f2.x, inv), q5 = quant4(f2.y, inv), q6 = quant4(f3.x, inv), q7 = quant4(f3.y, inv);
+                st_stream(dst + i * 32, nibbles(pack_s8(q1, q0, pack_s8(q3, q2, 0)), pack_s8(q5, q4, pack_s8(q7, q6, 0))));
             }
         }
     }

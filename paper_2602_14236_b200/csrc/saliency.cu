@@ -164,14 +164,18 @@ k_hysteresis(const uint32_t* __restrict__ bits_kept, uint32_t* __restrict__ bits
     for (int i = threadIdx.x; i < n; i += blockDim.x) ge[i] = E[i];
 }
 
-// ---- sRGB -> CIE L*a*b* (D65) in double; cube root = float seed + one Newton step in double.
+// ---- sRGB -> CIE L*a*b* (D65) in double.  Cube root: a hardware log2 / exp2 seed in single precision
+// (relative error below 1e-6) and one Newton step in double, y - (y^3 - t) / (3 y^2); the divisor only
+// scales a 1e-6 correction, so its single-precision reciprocal is enough and the result is good to ~1e-12.
 __device__ __forceinline__ double lab_f(double t) {
     const double d = 6.0 / 29.0;
-    if (t > d * d * d) {
-        double y = (double)cbrtf((float)t);          // relative error ~1e-7; one Newton step squares it
-        return y - (y * y * y - t) / (3.0 * y * y);
-    }
-    return t / (3.0 * d * d) + 4.0 / 29.0;
+    const float tf = fmaxf((float)t, 1e-6f);
+    const float y0 = exp2f(__log2f(tf) * (1.0f / 3.0f));
+    const float r = __frcp_rn(3.0f * y0 * y0);
+    const double y = (double)y0;
+    const double cube = y - (y * y * y - t) * (double)r;
+    const double lin = t * (1.0 / (3.0 * d * d)) + 4.0 / 29.0;
+    return t > d * d * d ? cube : lin;
 }
 __device__ __forceinline__ void rgb_to_lab(const double* __restrict__ lut, int R, int G, int B, double& L, double& a,
                                            double& b) {
@@ -179,7 +183,7 @@ __device__ __forceinline__ void rgb_to_lab(const double* __restrict__ lut, int R
     double X = 0.4124564 * r + 0.3575761 * g + 0.1804375 * bl;
     double Y = 0.2126729 * r + 0.7151522 * g + 0.0721750 * bl;
     double Z = 0.0193339 * r + 0.1191920 * g + 0.9503041 * bl;
-    double fx = lab_f(X / 0.95047), fy = lab_f(Y), fz = lab_f(Z / 1.08883);
+    double fx = lab_f(X * (1.0 / 0.95047)), fy = lab_f(Y), fz = lab_f(Z * (1.0 / 1.08883));
     L = 116.0 * fy - 16.0;
     a = 500.0 * (fx - fy);
     b = 200.0 * (fy - fz);
@@ -187,23 +191,48 @@ __device__ __forceinline__ void rgb_to_lab(const double* __restrict__ lut, int R
 
 // ---- colour branch + blend + patch mean.  One CTA per 2x2 patches (28x28 pixels), halo 3.
 // Variances are taken about the LAB value of the tile's first pixel (variance is shift invariant),
-// which keeps flat regions exactly zero and small contrasts accurate.
+// which keeps flat regions exactly zero and small contrasts accurate; the sums of x and x^2 stay in
+// double because mean(x^2) - mean(x)^2 cancels.
+//   phase 1  LAB of the 34x34 grown tile -> shared memory
+//   phase 2  one thread per (channel, row, run of 4 columns): 7-column sums of x and x^2
+//   phase 3  one thread per (column, run of 4 rows): 7-row sums, variance, C, blend with the edge bit,
+//            patch partial sums
+// Window sums of a run share their terms: the middle four once, then suffix sums to the left and prefix
+// sums to the right (11 additions for 4 windows).
 constexpr int ST = 28;
 constexpr int SR = 3;
 constexpr int SE = ST + 2 * SR;   // 34
+constexpr int SLP = SE + 2;       // lab row pitch (even: 16-byte loads of column pairs)
+constexpr int CRUN = 4;
+constexpr int CNQ = 2 * SR + CRUN;   // 10 values feed 4 windows
+
+// w[k] = q[k] + ... + q[k+6], k = 0..3
+__device__ __forceinline__ void window4(const double q[CNQ], double w[CRUN]) {
+    double mid = (q[3] + q[4]) + (q[5] + q[6]);
+    double s2 = q[2] + mid, s1 = q[1] + s2, s0 = q[0] + s1;
+    double p8 = q[7] + q[8], p9 = p8 + q[9];
+    w[0] = s0;
+    w[1] = s1 + q[7];
+    w[2] = s2 + p8;
+    w[3] = mid + p9;
+}
 
 __global__ void __launch_bounds__(256)
 k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom g, int patch,
               const double* __restrict__ lut, const uint32_t* __restrict__ bits_edge, int words, double inv_sigma,
               double w_edge, double w_color, float* __restrict__ s_out, const uint8_t* __restrict__ skip) {
-    extern __shared__ double cs[];
-    double (*lab)[SE][SE + 1] = reinterpret_cast<double (*)[SE][SE + 1]>(cs);                    // [3]
-    double (*hs)[SE][ST] = reinterpret_cast<double (*)[SE][ST]>(cs + 3 * SE * (SE + 1));          // [6]
+    extern __shared__ __align__(16) double cs[];
+    double (*lab)[SE][SLP] = reinterpret_cast<double (*)[SE][SLP]>(cs);                              // [3]
+    double2 (*hs)[SE][ST] = reinterpret_cast<double2 (*)[SE][ST]>(cs + 3 * SE * SLP);                 // [3] (sum x, sum x^2)
     __shared__ double psum[8][4];
+    __shared__ double slut[256];
     const int f = blockIdx.z, x0 = blockIdx.x * ST, y0 = blockIdx.y * ST;
     if (skip && skip[f]) return;
     const int h = g.H, w = g.W;
     const uint8_t* fr = frames + (size_t)f * frame_bytes;
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) slut[i] = lut[i];
+    __syncthreads();
+    lut = slut;
     double L0, a0, b0;
     {
         const uint8_t* p = fr + ((size_t)y0 * w + x0) * 3;
@@ -219,47 +248,65 @@ k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom 
         lab[2][ry][rx] = b - b0;
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < 3 * SE * ST; i += blockDim.x) {
-        int c = i / (SE * ST), r = i % (SE * ST);
-        int ry = r / ST, ox = r % ST;
-        double s1 = 0.0, s2 = 0.0;
+    for (int i = threadIdx.x; i < 3 * SE * (ST / CRUN); i += blockDim.x) {
+        const int run = i % (ST / CRUN), r = i / (ST / CRUN);
+        const int ry = r % SE, c = r / SE;
+        const int ox = CRUN * run;                         // windows ox .. ox+3 read columns ox .. ox+9 of the grown tile
+        const double2* src = reinterpret_cast<const double2*>(&lab[c][ry][ox]);
+        double q[CNQ], q2[CNQ];
 #pragma unroll
-        for (int k = 0; k < 2 * SR + 1; ++k) {
-            double v = lab[c][ry][ox + k];
-            s1 += v;
-            s2 += v * v;
+        for (int k = 0; k < CNQ / 2; ++k) {
+            double2 v = src[k];
+            q[2 * k] = v.x;
+            q[2 * k + 1] = v.y;
         }
-        hs[c][ry][ox] = s1;
-        hs[3 + c][ry][ox] = s2;
+#pragma unroll
+        for (int k = 0; k < CNQ; ++k) q2[k] = q[k] * q[k];
+        double w1[CRUN], w2[CRUN];
+        window4(q, w1);
+        window4(q2, w2);
+#pragma unroll
+        for (int k = 0; k < CRUN; ++k) hs[c][ry][ox + k] = make_double2(w1[k], w2[k]);
     }
     __syncthreads();
     const double inv_n = 1.0 / (double)((2 * SR + 1) * (2 * SR + 1));
     double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;   // the four patches of the tile
-    for (int i = threadIdx.x; i < ST * ST; i += blockDim.x) {
-        int oy = i / ST, ox = i % ST;
-        double V = 0.0;
+    if (threadIdx.x < ST * (ST / CRUN)) {
+        const int ox = threadIdx.x % ST, oy0 = CRUN * (threadIdx.x / ST);
+        double V[CRUN] = {0.0, 0.0, 0.0, 0.0};
 #pragma unroll
         for (int c = 0; c < 3; ++c) {
-            double s1 = 0.0, s2 = 0.0;
+            double q[CNQ], q2[CNQ];
 #pragma unroll
-            for (int k = 0; k < 2 * SR + 1; ++k) {
-                s1 += hs[c][oy + k][ox];
-                s2 += hs[3 + c][oy + k][ox];
+            for (int k = 0; k < CNQ; ++k) {
+                double2 v = hs[c][oy0 + k][ox];
+                q[k] = v.x;
+                q2[k] = v.y;
             }
-            double mean = s1 * inv_n;
-            V += s2 * inv_n - mean * mean;
+            double w1[CRUN], w2[CRUN];
+            window4(q, w1);
+            window4(q2, w2);
+#pragma unroll
+            for (int k = 0; k < CRUN; ++k) {
+                double mean = w1[k] * inv_n;
+                V[k] += w2[k] * inv_n - mean * mean;
+            }
         }
-        double C = sqrt(fmax(V, 0.0)) * inv_sigma;
-        C = fmin(C, 1.0);
-        int y = y0 + oy, x = x0 + ox;
-        uint32_t e = (bits_edge[((size_t)f * h + y) * words + (x >> 5)] >> (x & 31)) & 1u;
-        double S = w_edge * (double)e + w_color * C;
-        S = fmin(fmax(S, 0.0), 1.0);
-        bool lower = oy >= patch, right = ox >= patch;
-        acc0 += (!lower && !right) ? S : 0.0;
-        acc1 += (!lower && right) ? S : 0.0;
-        acc2 += (lower && !right) ? S : 0.0;
-        acc3 += (lower && right) ? S : 0.0;
+        const int x = x0 + ox;
+#pragma unroll
+        for (int k = 0; k < CRUN; ++k) {
+            const int oy = oy0 + k, y = y0 + oy;
+            double C = sqrt(fmax(V[k], 0.0)) * inv_sigma;
+            C = fmin(C, 1.0);
+            uint32_t e = (bits_edge[((size_t)f * h + y) * words + (x >> 5)] >> (x & 31)) & 1u;
+            double S = w_edge * (double)e + w_color * C;
+            S = fmin(fmax(S, 0.0), 1.0);
+            bool lower = oy >= patch, right = ox >= patch;
+            acc0 += (!lower && !right) ? S : 0.0;
+            acc1 += (!lower && right) ? S : 0.0;
+            acc2 += (lower && !right) ? S : 0.0;
+            acc3 += (lower && right) ? S : 0.0;
+        }
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) {
@@ -285,7 +332,7 @@ inline unsigned blocks_for(long long n, int threads) { return (unsigned)((n + th
 
 }  // namespace
 
-static size_t color_smem() { return (size_t)(3 * SE * (SE + 1) + 6 * SE * ST) * sizeof(double); }
+static size_t color_smem() { return (size_t)(3 * SE * SLP + 2 * 3 * SE * ST) * sizeof(double); }
 
 int sc_saliency_init(int max_h, int max_words) {
     SC_CHECK(cudaFuncSetAttribute(k_color_patch, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)color_smem()));
