@@ -154,7 +154,104 @@ __device__ __forceinline__ Unit decode_unit(long long u, const int* pre, int B, 
 }
 
 // ---- pack ---------------------------------------------------------------------------------------
-// ITERS = HD / 256: 16-byte loads per lane per row; groups per row = 2 * ITERS (<= 32, one per lane).
+// One row (or piece `part` of a row): ITERS 16-byte words per lane = 256 * ITERS elements = 2 * ITERS
+// quantisation groups (<= 32, one per lane).
+template <int ITERS>
+__device__ __forceinline__ void pack_piece(const uint4 (&v)[ITERS], const Unit& un, int part, const KvGeom& g,
+                                           const PoolPtrs& pp, int lane) {
+    const int src_lane = (lane & 1) << 4;                  // a lane of the half warp that reduced my group
+    const size_t prow = (size_t)un.plane * un.cap + un.row;
+    if (un.tier == 0) {
+        uint4* dst = reinterpret_cast<uint4*>(pp.fp16_pool + prow * (size_t)g.HD * 2) + part * (ITERS * 32) + lane;
+#pragma unroll
+        for (int i = 0; i < ITERS; ++i) st_stream(dst + i * 32, v[i]);
+    } else if (un.tier == 1) {
+        // INT8 symmetric: s = fp16(max|x| / 127), q = rint(x * (1/s)) clamped to [-127, 127]
+        uint32_t mine = 0;
+#pragma unroll
+        for (int i = 0; i < ITERS; ++i) {
+            __half2 m = __hmax2(__hmax2(__habs2(as_h2(v[i].x)), __habs2(as_h2(v[i].y))),
+                                __hmax2(__habs2(as_h2(v[i].z)), __habs2(as_h2(v[i].w))));
+#pragma unroll
+            for (int o = 8; o; o >>= 1) m = __hmax2(m, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(m), o)));
+            uint32_t sv = __shfl_sync(0xffffffffu, as_u32(m), src_lane);
+            if ((lane >> 1) == i) mine = sv;             // lane l owns group l = 2i + (l & 1)
+        }
+        float amax = fmaxf(__low2float(as_h2(mine)), __high2float(as_h2(mine)));
+        __half s16 = __float2half_rn(__fdiv_rn(amax, 127.0f));
+        if ((__half_as_ushort(s16) & 0x7fff) == 0) s16 = __ushort_as_half(0x3c00);
+        const float my_inv = __fdiv_rn(1.0f, __half2float(s16));
+        if (lane < 2 * ITERS)
+            reinterpret_cast<uint16_t*>(pp.int8_scale + prow * (size_t)g.ng * 2)[part * 2 * ITERS + lane] = __half_as_ushort(s16);
+        uint2* dst = reinterpret_cast<uint2*>(pp.int8_codes + prow * (size_t)g.HD) + part * (ITERS * 32) + lane;
+#pragma unroll
+        for (int i = 0; i < ITERS; ++i) {
+            const float inv = __shfl_sync(0xffffffffu, my_inv, 2 * i + (lane >> 4));
+            float2 f0 = __half22float2(as_h2(v[i].x)), f1 = __half22float2(as_h2(v[i].y));
+            float2 f2 = __half22float2(as_h2(v[i].z)), f3 = __half22float2(as_h2(v[i].w));
+            int q0 = __float2int_rn(__fmul_rn(f0.x, inv)), q1 = __float2int_rn(__fmul_rn(f0.y, inv));
+            int q2 = __float2int_rn(__fmul_rn(f1.x, inv)), q3 = __float2int_rn(__fmul_rn(f1.y, inv));
+            int q4 = __float2int_rn(__fmul_rn(f2.x, inv)), q5 = __float2int_rn(__fmul_rn(f2.y, inv));
+            int q6 = __float2int_rn(__fmul_rn(f3.x, inv)), q7 = __float2int_rn(__fmul_rn(f3.y, inv));
+            uint2 o;
+            o.x = __vmaxs4(pack_s8(q1, q0, pack_s8(q3, q2, 0)), 0x81818181u);
+            o.y = __vmaxs4(pack_s8(q5, q4, pack_s8(q7, q6, 0)), 0x81818181u);
+            st_stream(dst + i * 32, o);
+        }
+    } else {
+        // INT4 asymmetric: zero = min, s = fp16((max - min) / 15), q = rint((x - zero) * (1/s)) in [0, 15].
+        // One half2 carries (max, -min) so a single max-reduction serves both.
+        uint32_t mine = 0;
+#pragma unroll
+        for (int i = 0; i < ITERS; ++i) {
+            __half2 a = as_h2(v[i].x), b = as_h2(v[i].y), c = as_h2(v[i].z), d = as_h2(v[i].w);
+            __half2 mx = __hmax2(__hmax2(a, b), __hmax2(c, d));
+            __half2 nmn = __hneg2(__hmin2(__hmin2(a, b), __hmin2(c, d)));
+            __half2 m = __hmax2(as_h2(__byte_perm(as_u32(mx), as_u32(nmn), 0x5410)),
+                                as_h2(__byte_perm(as_u32(mx), as_u32(nmn), 0x7632)));   // (max, -min)
+#pragma unroll
+            for (int o = 8; o; o >>= 1) m = __hmax2(m, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(m), o)));
+            uint32_t sv = __shfl_sync(0xffffffffu, as_u32(m), src_lane);
+            if ((lane >> 1) == i) mine = sv;
+        }
+        const float fmx = __low2float(as_h2(mine));
+        float fmn = -__high2float(as_h2(mine));
+        __half z16 = __float2half_rn(fmn);                       // exact: fmn is an fp16 value
+        if (fmn == 0.0f) z16 = __ushort_as_half(0);              // a zero minimum is stored as +0
+        __half s16 = __float2half_rn(__fdiv_rn(__fsub_rn(fmx, fmn), 15.0f));
+        if ((__half_as_ushort(s16) & 0x7fff) == 0) s16 = __ushort_as_half(0x3c00);
+        const float my_inv = __fdiv_rn(1.0f, __half2float(s16));
+        const float my_z = __half2float(z16);
+        if (lane < 2 * ITERS)
+            reinterpret_cast<uint32_t*>(pp.int4_sz + prow * (size_t)g.ng * 4)[part * 2 * ITERS + lane] =
+                (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(z16) << 16);
+        uint32_t* dst = reinterpret_cast<uint32_t*>(pp.int4_codes + prow * (size_t)(g.HD / 2)) + part * (ITERS * 32) + lane;
+#pragma unroll
+        for (int i = 0; i < ITERS; ++i) {
+            const int owner = 2 * i + (lane >> 4);
+            const float inv = __shfl_sync(0xffffffffu, my_inv, owner);
+            const float z = __shfl_sync(0xffffffffu, my_z, owner);
+            const float2 f0 = sub_h2_f32(v[i].x, z), f1 = sub_h2_f32(v[i].y, z), f2 = sub_h2_f32(v[i].z, z), f3 = sub_h2_f32(v[i].w, z);
+            // x >= zero, so the product is >= 0; the upper clamp matters only for tiny ranges whose scale rounded down
+            int q0 = quant4(f0.x, inv), q1 = quant4(f0.y, inv), q2 = quant4(f1.x, inv), q3 = quant4(f1.y, inv);
+            int q4 = quant4(f2.x, inv), q5 = quant4(f2.y, inv), q6 = quant4(f3.x, inv), q7 = quant4(f3.y, inv);
+            st_stream(dst + i * 32, nibbles(pack_s8(q1, q0, pack_s8(q3, q2, 0)), pack_s8(q5, q4, pack_s8(q7, q6, 0))));
+        }
+    }
+}
+
+template <int ITERS>
+__device__ __forceinline__ void load_piece(uint4 (&v)[ITERS], const __half* K, const __half* V, const Unit& un, int part,
+                                           const KvGeom& g, int lane) {
+    const int layer = un.plane >> 1, kv = un.plane & 1;
+    const __half* src_h = (kv ? V : K) + (size_t)un.b * g.frame_stride + ((size_t)layer * g.n_tok + un.tok) * g.HD;
+    const uint4* src = reinterpret_cast<const uint4*>(src_h) + part * (ITERS * 32) + lane;
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) v[i] = ld_stream(src + i * 32);
+}
+
+// One warp per stored row: all 16-byte loads of the row are issued before any arithmetic, and the next
+// row's lookups (index list, row offset) run while they are in flight.
 template <int ITERS>
 __global__ void __launch_bounds__(KV_THREADS, 2)
 k_pack(const __half* __restrict__ K, const __half* __restrict__ V, KvGeom g, const int32_t* __restrict__ idx,
@@ -165,98 +262,20 @@ k_pack(const __half* __restrict__ K, const __half* __restrict__ V, KvGeom g, con
     const int planes = 2 * g.L;
     const long long n_units = (long long)pre[g.B] * planes;
     const int lane = threadIdx.x & 31;
-    const int src_lane = (lane & 1) << 4;                  // a lane of the half warp that reduced my group
     const long long warp0 = (long long)blockIdx.x * KV_WARPS + (threadIdx.x >> 5);
     const long long wstride = (long long)gridDim.x * KV_WARPS;
+    if (warp0 >= n_units) return;
+    Unit un = decode_unit(warp0, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp);
+    uint4 v[ITERS];
+    if (un.row >= 0) load_piece<ITERS>(v, K, V, un, 0, g, lane);
     for (long long u = warp0; u < n_units; u += wstride) {
-        Unit un = decode_unit(u, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp);
-        if (un.row < 0) {
-            if (lane == 0) atomicMin(status, SALICACHE_E_CAPACITY);
-            continue;
-        }
-        const int layer = un.plane >> 1, kv = un.plane & 1;
-        const __half* src_h = (kv ? V : K) + (size_t)un.b * g.frame_stride + ((size_t)layer * g.n_tok + un.tok) * g.HD;
-        const uint4* src = reinterpret_cast<const uint4*>(src_h) + lane;
-        uint4 v[ITERS];
-#pragma unroll
-        for (int i = 0; i < ITERS; ++i) v[i] = ld_stream(src + i * 32);
-        const size_t prow = (size_t)un.plane * un.cap + un.row;
-        if (un.tier == 0) {
-            uint4* dst = reinterpret_cast<uint4*>(pp.fp16_pool + prow * (size_t)g.HD * 2) + lane;
-#pragma unroll
-            for (int i = 0; i < ITERS; ++i) st_stream(dst + i * 32, v[i]);
-        } else if (un.tier == 1) {
-            // INT8 symmetric: s = fp16(max|x| / 127), q = rint(x * (1/s)) clamped to [-127, 127]
-            uint32_t mine = 0;
-#pragma unroll
-            for (int i = 0; i < ITERS; ++i) {
-                __half2 m = __hmax2(__hmax2(__habs2(as_h2(v[i].x)), __habs2(as_h2(v[i].y))),
-                                    __hmax2(__habs2(as_h2(v[i].z)), __habs2(as_h2(v[i].w))));
-#pragma unroll
-                for (int o = 8; o; o >>= 1) m = __hmax2(m, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(m), o)));
-                uint32_t sv = __shfl_sync(0xffffffffu, as_u32(m), src_lane);
-                if ((lane >> 1) == i) mine = sv;             // lane l owns group l = 2i + (l & 1)
-            }
-            float amax = fmaxf(__low2float(as_h2(mine)), __high2float(as_h2(mine)));
-            __half s16 = __float2half_rn(__fdiv_rn(amax, 127.0f));
-            if ((__half_as_ushort(s16) & 0x7fff) == 0) s16 = __ushort_as_half(0x3c00);
-            const float my_inv = __fdiv_rn(1.0f, __half2float(s16));
-            if (lane < g.ng) reinterpret_cast<uint16_t*>(pp.int8_scale + prow * (size_t)g.ng * 2)[lane] = __half_as_ushort(s16);
-            uint2* dst = reinterpret_cast<uint2*>(pp.int8_codes + prow * (size_t)g.HD) + lane;
-#pragma unroll
-            for (int i = 0; i < ITERS; ++i) {
-                const float inv = __shfl_sync(0xffffffffu, my_inv, 2 * i + (lane >> 4));
-                float2 f0 = __half22float2(as_h2(v[i].x)), f1 = __half22float2(as_h2(v[i].y));
-                float2 f2 = __half22float2(as_h2(v[i].z)), f3 = __half22float2(as_h2(v[i].w));
-                int q0 = __float2int_rn(__fmul_rn(f0.x, inv)), q1 = __float2int_rn(__fmul_rn(f0.y, inv));
-                int q2 = __float2int_rn(__fmul_rn(f1.x, inv)), q3 = __float2int_rn(__fmul_rn(f1.y, inv));
-                int q4 = __float2int_rn(__fmul_rn(f2.x, inv)), q5 = __float2int_rn(__fmul_rn(f2.y, inv));
-                int q6 = __float2int_rn(__fmul_rn(f3.x, inv)), q7 = __float2int_rn(__fmul_rn(f3.y, inv));
-                uint2 o;
-                o.x = __vmaxs4(pack_s8(q1, q0, pack_s8(q3, q2, 0)), 0x81818181u);
-                o.y = __vmaxs4(pack_s8(q5, q4, pack_s8(q7, q6, 0)), 0x81818181u);
-                st_stream(dst + i * 32, o);
-            }
-        } else {
-            // INT4 asymmetric: zero = min, s = fp16((max - min) / 15), q = rint((x - zero) * (1/s)) in [0, 15].
-            // One half2 carries (max, -min) so a single max-reduction serves both.
-            uint32_t mine = 0;
-#pragma unroll
-            for (int i = 0; i < ITERS; ++i) {
-                __half2 a = as_h2(v[i].x), b = as_h2(v[i].y), c = as_h2(v[i].z), d = as_h2(v[i].w);
-                __half2 mx = __hmax2(__hmax2(a, b), __hmax2(c, d));
-                __half2 nmn = __hneg2(__hmin2(__hmin2(a, b), __hmin2(c, d)));
-                __half2 m = __hmax2(as_h2(__byte_perm(as_u32(mx), as_u32(nmn), 0x5410)),
-                                    as_h2(__byte_perm(as_u32(mx), as_u32(nmn), 0x7632)));   // (max, -min)
-#pragma unroll
-                for (int o = 8; o; o >>= 1) m = __hmax2(m, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(m), o)));
-                uint32_t sv = __shfl_sync(0xffffffffu, as_u32(m), src_lane);
-                if ((lane >> 1) == i) mine = sv;
-            }
-            const float fmx = __low2float(as_h2(mine));
-            float fmn = -__high2float(as_h2(mine));
-            __half z16 = __float2half_rn(fmn);                       // exact: fmn is an fp16 value
-            if (fmn == 0.0f) z16 = __ushort_as_half(0);              // a zero minimum is stored as +0
-            __half s16 = __float2half_rn(__fdiv_rn(__fsub_rn(fmx, fmn), 15.0f));
-            if ((__half_as_ushort(s16) & 0x7fff) == 0) s16 = __ushort_as_half(0x3c00);
-            const float my_inv = __fdiv_rn(1.0f, __half2float(s16));
-            const float my_z = __half2float(z16);
-            if (lane < g.ng)
-                reinterpret_cast<uint32_t*>(pp.int4_sz + prow * (size_t)g.ng * 4)[lane] =
-                    (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(z16) << 16);
-            uint32_t* dst = reinterpret_cast<uint32_t*>(pp.int4_codes + prow * (size_t)(g.HD / 2)) + lane;
-#pragma unroll
-            for (int i = 0; i < ITERS; ++i) {
-                const int owner = 2 * i + (lane >> 4);
-                const float inv = __shfl_sync(0xffffffffu, my_inv, owner);
-                const float z = __shfl_sync(0xffffffffu, my_z, owner);
-                const float2 f0 = sub_h2_f32(v[i].x, z), f1 = sub_h2_f32(v[i].y, z), f2 = sub_h2_f32(v[i].z, z), f3 = sub_h2_f32(v[i].w, z);
-                // x >= zero, so the product is >= 0; the upper clamp matters only for tiny ranges whose scale rounded down
-                int q0 = quant4(f0.x, inv), q1 = quant4(f0.y, inv), q2 = quant4(f1.x, inv), q3 = quant4(f1.y, inv);
-                int q4 = quant4(f2.x, inv), q5 = quant4(f2.y, inv), q6 = quant4(f3.x, inv), q7 = quant4(f3.y, inv);
-                st_stream(dst + i * 32, nibbles(pack_s8(q1, q0, pack_s8(q3, q2, 0)), pack_s8(q5, q4, pack_s8(q7, q6, 0))));
-            }
-        }
+        const bool more = u + wstride < n_units;
+        Unit nxt = un;
+        if (more) nxt = decode_unit(u + wstride, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp);
+        if (un.row >= 0) pack_piece<ITERS>(v, un, 0, g, pp, lane);
+        else if (lane == 0) atomicMin(status, SALICACHE_E_CAPACITY);
+        if (more && nxt.row >= 0) load_piece<ITERS>(v, K, V, nxt, 0, g, lane);
+        un = nxt;
     }
 }
 
