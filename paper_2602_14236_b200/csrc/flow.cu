@@ -71,44 +71,81 @@ struct PolyW {
 };
 
 // ---- polynomial expansion, 5x5: planes r2 r3 r4 r5 r6 (b_x, b_y, A_xx, A_yy, 2 A_xy), stored as float.
-__global__ void k_poly_exp(const float* __restrict__ img, int h, int w, int n_frames, PolyW pw,
-                           float* __restrict__ coef) {
-    long long gid = blockIdx.x * (long long)blockDim.x + threadIdx.x;
-    size_t P = (size_t)h * w;
-    if (gid >= (long long)P * n_frames) return;
-    int f = (int)(gid / P);
-    int r = (int)(gid % P);
-    int y = r / w, x = r % w;
+// Separable, in double: a 32x32 tile grown by 2 is staged in shared memory, each grown row gets its three
+// horizontal moment sums (weights g, g*b, g*b^2), and each thread then walks down a column of 8 pixels
+// with the five rows of sums it needs in registers.
+constexpr int PX = 32, PY = 32, PH = 2;          // tile and halo
+constexpr int PEW = PX + 2 * PH, PEH = PY + 2 * PH;
+constexpr int PRUN = 8;                          // pixels per thread in the vertical pass
+
+__global__ void __launch_bounds__(256)
+k_poly_exp(const float* __restrict__ img, int h, int w, int n_frames, PolyW pw, float* __restrict__ coef) {
+    __shared__ double tile[PEH][PEW + 1];
+    __shared__ double hm[3][PEH][PX];
+    const int f = blockIdx.z, x0 = blockIdx.x * PX, y0 = blockIdx.y * PY;
+    const size_t P = (size_t)h * w;
     const float* s = img + (size_t)f * P;
-    int xs[5];
-#pragma unroll
-    for (int b = 0; b < 5; ++b) xs[b] = clampi(x + b - 2, 0, w - 1);
-    double m00 = 0, m10 = 0, m01 = 0, m20 = 0, m02 = 0, m11 = 0;
-#pragma unroll
-    for (int a = -2; a <= 2; ++a) {
-        const float* row = s + (size_t)clampi(y + a, 0, h - 1) * w;
+    for (int i = threadIdx.x; i < PEH * PEW; i += blockDim.x) {
+        const int ry = i / PEW, rx = i - ry * PEW;
+        tile[ry][rx] = (double)s[(size_t)clampi(y0 - PH + ry, 0, h - 1) * w + clampi(x0 - PH + rx, 0, w - 1)];
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < PEH * PX; i += blockDim.x) {
+        const int ry = i / PX, ox = i - ry * PX;
         double s0 = 0, s1 = 0, s2 = 0;
 #pragma unroll
         for (int b = -2; b <= 2; ++b) {
-            double v = pw.g[b + 2] * (double)row[xs[b + 2]];
+            const double v = pw.g[b + 2] * tile[ry][ox + PH + b];
             s0 += v;
             s1 += v * b;
             s2 += v * (b * b);
         }
-        double ga = pw.g[a + 2];
-        m00 += ga * s0;
-        m10 += ga * s1;
-        m20 += ga * s2;
-        m01 += ga * a * s0;
-        m11 += ga * a * s1;
-        m02 += ga * (a * a) * s0;
+        hm[0][ry][ox] = s0;
+        hm[1][ry][ox] = s1;
+        hm[2][ry][ox] = s2;
     }
-    float* c = coef + (size_t)f * 5 * P + r;
-    c[0 * P] = (float)(m10 * pw.inv_mu2);
-    c[1 * P] = (float)(m01 * pw.inv_mu2);
-    c[2 * P] = (float)((m20 - pw.mu2 * m00) * pw.inv_den);
-    c[3 * P] = (float)((m02 - pw.mu2 * m00) * pw.inv_den);
-    c[4 * P] = (float)(m11 * pw.inv_mu2sq);
+    __syncthreads();
+    if (threadIdx.x < PX * (PY / PRUN)) {
+        const int ox = threadIdx.x % PX, oy0 = PRUN * (threadIdx.x / PX);
+        const int x = x0 + ox;
+        if (x < w) {
+            double r0[5], r1[5], r2[5];              // sliding five rows of the three sums
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                r0[k + 1] = hm[0][oy0 + k][ox];
+                r1[k + 1] = hm[1][oy0 + k][ox];
+                r2[k + 1] = hm[2][oy0 + k][ox];
+            }
+#pragma unroll
+            for (int k = 0; k < PRUN; ++k) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { r0[j] = r0[j + 1]; r1[j] = r1[j + 1]; r2[j] = r2[j + 1]; }
+                r0[4] = hm[0][oy0 + k + 4][ox];
+                r1[4] = hm[1][oy0 + k + 4][ox];
+                r2[4] = hm[2][oy0 + k + 4][ox];
+                double m00 = 0, m10 = 0, m01 = 0, m20 = 0, m02 = 0, m11 = 0;
+#pragma unroll
+                for (int a = -2; a <= 2; ++a) {
+                    const double ga = pw.g[a + 2];
+                    m00 += ga * r0[a + 2];
+                    m10 += ga * r1[a + 2];
+                    m20 += ga * r2[a + 2];
+                    m01 += ga * a * r0[a + 2];
+                    m11 += ga * a * r1[a + 2];
+                    m02 += ga * (a * a) * r0[a + 2];
+                }
+                const int y = y0 + oy0 + k;
+                if (y < h) {
+                    float* c = coef + (size_t)f * 5 * P + (size_t)y * w + x;
+                    c[0 * P] = (float)(m10 * pw.inv_mu2);
+                    c[1 * P] = (float)(m01 * pw.inv_mu2);
+                    c[2 * P] = (float)((m20 - pw.mu2 * m00) * pw.inv_den);
+                    c[3 * P] = (float)((m02 - pw.mu2 * m00) * pw.inv_den);
+                    c[4 * P] = (float)(m11 * pw.inv_mu2sq);
+                }
+            }
+        }
+    }
 }
 
 // Bilinear corner set of a clamped continuous position.
@@ -444,9 +481,10 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
         for (int l = 1; l < 3; ++l)
             k_pyr_down<<<blocks_for((long long)hs[l] * ws[l] * nf, T), T, 0, st>>>(c->pyr[l - 1], hs[l - 1], ws[l - 1], nf,
                                                                                    c->pyr[l]);
-        for (int l = 0; l < 3; ++l)
-            k_poly_exp<<<blocks_for((long long)hs[l] * ws[l] * nf, T), T, 0, st>>>(c->pyr[l], hs[l], ws[l], nf, pw,
-                                                                                   c->coef[l]);
+        for (int l = 0; l < 3; ++l) {
+            dim3 gp((ws[l] + PX - 1) / PX, (hs[l] + PY - 1) / PY, nf);
+            k_poly_exp<<<gp, 256, 0, st>>>(c->pyr[l], hs[l], ws[l], nf, pw, c->coef[l]);
+        }
         c->launches += 5;
         const size_t fstride = 2 * P0, gstride = 5 * P0;
         double* d_lvl[2] = {c->flow_a, c->flow_b};

@@ -170,7 +170,8 @@ k_hysteresis(const uint32_t* __restrict__ bits_kept, uint32_t* __restrict__ bits
 __device__ __forceinline__ double lab_f(double t) {
     const double d = 6.0 / 29.0;
     const float tf = fmaxf((float)t, 1e-6f);
-    const float y0 = exp2f(__log2f(tf) * (1.0f / 3.0f));
+    float y0;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y0) : "f"(__log2f(tf) * (1.0f / 3.0f)));
     const float r = __frcp_rn(3.0f * y0 * y0);
     const double y = (double)y0;
     const double cube = y - (y * y * y - t) * (double)r;
@@ -194,9 +195,10 @@ __device__ __forceinline__ void rgb_to_lab(const double* __restrict__ lut, int R
 // which keeps flat regions exactly zero and small contrasts accurate; the sums of x and x^2 stay in
 // double because mean(x^2) - mean(x)^2 cancels.
 //   phase 1  LAB of the 34x34 grown tile -> shared memory
-//   phase 2  one thread per (channel, row, run of 4 columns): 7-column sums of x and x^2
-//   phase 3  one thread per (column, run of 4 rows): 7-row sums, variance, C, blend with the edge bit,
-//            patch partial sums
+//   then per channel (its row sums alone occupy shared memory, which keeps four CTAs on an SM):
+//   phase 2  one thread per (row, run of 4 columns): 7-column sums of x and x^2
+//   phase 3  one thread per (column, run of 4 rows): 7-row sums, variance added to the pixel's total
+//   last     C, blend with the edge bit, patch partial sums
 // Window sums of a run share their terms: the middle four once, then suffix sums to the left and prefix
 // sums to the right (11 additions for 4 windows).
 constexpr int ST = 28;
@@ -223,16 +225,12 @@ k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom 
               double w_edge, double w_color, float* __restrict__ s_out, const uint8_t* __restrict__ skip) {
     extern __shared__ __align__(16) double cs[];
     double (*lab)[SE][SLP] = reinterpret_cast<double (*)[SE][SLP]>(cs);                              // [3]
-    double2 (*hs)[SE][ST] = reinterpret_cast<double2 (*)[SE][ST]>(cs + 3 * SE * SLP);                 // [3] (sum x, sum x^2)
+    double2 (*hs)[ST] = reinterpret_cast<double2 (*)[ST]>(cs + 3 * SE * SLP);                        // [SE] (sum x, sum x^2) of one channel
     __shared__ double psum[8][4];
-    __shared__ double slut[256];
     const int f = blockIdx.z, x0 = blockIdx.x * ST, y0 = blockIdx.y * ST;
     if (skip && skip[f]) return;
     const int h = g.H, w = g.W;
     const uint8_t* fr = frames + (size_t)f * frame_bytes;
-    for (int i = threadIdx.x; i < 256; i += blockDim.x) slut[i] = lut[i];
-    __syncthreads();
-    lut = slut;
     double L0, a0, b0;
     {
         const uint8_t* p = fr + ((size_t)y0 * w + x0) * 3;
@@ -248,38 +246,37 @@ k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom 
         lab[2][ry][rx] = b - b0;
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < 3 * SE * (ST / CRUN); i += blockDim.x) {
-        const int run = i % (ST / CRUN), r = i / (ST / CRUN);
-        const int ry = r % SE, c = r / SE;
-        const int ox = CRUN * run;                         // windows ox .. ox+3 read columns ox .. ox+9 of the grown tile
-        const double2* src = reinterpret_cast<const double2*>(&lab[c][ry][ox]);
-        double q[CNQ], q2[CNQ];
-#pragma unroll
-        for (int k = 0; k < CNQ / 2; ++k) {
-            double2 v = src[k];
-            q[2 * k] = v.x;
-            q[2 * k + 1] = v.y;
-        }
-#pragma unroll
-        for (int k = 0; k < CNQ; ++k) q2[k] = q[k] * q[k];
-        double w1[CRUN], w2[CRUN];
-        window4(q, w1);
-        window4(q2, w2);
-#pragma unroll
-        for (int k = 0; k < CRUN; ++k) hs[c][ry][ox + k] = make_double2(w1[k], w2[k]);
-    }
-    __syncthreads();
     const double inv_n = 1.0 / (double)((2 * SR + 1) * (2 * SR + 1));
     double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;   // the four patches of the tile
-    if (threadIdx.x < ST * (ST / CRUN)) {
-        const int ox = threadIdx.x % ST, oy0 = CRUN * (threadIdx.x / ST);
-        double V[CRUN] = {0.0, 0.0, 0.0, 0.0};
+    const bool owner = threadIdx.x < ST * (ST / CRUN);          // phase 3: (column, run of 4 rows)
+    const int ox = threadIdx.x % ST, oy0 = CRUN * (threadIdx.x / ST);
+    double V[CRUN] = {0.0, 0.0, 0.0, 0.0};
+    for (int c = 0; c < 3; ++c) {                               // one channel's row sums in shared memory at a time
+        for (int i = threadIdx.x; i < SE * (ST / CRUN); i += blockDim.x) {
+            const int run = i % (ST / CRUN), ry = i / (ST / CRUN);
+            const int cx = CRUN * run;                          // windows cx .. cx+3 read columns cx .. cx+9 of the grown tile
+            const double2* src = reinterpret_cast<const double2*>(&lab[c][ry][cx]);
+            double q[CNQ], q2[CNQ];
 #pragma unroll
-        for (int c = 0; c < 3; ++c) {
+            for (int k = 0; k < CNQ / 2; ++k) {
+                double2 v = src[k];
+                q[2 * k] = v.x;
+                q[2 * k + 1] = v.y;
+            }
+#pragma unroll
+            for (int k = 0; k < CNQ; ++k) q2[k] = q[k] * q[k];
+            double w1[CRUN], w2[CRUN];
+            window4(q, w1);
+            window4(q2, w2);
+#pragma unroll
+            for (int k = 0; k < CRUN; ++k) hs[ry][cx + k] = make_double2(w1[k], w2[k]);
+        }
+        __syncthreads();
+        if (owner) {
             double q[CNQ], q2[CNQ];
 #pragma unroll
             for (int k = 0; k < CNQ; ++k) {
-                double2 v = hs[c][oy0 + k][ox];
+                double2 v = hs[oy0 + k][ox];
                 q[k] = v.x;
                 q2[k] = v.y;
             }
@@ -292,6 +289,9 @@ k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom 
                 V[k] += w2[k] * inv_n - mean * mean;
             }
         }
+        __syncthreads();
+    }
+    if (owner) {
         const int x = x0 + ox;
 #pragma unroll
         for (int k = 0; k < CRUN; ++k) {
@@ -332,7 +332,7 @@ inline unsigned blocks_for(long long n, int threads) { return (unsigned)((n + th
 
 }  // namespace
 
-static size_t color_smem() { return (size_t)(3 * SE * SLP + 2 * 3 * SE * ST) * sizeof(double); }
+static size_t color_smem() { return (size_t)(3 * SE * SLP + 2 * SE * ST) * sizeof(double); }
 
 int sc_saliency_init(int max_h, int max_words) {
     SC_CHECK(cudaFuncSetAttribute(k_color_patch, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)color_smem()));
