@@ -459,9 +459,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=3)
     ap.add_argument("--frames", type=int, default=0, help="use only the first N frames of the workload (profiling)")
-    ap.add_argument("--chunk", type=int, default=104, help="frames per internal pass of flow/saliency")
+    ap.add_argument("--chunk", type=int, default=304, help="frames per internal pass of flow/saliency")
     ap.add_argument("--ring", type=int, default=RING, help="K/V frame slabs resident on the device")
-    ap.add_argument("--segment", type=int, default=104, help="frames per pipeline segment (filter of one overlaps the store of the previous)")
+    ap.add_argument("--segment", type=int, default=304, help="frames per pipeline segment (filter of one overlaps the store of the previous)")
     ap.add_argument("--overlap", action="store_true", help="store of segment i on a second stream beside the filter of segment i+1")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

@@ -64,13 +64,6 @@ __device__ __forceinline__ uint32_t pack_s8(int a, int b, uint32_t c) {
     asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
     return d;
 }
-// d = (c << 8) | (sat_u4(a) << 4) | sat_u4(b)    (saturation to [0, 15])
-__device__ __forceinline__ uint32_t pack_u4(int a, int b, uint32_t c) {
-    uint32_t d;
-    asm("cvt.pack.sat.u4.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
-
 // Both halves of a word minus z, in binary32: the mixed-precision subtract converts the binary16 operand
 // exactly and rounds once, so it equals convert-then-subtract.
 __device__ __forceinline__ float2 sub_h2_f32(uint32_t w, float z) {
@@ -126,21 +119,21 @@ struct Unit {
     long long cap;
 };
 
-__device__ __forceinline__ Unit decode_unit(long long u, const int* pre, int B, int planes,
+__device__ __forceinline__ Unit decode_unit(uint32_t u, const int* pre, int B, uint32_t planes,
                                             const int32_t* __restrict__ counts, const int32_t* __restrict__ idx,
                                             const long long* __restrict__ row_offset, int n_tok, const PoolPtrs& pp) {
     Unit r;
-    int q = (int)(u / planes);          // lies in [pre[b], pre[b+1]) of exactly one frame
+    const uint32_t q = u / planes;      // lies in [pre[b], pre[b+1]) of exactly one frame
     int lo = 0, hi = B;                 // largest b with pre[b] <= q
     while (hi - lo > 1) {
         int mid = (lo + hi) >> 1;
-        if (pre[mid] <= q) lo = mid; else hi = mid;
+        if ((uint32_t)pre[mid] <= q) lo = mid; else hi = mid;
     }
     r.b = lo;
-    int stored = pre[lo + 1] - pre[lo];
-    long long local = u - (long long)pre[lo] * planes;
+    const uint32_t stored = (uint32_t)(pre[lo + 1] - pre[lo]);
+    const uint32_t local = u - (uint32_t)pre[lo] * planes;
     r.plane = (int)(local / stored);
-    int j = (int)(local % stored);
+    int j = (int)(local - (uint32_t)r.plane * stored);
     int n16 = counts[lo * 5 + SALICACHE_FP16], n8 = counts[lo * 5 + SALICACHE_INT8];
     if (j < n16) { r.tier = 0; r.cap = pp.cap0; }
     else if (j < n16 + n8) { r.tier = 1; j -= n16; r.cap = pp.cap1; }
@@ -154,12 +147,40 @@ __device__ __forceinline__ Unit decode_unit(long long u, const int* pre, int B, 
 }
 
 // ---- pack ---------------------------------------------------------------------------------------
+template <int N> struct ILog2 { static constexpr int v = 1 + ILog2<N / 2>::v; };
+template <> struct ILog2<1> { static constexpr int v = 0; };
+
+// m[i] holds this lane's partial (a half2, reduced with max) of the group that the lane's half warp reads
+// in iteration i.  Reduces every m[i] over the 16 lanes of the half warp with a transposing butterfly:
+// each step a lane hands half of its values to its partner and keeps the other half, so ITERS values
+// cost ITERS - 1 exchanges instead of 4 * ITERS.  On return the lane whose low four bits are
+// i << (4 - log2 ITERS) (and its neighbours above it) holds the reduced value of iteration i.
+template <int ITERS>
+__device__ __forceinline__ uint32_t half_warp_max_transpose(uint32_t (&m)[ITERS], int lane) {
+    int s = 8;
+#pragma unroll
+    for (int n = ITERS; n > 1; n >>= 1, s >>= 1) {
+        const bool up = lane & s;
+#pragma unroll
+        for (int j = 0; j < n / 2; ++j) {
+            const uint32_t send = up ? m[j] : m[j + n / 2];
+            const uint32_t keep = up ? m[j + n / 2] : m[j];
+            m[j] = as_u32(__hmax2(as_h2(keep), as_h2(__shfl_xor_sync(0xffffffffu, send, s))));
+        }
+    }
+#pragma unroll
+    for (; s >= 1; s >>= 1) m[0] = as_u32(__hmax2(as_h2(m[0]), as_h2(__shfl_xor_sync(0xffffffffu, m[0], s))));
+    return m[0];
+}
 // One row (or piece `part` of a row): ITERS 16-byte words per lane = 256 * ITERS elements = 2 * ITERS
 // quantisation groups (<= 32, one per lane).
 template <int ITERS>
 __device__ __forceinline__ void pack_piece(const uint4 (&v)[ITERS], const Unit& un, int part, const KvGeom& g,
                                            const PoolPtrs& pp, int lane) {
-    const int src_lane = (lane & 1) << 4;                  // a lane of the half warp that reduced my group
+    // after the transposing reduction the lanes with low bits (i << SH) of each half warp hold iteration i's group
+    constexpr int SH = 4 - ILog2<ITERS>::v;
+    const bool owns = (lane & ((1 << SH) - 1)) == 0;
+    const int my_group = 2 * ((lane & 15) >> SH) + (lane >> 4);
     const size_t prow = (size_t)un.plane * un.cap + un.row;
     if (un.tier == 0) {
         uint4* dst = reinterpret_cast<uint4*>(pp.fp16_pool + prow * (size_t)g.HD * 2) + part * (ITERS * 32) + lane;
@@ -167,6 +188,8 @@ __device__ __forceinline__ void pack_piece(const uint4 (&v)[ITERS], const Unit& 
         for (int i = 0; i < ITERS; ++i) st_stream(dst + i * 32, v[i]);
     } else if (un.tier == 1) {
         // INT8 symmetric: s = fp16(max|x| / 127), q = rint(x * (1/s)) clamped to [-127, 127]
+        // (this tier runs at the memory limit: the plain butterfly, whose result every lane of the half warp
+        // sees, then one pick per iteration by the lane that will own the group)
         uint32_t mine = 0;
 #pragma unroll
         for (int i = 0; i < ITERS; ++i) {
@@ -174,19 +197,18 @@ __device__ __forceinline__ void pack_piece(const uint4 (&v)[ITERS], const Unit& 
                                 __hmax2(__habs2(as_h2(v[i].z)), __habs2(as_h2(v[i].w))));
 #pragma unroll
             for (int o = 8; o; o >>= 1) m = __hmax2(m, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(m), o)));
-            uint32_t sv = __shfl_sync(0xffffffffu, as_u32(m), src_lane);
-            if ((lane >> 1) == i) mine = sv;             // lane l owns group l = 2i + (l & 1)
+            if (((lane & 15) >> SH) == i) mine = as_u32(m);
         }
         float amax = fmaxf(__low2float(as_h2(mine)), __high2float(as_h2(mine)));
         __half s16 = __float2half_rn(__fdiv_rn(amax, 127.0f));
         if ((__half_as_ushort(s16) & 0x7fff) == 0) s16 = __ushort_as_half(0x3c00);
         const float my_inv = __fdiv_rn(1.0f, __half2float(s16));
-        if (lane < 2 * ITERS)
-            reinterpret_cast<uint16_t*>(pp.int8_scale + prow * (size_t)g.ng * 2)[part * 2 * ITERS + lane] = __half_as_ushort(s16);
+        if (owns)
+            reinterpret_cast<uint16_t*>(pp.int8_scale + prow * (size_t)g.ng * 2)[part * 2 * ITERS + my_group] = __half_as_ushort(s16);
         uint2* dst = reinterpret_cast<uint2*>(pp.int8_codes + prow * (size_t)g.HD) + part * (ITERS * 32) + lane;
 #pragma unroll
         for (int i = 0; i < ITERS; ++i) {
-            const float inv = __shfl_sync(0xffffffffu, my_inv, 2 * i + (lane >> 4));
+            const float inv = __shfl_sync(0xffffffffu, my_inv, (lane & 16) | (i << SH));
             float2 f0 = __half22float2(as_h2(v[i].x)), f1 = __half22float2(as_h2(v[i].y));
             float2 f2 = __half22float2(as_h2(v[i].z)), f3 = __half22float2(as_h2(v[i].w));
             int q0 = __float2int_rn(__fmul_rn(f0.x, inv)), q1 = __float2int_rn(__fmul_rn(f0.y, inv));
@@ -201,19 +223,16 @@ __device__ __forceinline__ void pack_piece(const uint4 (&v)[ITERS], const Unit& 
     } else {
         // INT4 asymmetric: zero = min, s = fp16((max - min) / 15), q = rint((x - zero) * (1/s)) in [0, 15].
         // One half2 carries (max, -min) so a single max-reduction serves both.
-        uint32_t mine = 0;
+        uint32_t ext[ITERS];
 #pragma unroll
         for (int i = 0; i < ITERS; ++i) {
             __half2 a = as_h2(v[i].x), b = as_h2(v[i].y), c = as_h2(v[i].z), d = as_h2(v[i].w);
             __half2 mx = __hmax2(__hmax2(a, b), __hmax2(c, d));
             __half2 nmn = __hneg2(__hmin2(__hmin2(a, b), __hmin2(c, d)));
-            __half2 m = __hmax2(as_h2(__byte_perm(as_u32(mx), as_u32(nmn), 0x5410)),
-                                as_h2(__byte_perm(as_u32(mx), as_u32(nmn), 0x7632)));   // (max, -min)
-#pragma unroll
-            for (int o = 8; o; o >>= 1) m = __hmax2(m, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(m), o)));
-            uint32_t sv = __shfl_sync(0xffffffffu, as_u32(m), src_lane);
-            if ((lane >> 1) == i) mine = sv;
+            ext[i] = as_u32(__hmax2(as_h2(__byte_perm(as_u32(mx), as_u32(nmn), 0x5410)),
+                                     as_h2(__byte_perm(as_u32(mx), as_u32(nmn), 0x7632))));   // (max, -min)
         }
+        const uint32_t mine = half_warp_max_transpose<ITERS>(ext, lane);
         const float fmx = __low2float(as_h2(mine));
         float fmn = -__high2float(as_h2(mine));
         __half z16 = __float2half_rn(fmn);                       // exact: fmn is an fp16 value
@@ -222,13 +241,13 @@ __device__ __forceinline__ void pack_piece(const uint4 (&v)[ITERS], const Unit& 
         if ((__half_as_ushort(s16) & 0x7fff) == 0) s16 = __ushort_as_half(0x3c00);
         const float my_inv = __fdiv_rn(1.0f, __half2float(s16));
         const float my_z = __half2float(z16);
-        if (lane < 2 * ITERS)
-            reinterpret_cast<uint32_t*>(pp.int4_sz + prow * (size_t)g.ng * 4)[part * 2 * ITERS + lane] =
+        if (owns)
+            reinterpret_cast<uint32_t*>(pp.int4_sz + prow * (size_t)g.ng * 4)[part * 2 * ITERS + my_group] =
                 (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(z16) << 16);
         uint32_t* dst = reinterpret_cast<uint32_t*>(pp.int4_codes + prow * (size_t)(g.HD / 2)) + part * (ITERS * 32) + lane;
 #pragma unroll
         for (int i = 0; i < ITERS; ++i) {
-            const int owner = 2 * i + (lane >> 4);
+            const int owner = (lane & 16) | (i << SH);
             const float inv = __shfl_sync(0xffffffffu, my_inv, owner);
             const float z = __shfl_sync(0xffffffffu, my_z, owner);
             const float2 f0 = sub_h2_f32(v[i].x, z), f1 = sub_h2_f32(v[i].y, z), f2 = sub_h2_f32(v[i].z, z), f3 = sub_h2_f32(v[i].w, z);
@@ -259,16 +278,16 @@ k_pack(const __half* __restrict__ K, const __half* __restrict__ V, KvGeom g, con
        int* __restrict__ status) {
     extern __shared__ int pre[];
     build_prefix(counts, g.B, pre);
-    const int planes = 2 * g.L;
-    const long long n_units = (long long)pre[g.B] * planes;
+    const uint32_t planes = 2u * (uint32_t)g.L;
+    const uint32_t n_units = (uint32_t)pre[g.B] * planes;      // < 2^31: checked on the host
     const int lane = threadIdx.x & 31;
-    const long long warp0 = (long long)blockIdx.x * KV_WARPS + (threadIdx.x >> 5);
-    const long long wstride = (long long)gridDim.x * KV_WARPS;
+    const uint32_t warp0 = blockIdx.x * KV_WARPS + (threadIdx.x >> 5);
+    const uint32_t wstride = gridDim.x * KV_WARPS;
     if (warp0 >= n_units) return;
     Unit un = decode_unit(warp0, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp);
     uint4 v[ITERS];
     if (un.row >= 0) load_piece<ITERS>(v, K, V, un, 0, g, lane);
-    for (long long u = warp0; u < n_units; u += wstride) {
+    for (uint32_t u = warp0; u < n_units; u += wstride) {
         const bool more = u + wstride < n_units;
         Unit nxt = un;
         if (more) nxt = decode_unit(u + wstride, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp);
@@ -287,12 +306,12 @@ k_unpack(__half* __restrict__ K, __half* __restrict__ V, KvGeom g, const int32_t
          int* __restrict__ status) {
     extern __shared__ int pre[];
     build_prefix(counts, g.B, pre);
-    const int planes = 2 * g.L;
-    const long long n_units = (long long)pre[g.B] * planes;
+    const uint32_t planes = 2u * (uint32_t)g.L;
+    const uint32_t n_units = (uint32_t)pre[g.B] * planes;      // < 2^31: checked on the host
     const int lane = threadIdx.x & 31;
-    const long long warp0 = (long long)blockIdx.x * KV_WARPS + (threadIdx.x >> 5);
-    const long long wstride = (long long)gridDim.x * KV_WARPS;
-    for (long long u = warp0; u < n_units; u += wstride) {
+    const uint32_t warp0 = blockIdx.x * KV_WARPS + (threadIdx.x >> 5);
+    const uint32_t wstride = gridDim.x * KV_WARPS;
+    for (uint32_t u = warp0; u < n_units; u += wstride) {
         Unit un = decode_unit(u, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp);
         if (un.row < 0) {
             if (lane == 0) atomicMin(status, SALICACHE_E_CAPACITY);
@@ -402,9 +421,13 @@ int sc_kv_max_batch() { return MAX_PREFIX; }
 // Row lengths the kernels are instantiated for (HD = 256 * ITERS).
 bool sc_kv_supported_hd(int HD) { return HD == 4096 || HD == 2048 || HD == 1024 || HD == 512 || HD == 256; }
 
+// Work units of one call are counted in 32 bits on the device.
+static bool units_fit(const salicache_ctx* c, int B) { return (long long)B * c->n_tok * 2 * c->p.L < (1ll << 31); }
+
 int sc_pack(salicache_ctx* c, const void* d_K, const void* d_V, int64_t frame_stride, const int32_t* d_idx,
             const int32_t* d_counts, const int64_t* d_row_offset, int B, const salicache_pools* pools, cudaStream_t st) {
     if (B == 0) return SALICACHE_OK;
+    if (!units_fit(c, B)) return SALICACHE_E_SHAPE;
     const int HD = c->p.heads * c->p.head_dim;
     KvGeom g{c->p.L, c->n_tok, HD, HD / 128, frame_stride, B};
     const int grid = c->sm_count * 2;
@@ -430,6 +453,7 @@ int sc_unpack(salicache_ctx* c, const salicache_pools* pools, const int32_t* d_i
               const uint8_t* d_decision, const int64_t* d_row_offset, int B, int zero_fill_pruned, void* d_K_out,
               void* d_V_out, int64_t frame_stride, cudaStream_t st) {
     if (B == 0) return SALICACHE_OK;
+    if (!units_fit(c, B)) return SALICACHE_E_SHAPE;
     const int HD = c->p.heads * c->p.head_dim;
     KvGeom g{c->p.L, c->n_tok, HD, HD / 128, frame_stride, B};
     const int grid = c->sm_count * 2;
