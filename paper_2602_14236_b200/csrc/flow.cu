@@ -176,43 +176,57 @@ __device__ __forceinline__ double bilin_fetch(const T* __restrict__ p, const Bil
 
 // Normal-equation terms of one pixel for the prior (du, dv): G = A^T A (g11 g12 g22), hv = A^T db,
 //   A = (A1(x) + A2(x~))/2,  db = -(b2(x~) - b1(x))/2 + A d~,  x~ = clamp(x + d~), bilinear fetch.
-// The sampling position is exact: floor and fraction of d~ are taken in double and the integer part is
-// added to the pixel index (a single-precision x + d~ would move the sample by up to 2e-5 px at
-// x ~ 300); the interpolation and the products run in single precision on the single-precision
-// coefficients, whose rounding already bounds what they can deliver.
+// The sampling position is exact: floor and fraction of d~ are taken in the precision d~ comes in and the
+// integer part is added to the pixel index (x + d~ in single precision would move the sample by up to
+// 2e-5 px at x ~ 300); the interpolation and the products run in single precision on the
+// single-precision coefficients, whose rounding already bounds what they can deliver.
+// The four taps are read at i, i+1, i+w, i+w+1 without clamping the far ones: where the position is
+// clamped to the last column or row the fraction is zero, so the far tap is multiplied by zero, and it
+// is a finite number (the next row, the next plane, or the zeroed pad behind the last plane).
+template <typename R>
 __device__ __forceinline__ void normal_terms(const float* __restrict__ c1, const float* __restrict__ c2, size_t P,
-                                             int h, int w, int y, int x, double du, double dv, float out[5]) {
+                                             int h, int w, int y, int x, R du, R dv, float out[5]) {
     const int p = y * w + x;
-    // x~ = clamp(x + du): integer part and fraction of du in double, the integer add is exact
-    const double fdu = floor(du), fdv = floor(dv);
+    const R fdu = floor(du), fdv = floor(dv);
     int x0 = x + (int)fdu, y0 = y + (int)fdv;
     float fx = (float)(du - fdu), fy = (float)(dv - fdv);
     if (x0 < 0) { x0 = 0; fx = 0.0f; }
     if (x0 >= w - 1) { x0 = w - 1; fx = 0.0f; }
     if (y0 < 0) { y0 = 0; fy = 0.0f; }
     if (y0 >= h - 1) { y0 = h - 1; fy = 0.0f; }
-    const int x1 = min(x0 + 1, w - 1), y1 = min(y0 + 1, h - 1);
     const float gx = 1.0f - fx, gy = 1.0f - fy;
-    const int i00 = y0 * w + x0, i01 = y0 * w + x1, i10 = y1 * w + x0, i11 = y1 * w + x1;
-    float v[5];
+    const float* q = c2 + (y0 * w + x0);
+    const float* a = c1 + p;
+    float v[5], u[5];
 #pragma unroll
     for (int c = 0; c < 5; ++c) {
-        const float* q = c2 + c * P;
-        const float top = q[i00] * gx + q[i01] * fx;
-        const float bot = q[i10] * gx + q[i11] * fx;
+        const float top = q[0] * gx + q[1] * fx;
+        const float bot = q[w] * gx + q[w + 1] * fx;
         v[c] = top * gy + bot * fy;
+        u[c] = a[0];
+        q += P;
+        a += P;
     }
     const float duf = (float)du, dvf = (float)dv;
-    const float axx = 0.5f * (c1[2 * P + p] + v[2]);
-    const float ayy = 0.5f * (c1[3 * P + p] + v[3]);
-    const float axy = 0.5f * (0.5f * c1[4 * P + p] + 0.5f * v[4]);
-    const float dbx = -0.5f * (v[0] - c1[p]) + (axx * duf + axy * dvf);
-    const float dby = -0.5f * (v[1] - c1[P + p]) + (axy * duf + ayy * dvf);
+    const float axx = 0.5f * (u[2] + v[2]);
+    const float ayy = 0.5f * (u[3] + v[3]);
+    const float axy = 0.5f * (0.5f * u[4] + 0.5f * v[4]);
+    const float dbx = -0.5f * (v[0] - u[0]) + (axx * duf + axy * dvf);
+    const float dby = -0.5f * (v[1] - u[1]) + (axy * duf + ayy * dvf);
     out[0] = axx * axx + axy * axy;
     out[1] = axx * axy + axy * ayy;
     out[2] = axy * axy + ayy * ayy;
     out[3] = axx * dbx + axy * dby;
     out[4] = axy * dbx + ayy * dby;
+}
+
+// a*d - b*c with one rounding error of each product recovered by a fused multiply-add (Kahan): good to
+// about 1.5 ulp even when the products cancel.
+__device__ __forceinline__ float det2(float a, float b, float c, float d) {
+    const float w = b * c;
+    const float e = fmaf(-b, c, w);
+    const float f = fmaf(a, d, -w);
+    return f + e;
 }
 
 // ---- (G, h) of the first update of a level.  Prior: zero at the coarsest level, else the coarser
@@ -275,10 +289,11 @@ k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, d
               PlaneGeom g) {
     using G = UpdGeom<TW>;
     constexpr int RUN = G::RUN, EW = G::EW, S = G::S, NQ = G::NQ;
+    constexpr int DSM_DOUBLES = (TH * (TW + 1) + 1) / 2 * 2 > UPD_THREADS + TW ? (TH * (TW + 1) + 1) / 2 * 2 : UPD_THREADS + TW + 2;
     extern __shared__ __align__(16) double upd_smem[];
-    double (*dsm)[TW + 1][2] = reinterpret_cast<double (*)[TW + 1][2]>(upd_smem);      // [TH] (du, dv); the odd row pitch
+    float2 (*dsm)[TW + 1] = reinterpret_cast<float2 (*)[TW + 1]>(upd_smem);            // [TH] (du, dv); the odd row pitch
                                                                                        // spreads phase 2's stores over the banks
-    float (*vs)[TH][S] = reinterpret_cast<float (*)[TH][S]>(upd_smem + TH * (TW + 1) * 2);   // [5] 15-row sums
+    float (*vs)[TH][S] = reinterpret_cast<float (*)[TH][S]>(upd_smem + DSM_DOUBLES);   // [5] 15-row sums
     const int f = blockIdx.z;
     const int x0 = blockIdx.x * TW, y0 = blockIdx.y * TH;
     const size_t P = (size_t)h * w;
@@ -346,15 +361,12 @@ k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, d
                 s[c][k] += pre;
             }
         }
-        // the 2x2 solve in double: the determinant cancels
+        // the 2x2 solve: determinant and numerators cancel, so each is formed with compensated products
 #pragma unroll
         for (int k = 0; k < RUN; ++k) {
-            const double g11 = s[0][k], g12 = s[1][k], g22 = s[2][k], h1 = s[3][k], h2 = s[4][k];
-            const double inv = 1.0 / (g11 * g22 - g12 * g12 + eps);
-            double2 d;
-            d.x = (g22 * h1 - g12 * h2) * inv;
-            d.y = (g11 * h2 - g12 * h1) * inv;
-            *reinterpret_cast<double2*>(&dsm[row][col0 + k][0]) = d;
+            const float g11 = s[0][k], g12 = s[1][k], g22 = s[2][k], h1 = s[3][k], h2 = s[4][k];
+            const float inv = __frcp_rn(det2(g11, g12, g12, g22) + (float)eps);
+            dsm[row][col0 + k] = make_float2(det2(g22, g12, h2, h1) * inv, det2(g11, g12, h1, h2) * inv);
         }
     }
     __syncthreads();
@@ -367,12 +379,12 @@ k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, d
         const int i = t + j * UPD_THREADS;
         if (i >= TH * TW) break;
         const int oy = i / TW, ox = i - oy * TW;
-        const double2 d = *reinterpret_cast<const double2*>(&dsm[oy][ox][0]);
+        const float2 d = dsm[oy][ox];
         const int y = y0 + oy, x = x0 + ox, p = y * w + x;
         if (FLAGS & EMIT_D) {
             double* o = d_out + (size_t)f * flow_stride;
-            o[p] = d.x;
-            o[P + p] = d.y;
+            o[p] = (double)d.x;
+            o[P + p] = (double)d.y;
         }
         if (FLAGS & EMIT_NEXT) {
             float tm[5];
@@ -381,7 +393,7 @@ k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, d
 #pragma unroll
             for (int c = 0; c < 5; ++c) o[c * P] = tm[c];
         }
-        if (FLAGS & EMIT_DP) acc += d.x * d.x + d.y * d.y;
+        if (FLAGS & EMIT_DP) acc += (double)d.x * (double)d.x + (double)d.y * (double)d.y;
     }
     if (FLAGS & EMIT_DP) {     // Eq. 5 (flow reading): dP_i = sqrt(mean over the patch of u^2 + v^2)
         double* part = upd_smem;                   // (du, dv) are no longer needed once every thread is here
@@ -407,7 +419,9 @@ k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, d
 
 template <int TW>
 constexpr size_t upd_smem_bytes() {
-    return (size_t)TH * (TW + 1) * 2 * sizeof(double) + (size_t)5 * TH * UpdGeom<TW>::S * sizeof(float);
+    // (du, dv) as float2, reused as UPD_THREADS + TW doubles by the patch reduction; then the row sums
+    constexpr size_t d = (TH * (TW + 1) + 1) / 2 * 2 > UPD_THREADS + TW ? (TH * (TW + 1) + 1) / 2 * 2 : UPD_THREADS + TW + 2;
+    return d * sizeof(double) + (size_t)5 * TH * UpdGeom<TW>::S * sizeof(float);
 }
 
 template <int TW>
