@@ -290,7 +290,7 @@ def run_ours(args):
         "metric": "frames/s through flow+saliency+select+KV-pack at LLaVA-1.6-7B shape", "value": round(fps, 2),
         "unit": "frames/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": round(ms_per_step, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f16->i8/i4 (store), f64 (scores)", "data": "synthetic",
+        "dtype": "f16->i4/i8 (store), f32+f64 (scores)", "data": "synthetic",
         "config": {"workload": f"configs[{wl.index - 1}]: {wl.description}", "frames": T, "tokens_per_frame": n_tok,
                    "layers": L, "heads": wl.heads, "head_dim": wl.head_dim, "background": wl.background,
                    "kv_ring_slabs": ring, "pipeline_segment_frames": seg, "l2_policy": "inputs larger than L2 (K/V ring of %.1f GB)" % (2 * Kring.numel() * 2 / 1e9),
@@ -441,7 +441,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": "frames/s through flow+saliency+select+KV-pack at LLaVA-1.6-7B shape",
             "value": round(fps, 4), "unit": "frames/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": round(secs * 1e3, 1), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f16->i8/i4 (store), f64 (scores)", "data": "synthetic",
+            "dtype": "f16->i4/i8 (store), f32+f64 (scores)", "data": "synthetic",
             "config": {"workload": f"configs[{wl.index - 1}]: {wl.description}", "frames": T,
                        "tokens_per_frame": wl.n_tok, "layers": wl.L, "background": wl.background},
             "cpu_baseline": {"value": round(fps, 4), "unit": "frames/s", "cores": oracle.num_threads(),
@@ -466,7 +466,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=1)
-    ap.add_argument("--cpu-sample", type=int, default=6)
+    ap.add_argument("--cpu-sample", type=int, default=100, help="frames of the workload the oracle is timed on (about 15 s)")
     ap.add_argument("--ref-sample", type=int, default=4)
     args = ap.parse_args()
     if args.impl == "reference":

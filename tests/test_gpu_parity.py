@@ -301,6 +301,39 @@ def test_pack_special_values():
         _assert_pools_equal(pools, ref, (0, 576, 576))
 
 
+@pytest.mark.parametrize("heads", [8, 2])
+def test_pack_other_row_lengths(heads):
+    """8 KV heads x 128 (the grouped-query shape of the paper's model) and a 256-element row."""
+    import torch
+    L, n_tok, HD = 2, 576, heads * 128
+    ctx = _ctx(L=L, heads=heads, **synth.thresholds("four"))
+    rng = np.random.default_rng(7)
+    s = rng.uniform(0.0, 0.6, (2, n_tok)).astype(np.float32)
+    K = rng.standard_normal((2, L, n_tok, HD)).astype(np.float16)
+    V = rng.standard_normal((2, L, n_tok, HD)).astype(np.float16)
+    dec, idx, counts, red, off = gu.oracle_select_all(None, s, gu.oracle_params(ctx.params))
+    caps = tuple(int(c) + 1 for c in counts[:, [4, 3, 2]].sum(axis=0))
+    ref = oracle.Pools(L, HD, 128, *caps)
+    for t in range(2):
+        oracle.pack_frame(K[t].view(np.uint16), V[t].view(np.uint16), idx[t], counts[t], off[t], ref)
+    out = gu.gpu_select(ctx, None, s)
+    pools = sc.PoolSet(L, HD, *caps)
+    sc.salicache_pack_kv(ctx, torch.from_numpy(K).cuda(), torch.from_numpy(V).cuda(), L * n_tok * HD, out["idx"],
+                         out["counts"], out["row_offset"], 2, pools.c)
+    torch.cuda.synchronize()
+    _assert_pools_equal(pools, ref, caps)
+    Ko = np.zeros(K.shape, np.uint16)
+    Vo = np.zeros(K.shape, np.uint16)
+    for t in range(2):
+        oracle.unpack_frame(n_tok, idx[t], counts[t], dec[t], off[t], ref, True, Ko[t], Vo[t])
+    gK = torch.zeros(K.shape, dtype=torch.float16, device="cuda")
+    gV = gK.clone()
+    sc.salicache_unpack_kv(ctx, pools.c, out["idx"], out["counts"], out["decision"], out["row_offset"], 2, True, gK, gV,
+                           L * n_tok * HD)
+    torch.cuda.synchronize()
+    assert np.array_equal(gK.cpu().numpy().view(np.uint16), Ko) and np.array_equal(gV.cpu().numpy().view(np.uint16), Vo)
+
+
 def test_dequantised_values_within_the_stated_bound_of_the_oracle():
     import torch
     ctx, (K, V, dec, idx, counts, off, ref), (out, pools, dK, dV) = _pack_case("four", L=1, T=1, seed=3)
