@@ -29,7 +29,7 @@ PAPER_CONTEXT = {"compression_ratio": 2.20, "time_per_frame_s": 0.068, "baseline
                  "hardware": "1x RTX 3090 24 GB, LLaVA-1.6 Mistral-7B, fp16 (paper Tables I and III)"}
 # DRAM bytes of the pack kernel per algorithmic byte, from the ncu capture summarised in
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over the algorithmic bytes of the same launch).
-NCU_TRAFFIC_RATIO = None
+NCU_TRAFFIC_RATIO = 0.969
 
 
 def _peaks():
