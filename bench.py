@@ -408,7 +408,7 @@ def cpu_baseline(args, wl, T, frames_np, Kring, Vring, th):
     Vh = Vring.cpu().numpy().view(np.uint16)
     secs, stored = _oracle_sample(wl, T, frames_np, Kh, Vh, th, sample)
     return {"value": round(len(sample) / secs, 4), "unit": "frames/s", "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"{len(sample)} evenly spaced frames {sample} of the {T}-frame workload "
+            "sample": f"{len(sample)} evenly spaced frames ({sample[0]}, {sample[1] if len(sample) > 1 else sample[0]}, ..., {sample[-1]}) of the {T}-frame workload "
                       f"({stored} stored token rows x {2 * wl.L} planes), {secs:.1f} s",
             "seconds": round(secs, 2)}
 

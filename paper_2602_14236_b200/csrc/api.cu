@@ -115,8 +115,8 @@ int salicache_create(salicache_ctx** out, const salicache_params* p) {
     }
     ok = ok && cudaMalloc(&c->gh_a, (size_t)c->chunk * 5 * P0 * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->gh_b, (size_t)c->chunk * 5 * P0 * sizeof(float)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->flow_a, (size_t)c->chunk * 2 * P0 * sizeof(double)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->flow_b, (size_t)c->chunk * 2 * P0 * sizeof(double)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->flow_a, (size_t)c->chunk * 2 * P0 * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->flow_b, (size_t)c->chunk * 2 * P0 * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->bits_kept, (size_t)c->chunk * p->H * words * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->bits_edge, (size_t)c->chunk * p->H * words * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->lut, 256 * sizeof(double)) == cudaSuccess;

@@ -39,8 +39,8 @@ struct salicache_ctx {
     float* coef[3];            // [2*chunk][5][h_l*w_l] expansion planes
     float* gh_a;               // [chunk][5][H*W] normal-equation terms, ping
     float* gh_b;               //                                         pong
-    double* flow_a;            // [chunk][2][H*W] displacement carried between levels
-    double* flow_b;
+    float* flow_a;             // [chunk][2][H*W] displacement carried between levels
+    float* flow_b;
     // saliency scratch
     uint32_t* bits_kept;       // [chunk][H][Ww]  NMS-kept weak or strong pixels
     uint32_t* bits_edge;       // [chunk][H][Ww]  strong pixels, grown to the edge map E

@@ -148,15 +148,16 @@ k_poly_exp(const float* __restrict__ img, int h, int w, int n_frames, PolyW pw, 
     }
 }
 
-// Bilinear corner set of a clamped continuous position.
+// Bilinear corner set of a clamped continuous position (the coarse-to-fine transfer samples at multiples of
+// 1/4, which single precision holds exactly).
 struct Bilin {
     int i00, i01, i10, i11;
-    double fx, fy;
+    float fx, fy;
 };
-__device__ __forceinline__ Bilin bilin_at(double y, double x, int h, int w) {
-    x = fmin(fmax(x, 0.0), (double)(w - 1));
-    y = fmin(fmax(y, 0.0), (double)(h - 1));
-    int x0 = (int)floor(x), y0 = (int)floor(y);
+__device__ __forceinline__ Bilin bilin_at(float y, float x, int h, int w) {
+    x = fminf(fmaxf(x, 0.0f), (float)(w - 1));
+    y = fminf(fmaxf(y, 0.0f), (float)(h - 1));
+    int x0 = (int)floorf(x), y0 = (int)floorf(y);
     int x1 = min(x0 + 1, w - 1), y1 = min(y0 + 1, h - 1);
     Bilin b;
     b.fx = x - x0;
@@ -167,11 +168,10 @@ __device__ __forceinline__ Bilin bilin_at(double y, double x, int h, int w) {
     b.i11 = y1 * w + x1;
     return b;
 }
-template <typename T>
-__device__ __forceinline__ double bilin_fetch(const T* __restrict__ p, const Bilin& b) {
-    double top = (double)p[b.i00] * (1.0 - b.fx) + (double)p[b.i01] * b.fx;
-    double bot = (double)p[b.i10] * (1.0 - b.fx) + (double)p[b.i11] * b.fx;
-    return top * (1.0 - b.fy) + bot * b.fy;
+__device__ __forceinline__ float bilin_fetch(const float* __restrict__ p, const Bilin& b) {
+    float top = p[b.i00] * (1.0f - b.fx) + p[b.i01] * b.fx;
+    float bot = p[b.i10] * (1.0f - b.fx) + p[b.i11] * b.fx;
+    return top * (1.0f - b.fy) + bot * b.fy;
 }
 
 // Normal-equation terms of one pixel for the prior (du, dv): G = A^T A (g11 g12 g22), hv = A^T db,
@@ -233,20 +233,20 @@ __device__ __forceinline__ float det2(float a, float b, float c, float d) {
 // level's field carried over as d = 2 * bilinear(d_coarse) at ((x+1/2)/2 - 1/2, (y+1/2)/2 - 1/2).
 __global__ void __launch_bounds__(256)
 k_flow_gh(const float* __restrict__ coef1, const float* __restrict__ coef2, size_t coef_stride, int h, int w,
-          const double* __restrict__ d_coarse, size_t flow_stride, float* __restrict__ gh, size_t gh_stride,
+          const float* __restrict__ d_coarse, size_t flow_stride, float* __restrict__ gh, size_t gh_stride,
           int n_pairs) {
     const size_t P = (size_t)h * w;
     long long gid = blockIdx.x * (long long)blockDim.x + threadIdx.x;
     if (gid >= (long long)P * n_pairs) return;
     const int f = (int)(gid / P), r = (int)(gid % P);
     const int y = r / w, x = r % w;
-    double du = 0.0, dv = 0.0;
+    float du = 0.0f, dv = 0.0f;
     if (d_coarse) {
         const int hc = h / 2, wc = w / 2;
-        Bilin b = bilin_at((y + 0.5) * 0.5 - 0.5, (x + 0.5) * 0.5 - 0.5, hc, wc);
-        const double* c = d_coarse + (size_t)f * flow_stride;
-        du = 2.0 * bilin_fetch(c, b);
-        dv = 2.0 * bilin_fetch(c + (size_t)hc * wc, b);
+        Bilin b = bilin_at((y + 0.5f) * 0.5f - 0.5f, (x + 0.5f) * 0.5f - 0.5f, hc, wc);
+        const float* c = d_coarse + (size_t)f * flow_stride;
+        du = 2.0f * bilin_fetch(c, b);
+        dv = 2.0f * bilin_fetch(c + (size_t)hc * wc, b);
     }
     float t[5];
     normal_terms(coef1 + (size_t)f * coef_stride, coef2 + (size_t)f * coef_stride, P, h, w, y, x, du, dv, t);
@@ -268,7 +268,7 @@ constexpr int TH = 14;             // tile height = 1 patch
 constexpr int BR = 7;              // window radius (window 15)
 constexpr int ER = TH + 2 * BR;    // 28 rows loaded
 constexpr int UPD_THREADS = 224;
-constexpr int EMIT_NEXT = 1, EMIT_D = 2, EMIT_DP = 4;
+constexpr int EMIT_NEXT = 1, EMIT_D = 2, EMIT_DP = 4, EMIT_D64 = 8;
 
 template <int TW>
 struct UpdGeom {
@@ -285,8 +285,8 @@ template <int TW, int FLAGS>
 __global__ void __launch_bounds__(UPD_THREADS, 4)
 k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, double eps,
               const float* __restrict__ coef1, const float* __restrict__ coef2, size_t coef_stride,
-              float* __restrict__ gh_out, double* __restrict__ d_out, size_t flow_stride, float* __restrict__ dP,
-              PlaneGeom g) {
+              float* __restrict__ gh_out, float* __restrict__ d_out, double* __restrict__ d_out64, size_t flow_stride,
+              float* __restrict__ dP, PlaneGeom g) {
     using G = UpdGeom<TW>;
     constexpr int RUN = G::RUN, EW = G::EW, S = G::S, NQ = G::NQ;
     constexpr int DSM_DOUBLES = (TH * (TW + 1) + 1) / 2 * 2 > UPD_THREADS + TW ? (TH * (TW + 1) + 1) / 2 * 2 : UPD_THREADS + TW + 2;
@@ -382,7 +382,12 @@ k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, d
         const float2 d = dsm[oy][ox];
         const int y = y0 + oy, x = x0 + ox, p = y * w + x;
         if (FLAGS & EMIT_D) {
-            double* o = d_out + (size_t)f * flow_stride;
+            float* o = d_out + (size_t)f * flow_stride;
+            o[p] = d.x;
+            o[P + p] = d.y;
+        }
+        if (FLAGS & EMIT_D64) {
+            double* o = d_out64 + (size_t)f * flow_stride;
             o[p] = (double)d.x;
             o[P + p] = (double)d.y;
         }
@@ -427,24 +432,25 @@ constexpr size_t upd_smem_bytes() {
 template <int TW>
 int init_update() {
 #define SC_UPD(F) SC_CHECK(cudaFuncSetAttribute(k_flow_update<TW, F>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)upd_smem_bytes<TW>()));
-    SC_UPD(EMIT_NEXT) SC_UPD(EMIT_D) SC_UPD(EMIT_DP | EMIT_D)
+    SC_UPD(EMIT_NEXT) SC_UPD(EMIT_D) SC_UPD(EMIT_DP) SC_UPD(EMIT_DP | EMIT_D64)
 #undef SC_UPD
     return SALICACHE_OK;
 }
 
 template <int TW>
 void launch_update(dim3 grid, cudaStream_t st, int flags, const float* gin, size_t gstride, int h, int w, double eps,
-                   const float* c1, const float* c2, size_t cstride, float* gout, double* dout, size_t fstride,
-                   float* dP, const PlaneGeom& g) {
+                   const float* c1, const float* c2, size_t cstride, float* gout, float* dout, double* dout64,
+                   size_t fstride, float* dP, const PlaneGeom& g) {
 #define SC_UPD(F)                                                                                                   \
     case F:                                                                                                         \
         k_flow_update<TW, F><<<grid, UPD_THREADS, upd_smem_bytes<TW>(), st>>>(gin, gstride, h, w, eps, c1, c2,     \
-                                                                               cstride, gout, dout, fstride, dP, g); \
+                                                                               cstride, gout, dout, dout64, fstride, dP, g); \
         break;
     switch (flags) {
         SC_UPD(EMIT_NEXT)
         SC_UPD(EMIT_D)
-        SC_UPD(EMIT_DP | EMIT_D)
+        SC_UPD(EMIT_DP)
+        SC_UPD(EMIT_DP | EMIT_D64)
         default: break;
     }
 #undef SC_UPD
@@ -501,12 +507,12 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
         }
         c->launches += 5;
         const size_t fstride = 2 * P0, gstride = 5 * P0;
-        double* d_lvl[2] = {c->flow_a, c->flow_b};
-        const double* coarse = nullptr;
+        float* d_lvl[2] = {c->flow_a, c->flow_b};
+        const float* coarse = nullptr;
         for (int l = 2; l >= 0; --l) {
             const size_t Pl = (size_t)hs[l] * ws[l];
             const size_t cstride = 5 * Pl;
-            double* dl = d_lvl[l & 1];
+            float* dl = d_lvl[l & 1];
             const int tw = ws[l] % 56 == 0 ? 56 : 28;
             {
                 const int z0 = 0, nz = nb;
@@ -521,19 +527,23 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
                 for (int it = 0; it < p.iters; ++it) {
                     const bool last = it == p.iters - 1;
                     int flags = last ? 0 : EMIT_NEXT;
-                    double* dout = dl + (size_t)z0 * fstride;
+                    float* dout = dl + (size_t)z0 * fstride;
+                    double* dout64 = nullptr;
                     if (last && l > 0) flags |= EMIT_D;
-                    if (last && l == 0) {      // the field goes to the caller's buffer if there is one, else to scratch
-                        flags |= EMIT_DP | EMIT_D;
-                        if (d_flow_or_null) dout = d_flow_or_null + (size_t)(b0 + z0) * fstride;
+                    if (last && l == 0) {      // the field goes to the caller's buffer if there is one
+                        flags |= EMIT_DP;
+                        if (d_flow_or_null) {
+                            flags |= EMIT_D64;
+                            dout64 = d_flow_or_null + (size_t)(b0 + z0) * fstride;
+                        }
                     }
                     float* dp = d_deltaP + (size_t)(b0 + z0) * g.n_tok;
                     if (tw == 56)
                         launch_update<56>(grid, st, flags, gin, gstride, hs[l], ws[l], p.eps_det, c1, c2, cstride, gout, dout,
-                                          fstride, dp, g);
+                                          dout64, fstride, dp, g);
                     else
                         launch_update<28>(grid, st, flags, gin, gstride, hs[l], ws[l], p.eps_det, c1, c2, cstride, gout, dout,
-                                          fstride, dp, g);
+                                          dout64, fstride, dp, g);
                     c->launches++;
                     float* t = gin; gin = gout; gout = t;
                 }
