@@ -84,7 +84,8 @@ typedef struct salicache_params {
     int32_t patch_reuse;     /* 1: static patches of a non-redundant frame are REUSE (Fig. 3)        */
     /* K/V shape and quantiser */
     int32_t L, heads, head_dim;   /* layers, heads, head size; heads*head_dim = row length HD        */
-    int32_t group;           /* elements per quantisation group: 128 (only value supported)          */
+    int32_t group;           /* elements per quantisation group: 128 (one head), or heads*head_dim    */
+                             /* (one scale, and zero, per token row)                                  */
 } salicache_params;
 
 /* Fills *p with the defaults listed above for a 336x336, L=32, 32x128 configuration. */

@@ -67,7 +67,7 @@ int salicache_create(salicache_ctx** out, const salicache_params* p) {
     if (!out || !p) return SALICACHE_E_NULL;
     *out = nullptr;
     if (p->pyr_levels != 3 || p->poly_n != 5 || p->win != 15 || p->var_radius != 3 || p->patch != 14 ||
-        p->group != 128 || p->iters < 1 || p->iters > 64 || !(p->poly_sigma > 0) || !(p->sigma_ref > 0) ||
+        (p->group != 128 && p->group != p->heads * p->head_dim) || p->iters < 1 || p->iters > 64 || !(p->poly_sigma > 0) || !(p->sigma_ref > 0) ||
         p->canny_lo < 0 || p->canny_hi < p->canny_lo || p->canny_hi > 1442 || p->hyst_max_iters < 1 ||
         (p->n_images != 1 && p->n_images != 5) || p->L < 1 || p->heads < 1 || p->head_dim < 1)
         return SALICACHE_E_PARAM;

@@ -13,9 +13,10 @@ constexpr int KV_WARPS = KV_THREADS / 32;
 constexpr int MAX_PREFIX = 4096;   // frames per call whose row prefix fits the shared-memory table
 
 struct KvGeom {
-    int L, n_tok, HD, ng;          // ng = HD / 128
+    int L, n_tok, HD, ng;          // ng = groups per row: HD / 128, or 1 when the whole row is one group
     long long frame_stride;        // fp16 elements between frames
     int B;
+    int row_group;                 // 1: one quantisation group per row (ng == 1)
 };
 
 struct PoolPtrs {
@@ -173,8 +174,8 @@ __device__ __forceinline__ uint32_t half_warp_max_transpose(uint32_t (&m)[ITERS]
     return m[0];
 }
 // One row (or piece `part` of a row): ITERS 16-byte words per lane = 256 * ITERS elements = 2 * ITERS
-// quantisation groups (<= 32, one per lane).
-template <int ITERS>
+// quantisation groups (<= 32, one per lane), or one group for the whole row when RG.
+template <int ITERS, bool RG>
 __device__ __forceinline__ void pack_piece(const uint4 (&v)[ITERS], const Unit& un, int part, const KvGeom& g,
                                            const PoolPtrs& pp, int lane) {
     // after the transposing reduction the lanes with low bits (i << SH) of each half warp hold iteration i's group
@@ -191,24 +192,36 @@ __device__ __forceinline__ void pack_piece(const uint4 (&v)[ITERS], const Unit& 
         // (this tier runs at the memory limit: the plain butterfly, whose result every lane of the half warp
         // sees, then one pick per iteration by the lane that will own the group)
         uint32_t mine = 0;
+        if (RG) {                         // one group: every lane ends with the row's maximum
+            __half2 m = __floats2half2_rn(0.0f, 0.0f);
 #pragma unroll
-        for (int i = 0; i < ITERS; ++i) {
-            __half2 m = __hmax2(__hmax2(__habs2(as_h2(v[i].x)), __habs2(as_h2(v[i].y))),
-                                __hmax2(__habs2(as_h2(v[i].z)), __habs2(as_h2(v[i].w))));
+            for (int i = 0; i < ITERS; ++i)
+                m = __hmax2(m, __hmax2(__hmax2(__habs2(as_h2(v[i].x)), __habs2(as_h2(v[i].y))),
+                                       __hmax2(__habs2(as_h2(v[i].z)), __habs2(as_h2(v[i].w)))));
 #pragma unroll
-            for (int o = 8; o; o >>= 1) m = __hmax2(m, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(m), o)));
-            if (((lane & 15) >> SH) == i) mine = as_u32(m);
+            for (int o = 16; o; o >>= 1) m = __hmax2(m, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(m), o)));
+            mine = as_u32(m);
+        } else {
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) {
+                __half2 m = __hmax2(__hmax2(__habs2(as_h2(v[i].x)), __habs2(as_h2(v[i].y))),
+                                    __hmax2(__habs2(as_h2(v[i].z)), __habs2(as_h2(v[i].w))));
+#pragma unroll
+                for (int o = 8; o; o >>= 1) m = __hmax2(m, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(m), o)));
+                if (((lane & 15) >> SH) == i) mine = as_u32(m);
+            }
         }
         float amax = fmaxf(__low2float(as_h2(mine)), __high2float(as_h2(mine)));
         __half s16 = __float2half_rn(__fdiv_rn(amax, 127.0f));
         if ((__half_as_ushort(s16) & 0x7fff) == 0) s16 = __ushort_as_half(0x3c00);
         const float my_inv = __fdiv_rn(1.0f, __half2float(s16));
-        if (owns)
-            reinterpret_cast<uint16_t*>(pp.int8_scale + prow * (size_t)g.ng * 2)[part * 2 * ITERS + my_group] = __half_as_ushort(s16);
+        if (RG ? lane == 0 : owns)
+            reinterpret_cast<uint16_t*>(pp.int8_scale + prow * (size_t)g.ng * 2)[RG ? 0 : part * 2 * ITERS + my_group] =
+                __half_as_ushort(s16);
         uint2* dst = reinterpret_cast<uint2*>(pp.int8_codes + prow * (size_t)g.HD) + part * (ITERS * 32) + lane;
 #pragma unroll
         for (int i = 0; i < ITERS; ++i) {
-            const float inv = __shfl_sync(0xffffffffu, my_inv, (lane & 16) | (i << SH));
+            const float inv = RG ? my_inv : __shfl_sync(0xffffffffu, my_inv, (lane & 16) | (i << SH));
             float2 f0 = __half22float2(as_h2(v[i].x)), f1 = __half22float2(as_h2(v[i].y));
             float2 f2 = __half22float2(as_h2(v[i].z)), f3 = __half22float2(as_h2(v[i].w));
             int q0 = __float2int_rn(__fmul_rn(f0.x, inv)), q1 = __float2int_rn(__fmul_rn(f0.y, inv));
@@ -232,7 +245,17 @@ __device__ __forceinline__ void pack_piece(const uint4 (&v)[ITERS], const Unit& 
             ext[i] = as_u32(__hmax2(as_h2(__byte_perm(as_u32(mx), as_u32(nmn), 0x5410)),
                                      as_h2(__byte_perm(as_u32(mx), as_u32(nmn), 0x7632))));   // (max, -min)
         }
-        const uint32_t mine = half_warp_max_transpose<ITERS>(ext, lane);
+        uint32_t mine;
+        if (RG) {
+            __half2 m = as_h2(ext[0]);
+#pragma unroll
+            for (int i = 1; i < ITERS; ++i) m = __hmax2(m, as_h2(ext[i]));
+#pragma unroll
+            for (int o = 16; o; o >>= 1) m = __hmax2(m, as_h2(__shfl_xor_sync(0xffffffffu, as_u32(m), o)));
+            mine = as_u32(m);
+        } else {
+            mine = half_warp_max_transpose<ITERS>(ext, lane);
+        }
         const float fmx = __low2float(as_h2(mine));
         float fmn = -__high2float(as_h2(mine));
         __half z16 = __float2half_rn(fmn);                       // exact: fmn is an fp16 value
@@ -241,15 +264,15 @@ __device__ __forceinline__ void pack_piece(const uint4 (&v)[ITERS], const Unit& 
         if ((__half_as_ushort(s16) & 0x7fff) == 0) s16 = __ushort_as_half(0x3c00);
         const float my_inv = __fdiv_rn(1.0f, __half2float(s16));
         const float my_z = __half2float(z16);
-        if (owns)
-            reinterpret_cast<uint32_t*>(pp.int4_sz + prow * (size_t)g.ng * 4)[part * 2 * ITERS + my_group] =
+        if (RG ? lane == 0 : owns)
+            reinterpret_cast<uint32_t*>(pp.int4_sz + prow * (size_t)g.ng * 4)[RG ? 0 : part * 2 * ITERS + my_group] =
                 (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(z16) << 16);
         uint32_t* dst = reinterpret_cast<uint32_t*>(pp.int4_codes + prow * (size_t)(g.HD / 2)) + part * (ITERS * 32) + lane;
 #pragma unroll
         for (int i = 0; i < ITERS; ++i) {
             const int owner = (lane & 16) | (i << SH);
-            const float inv = __shfl_sync(0xffffffffu, my_inv, owner);
-            const float z = __shfl_sync(0xffffffffu, my_z, owner);
+            const float inv = RG ? my_inv : __shfl_sync(0xffffffffu, my_inv, owner);
+            const float z = RG ? my_z : __shfl_sync(0xffffffffu, my_z, owner);
             const float2 f0 = sub_h2_f32(v[i].x, z), f1 = sub_h2_f32(v[i].y, z), f2 = sub_h2_f32(v[i].z, z), f3 = sub_h2_f32(v[i].w, z);
             // x >= zero, so the product is >= 0; the upper clamp matters only for tiny ranges whose scale rounded down
             int q0 = quant4(f0.x, inv), q1 = quant4(f0.y, inv), q2 = quant4(f1.x, inv), q3 = quant4(f1.y, inv);
@@ -271,7 +294,7 @@ __device__ __forceinline__ void load_piece(uint4 (&v)[ITERS], const __half* K, c
 
 // One warp per stored row: all 16-byte loads of the row are issued before any arithmetic, and the next
 // row's lookups (index list, row offset) run while they are in flight.
-template <int ITERS>
+template <int ITERS, bool RG>
 __global__ void __launch_bounds__(KV_THREADS, 2)
 k_pack(const __half* __restrict__ K, const __half* __restrict__ V, KvGeom g, const int32_t* __restrict__ idx,
        const int32_t* __restrict__ counts, const long long* __restrict__ row_offset, PoolPtrs pp,
@@ -291,7 +314,7 @@ k_pack(const __half* __restrict__ K, const __half* __restrict__ V, KvGeom g, con
         const bool more = u + wstride < n_units;
         Unit nxt = un;
         if (more) nxt = decode_unit(u + wstride, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp);
-        if (un.row >= 0) pack_piece<ITERS>(v, un, 0, g, pp, lane);
+        if (un.row >= 0) pack_piece<ITERS, RG>(v, un, 0, g, pp, lane);
         else if (lane == 0) atomicMin(status, SALICACHE_E_CAPACITY);
         if (more && nxt.row >= 0) load_piece<ITERS>(v, K, V, nxt, 0, g, lane);
         un = nxt;
@@ -338,7 +361,7 @@ k_unpack(__half* __restrict__ K, __half* __restrict__ V, KvGeom g, const int32_t
             const float my_s = __half2float(__ushort_as_half((uint16_t)my_scale));
 #pragma unroll
             for (int i = 0; i < ITERS; ++i) {
-                const float s = __shfl_sync(0xffffffffu, my_s, 2 * i + (lane >> 4));
+                const float s = __shfl_sync(0xffffffffu, my_s, g.row_group ? 0 : 2 * i + (lane >> 4));
                 const uint32_t w[2] = {c[i].x, c[i].y};
                 uint32_t o[4];
 #pragma unroll
@@ -360,7 +383,7 @@ k_unpack(__half* __restrict__ K, __half* __restrict__ V, KvGeom g, const int32_t
             const float my_z = __half2float(__ushort_as_half((uint16_t)(my_sz >> 16)));
 #pragma unroll
             for (int i = 0; i < ITERS; ++i) {
-                const int owner = 2 * i + (lane >> 4);
+                const int owner = g.row_group ? 0 : 2 * i + (lane >> 4);
                 const float s = __shfl_sync(0xffffffffu, my_s, owner);
                 const float z = __shfl_sync(0xffffffffu, my_z, owner);
                 uint32_t o[4];
@@ -406,7 +429,8 @@ PoolPtrs make_pools(const salicache_pools* p) {
 template <int ITERS>
 void launch_pack(int grid, size_t smem, cudaStream_t st, const __half* K, const __half* V, const KvGeom& g,
                  const int32_t* idx, const int32_t* counts, const long long* off, const PoolPtrs& pp, int* status) {
-    k_pack<ITERS><<<grid, KV_THREADS, smem, st>>>(K, V, g, idx, counts, off, pp, status);
+    if (g.row_group) k_pack<ITERS, true><<<grid, KV_THREADS, smem, st>>>(K, V, g, idx, counts, off, pp, status);
+    else k_pack<ITERS, false><<<grid, KV_THREADS, smem, st>>>(K, V, g, idx, counts, off, pp, status);
 }
 template <int ITERS>
 void launch_unpack(int grid, size_t smem, cudaStream_t st, __half* K, __half* V, const KvGeom& g, const int32_t* idx,
@@ -429,7 +453,8 @@ int sc_pack(salicache_ctx* c, const void* d_K, const void* d_V, int64_t frame_st
     if (B == 0) return SALICACHE_OK;
     if (!units_fit(c, B)) return SALICACHE_E_SHAPE;
     const int HD = c->p.heads * c->p.head_dim;
-    KvGeom g{c->p.L, c->n_tok, HD, HD / 128, frame_stride, B};
+    const int row_group = c->p.group == HD ? 1 : 0;
+    KvGeom g{c->p.L, c->n_tok, HD, row_group ? 1 : HD / 128, frame_stride, B, row_group};
     const int grid = c->sm_count * 2;
     const size_t smem = (size_t)(B + 1) * sizeof(int);
     const __half* K = (const __half*)d_K;
@@ -455,7 +480,8 @@ int sc_unpack(salicache_ctx* c, const salicache_pools* pools, const int32_t* d_i
     if (B == 0) return SALICACHE_OK;
     if (!units_fit(c, B)) return SALICACHE_E_SHAPE;
     const int HD = c->p.heads * c->p.head_dim;
-    KvGeom g{c->p.L, c->n_tok, HD, HD / 128, frame_stride, B};
+    const int row_group = c->p.group == HD ? 1 : 0;
+    KvGeom g{c->p.L, c->n_tok, HD, row_group ? 1 : HD / 128, frame_stride, B, row_group};
     const int grid = c->sm_count * 2;
     const size_t smem = (size_t)(B + 1) * sizeof(int);
     __half* K = (__half*)d_K_out;

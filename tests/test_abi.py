@@ -47,6 +47,8 @@ def test_host_side_argument_checks_need_no_device():
     h = ctypes.c_void_p()
     bad = binding.salicache_default_params(win=7)
     assert lib.salicache_create(ctypes.byref(h), ctypes.byref(bad)) == binding.E_PARAM
+    bad = binding.salicache_default_params(group=256)
+    assert lib.salicache_create(ctypes.byref(h), ctypes.byref(bad)) == binding.E_PARAM
     bad = binding.salicache_default_params(H=300)
     assert lib.salicache_create(ctypes.byref(h), ctypes.byref(bad)) == binding.E_SHAPE
     assert lib.salicache_destroy(None) == binding.E_NULL

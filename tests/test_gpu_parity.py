@@ -334,6 +334,41 @@ def test_pack_other_row_lengths(heads):
     assert np.array_equal(gK.cpu().numpy().view(np.uint16), Ko) and np.array_equal(gV.cpu().numpy().view(np.uint16), Vo)
 
 
+def test_pack_with_one_group_per_token_row():
+    """group = heads * head_dim: a single scale (and zero) per token row."""
+    import torch
+    L, n_tok, HD = 1, 576, 4096
+    ctx = _ctx(L=L, group=HD, **synth.thresholds("four"))
+    rng = np.random.default_rng(11)
+    s = rng.uniform(0.0, 0.6, (2, n_tok)).astype(np.float32)
+    KV = [synth.kv_numpy(2, t, L=L) for t in range(2)]
+    K = np.stack([k for k, _ in KV])
+    V = np.stack([v for _, v in KV])
+    K[0, 0, 3] = 0.0                                   # an all-zero row: scale 1, codes 0
+    dec, idx, counts, red, off = gu.oracle_select_all(None, s, gu.oracle_params(ctx.params))
+    caps = tuple(int(c) + 1 for c in counts[:, [4, 3, 2]].sum(axis=0))
+    ref = oracle.Pools(L, HD, HD, *caps)
+    for t in range(2):
+        oracle.pack_frame(K[t].view(np.uint16), V[t].view(np.uint16), idx[t], counts[t], off[t], ref)
+    out = gu.gpu_select(ctx, None, s)
+    pools = sc.PoolSet(L, HD, *caps, G=HD)
+    assert pools.int8_scale.shape[-1] == 1 and pools.int4_sz.shape[-2] == 1
+    sc.salicache_pack_kv(ctx, torch.from_numpy(K).cuda(), torch.from_numpy(V).cuda(), L * n_tok * HD, out["idx"],
+                         out["counts"], out["row_offset"], 2, pools.c)
+    torch.cuda.synchronize()
+    _assert_pools_equal(pools, ref, caps)
+    Ko = np.zeros(K.shape, np.uint16)
+    Vo = np.zeros(K.shape, np.uint16)
+    for t in range(2):
+        oracle.unpack_frame(n_tok, idx[t], counts[t], dec[t], off[t], ref, True, Ko[t], Vo[t])
+    gK = torch.zeros(K.shape, dtype=torch.float16, device="cuda")
+    gV = gK.clone()
+    sc.salicache_unpack_kv(ctx, pools.c, out["idx"], out["counts"], out["decision"], out["row_offset"], 2, True, gK, gV,
+                           L * n_tok * HD)
+    torch.cuda.synchronize()
+    assert np.array_equal(gK.cpu().numpy().view(np.uint16), Ko) and np.array_equal(gV.cpu().numpy().view(np.uint16), Vo)
+
+
 def test_dequantised_values_within_the_stated_bound_of_the_oracle():
     import torch
     ctx, (K, V, dec, idx, counts, off, ref), (out, pools, dK, dV) = _pack_case("four", L=1, T=1, seed=3)
