@@ -155,6 +155,20 @@ SALICACHE_API int salicache_select(salicache_ctx* ctx, const float* d_deltaP, co
                      uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts, uint8_t* d_frame_redundant,
                      int64_t* d_row_offset, int64_t* d_fill, void* cuda_stream);
 
+/*
+ * Source-frame table (Alg. 1 line 7: a reused entry is a pointer to the previous frame's entry; Fig. 3
+ * counts reuse per patch).  For the B frames first_frame .. first_frame+B-1 of a video:
+ *   d_src[b][i] = d_src[b-1][i] if decision[b][i] == SALICACHE_REUSE, else first_frame + b,
+ * chains resolved, so that every token names the frame whose stored (or pruned) entry it uses.
+ *   d_decision  DEVICE u8  [B][N_tok]  from salicache_select
+ *   d_carry     DEVICE i32 [N_tok]     in: sources of frame first_frame-1 (ignored where frame 0 cannot
+ *                                      reuse); out: sources of the batch's last frame, for the next call
+ *   d_src       DEVICE i32 [B][N_tok]  written
+ * Errors: E_NULL, E_SHAPE, E_CUDA.
+ */
+SALICACHE_API int salicache_source_frames(salicache_ctx* ctx, const uint8_t* d_decision, int B, int first_frame,
+                                          int32_t* d_carry, int32_t* d_src, void* cuda_stream);
+
 /* Per-tier pools of the mixed-precision store (device memory, caller-owned).  Axis 2 of the
  * second dimension: 0 = K, 1 = V.  ng = HD / group.
  *   fp16_pool   f16 [L][2][cap_fp16][HD]

@@ -224,6 +224,16 @@ def select(dP, s, has_prev: bool, p: Params = Params()):
     return dec, idx, counts, int(red[0]), float(R[0])
 
 
+def source_frames(decision: np.ndarray, first: int = 0, prev=None) -> np.ndarray:
+    """decision u8 [T][n_tok] -> int32 [T][n_tok]: the frame whose entry each token uses (reuse chains resolved)."""
+    decision = _c(decision, np.uint8)
+    T, n = decision.shape
+    prev = _c(prev if prev is not None else np.full(n, -1, np.int32), np.int32)
+    src = np.empty((T, n), np.int32)
+    lib().oracle_source_frames(_p(decision), C.c_int(T), C.c_int(n), C.c_int(first), _p(prev), _p(src))
+    return src
+
+
 def half_to_float(bits: np.ndarray) -> np.ndarray:
     bits = _c(bits, np.uint16).ravel()
     f = lib().oracle_half_to_float

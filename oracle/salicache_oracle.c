@@ -508,6 +508,21 @@ EXPORT void oracle_select(const float* dP, const float* s, int n_tok, int has_pr
 }
 
 /* ------------------------------------------------------------------------- */
+/* Source-frame table (Alg. 1 line 7: C[t] <- Pointer(C[t-1]); Fig. 3 counts    */
+/* reuse per patch).  src[t][i] = src[t-1][i] when token i of frame t is REUSE, */
+/* else t: every token names the frame whose entry it uses, chains resolved.   */
+/* prev = sources of the frame before frame `first` (unused for tokens that do */
+/* not reuse).                                                                 */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_source_frames(const uint8_t* decision, int T, int n_tok, int first, const int32_t* prev, int32_t* src) {
+    for (int i = 0; i < n_tok; ++i)
+        for (int t = 0; t < T; ++t) {
+            int32_t before = t == 0 ? prev[i] : src[(size_t)(t - 1) * n_tok + i];
+            src[(size_t)t * n_tok + i] = decision[(size_t)t * n_tok + i] == 0 ? before : first + t;
+        }
+}
+
+/* ------------------------------------------------------------------------- */
 /* binary16 <-> binary32, written out on the bits (round to nearest even).     */
 /* ------------------------------------------------------------------------- */
 EXPORT float oracle_half_to_float(uint16_t hbits) {

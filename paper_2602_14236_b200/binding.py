@@ -49,7 +49,7 @@ EXPORTS = [
     "salicache_default_params", "salicache_create", "salicache_destroy", "salicache_strerror",
     "salicache_tokens_per_frame", "salicache_launch_count", "salicache_flow_score", "salicache_saliency", "salicache_select",
     "salicache_pack_kv", "salicache_unpack_kv", "salicache_poll_status", "salicache_saliency_noalloc",
-    "salicache_frame_redundancy",
+    "salicache_frame_redundancy", "salicache_source_frames",
 ]
 
 _lib = None
@@ -78,6 +78,7 @@ def lib():
         _lib.salicache_flow_score.argtypes = [vp, vp, vp, i32, vp, vp, vp]
         _lib.salicache_saliency.argtypes = [vp, vp, i32, vp, vp, vp]
         _lib.salicache_frame_redundancy.argtypes = [vp, vp, i32, i32, vp, vp]
+        _lib.salicache_source_frames.argtypes = [vp, vp, i32, i32, vp, vp, vp]
         _lib.salicache_select.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         _lib.salicache_pack_kv.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, C.POINTER(Pools), vp]
         _lib.salicache_unpack_kv.argtypes = [vp, C.POINTER(Pools), vp, vp, vp, vp, i32, i32, vp, vp, i64, vp]
@@ -164,6 +165,11 @@ def salicache_saliency_noalloc(params: Params, d_frames, B: int, d_s, d_status=N
 
 
 NOALLOC_MAX_FRAMES, NOALLOC_MAX_SIDE = 8, 336
+
+
+def salicache_source_frames(ctx: Context, d_decision, B: int, first_frame: int, d_carry, d_src, stream=None):
+    _check(lib().salicache_source_frames(ctx.handle, _ptr(d_decision), B, first_frame, _ptr(d_carry), _ptr(d_src),
+                                         _stream(stream)), "salicache_source_frames")
 
 
 def salicache_select(ctx: Context, d_deltaP, d_s, B: int, first_has_no_prev: bool, d_decision, d_idx, d_counts,

@@ -231,6 +231,13 @@ int salicache_select(salicache_ctx* c, const float* d_deltaP, const float* d_s, 
                      d_row_offset, d_fill, (cudaStream_t)cuda_stream);
 }
 
+int salicache_source_frames(salicache_ctx* c, const uint8_t* d_decision, int B, int first_frame, int32_t* d_carry,
+                            int32_t* d_src, void* cuda_stream) {
+    if (!c || !d_decision || !d_carry || !d_src) return SALICACHE_E_NULL;
+    if (B < 0 || B > c->p.max_batch || first_frame < 0) return SALICACHE_E_SHAPE;
+    return sc_sources(c, d_decision, B, first_frame, d_carry, d_src, (cudaStream_t)cuda_stream);
+}
+
 static int check_pools(const salicache_pools* p) {
     if (!p) return SALICACHE_E_NULL;
     if (p->cap_fp16 < 0 || p->cap_int8 < 0 || p->cap_int4 < 0) return SALICACHE_E_SHAPE;

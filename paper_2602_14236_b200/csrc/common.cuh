@@ -64,6 +64,8 @@ int sc_box_down2(const uint8_t* d_src, int H, int W, int B, uint8_t* d_dst, cuda
 int sc_select(salicache_ctx* c, const float* d_deltaP, const float* d_s, int B, int first_has_no_prev,
               uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts, uint8_t* d_frame_redundant,
               int64_t* d_row_offset, int64_t* d_fill, cudaStream_t st);
+int sc_sources(salicache_ctx* c, const uint8_t* d_decision, int B, int first_frame, int32_t* d_carry, int32_t* d_src,
+               cudaStream_t st);
 int sc_frame_redundancy(salicache_ctx* c, const float* d_deltaP, int B, int first_has_no_prev, uint8_t* d_frame_redundant,
                         cudaStream_t st);
 // kv.cu

@@ -113,6 +113,21 @@ k_frame_redundancy(const float* __restrict__ dP, int n_tok, int first_has_no_pre
     }
 }
 
+// Source-frame table (Alg. 1 line 7, C[t] <- Pointer(C[t-1]), extended to patches): one thread per token
+// walks the batch in frame order; a REUSE token inherits its predecessor's source, any other token is its
+// own source.  `carry` holds the sources of the frame before the batch and receives those of its last frame.
+__global__ void k_sources(const uint8_t* __restrict__ decision, int n_tok, int B, int first_frame, int32_t* __restrict__ carry,
+                          int32_t* __restrict__ src) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_tok) return;
+    int cur = carry[i];
+    for (int b = 0; b < B; ++b) {
+        if (decision[(size_t)b * n_tok + i] != SALICACHE_REUSE) cur = first_frame + b;
+        src[(size_t)b * n_tok + i] = cur;
+    }
+    carry[i] = cur;
+}
+
 // Pool row offsets: exclusive scan over the frames of the batch, continuing from the running fill.
 __global__ void k_row_offsets(const int32_t* __restrict__ counts, int B, int64_t* __restrict__ row_offset,
                               int64_t* __restrict__ fill) {
@@ -134,6 +149,15 @@ int sc_frame_redundancy(salicache_ctx* c, const float* d_deltaP, int B, int firs
     if (B == 0) return SALICACHE_OK;
     k_frame_redundancy<<<B, SEL_THREADS, 0, st>>>(d_deltaP, c->n_tok, first_has_no_prev, c->p.tau_t, c->p.theta_R,
                                                   d_frame_redundant);
+    c->launches++;
+    SC_CHECK(cudaGetLastError());
+    return SALICACHE_OK;
+}
+
+int sc_sources(salicache_ctx* c, const uint8_t* d_decision, int B, int first_frame, int32_t* d_carry, int32_t* d_src,
+               cudaStream_t st) {
+    if (B == 0) return SALICACHE_OK;
+    k_sources<<<(c->n_tok + 255) / 256, 256, 0, st>>>(d_decision, c->n_tok, B, first_frame, d_carry, d_src);
     c->launches++;
     SC_CHECK(cudaGetLastError());
     return SALICACHE_OK;

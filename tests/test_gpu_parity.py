@@ -163,6 +163,23 @@ def test_pipeline_decisions_match_oracle_up_to_near_threshold_tokens(wl1_frames,
     assert len(set(np.unique(dec))) >= 4              # the case exercises several categories
 
 
+def test_source_frames_table_in_two_batches():
+    import torch
+    ctx = _ctx()
+    rng = np.random.default_rng(9)
+    dec = rng.integers(0, 5, (12, 576)).astype(np.uint8)
+    dec[0][dec[0] == 0] = 1
+    want = oracle.source_frames(dec)
+    d_dec = torch.from_numpy(dec).cuda()
+    carry = torch.full((576,), -1, dtype=torch.int32, device="cuda")
+    src = torch.full((12, 576), -9, dtype=torch.int32, device="cuda")
+    sc.salicache_source_frames(ctx, d_dec, 7, 0, carry, src)
+    sc.salicache_source_frames(ctx, d_dec[7:], 5, 7, carry, src[7:])
+    torch.cuda.synchronize()
+    assert np.array_equal(src.cpu().numpy(), want)
+    assert np.array_equal(carry.cpu().numpy(), want[-1])
+
+
 def test_select_without_temporal_scores_and_empty_batch():
     ctx = _ctx()
     s = np.random.default_rng(0).uniform(0, 0.6, (3, 576)).astype(np.float32)

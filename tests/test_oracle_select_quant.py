@@ -266,3 +266,28 @@ def test_accounting_closed_form_and_the_paper_tier_mix():
     ratio = oracle.raw_bytes(100, L, HD, n_tok) / oracle.stored_bytes(mix, L, HD, G, n_tok)
     assert ratio == pytest.approx(1 / (0.317 + 0.071 * (0.5 + 1 / 128) + 0.214 * (0.25 + 1 / 64)), rel=2e-4)
     assert 2.40 < ratio < 2.48
+
+
+def test_source_frames_resolve_reuse_chains():
+    """Alg. 1 line 7: a chain of reused entries ends at the last frame that stored (or pruned) the token."""
+    dec = np.array([[4, 1, 2, 3],      # frame 0: nothing can be reused
+                    [0, 0, 4, 0],
+                    [0, 2, 0, 0],
+                    [4, 0, 0, 0]], np.uint8)
+    src = oracle.source_frames(dec)
+    assert src.tolist() == [[0, 0, 0, 0], [0, 0, 1, 0], [0, 2, 1, 0], [3, 2, 1, 0]]
+    # brute force on random decisions: walk back until a non-reuse entry
+    rng = np.random.default_rng(5)
+    dec = rng.integers(0, 5, (40, 64)).astype(np.uint8)
+    dec[0][dec[0] == 0] = 1
+    src = oracle.source_frames(dec)
+    for t in range(40):
+        for i in range(64):
+            k = t
+            while dec[k, i] == 0:
+                k -= 1
+            assert src[t, i] == k
+    # a stream cut in two continues through the carried row
+    a = oracle.source_frames(dec[:17])
+    b = oracle.source_frames(dec[17:], first=17, prev=a[-1])
+    assert np.array_equal(np.concatenate([a, b]), src)
