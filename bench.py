@@ -284,6 +284,10 @@ def run_ours(args):
         e2e = run_e2e(args, sc, ctx, wl, T, frames_np, Kring, Vring, pools, dev,
                       (dP, s, dec, idx, counts, red, off, fill), world)
 
+    extras = None
+    if not args.no_extras and world == 1:
+        extras = run_extras(sc, synth, ctx, wl, T, frames, dP, dev, peak)
+
     raw = 2 * L * T * n_tok * HD * 2
     stored = wr + T * (n_tok + 52) + 4 * int(tot.sum())     # payload + decisions, tables, index lists
     line = {
@@ -302,11 +306,71 @@ def run_ours(args):
         "tier_counts": {"reuse": int(counts_h[:, 0].sum()), "prune": int(counts_h[:, 1].sum()),
                         "int4": int(counts_h[:, 2].sum()), "int8": int(counts_h[:, 3].sum()),
                         "fp16": int(counts_h[:, 4].sum()), "frames_redundant": int(red.sum().item())},
-        "paper_context": PAPER_CONTEXT,
+        "extras": extras, "paper_context": PAPER_CONTEXT,
     }
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_extras(sc, synth, ctx, wl, T, frames, dP, dev, peak):
+    """Measurements beside the headline, outside its timed region: the unpack kernel on the stored cache of
+    this workload's layout, the literal Eq. 5 temporal score, and the four-tier breakdown on workload 2."""
+    import torch
+    out = {}
+
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # larger than L2
+
+    def timed(fn, reps=10):
+        fn()
+        ms = 0.0
+        for _ in range(reps):
+            flush.fill_(1)                                                 # evict the inputs between repetitions
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ms += e0.elapsed_time(e1)
+        return ms / reps
+
+    if T > 1:
+        d2 = torch.zeros_like(dP)
+        ms = timed(lambda: sc.salicache_diff_score(ctx, frames[:-1], frames[1:], T - 1, d2[1:]))
+        nbytes = int(frames.numel())                        # every frame is needed once
+        out["diff_score"] = {"what": "Eq. 5 read literally (RMS pixel difference per patch), all frame pairs",
+                             "ms": round(ms, 4), "l2": "flushed between repetitions", "algorithmic_GBps": round(nbytes / ms / 1e6, 1),
+                             "frac_of_hbm_peak": round(nbytes / ms / 1e6 / peak, 4)}
+    # Fig. 3 style breakdown: workload 2 frames under the four-tier rule
+    wl2 = synth.WORKLOADS[2]
+    p2 = sc.salicache_default_params(max_batch=wl2.T, chunk_frames=wl2.T, L=1, **synth.thresholds("four"))
+    c2 = sc.Context(p2)
+    fr2 = torch.from_numpy(synth.frames(2)).to(dev)
+    n = wl2.n_tok
+    dP2 = torch.zeros((wl2.T, n), dtype=torch.float32, device=dev)
+    s2 = torch.zeros_like(dP2)
+    red2 = torch.zeros((wl2.T,), dtype=torch.uint8, device=dev)
+    dec2 = torch.zeros((wl2.T, n), dtype=torch.uint8, device=dev)
+    idx2 = torch.zeros((wl2.T, 3, n), dtype=torch.int32, device=dev)
+    cnt2 = torch.zeros((wl2.T, 5), dtype=torch.int32, device=dev)
+    off2 = torch.zeros((wl2.T, 3), dtype=torch.int64, device=dev)
+    fill2 = torch.zeros((3,), dtype=torch.int64, device=dev)
+    sc.salicache_flow_score(c2, fr2[:-1], fr2[1:], wl2.T - 1, dP2[1:])
+    sc.salicache_frame_redundancy(c2, dP2, wl2.T, True, red2)
+    sc.salicache_saliency(c2, fr2, wl2.T, s2, red2)
+    sc.salicache_select(c2, dP2, s2, wl2.T, True, dec2, idx2, cnt2, red2, off2, fill2)
+    torch.cuda.synchronize()
+    c = cnt2.sum(dim=0).cpu().numpy().astype(float)
+    tot = c.sum()
+    ng = wl2.HD // 128
+    per_tok = wl2.HD * 2
+    stored = c[4] * per_tok + c[3] * (wl2.HD + 2 * ng) + c[2] * (wl2.HD // 2 + 4 * ng)
+    out["four_tier_workload2"] = {
+        "what": "workload 2 frames, four-tier rule (Eq. 8); paper Fig. 3: skipped 26.7, pruned 13.1, INT4 21.4, INT8 7.1, FP16 31.7 %",
+        "percent": {k: round(100 * c[i] / tot, 2) for k, i in (("reuse", 0), ("prune", 1), ("int4", 2), ("int8", 3), ("fp16", 4))},
+        "compression_ratio_payload": round(tot * per_tok / stored, 3) if stored > 0 else None}
+    c2.close()
+    return out
 
 
 def run_e2e(args, sc, ctx, wl, T, frames_np, Kring, Vring, pools, dev, bufs, world):
@@ -465,6 +529,7 @@ def main():
     ap.add_argument("--overlap", action="store_true", help="store of segment i on a second stream beside the filter of segment i+1")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--cpu-sample", type=int, default=100, help="frames of the workload the oracle is timed on (about 15 s)")
     ap.add_argument("--ref-sample", type=int, default=4)

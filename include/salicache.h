@@ -116,6 +116,16 @@ SALICACHE_API int salicache_flow_score(salicache_ctx* ctx, const uint8_t* d_prev
                          float* d_deltaP, double* d_flow_or_null, void* cuda_stream);
 
 /*
+ * Temporal score, Eq. 5 read literally (no optical flow): d_deltaP[b][i] = L2 norm of the pixel difference
+ * d_cur[b] - d_prev[b] over patch i, divided by sqrt(3 * patch * patch): the RMS difference in grey levels,
+ * summed exactly in integers.  A cheap alternative to salicache_flow_score (one pass over the two frames);
+ * tau_t is then a grey-level threshold instead of pixels of motion.  Same arguments and errors as
+ * salicache_flow_score (no flow field).
+ */
+SALICACHE_API int salicache_diff_score(salicache_ctx* ctx, const uint8_t* d_prev, const uint8_t* d_cur, int B,
+                                       float* d_deltaP, void* cuda_stream);
+
+/*
  * Spatial score (Sec. III-B, Eq. 7): Canny edge map E and LAB local colour variance C give
  * S = clamp(w_edge E + w_color C, 0, 1); d_s[b][i] = mean of S over patch i.
  * d_frames: B frames.  d_skip_or_null: DEVICE u8 [B] or NULL; frames with a non-zero entry are not

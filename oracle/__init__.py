@@ -163,6 +163,16 @@ def flow_score(prev: np.ndarray, cur: np.ndarray, p: Params = Params(), want_flo
     return (dP, fl) if want_flow else dP
 
 
+def diff_score(prev: np.ndarray, cur: np.ndarray, patch: int = 14) -> np.ndarray:
+    """Eq. 5 read literally.  prev, cur: [B][h][w][3] uint8 -> dP [B][n_patches] float64 (RMS grey-level difference)."""
+    prev, cur = _c(prev, np.uint8), _c(cur, np.uint8)
+    B, h, w, _ = prev.shape
+    out = np.empty((B, (h // patch) * (w // patch)), np.float64)
+    for b in range(B):
+        lib().oracle_diff_score(_p(prev[b]), _p(cur[b]), C.c_int(h), C.c_int(w), C.c_int(patch), _p(out[b]))
+    return out
+
+
 def canny(g: np.ndarray, lo: int = 50, hi: int = 150, want_cls: bool = False):
     g = _c(g, np.uint8)
     h, w = g.shape

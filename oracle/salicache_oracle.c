@@ -274,6 +274,26 @@ EXPORT void oracle_delta_p(const double* flow, int h, int w, int patch, double* 
         }
 }
 
+/* ------------------------------------------------------------------------- */
+/* Eq. 5 exactly as printed: dP_i = || F^N_i - F^{N-1}_i ||_2 over the pixels   */
+/* (all three channels) of patch i.  Reading: divided by sqrt(3 patch^2), so    */
+/* that it is an RMS difference in grey levels (the paper gives no scale).      */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_diff_score(const uint8_t* prev, const uint8_t* cur, int h, int w, int patch, double* dP) {
+    int gh = h / patch, gw = w / patch;
+    for (int py = 0; py < gh; ++py)
+        for (int px = 0; px < gw; ++px) {
+            double acc = 0.0;
+            for (int y = py * patch; y < (py + 1) * patch; ++y)
+                for (int x = px * patch; x < (px + 1) * patch; ++x)
+                    for (int c = 0; c < 3; ++c) {
+                        double d = (double)cur[((size_t)y * w + x) * 3 + c] - (double)prev[((size_t)y * w + x) * 3 + c];
+                        acc += d * d;
+                    }
+            dP[py * gw + px] = sqrt(acc / (3.0 * patch * patch));
+        }
+}
+
 /* Frame pairs -> dP, B pairs in parallel over host threads.  dP: [B][n_patches]. */
 EXPORT void oracle_flow_score_batch(const uint8_t* prev, const uint8_t* cur, int B, int h, int w, int patch,
                                     int levels, int poly_n, double poly_sigma, int win, int iters, double eps,

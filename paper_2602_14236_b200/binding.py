@@ -49,7 +49,7 @@ EXPORTS = [
     "salicache_default_params", "salicache_create", "salicache_destroy", "salicache_strerror",
     "salicache_tokens_per_frame", "salicache_launch_count", "salicache_flow_score", "salicache_saliency", "salicache_select",
     "salicache_pack_kv", "salicache_unpack_kv", "salicache_poll_status", "salicache_saliency_noalloc",
-    "salicache_frame_redundancy", "salicache_source_frames",
+    "salicache_frame_redundancy", "salicache_source_frames", "salicache_diff_score",
 ]
 
 _lib = None
@@ -77,6 +77,7 @@ def lib():
         vp, i32, i64 = C.c_void_p, C.c_int, C.c_int64
         _lib.salicache_flow_score.argtypes = [vp, vp, vp, i32, vp, vp, vp]
         _lib.salicache_saliency.argtypes = [vp, vp, i32, vp, vp, vp]
+        _lib.salicache_diff_score.argtypes = [vp, vp, vp, i32, vp, vp]
         _lib.salicache_frame_redundancy.argtypes = [vp, vp, i32, i32, vp, vp]
         _lib.salicache_source_frames.argtypes = [vp, vp, i32, i32, vp, vp, vp]
         _lib.salicache_select.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
@@ -144,6 +145,11 @@ class Context:
 def salicache_flow_score(ctx: Context, d_prev, d_cur, B: int, d_deltaP, d_flow=None, stream=None):
     _check(lib().salicache_flow_score(ctx.handle, _ptr(d_prev), _ptr(d_cur), B, _ptr(d_deltaP), _ptr(d_flow),
                                       _stream(stream)), "salicache_flow_score")
+
+
+def salicache_diff_score(ctx: Context, d_prev, d_cur, B: int, d_deltaP, stream=None):
+    _check(lib().salicache_diff_score(ctx.handle, _ptr(d_prev), _ptr(d_cur), B, _ptr(d_deltaP), _stream(stream)),
+           "salicache_diff_score")
 
 
 def salicache_saliency(ctx: Context, d_frames, B: int, d_s, d_skip=None, stream=None):

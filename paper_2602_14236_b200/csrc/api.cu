@@ -198,6 +198,33 @@ int salicache_flow_score(salicache_ctx* c, const uint8_t* d_prev, const uint8_t*
     return SALICACHE_OK;
 }
 
+int salicache_diff_score(salicache_ctx* c, const uint8_t* d_prev, const uint8_t* d_cur, int B, float* d_deltaP,
+                         void* cuda_stream) {
+    if (!c || !d_prev || !d_cur || !d_deltaP) return SALICACHE_E_NULL;
+    if (B < 0 || B > c->p.max_batch) return SALICACHE_E_SHAPE;
+    if (!aligned16(d_prev) || !aligned16(d_cur) || !aligned16(d_deltaP)) return SALICACHE_E_ALIGN;
+    if (B == 0) return SALICACHE_OK;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const size_t fb = (size_t)c->p.H * c->p.W * 3;
+    int rc = sc_diff_score(c, c->plane[0], d_prev, d_cur, fb, B, d_deltaP, st);
+    if (rc != SALICACHE_OK || c->n_planes == 1) return rc;
+    // anyres base image: 2x2 box mean of both frames of every pair, in passes that fit the base buffer
+    const size_t fbb = fb / 4;
+    uint8_t* base = c->base_frames;
+    for (int b0 = 0; b0 < B;) {
+        int nb = (c->p.max_batch + 1) / 2;
+        if (nb > B - b0) nb = B - b0;
+        rc = sc_box_down2(d_prev + (size_t)b0 * fb, c->p.H, c->p.W, nb, base, st);
+        if (rc == SALICACHE_OK) rc = sc_box_down2(d_cur + (size_t)b0 * fb, c->p.H, c->p.W, nb, base + (size_t)nb * fbb, st);
+        c->launches += 2;
+        if (rc == SALICACHE_OK)
+            rc = sc_diff_score(c, c->plane[1], base, base + (size_t)nb * fbb, fbb, nb, d_deltaP + (size_t)b0 * c->n_tok, st);
+        if (rc != SALICACHE_OK) return rc;
+        b0 += nb;
+    }
+    return SALICACHE_OK;
+}
+
 int salicache_frame_redundancy(salicache_ctx* c, const float* d_deltaP, int B, int first_has_no_prev,
                                uint8_t* d_frame_redundant, void* cuda_stream) {
     if (!c || !d_frame_redundant) return SALICACHE_E_NULL;

@@ -56,6 +56,8 @@ struct salicache_ctx {
 // flow.cu
 int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, const uint8_t* d_cur, size_t frame_bytes,
                   int B, bool sequence, float* d_deltaP, double* d_flow_or_null, cudaStream_t st);
+int sc_diff_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, const uint8_t* d_cur, size_t frame_bytes,
+                  int B, float* d_deltaP, cudaStream_t st);
 // saliency.cu
 int sc_saliency(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_frames, size_t frame_bytes, int B, float* d_s,
                 const uint8_t* d_skip, cudaStream_t st);

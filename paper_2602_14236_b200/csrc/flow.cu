@@ -456,6 +456,46 @@ void launch_update(dim3 grid, cudaStream_t st, int flags, const float* gin, size
 #undef SC_UPD
 }
 
+// ---- Eq. 5 read literally: dP_i = L2 norm of the pixel difference over patch i, normalised by the patch's
+// 3 * 14 * 14 values so that it is an RMS in grey levels.  One CTA per (band of 14 image rows, frame pair):
+// both bands are read once with 16-byte loads, squared byte differences are summed exactly in integers
+// (a 16-byte chunk straddles at most two patches: 42 bytes per patch row), one shared-memory counter per patch.
+constexpr int DIFF_THREADS = 256;
+__global__ void __launch_bounds__(DIFF_THREADS)
+k_diff_score(const uint8_t* __restrict__ prev, const uint8_t* __restrict__ cur, size_t frame_bytes, PlaneGeom g,
+             float* __restrict__ dP) {
+    __shared__ unsigned int acc[64];                          // patches per band (<= 48)
+    const int f = blockIdx.y, py = blockIdx.x;
+    const int row_bytes = g.W * 3, chunks = row_bytes / 16;   // W is a multiple of 16
+    for (int i = threadIdx.x; i < g.gw; i += DIFF_THREADS) acc[i] = 0;
+    __syncthreads();
+    const uint8_t* a = prev + (size_t)f * frame_bytes + (size_t)py * 14 * row_bytes;
+    const uint8_t* b = cur + (size_t)f * frame_bytes + (size_t)py * 14 * row_bytes;
+    for (int i = threadIdx.x; i < 14 * chunks; i += DIFF_THREADS) {
+        const int r = i / chunks, k = i - r * chunks;
+        const uint4 va = __ldg(reinterpret_cast<const uint4*>(a + (size_t)r * row_bytes) + k);
+        const uint4 vb = __ldg(reinterpret_cast<const uint4*>(b + (size_t)r * row_bytes) + k);
+        const int b0 = 16 * k, p0 = b0 / 42;
+        const int m = 42 * (p0 + 1) - b0;                     // bytes of this chunk that belong to patch p0 (>= 1)
+        const uint32_t wa[4] = {va.x, va.y, va.z, va.w}, wb[4] = {vb.x, vb.y, vb.z, vb.w};
+        unsigned int lo = 0, hi = 0;
+#pragma unroll
+        for (int w4 = 0; w4 < 4; ++w4) {
+            const uint32_t d = __vabsdiffu4(wa[w4], wb[w4]);
+            const int n = m - 4 * w4;                         // bytes of this word in patch p0
+            const uint32_t mask = n >= 4 ? 0xffffffffu : (n <= 0 ? 0u : ((1u << (8 * n)) - 1u));
+            const uint32_t dl = d & mask, dh = d & ~mask;
+            lo = __dp4a(dl, dl, lo);
+            hi = __dp4a(dh, dh, hi);
+        }
+        atomicAdd(&acc[p0], lo);
+        if (hi) atomicAdd(&acc[p0 + 1], hi);
+    }
+    __syncthreads();
+    for (int px = threadIdx.x; px < g.gw; px += DIFF_THREADS)
+        dP[(size_t)f * g.n_tok + patch_token(g, py, px)] = (float)sqrt((double)acc[px] / (double)(3 * 14 * 14));
+}
+
 inline unsigned blocks_for(long long n, int threads) { return (unsigned)((n + threads - 1) / threads); }
 
 }  // namespace
@@ -463,6 +503,16 @@ inline unsigned blocks_for(long long n, int threads) { return (unsigned)((n + th
 int sc_flow_init() {
     int rc = init_update<56>();
     return rc != SALICACHE_OK ? rc : init_update<28>();
+}
+
+int sc_diff_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, const uint8_t* d_cur, size_t frame_bytes,
+                  int B, float* d_deltaP, cudaStream_t st) {
+    if (B == 0) return SALICACHE_OK;
+    dim3 grid(g.gh, B);
+    k_diff_score<<<grid, DIFF_THREADS, 0, st>>>(d_prev, d_cur, frame_bytes, g, d_deltaP);
+    c->launches++;
+    SC_CHECK(cudaGetLastError());
+    return SALICACHE_OK;
 }
 
 int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, const uint8_t* d_cur, size_t frame_bytes,

@@ -175,3 +175,21 @@ def test_workload_3_full_shape_in_the_benchmark_launch_configuration():
     assert np.array_equal(pools.int4_codes.cpu().numpy(), ref.int4_codes)
     assert np.array_equal(pools.int4_sz.cpu().numpy().view(np.uint16), ref.int4_sz)
     assert np.array_equal(pools.fp16_pool.cpu().numpy().view(np.uint16), ref.fp16_pool)
+
+
+def test_literal_eq5_difference_score_matches_the_oracle():
+    """The frame-difference reading of Eq. 5: exact integer sums, so the float32 scores are the oracle's, rounded."""
+    import torch
+    for wl, kw in ((1, {}), (3, {}), (4, dict(H=672, W=672, n_images=5))):
+        fr = synth.frames(wl, T=4, t0=118 if wl == 3 else 1)
+        ctx = sc.Context(sc.salicache_default_params(max_batch=4, chunk_frames=2, L=1, **kw))
+        d = torch.from_numpy(fr).cuda()
+        dP = torch.full((3, ctx.n_tok), -1.0, dtype=torch.float32, device="cuda")
+        sc.salicache_diff_score(ctx, d[:-1], d[1:], 3, dP)
+        torch.cuda.synchronize()
+        want = oracle.diff_score(fr[:-1], fr[1:])
+        if wl == 4:
+            base = np.stack([oracle.box_down2(f) for f in fr])
+            wb = oracle.diff_score(base[:-1], base[1:])
+            want = np.stack([_anyres_tokens(want[t], wb[t]) for t in range(3)])
+        assert np.array_equal(dP.cpu().numpy(), want.astype(np.float32)), wl

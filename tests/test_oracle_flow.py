@@ -223,3 +223,23 @@ def test_flow_score_batch_matches_single_calls():
     dP = oracle.flow_score(fr[:-1], fr[1:])
     for b in range(2):
         assert np.array_equal(dP[b], oracle.delta_p(oracle.flow(fr[b], fr[b + 1]), 14))
+
+
+def test_literal_eq5_frame_difference_score():
+    """Eq. 5 as printed: closed forms and the library norm."""
+    rng = np.random.default_rng(2)
+    a = rng.integers(0, 256, (1, 28, 42, 3)).astype(np.uint8)
+    assert np.array_equal(oracle.diff_score(a, a), np.zeros((1, 6)))
+    b = np.clip(a.astype(int), 0, 250).astype(np.uint8)
+    assert np.allclose(oracle.diff_score(b, b + 5), 5.0, atol=1e-12)                 # uniform offset k -> k
+    c = a.copy()
+    c[0, 3, 20, 1] = np.uint8((int(a[0, 3, 20, 1]) + 100) % 256)                     # one value in patch (0, 1)
+    d = abs(int(c[0, 3, 20, 1]) - int(a[0, 3, 20, 1]))
+    got = oracle.diff_score(a, c)[0]
+    assert got[1] == pytest.approx(d / np.sqrt(588.0), abs=1e-12) and got[[0, 2, 3, 4, 5]].max() == 0.0
+    e = rng.integers(0, 256, (1, 28, 42, 3)).astype(np.uint8)
+    diff = e.astype(np.float64) - a.astype(np.float64)
+    want = [np.linalg.norm(diff[0, 14 * py:14 * py + 14, 14 * px:14 * px + 14]) / np.sqrt(588.0)
+            for py in range(2) for px in range(3)]
+    assert np.allclose(oracle.diff_score(a, e)[0], want, rtol=1e-13)
+    assert np.allclose(oracle.diff_score(e, a), oracle.diff_score(a, e))             # symmetric
