@@ -263,12 +263,13 @@ def run_ours(args):
     pack_s = pack_ms / 1e3
     achieved = (rd + wr) * args.steps / pack_s / 1e9 if pack_s > 0 else 0.0
     roofline = {"kernel": "k_pack", "bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
-                "frac": round(achieved / peak, 4), "peak_source": peak_src,
+                "frac": round(achieved / peak, 4), "peak_source": peak_src, "frac_of_nominal_8000": round(achieved / 8000.0, 4),
                 "traffic": (None if NCU_TRAFFIC_RATIO is None else int(NCU_TRAFFIC_RATIO * (rd + wr) / n_chunks)),
                 "algorithmic_bytes_per_launch": int((rd + wr) / n_chunks), "launches_per_step": n_chunks,
                 "avg_launch_ms": round(pack_ms / pack_launches, 4),
                 "pack_ms_per_step": round(pack_ms / args.steps, 3), "filter_ms_per_step": round(filt_ms / args.steps, 3),
-                "pipeline_frac_of_peak": round((rd + wr) / (ms_per_step / 1e3) / 1e9 / peak, 4)}
+                "pipeline_frac_of_peak": round((rd + wr) / (ms_per_step / 1e3) / 1e9 / peak, 4),
+                "pipeline_frac_of_nominal_8000": round((rd + wr) / (ms_per_step / 1e3) / 1e9 / 8000.0, 4)}
 
     if rank != 0:
         if world > 1:
@@ -278,7 +279,8 @@ def run_ours(args):
     # ---- end to end: host buffers in, decisions out; copies inside the timed region (single rank)
     cpu = None
     if not args.no_cpu and world == 1:
-        cpu = cpu_baseline(args, wl, T, frames_np, Kring, Vring, th)
+        cpu = cpu_baseline(args, wl, T, frames_np, Kring, Vring, th,
+                           gpu=(dP.cpu().numpy(), s.cpu().numpy(), dec.cpu().numpy(), red.cpu().numpy()))
     e2e = None
     if not args.no_e2e:
         e2e = run_e2e(args, sc, ctx, wl, T, frames_np, Kring, Vring, pools, dev,
@@ -341,6 +343,11 @@ def run_extras(sc, synth, ctx, wl, T, frames, dP, dev, peak):
         out["diff_score"] = {"what": "Eq. 5 read literally (RMS pixel difference per patch), all frame pairs",
                              "ms": round(ms, 4), "l2": "flushed between repetitions", "algorithmic_GBps": round(nbytes / ms / 1e6, 1),
                              "frac_of_hbm_peak": round(nbytes / ms / 1e6 / peak, 4)}
+        ms = timed(lambda: sc.salicache_flow_score(ctx, frames[:-1], frames[1:], T - 1, d2[1:]), reps=5)
+        gflop = 0.13 * (T - 1) * (wl.H * wl.W) / (336 * 336)      # about 0.13 GFLOP per 336x336 pair
+        out["flow_score"] = {"what": "dense flow + patch scores, all frame pairs", "ms": round(ms, 3),
+                             "us_per_pair": round(1e3 * ms / (T - 1), 2), "algorithmic_TFLOPs": round(gflop / ms, 2),
+                             "fp32_peak_TFLOPs_nominal": 74.0, "note": "bound by L1 / shared memory and HBM, not by the ALUs"}
     # Fig. 3 style breakdown: workload 2 frames under the four-tier rule
     wl2 = synth.WORKLOADS[2]
     p2 = sc.salicache_default_params(max_batch=wl2.T, chunk_frames=wl2.T, L=1, **synth.thresholds("four"))
@@ -455,23 +462,45 @@ def _oracle_sample(wl, T, frames_np, Kring_h, Vring_h, th, sample):
     pools = oracle.Pools(wl.L, wl.HD, 128, caps, caps, caps)
     off = np.zeros(3, np.int64)
     stored = 0
+    decs, reds = [], []
     for i, t in enumerate(sample):
         d, idx, counts, r, _ = oracle.select(dP[i], s[i], t > 0, p)
+        decs.append(d)
+        reds.append(r)
         slot = t % Kring_h.shape[0]
         oracle.pack_frame(Kring_h[slot], Vring_h[slot], idx, counts, off, pools)
         off += counts[[4, 3, 2]]
         stored += int(counts[[4, 3, 2]].sum())
-    return time.perf_counter() - t0, stored
+    return time.perf_counter() - t0, stored, (dP, s, np.stack(decs), np.array(reds), p)
 
 
-def cpu_baseline(args, wl, T, frames_np, Kring, Vring, th):
+def cpu_baseline(args, wl, T, frames_np, Kring, Vring, th, gpu=None):
+    """Times the oracle on a sample of the workload and, with the device's scores and decisions of the same
+    frames at hand, reports how they compare (the parity tests do this with assertions; this is the full-size
+    record: worst score error over its tolerance, tokens within 1e-4 of a threshold, decisions that differ)."""
     import oracle
     n = min(args.cpu_sample, T)
     sample = sorted(set(int(round(x)) for x in np.linspace(0, T - 1, n)))
-    Kh = Kring.cpu().numpy().view(np.uint16)
-    Vh = Vring.cpu().numpy().view(np.uint16)
-    secs, stored = _oracle_sample(wl, T, frames_np, Kh, Vh, th, sample)
-    return {"value": round(len(sample) / secs, 4), "unit": "frames/s", "cores": oracle.num_threads(), "kind": "oracle",
+    Kh = Kring[:8].cpu().numpy().view(np.uint16)      # K/V values are i.i.d.: eight slabs serve every sampled frame
+    Vh = Vring[:8].cpu().numpy().view(np.uint16)
+    secs, stored, (o_dP, o_s, o_dec, o_red, p) = _oracle_sample(wl, T, frames_np, Kh, Vh, th, sample)
+    parity = None
+    if gpu is not None:
+        g_dP, g_s, g_dec, g_red = (x[sample] for x in gpu)
+        ratio = lambda g, r: float((np.abs(g.astype(np.float64) - r) / (1e-6 + 1e-4 * np.abs(r))).max()) if r.size else 0.0
+        has_prev = np.array([t > 0 for t in sample])
+        scored = o_red == 0
+        near = np.zeros(o_s.shape, bool)
+        for tau in (p.tau_high, p.tau_med, p.tau_low):
+            near |= np.abs(o_s - tau) <= 1e-4 * abs(tau)
+        near |= (np.abs(o_dP - p.tau_t) <= 1e-4 * p.tau_t) & has_prev[:, None]
+        diff = g_dec != o_dec
+        parity = {"frames_compared": len(sample), "dP_error_over_tolerance": round(ratio(g_dP[has_prev], o_dP[has_prev]), 4),
+                  "s_error_over_tolerance": round(ratio(g_s[scored], o_s[scored]), 4),
+                  "tokens_near_a_threshold": int(near.sum()), "decisions_differing": int(diff.sum()),
+                  "decisions_differing_away_from_thresholds": int((diff & ~near).sum()),
+                  "frame_redundancy_flags_differing": int((g_red != o_red).sum())}
+    return {"parity_vs_oracle": parity, "value": round(len(sample) / secs, 4), "unit": "frames/s", "cores": oracle.num_threads(), "kind": "oracle",
             "sample": f"{len(sample)} evenly spaced frames ({sample[0]}, {sample[1] if len(sample) > 1 else sample[0]}, ..., {sample[-1]}) of the {T}-frame workload "
                       f"({stored} stored token rows x {2 * wl.L} planes), {secs:.1f} s",
             "seconds": round(secs, 2)}
@@ -496,7 +525,7 @@ def run_reference(args):
     sample = sorted(set(int(round(x)) for x in np.linspace(0, T - 1, n)))
     times = []
     for k in range(args.warmup + args.steps):
-        secs, stored = _oracle_sample(wl, T, frames_np, Kh, Vh, th, sample)
+        secs, stored, _ = _oracle_sample(wl, T, frames_np, Kh, Vh, th, sample)
         if k >= args.warmup:
             times.append(secs)
     secs = float(np.mean(times))
