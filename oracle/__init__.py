@@ -332,6 +332,20 @@ def unpack_frame(n_tok: int, idx, counts, decision, off, pools: Pools, zero_fill
         C.c_int(int(zero_fill_pruned)), _p(K_out), _p(V_out)))
 
 
+def attend(q16: np.ndarray, pools: "Pools", n_rows) -> np.ndarray:
+    """Decode attention over the rows the pools hold (n_rows = rows used in the FP16, INT8, INT4 pool).
+    q16: fp16 bits [L][H][D].  Returns float64 [L][H][D]."""
+    q16 = _c(q16, np.uint16)
+    L, H, D = q16.shape
+    out = np.empty((L, H, D), np.float64)
+    n16, n8, n4 = (int(x) for x in n_rows)
+    lib().oracle_attend(_p(q16), C.c_int(L), C.c_int(H), C.c_int(D), C.c_int(pools.G), _p(pools.fp16_pool),
+                        C.c_int64(pools.cap16), C.c_int64(n16), _p(pools.int8_codes), _p(pools.int8_scale),
+                        C.c_int64(pools.cap8), C.c_int64(n8), _p(pools.int4_codes), _p(pools.int4_sz),
+                        C.c_int64(pools.cap4), C.c_int64(n4), _p(out))
+    return out
+
+
 def stored_bytes(counts_all: np.ndarray, L: int, HD: int, G: int, n_tok: int) -> int:
     """Bytes the mixed-precision store holds for frames with the given per-code counts [T][5]
     (Eq. 3 applied per tier, plus all metadata: scales/zeros, index lists, decision bytes,

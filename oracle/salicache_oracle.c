@@ -754,3 +754,67 @@ EXPORT int oracle_unpack_frame(int L, int n_tok, int HD, int G, const int32_t* i
         }
     return status;
 }
+
+/* ------------------------------------------------------------------------- */
+/* Decode attention over the mixed-precision store with just-in-time           */
+/* dequantisation (Eq. 2; Sec. III-C: dequantisation happens inside the        */
+/* attention computation).  One query vector per layer and head; the keys and  */
+/* values are the rows the store holds: rows [0, n16) of the FP16 pool, [0, n8)*/
+/* of the INT8 pool, [0, n4) of the INT4 pool (pruned tokens have no row).     */
+/*   score_j = q_h . K^_{j,h} / sqrt(D),  p = softmax_j(score),                */
+/*   out_h   = sum_j p_j V^_{j,h}                                              */
+/* with K^, V^ the dequantised values in exact arithmetic (q * s, q * s + z:   */
+/* no rounding to binary16 in between, as in a fused kernel), everything in    */
+/* double.  q: fp16 bits [L][H][D]; out: double [L][H][D]; zero rows -> zeros. */
+/* ------------------------------------------------------------------------- */
+static double pool_value(int tier, size_t prow, int h, int d, int HD, int D, int G, const uint16_t* fp16_pool,
+                         const int8_t* int8_codes, const uint16_t* int8_scale, const uint8_t* int4_codes,
+                         const uint16_t* int4_sz) {
+    int e = h * D + d, ng = HD / G;
+    if (tier == 0) return (double)oracle_half_to_float(fp16_pool[prow * HD + e]);
+    if (tier == 1)
+        return (double)int8_codes[prow * HD + e] * (double)oracle_half_to_float(int8_scale[prow * ng + e / G]);
+    uint8_t byte = int4_codes[prow * (HD / 2) + e / 2];
+    int q = (e & 1) ? (byte >> 4) : (byte & 15);
+    return (double)q * (double)oracle_half_to_float(int4_sz[(prow * ng + e / G) * 2]) +
+           (double)oracle_half_to_float(int4_sz[(prow * ng + e / G) * 2 + 1]);
+}
+
+EXPORT void oracle_attend(const uint16_t* q, int L, int H, int D, int G, const uint16_t* fp16_pool, int64_t cap16,
+                          int64_t n16, const int8_t* int8_codes, const uint16_t* int8_scale, int64_t cap8, int64_t n8,
+                          const uint8_t* int4_codes, const uint16_t* int4_sz, int64_t cap4, int64_t n4, double* out) {
+    int HD = H * D;
+    int64_t caps[3] = {cap16, cap8, cap4}, ns[3] = {n16, n8, n4};
+    int64_t R = n16 + n8 + n4;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int l = 0; l < L; ++l)
+        for (int h = 0; h < H; ++h) {
+            double* o = out + ((size_t)l * H + h) * D;
+            for (int d = 0; d < D; ++d) o[d] = 0.0;
+            if (R == 0) continue;
+            double* sc = (double*)malloc((size_t)R * sizeof(double));
+            double mx = -INFINITY;
+            int64_t j = 0;
+            for (int t = 0; t < 3; ++t)
+                for (int64_t r = 0; r < ns[t]; ++r, ++j) {
+                    size_t prow = (size_t)(2 * l) * caps[t] + r;            /* K plane of layer l */
+                    double dot = 0.0;
+                    for (int d = 0; d < D; ++d)
+                        dot += (double)oracle_half_to_float(q[((size_t)l * H + h) * D + d]) *
+                               pool_value(t, prow, h, d, HD, D, G, fp16_pool, int8_codes, int8_scale, int4_codes, int4_sz);
+                    sc[j] = dot / sqrt((double)D);
+                    if (sc[j] > mx) mx = sc[j];
+                }
+            double den = 0.0;
+            for (j = 0; j < R; ++j) { sc[j] = exp(sc[j] - mx); den += sc[j]; }
+            j = 0;
+            for (int t = 0; t < 3; ++t)
+                for (int64_t r = 0; r < ns[t]; ++r, ++j) {
+                    size_t prow = (size_t)(2 * l + 1) * caps[t] + r;        /* V plane */
+                    double p = sc[j] / den;
+                    for (int d = 0; d < D; ++d)
+                        o[d] += p * pool_value(t, prow, h, d, HD, D, G, fp16_pool, int8_codes, int8_scale, int4_codes, int4_sz);
+                }
+            free(sc);
+        }
+}
