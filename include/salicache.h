@@ -259,6 +259,22 @@ SALICACHE_API int salicache_unpack_kv(salicache_ctx* ctx, const salicache_pools*
 SALICACHE_API int salicache_saliency_noalloc(const salicache_params* p, const uint8_t* d_frames, int B, float* d_s,
                                              int32_t* d_status_or_null, void* cuda_stream);
 
+/*
+ * Decode attention straight from the mixed-precision store (Eq. 2 with the just-in-time dequantisation of
+ * Sec. III-C fused in): for every layer l and head h,
+ *   score_j = q[l][h] . K^_j / sqrt(head_dim),  p = softmax_j(score),  out[l][h] = sum_j p_j V^_j,
+ * over the rows j the pools hold: rows [0, min(fill, cap)) of the FP16, INT8 and INT4 pool (pruned tokens
+ * have no row; a reused token is attended through the row it points to, once).  K^, V^ are the dequantised
+ * values q*s and q*s + zero in single precision, not rounded to binary16 in between.
+ *   d_q     DEVICE f16 [L][heads][head_dim], 16-byte aligned
+ *   pools   as for salicache_pack_kv;  d_fill DEVICE i64 [3]: rows written per pool (salicache_select's d_fill)
+ *   d_out   DEVICE f32 [L][heads][head_dim], written; zeros when the store is empty
+ * Needs head_dim == 128 and group == 128 or heads*head_dim (E_PARAM otherwise); pool capacities below 2^28
+ * rows.  Errors: E_NULL, E_ALIGN, E_PARAM, E_SHAPE, E_CUDA.
+ */
+SALICACHE_API int salicache_attend(salicache_ctx* ctx, const void* d_q, const salicache_pools* pools, const int64_t* d_fill,
+                                   float* d_out, void* cuda_stream);
+
 /* Synchronises `cuda_stream`, returns the deferred device status (0, E_CAPACITY or
  * E_NOCONVERGE; E_CUDA if the stream reports an error) and clears it. */
 SALICACHE_API int salicache_poll_status(salicache_ctx* ctx, void* cuda_stream);

@@ -49,7 +49,7 @@ EXPORTS = [
     "salicache_default_params", "salicache_create", "salicache_destroy", "salicache_strerror",
     "salicache_tokens_per_frame", "salicache_launch_count", "salicache_flow_score", "salicache_saliency", "salicache_select",
     "salicache_pack_kv", "salicache_unpack_kv", "salicache_poll_status", "salicache_saliency_noalloc",
-    "salicache_frame_redundancy", "salicache_source_frames", "salicache_diff_score",
+    "salicache_frame_redundancy", "salicache_source_frames", "salicache_diff_score", "salicache_attend",
 ]
 
 _lib = None
@@ -84,6 +84,7 @@ def lib():
         _lib.salicache_pack_kv.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, C.POINTER(Pools), vp]
         _lib.salicache_unpack_kv.argtypes = [vp, C.POINTER(Pools), vp, vp, vp, vp, i32, i32, vp, vp, i64, vp]
         _lib.salicache_poll_status.argtypes = [vp, vp]
+        _lib.salicache_attend.argtypes = [vp, vp, C.POINTER(Pools), vp, vp, vp]
         _lib.salicache_saliency_noalloc.argtypes = [C.POINTER(Params), vp, i32, vp, vp, vp]
     return _lib
 
@@ -196,6 +197,11 @@ def salicache_unpack_kv(ctx: Context, pools: Pools, d_idx, d_counts, d_decision,
     _check(lib().salicache_unpack_kv(ctx.handle, C.byref(pools), _ptr(d_idx), _ptr(d_counts), _ptr(d_decision),
                                      _ptr(d_row_offset), B, int(zero_fill_pruned), _ptr(d_K_out), _ptr(d_V_out),
                                      frame_stride, _stream(stream)), "salicache_unpack_kv")
+
+
+def salicache_attend(ctx: Context, d_q, pools: Pools, d_fill, d_out, stream=None):
+    _check(lib().salicache_attend(ctx.handle, _ptr(d_q), C.byref(pools), _ptr(d_fill), _ptr(d_out), _stream(stream)),
+           "salicache_attend")
 
 
 def salicache_poll_status(ctx: Context, stream=None) -> int:

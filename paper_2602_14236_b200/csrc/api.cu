@@ -28,6 +28,7 @@ void free_scratch(salicache_ctx* c) {
     if (c->lut) cudaFree(c->lut);
     if (c->base_frames) cudaFree(c->base_frames);
     if (c->row_prefix) cudaFree(c->row_prefix);
+    if (c->attend_ws) cudaFree(c->attend_ws);
     if (c->d_status) cudaFree(c->d_status);
 }
 
@@ -122,6 +123,7 @@ int salicache_create(salicache_ctx** out, const salicache_params* p) {
     ok = ok && cudaMalloc(&c->lut, 256 * sizeof(double)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->row_prefix, ((size_t)p->max_batch + 1) * sizeof(int64_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_status, sizeof(int)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->attend_ws, sc_attend_workspace_bytes(p->L, p->heads)) == cudaSuccess;
     if (ok && p->n_images == 5)
         ok = cudaMalloc(&c->base_frames, ((size_t)p->max_batch + 1) * (P0 / 4) * 3) == cudaSuccess;
     if (!ok) {
@@ -303,6 +305,15 @@ int salicache_unpack_kv(salicache_ctx* c, const salicache_pools* pools, const in
     if (!aligned16(d_K_out) || !aligned16(d_V_out)) return SALICACHE_E_ALIGN;
     return sc_unpack(c, pools, d_idx, d_counts, d_decision, d_row_offset, B, zero_fill_pruned, d_K_out, d_V_out,
                      frame_stride, (cudaStream_t)cuda_stream);
+}
+
+int salicache_attend(salicache_ctx* c, const void* d_q, const salicache_pools* pools, const int64_t* d_fill, float* d_out,
+                     void* cuda_stream) {
+    if (!c || !d_q || !d_fill || !d_out) return SALICACHE_E_NULL;
+    int rc = check_pools(pools);
+    if (rc != SALICACHE_OK) return rc;
+    if (!aligned16(d_q) || !aligned16(d_out)) return SALICACHE_E_ALIGN;
+    return sc_attend(c, d_q, pools, d_fill, d_out, (cudaStream_t)cuda_stream);
 }
 
 int salicache_poll_status(salicache_ctx* c, void* cuda_stream) {

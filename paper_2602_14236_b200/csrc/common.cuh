@@ -48,6 +48,7 @@ struct salicache_ctx {
     uint8_t* base_frames;      // anyres only: [chunk+1][336*336*3]
     // select / pack scratch
     int64_t* row_prefix;       // [max_batch+1] stored rows before each frame of the batch
+    float* attend_ws;          // partial attention results [L][heads][64][head_dim + 2]
     int* d_status;             // deferred status word
     int sm_count;
     long long launches;        // kernels launched through this context so far
@@ -70,6 +71,10 @@ int sc_sources(salicache_ctx* c, const uint8_t* d_decision, int B, int first_fra
                cudaStream_t st);
 int sc_frame_redundancy(salicache_ctx* c, const float* d_deltaP, int B, int first_has_no_prev, uint8_t* d_frame_redundant,
                         cudaStream_t st);
+// attend.cu
+size_t sc_attend_workspace_bytes(int L, int H);
+int sc_attend(salicache_ctx* c, const void* d_q, const salicache_pools* pools, const int64_t* d_fill, float* d_out,
+              cudaStream_t st);
 // kv.cu
 int sc_pack(salicache_ctx* c, const void* d_K, const void* d_V, int64_t frame_stride, const int32_t* d_idx,
             const int32_t* d_counts, const int64_t* d_row_offset, int B, const salicache_pools* pools, cudaStream_t st);

@@ -1,0 +1,101 @@
+"""GPU parity of the decode attention with fused dequantisation against the oracle, through the C ABI.
+
+Tolerance: the device accumulates 128-term dot products and up to tens of thousands of weighted rows in
+binary32; with |q|, |k|, |v| ~ 1 the scores carry an absolute error of a few 1e-6, the softmax weights the
+same relative error, and the outputs stay within 2e-5 + 1e-4 |out| of the double-precision oracle."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2602_14236_b200 import binding as sc
+from paper_2602_14236_b200 import synth
+
+import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+ATOL, RTOL = 2e-5, 1e-4
+
+
+def _store(L, heads, T, background, group=128, seed=0, s_lo=0.0):
+    """Random scores -> decisions -> pools on both sides (the pools are bit-identical, checked elsewhere)."""
+    import torch
+    HD, n_tok = heads * 128, 576
+    ctx = sc.Context(sc.salicache_default_params(max_batch=8, chunk_frames=4, L=L, heads=heads, group=group,
+                                                 **synth.thresholds(background)))
+    rng = np.random.default_rng(seed)
+    s = rng.uniform(s_lo, 0.6, (T, n_tok)).astype(np.float32)
+    out = gu.gpu_select(ctx, None, s, first_has_no_prev=False)
+    counts = out["counts"].cpu().numpy()
+    caps = tuple(int(c) + 3 for c in counts[:, [4, 3, 2]].sum(axis=0))
+    K = rng.standard_normal((T, L, n_tok, HD)).astype(np.float16)
+    V = rng.standard_normal((T, L, n_tok, HD)).astype(np.float16)
+    pools = sc.PoolSet(L, HD, *caps, G=group)
+    sc.salicache_pack_kv(ctx, torch.from_numpy(K).cuda(), torch.from_numpy(V).cuda(), L * n_tok * HD, out["idx"],
+                         out["counts"], out["row_offset"], T, pools.c)
+    torch.cuda.synchronize()
+    ref = oracle.Pools(L, HD, group, *caps)
+    g = lambda t: t.cpu().numpy()
+    ref.fp16_pool[:] = g(pools.fp16_pool).view(np.uint16)
+    ref.int8_codes[:] = g(pools.int8_codes)
+    ref.int8_scale[:] = g(pools.int8_scale).view(np.uint16)
+    ref.int4_codes[:] = g(pools.int4_codes)
+    ref.int4_sz[:] = g(pools.int4_sz).view(np.uint16)
+    return ctx, pools, ref, out["fill"], rng
+
+
+def _check(ctx, pools, ref, fill, q):
+    import torch
+    L, H, D = q.shape
+    d_out = torch.full((L, H, D), 7.0, dtype=torch.float32, device="cuda")
+    sc.salicache_attend(ctx, torch.from_numpy(q).cuda(), pools.c, fill, d_out)
+    torch.cuda.synchronize()
+    n = np.minimum(fill.cpu().numpy(), [ref.cap16, ref.cap8, ref.cap4])
+    want = oracle.attend(q.view(np.uint16), ref, n)
+    got = d_out.cpu().numpy().astype(np.float64)
+    err = np.abs(got - want)
+    assert (err <= ATOL + RTOL * np.abs(want)).all(), f"worst {err.max():.3e} at |out| {np.abs(want).ravel()[err.argmax()]:.3e}"
+    return got, want
+
+
+@pytest.mark.parametrize("background,group", [("four", 128), ("int4", 128), ("int8", 128), ("four", 4096)])
+def test_attention_over_all_tiers_matches_the_oracle(background, group):
+    ctx, pools, ref, fill, rng = _store(L=2, heads=32, T=3, background=background, group=group, seed=3)
+    q = rng.standard_normal((2, 32, 128)).astype(np.float16)
+    _check(ctx, pools, ref, fill, q)
+    # a peaked query: one row dominates the softmax
+    k0 = ref.fp16_pool.view(np.float16)[:, 0, 0].reshape(2, 32, 128)
+    _check(ctx, pools, ref, fill, (4 * k0).astype(np.float16))
+
+
+def test_attention_edge_cases():
+    import torch
+    ctx, pools, ref, fill, rng = _store(L=1, heads=8, T=1, background="four", seed=5)
+    q = rng.standard_normal((1, 8, 128)).astype(np.float16)
+    # an empty store gives zeros
+    zero = torch.zeros(3, dtype=torch.int64, device="cuda")
+    got, _ = _check(ctx, pools, ref, zero, q)
+    assert (got == 0).all()
+    # a single row returns that row's values (exactly: the weight is 1)
+    one = torch.tensor([1, 0, 0], dtype=torch.int64, device="cuda")
+    got, want = _check(ctx, pools, ref, one, q)
+    assert np.array_equal(got, want)
+    # fewer rows than chunks, a zero query (uniform weights), a fill beyond the capacity (ring pools hold cap rows)
+    few = torch.tensor([3, 5, 2], dtype=torch.int64, device="cuda")
+    _check(ctx, pools, ref, few, q)
+    _check(ctx, pools, ref, fill, np.zeros_like(q))
+    over = fill + 10 ** 6
+    _check(ctx, pools, ref, over, q)
+    lib = sc.lib()
+    import ctypes
+    assert lib.salicache_attend(ctx.handle, None, ctypes.byref(pools.c), fill.data_ptr(), 16, None) == sc.E_NULL
+    bad = sc.Context(sc.salicache_default_params(L=1, heads=16, head_dim=256))
+    d = torch.zeros(16, 256, dtype=torch.float32, device="cuda")
+    assert lib.salicache_attend(bad.handle, d.data_ptr(), ctypes.byref(pools.c), fill.data_ptr(), d.data_ptr(), None) == sc.E_PARAM
+
+
+def test_attention_at_the_benchmark_shape():
+    """32 layers x 32 heads over the cache of eight frames of workload 3 (all INT4 but a few FP16 rows)."""
+    ctx, pools, ref, fill, rng = _store(L=32, heads=32, T=2, background="int4", seed=9, s_lo=0.3)
+    q = rng.standard_normal((32, 32, 128)).astype(np.float16)
+    _check(ctx, pools, ref, fill, q)
