@@ -193,3 +193,55 @@ def test_literal_eq5_difference_score_matches_the_oracle():
             wb = oracle.diff_score(base[:-1], base[1:])
             want = np.stack([_anyres_tokens(want[t], wb[t]) for t in range(3)])
         assert np.array_equal(dP.cpu().numpy(), want.astype(np.float32)), wl
+
+
+@pytest.mark.parametrize("wl_index,T,L", [(2, 2, 32), (4, 1, 2)])
+def test_store_on_the_other_workloads_kv(wl_index, T, L):
+    """Workload 2 (32 layers, 1 % of the elements x8: the scale follows the outlier) and workload 4
+    (2880 tokens per frame), INT8 background: pools bit-exact, dequantised values within the target's 1e-3
+    of the oracle's (they are equal) and the INT8 error bound s/2 against the input."""
+    import torch
+    wl = synth.WORKLOADS[wl_index]
+    n_tok, HD = wl.n_tok, wl.HD
+    th = synth.thresholds(wl.background)
+    ctx = sc.Context(sc.salicache_default_params(H=wl.H, W=wl.W, n_images=wl.n_images, max_batch=4, chunk_frames=2, L=L, **th))
+    rng = np.random.default_rng(wl_index)
+    s = rng.uniform(0.2, 0.6, (T, n_tok)).astype(np.float32)
+    out = gu.gpu_select(ctx, None, s, first_has_no_prev=False)
+    counts, idx, off, dec = (out[k].cpu().numpy() for k in ("counts", "idx", "row_offset", "decision"))
+    K = torch.empty((T, L, n_tok, HD), dtype=torch.float16, device="cuda")
+    V = torch.empty_like(K)
+    for t in range(T):
+        k, v = synth.kv_torch(wl_index, t, "cuda", L=L)
+        K[t].copy_(k)
+        V[t].copy_(v)
+    caps = tuple(int(c) + 1 for c in counts[:, [4, 3, 2]].sum(axis=0))
+    pools = sc.PoolSet(L, HD, *caps)
+    sc.salicache_pack_kv(ctx, K, V, L * n_tok * HD, out["idx"], out["counts"], out["row_offset"], T, pools.c)
+    gK = torch.zeros_like(K)
+    gV = torch.zeros_like(V)
+    sc.salicache_unpack_kv(ctx, pools.c, out["idx"], out["counts"], out["decision"], out["row_offset"], T, True, gK, gV,
+                           L * n_tok * HD)
+    torch.cuda.synchronize()
+    assert sc.salicache_poll_status(ctx) == 0
+    hK, hV = K.cpu().numpy(), V.cpu().numpy()
+    ref = oracle.Pools(L, HD, 128, *caps)
+    Ko = np.zeros(hK.shape, np.uint16)
+    Vo = np.zeros(hK.shape, np.uint16)
+    for t in range(T):
+        oracle.pack_frame(hK[t].view(np.uint16), hV[t].view(np.uint16), idx[t], counts[t], off[t], ref)
+        oracle.unpack_frame(n_tok, idx[t], counts[t], dec[t], off[t], ref, True, Ko[t], Vo[t])
+    assert counts[:, 3].sum() > 100 and counts[:, 4].sum() > 100
+    assert np.array_equal(pools.int8_codes.cpu().numpy(), ref.int8_codes)
+    assert np.array_equal(pools.int8_scale.cpu().numpy().view(np.uint16), ref.int8_scale)
+    assert np.array_equal(pools.fp16_pool.cpu().numpy().view(np.uint16), ref.fp16_pool)
+    g = gK.cpu().numpy()
+    assert np.array_equal(g.view(np.uint16), Ko) and np.array_equal(gV.cpu().numpy().view(np.uint16), Vo)
+    # error bound of the symmetric quantiser on the INT8 rows of frame 0, layer 0: |x^ - x| <= s/2 + half an fp16 ulp of x^
+    rows = idx[0, 1, :counts[0, 3]]
+    x = hK[0, 0, rows].astype(np.float64).reshape(len(rows), HD // 128, 128)
+    xh = g[0, 0, rows].astype(np.float64).reshape(x.shape)
+    sc8 = ref.int8_scale[0, 0, off[0, 1]:off[0, 1] + len(rows)].view(np.float16).astype(np.float64)
+    assert (np.abs(xh - x) <= sc8[..., None] * (0.5 + 2.0 ** -11) + np.abs(xh) * 2.0 ** -11).all()
+    if wl.outlier_frac:
+        assert np.abs(x).max() > 12.0                      # the x8 outliers are there
