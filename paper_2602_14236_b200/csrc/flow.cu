@@ -22,10 +22,9 @@ __device__ __forceinline__ int clampi(int v, int lo, int hi) { return v < lo ? l
 // three 16-byte loads of the interleaved RGB bytes.
 __global__ void k_gray(const uint8_t* __restrict__ frames, size_t frame_bytes, int n_px, int n_frames,
                        float* __restrict__ out) {
-    int groups = n_px / 16;
-    long long gid = blockIdx.x * (long long)blockDim.x + threadIdx.x;
-    if (gid >= (long long)groups * n_frames) return;
-    int f = (int)(gid / groups), gidx = (int)(gid % groups);
+    const int groups = n_px / 16;
+    const int f = blockIdx.y, gidx = blockIdx.x * blockDim.x + threadIdx.x;      // grid: (groups of a frame, frames)
+    if (gidx >= groups || f >= n_frames) return;
     const uint4* src = reinterpret_cast<const uint4*>(frames + (size_t)f * frame_bytes) + (size_t)gidx * 3;
     uint4 v0 = __ldg(src), v1 = __ldg(src + 1), v2 = __ldg(src + 2);
     uint32_t w[12] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w, v2.x, v2.y, v2.z, v2.w};
@@ -47,9 +46,8 @@ __global__ void k_gray(const uint8_t* __restrict__ frames, size_t frame_bytes, i
 // dyadic rationals with at most 24 significant bits, so float holds them exactly.
 __global__ void k_pyr_down(const float* __restrict__ src, int h, int w, int n_frames, float* __restrict__ dst) {
     int h2 = h / 2, w2 = w / 2;
-    long long gid = blockIdx.x * (long long)blockDim.x + threadIdx.x;
-    if (gid >= (long long)h2 * w2 * n_frames) return;
-    int f = (int)(gid / (h2 * w2)), r = (int)(gid % (h2 * w2));
+    const int f = blockIdx.y, r = blockIdx.x * blockDim.x + threadIdx.x;        // grid: (pixels of a level, frames)
+    if (r >= h2 * w2 || f >= n_frames) return;
     int y = r / w2, x = r % w2;
     const float* s = src + (size_t)f * h * w;
     const float k[5] = {1.f, 4.f, 6.f, 4.f, 1.f};
@@ -236,9 +234,8 @@ k_flow_gh(const float* __restrict__ coef1, const float* __restrict__ coef2, size
           const float* __restrict__ d_coarse, size_t flow_stride, float* __restrict__ gh, size_t gh_stride,
           int n_pairs) {
     const size_t P = (size_t)h * w;
-    long long gid = blockIdx.x * (long long)blockDim.x + threadIdx.x;
-    if (gid >= (long long)P * n_pairs) return;
-    const int f = (int)(gid / P), r = (int)(gid % P);
+    const int f = blockIdx.y, r = blockIdx.x * blockDim.x + threadIdx.x;        // grid: (pixels of the level, pairs)
+    if (r >= (int)P || f >= n_pairs) return;
     const int y = r / w, x = r % w;
     float du = 0.0f, dv = 0.0f;
     if (d_coarse) {
@@ -545,12 +542,12 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
             const uint8_t* src = (part == 0 ? d_prev : d_cur) + (size_t)b0 * frame_bytes;
             int n = sequence ? nf : nb;
             float* dst = c->pyr[0] + (size_t)part * nb * P0;
-            k_gray<<<blocks_for((long long)(P0 / 16) * n, T), T, 0, st>>>(src, frame_bytes, (int)P0, n, dst);
+            k_gray<<<dim3(blocks_for((long long)(P0 / 16), T), n), T, 0, st>>>(src, frame_bytes, (int)P0, n, dst);
             c->launches++;
         }
         for (int l = 1; l < 3; ++l)
-            k_pyr_down<<<blocks_for((long long)hs[l] * ws[l] * nf, T), T, 0, st>>>(c->pyr[l - 1], hs[l - 1], ws[l - 1], nf,
-                                                                                   c->pyr[l]);
+            k_pyr_down<<<dim3(blocks_for((long long)hs[l] * ws[l], T), nf), T, 0, st>>>(c->pyr[l - 1], hs[l - 1], ws[l - 1], nf,
+                                                                                        c->pyr[l]);
         for (int l = 0; l < 3; ++l) {
             dim3 gp((ws[l] + PX - 1) / PX, (hs[l] + PY - 1) / PY, nf);
             k_poly_exp<<<gp, 256, 0, st>>>(c->pyr[l], hs[l], ws[l], nf, pw, c->coef[l]);
@@ -570,7 +567,7 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
                 const float* c2 = c1 + (sequence ? cstride : (size_t)nb * cstride);
                 float* gin = c->gh_a + (size_t)z0 * gstride;
                 float* gout = c->gh_b + (size_t)z0 * gstride;
-                k_flow_gh<<<blocks_for((long long)Pl * nz, 256), 256, 0, st>>>(
+                k_flow_gh<<<dim3(blocks_for((long long)Pl, 256), nz), 256, 0, st>>>(
                     c1, c2, cstride, hs[l], ws[l], coarse ? coarse + (size_t)z0 * fstride : nullptr, fstride, gin, gstride, nz);
                 c->launches++;
                 dim3 grid(ws[l] / tw, hs[l] / TH, nz);
