@@ -29,7 +29,7 @@ PAPER_CONTEXT = {"compression_ratio": 2.20, "time_per_frame_s": 0.068, "baseline
                  "hardware": "1x RTX 3090 24 GB, LLaVA-1.6 Mistral-7B, fp16 (paper Tables I and III)"}
 # DRAM bytes of the pack kernel per algorithmic byte, from the ncu capture summarised in
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over the algorithmic bytes of the same launch).
-NCU_TRAFFIC_RATIO = 0.969
+NCU_TRAFFIC_RATIO = 0.968
 
 
 def _peaks():
@@ -574,7 +574,7 @@ def main():
     ap.add_argument("--frames", type=int, default=0, help="use only the first N frames of the workload (profiling)")
     ap.add_argument("--chunk", type=int, default=304, help="frames per internal pass of flow/saliency")
     ap.add_argument("--ring", type=int, default=RING, help="K/V frame slabs resident on the device")
-    ap.add_argument("--segment", type=int, default=304, help="frames per pipeline segment (filter of one overlaps the store of the previous)")
+    ap.add_argument("--segment", type=int, default=320, help="frames per pipeline segment (filter of one overlaps the store of the previous)")
     ap.add_argument("--overlap", action="store_true", help="store of segment i on a second stream beside the filter of segment i+1")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
