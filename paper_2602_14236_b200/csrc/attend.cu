@@ -19,6 +19,7 @@ constexpr int AT_D = 128;           // head size = threads per CTA = quantisatio
 constexpr int AT_WARPS = AT_D / 32;
 constexpr int AT_CHUNKS = 64;       // partial results per (layer, head)
 constexpr int AT_REC = AT_D + 2;    // partial record: 128 sums, running maximum, running denominator
+constexpr int AT_RECS = 2 * AT_CHUNKS;   // records per (layer, head): AT_CHUNKS of each of the two partial kernels
 
 struct AtPools {
     const uint8_t* fp16_pool;
@@ -51,7 +52,11 @@ __device__ __forceinline__ uint32_t hsub2u(uint32_t a, uint32_t b) {
 // Four INT4 code pairs of a word of 8 nibbles e0..e7: (e0,e4) (e1,e5) (e2,e6) (e3,e7).
 __device__ __forceinline__ void nibbles_to_h2(uint32_t x, uint32_t out[4]) {
 #pragma unroll
-    for (int k = 0; k < 4; ++k) out[k] = hsub2u(((x >> (4 * k)) & 0x000f000fu) | 0x64006400u, 0x64006400u);
+    for (int k = 0; k < 4; k += 2) {
+        const uint32_t y = x >> (4 * k);
+        out[k] = hsub2u((y & 0x000f000fu) | 0x64006400u, 0x64006400u);
+        out[k + 1] = hsub2u((y & 0x00f000f0u) | 0x54005400u, 0x54005400u);      // 64 + nibble: unit in the last place 1/16
+    }
 }
 // Two INT8 code pairs of a word of 4 bytes b0..b3: (b0,b1) (b2,b3).  The bytes are biased by 128 first.
 __device__ __forceinline__ void bytes_to_h2(uint32_t w, uint32_t out[2]) {
@@ -85,7 +90,7 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 
 __global__ void __launch_bounds__(AT_D)
 k_attend_partial(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int ng,
-                 float* __restrict__ ws) {
+                 int with_int4, float* __restrict__ ws) {
     __shared__ __align__(16) float qs[AT_D];        // the query as binary32 (for sum(q))
     __shared__ __align__(16) __half qn[AT_D];       // the query in natural order
     __shared__ __align__(16) __half qp[AT_D];       // the query with every 8 elements ordered 0 4 1 5 2 6 3 7 (INT4 pairs)
@@ -97,7 +102,8 @@ k_attend_partial(const __half* __restrict__ q, AtPools pp, const long long* __re
     const int h = blockIdx.x, c = blockIdx.y, l = blockIdx.z, t = threadIdx.x;
     const int lane = t & 31, wid = t >> 5;
     const int HD = H * AT_D;
-    const long long n16 = min(fill[0], pp.cap16), n8 = min(fill[1], pp.cap8), n4 = min(fill[2], pp.cap4);
+    const long long n16 = min(fill[0], pp.cap16), n8 = min(fill[1], pp.cap8);
+    const long long n4 = with_int4 ? min(fill[2], pp.cap4) : 0;      // the INT4 rows may be left to k_attend_int4
     const long long R = n16 + n8 + n4;
     const long long per = (R + AT_CHUNKS - 1) / AT_CHUNKS;
     const long long r0 = (long long)c * per, r1 = min(R, r0 + per);
@@ -235,7 +241,7 @@ k_attend_partial(const __half* __restrict__ q, AtPools pp, const long long* __re
 #pragma unroll
     for (int k = 0; k < 4; ++k) part[wid][4 * lane + k] = acc[k] + zacc;
     __syncthreads();
-    float* rec = ws + (((size_t)l * H + h) * AT_CHUNKS + c) * AT_REC;
+    float* rec = ws + (((size_t)l * H + h) * AT_RECS + c) * AT_REC;
     float sum = 0.0f;
 #pragma unroll
     for (int k = 0; k < AT_WARPS; ++k) sum += part[k][t];
@@ -246,16 +252,302 @@ k_attend_partial(const __half* __restrict__ q, AtPools pp, const long long* __re
     }
 }
 
+// ---- INT4 rows on the tensor cores.  A single query is a matrix-vector product, but forming it with
+// 16x8x16 matrix instructions (most of the 8 columns idle) still costs far fewer instructions per multiply-add
+// than scalar code, which is what this stage is short of: it is bound by instruction issue, not by arithmetic.
+//   scores  A = 16 key rows x 16 dimensions (codes expanded to binary16), B = the query in column 0
+//   values  A = 16 dimensions x 16 value rows (codes, transposed), B = the 16 softmax weights (times the
+//           value scale) in column 0 (high half) and column 1 (low half of a two-term binary16 split, so that
+//           the weights keep 22 bits)
+// One warp walks 16-row tiles with its own online softmax; the four warps of a CTA are merged at the end.
+// The k index of a matrix instruction may be permuted freely as long as A and B agree, and so may the
+// assignment of the 16 rows of A to dimensions; both are chosen so that a lane reads contiguous bytes.
+__device__ __forceinline__ uint4 ld_stream16(const uint8_t* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint2 ld_stream8(const uint8_t* p) {
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+// Low / high nibbles of bytes 0 and 2 as a binary16 pair.  The high nibble needs no shift: 64 (0x5400) has its
+// unit in the last place at 1/16, so a nibble in bits 4..7 of the mantissa adds exactly its value.
+__device__ __forceinline__ uint32_t nib_lo_pair(uint32_t t) { return hsub2u((t & 0x000f000fu) | 0x64006400u, 0x64006400u); }
+__device__ __forceinline__ uint32_t nib_hi_pair(uint32_t t) { return hsub2u((t & 0x00f000f0u) | 0x54005400u, 0x54005400u); }
+
+// What one lane loads of a tile of 16 INT4 rows: the keys of rows g8 and g8 + 8 (32 dimensions at 32 * c4), the
+// values of rows 2 c4, 2 c4 + 1, 2 c4 + 8, 2 c4 + 9 (16 dimensions at 16 * g8) and the (scale, zero) pairs of
+// rows g8 and g8 + 8.
+struct I4Tile {
+    uint4 ka, kb;
+    uint2 v0, v1, v2, v3;
+    uint32_t ksa, ksb, vsa, vsb;
+};
+// The lane's addresses of a tile: row 0 of its part of the chunk plus a running byte offset.
+struct I4Addr {
+    const uint8_t* k;        // key codes of row g8
+    const uint8_t* v;        // value codes of row 2 c4
+    const uint32_t* ks;      // key (scale, zero) of row g8
+    const uint32_t* vs;      // value (scale, zero) of row g8
+    size_t pitch;            // bytes per row of codes
+    size_t ng;               // (scale, zero) pairs per row
+};
+// FULL: all 16 rows exist.  Otherwise rows at or beyond r1 read as zero codes and are not touched.
+template <bool FULL>
+__device__ __forceinline__ void i4_load(I4Tile& x, const I4Addr& a, long long tile, long long t0, long long r1, int g8, int c4) {
+    const size_t d = (size_t)(tile - t0);
+    const uint8_t* k = a.k + d * a.pitch;
+    const uint8_t* v = a.v + d * a.pitch;
+    const uint32_t* ks = a.ks + d * a.ng;
+    const uint32_t* vs = a.vs + d * a.ng;
+    if (FULL) {
+        x.ka = ld_stream16(k);
+        x.kb = ld_stream16(k + 8 * a.pitch);
+        x.v0 = ld_stream8(v);
+        x.v1 = ld_stream8(v + a.pitch);
+        x.v2 = ld_stream8(v + 8 * a.pitch);
+        x.v3 = ld_stream8(v + 9 * a.pitch);
+        x.ksa = __ldg(ks);
+        x.ksb = __ldg(ks + 8 * a.ng);
+        x.vsa = __ldg(vs);
+        x.vsb = __ldg(vs + 8 * a.ng);
+    } else {
+        x.ka = x.kb = make_uint4(0, 0, 0, 0);
+        x.v0 = x.v1 = x.v2 = x.v3 = make_uint2(0, 0);
+        x.ksa = x.ksb = x.vsa = x.vsb = 0;
+        const long long ra = tile + g8, rv = tile + 2 * c4;
+        if (ra < r1) {
+            x.ka = ld_stream16(k);
+            x.ksa = __ldg(ks);
+            x.vsa = __ldg(vs);
+        }
+        if (ra + 8 < r1) {
+            x.kb = ld_stream16(k + 8 * a.pitch);
+            x.ksb = __ldg(ks + 8 * a.ng);
+            x.vsb = __ldg(vs + 8 * a.ng);
+        }
+        if (rv < r1) x.v0 = ld_stream8(v);
+        if (rv + 1 < r1) x.v1 = ld_stream8(v + a.pitch);
+        if (rv + 8 < r1) x.v2 = ld_stream8(v + 8 * a.pitch);
+        if (rv + 9 < r1) x.v3 = ld_stream8(v + 9 * a.pitch);
+    }
+}
+__device__ __forceinline__ void i4_fetch(I4Tile& x, const I4Addr& a, long long tile, long long t0, long long r1, int g8, int c4) {
+    if (tile + 16 <= r1) i4_load<true>(x, a, tile, t0, r1, g8, c4);
+    else i4_load<false>(x, a, tile, t0, r1, g8, c4);      // loads nothing at all once tile >= r1
+}
+
+// Running state of a warp: m is its maximum (the same in every lane); den and zacc are per-lane partial sums;
+// acc[b] holds, in the lanes with c4 == 0, dimensions 16 g8 + 2 b (.x high, .y low) and 16 g8 + 2 b + 1 (.z, .w).
+struct I4State {
+    float acc[8][4];
+    float m, den, zacc, F;
+};
+
+__device__ __forceinline__ void i4_tile(I4State& st, const I4Tile& x, const uint32_t (&qf)[8][2], long long tile, long long r1,
+                                        float rs, float qsum, int g8, int c4) {
+    // ---- scores of rows tile + g8 and tile + g8 + 8
+    const bool va = tile + g8 < r1, vb = tile + g8 + 8 < r1;
+    float sc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    {
+        const uint32_t wa[4] = {x.ka.x, x.ka.y, x.ka.z, x.ka.w}, wb[4] = {x.kb.x, x.kb.y, x.kb.z, x.kb.w};
+#pragma unroll
+        for (int w4 = 0; w4 < 4; ++w4) {
+            uint32_t pa[4], pb[4];
+            nibbles_to_h2(wa[w4], pa);
+            nibbles_to_h2(wb[w4], pb);
+            mma16816(sc, pa[0], pb[0], pa[1], pb[1], qf[2 * w4][0], qf[2 * w4][1]);
+            mma16816(sc, pa[2], pb[2], pa[3], pb[3], qf[2 * w4 + 1][0], qf[2 * w4 + 1][1]);
+        }
+    }
+    // column 0 (lanes with c4 == 0) holds the dot products of rows g8 (sc[0]) and g8 + 8 (sc[2])
+    const bool own = c4 == 0;
+    const float2 kza = w2f(x.ksa), kzb = w2f(x.ksb), vza = w2f(x.vsa), vzb = w2f(x.vsb);      // (scale, zero)
+    const float sa = own && va ? rs * (sc[0] * kza.x + qsum * kza.y) : -INFINITY;
+    const float sb = own && vb ? rs * (sc[2] * kzb.x + qsum * kzb.y) : -INFINITY;
+    // ---- online softmax of this warp.  The maximum rarely moves after the first tiles and the scale F
+    // almost never: one vote decides whether the reductions and the rescaling of the sums are needed.
+    const float sm = fmaxf(sa, sb), sv = fmaxf(vza.x, vzb.x);       // scales of absent rows are 0
+    if (__any_sync(0xffffffffu, sm > st.m || sv * st.F >= 32768.0f)) {
+        const float m_new = fmaxf(st.m, warp_max(sm));
+        const float corr = st.m == -INFINITY ? 0.0f : __expf(st.m - m_new);
+        st.m = m_new;
+        // keep weight * scale * F below 32768 (binary16): F only ever shrinks, by powers of two
+        const float smax = warp_max(sv);
+        float Fn = st.F;
+        for (int k = 0; k < 40 && smax * Fn >= 32768.0f; ++k) Fn *= 0.5f;
+        const float rescale = corr * (Fn / st.F);
+        st.F = Fn;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) st.acc[b][i] *= rescale;
+        }
+        st.den *= corr;
+        st.zacc *= corr;
+    }
+    const float pa_ = __expf(sa - st.m), pb_ = __expf(sb - st.m);      // 0 for rows that are not this lane's
+    st.den += pa_ + pb_;
+    st.zacc += pa_ * vza.y + pb_ * vzb.y;
+    // weights as a two-term binary16 split (high, low), packed per row
+    uint32_t packa, packb;
+    {
+        const float wa_ = pa_ * vza.x * st.F, wb_ = pb_ * vzb.x * st.F;
+        const __half ha = __float2half_rn(wa_), hb = __float2half_rn(wb_);
+        const __half la = __float2half_rn(wa_ - __half2float(ha)), lb = __float2half_rn(wb_ - __half2float(hb));
+        packa = (uint32_t)__half_as_ushort(ha) | ((uint32_t)__half_as_ushort(la) << 16);
+        packb = (uint32_t)__half_as_ushort(hb) | ((uint32_t)__half_as_ushort(lb) << 16);
+    }
+    // B fragment of the second product: column 0 = high halves, column 1 = low halves, k = tile rows as loaded.
+    // Row r of the tile was scored by lane 4 * (r % 8).
+    const uint32_t x1 = __shfl_sync(0xffffffffu, packa, 8 * c4), x2 = __shfl_sync(0xffffffffu, packa, 8 * c4 + 4);
+    const uint32_t y1 = __shfl_sync(0xffffffffu, packb, 8 * c4), y2 = __shfl_sync(0xffffffffu, packb, 8 * c4 + 4);
+    const uint32_t psel = g8 == 0 ? 0x5410u : 0x7632u;
+    const uint32_t b0 = g8 < 2 ? __byte_perm(x1, x2, psel) : 0u, b1 = g8 < 2 ? __byte_perm(y1, y2, psel) : 0u;
+    // ---- values: instruction b takes byte b of the lane's 8 bytes of each row: dimensions 16 g8 + 2 b (A row g8)
+    // and 16 g8 + 2 b + 1 (A row g8 + 8)
+    {
+        const uint32_t w0[2] = {x.v0.x, x.v0.y}, w1[2] = {x.v1.x, x.v1.y}, w2[2] = {x.v2.x, x.v2.y}, w3[2] = {x.v3.x, x.v3.y};
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            const uint32_t sel = (uint32_t)((b & 3) | ((b & 3) << 4) | ((4 + (b & 3)) << 8) | ((4 + (b & 3)) << 12));
+            const uint32_t t1 = __byte_perm(w0[b >> 2], w1[b >> 2], sel);      // bytes (row 2 c4: b, -, row 2 c4 + 1: b, -)
+            const uint32_t t2 = __byte_perm(w2[b >> 2], w3[b >> 2], sel);
+            mma16816(st.acc[b], nib_lo_pair(t1), nib_hi_pair(t1), nib_lo_pair(t2), nib_hi_pair(t2), b0, b1);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(AT_D)
+k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int ng,
+              float* __restrict__ ws) {
+    __shared__ __align__(16) float qs[AT_D];
+    __shared__ __align__(16) __half qp[AT_D];       // every 8 elements ordered 0 4 1 5 2 6 3 7
+    __shared__ float red[AT_WARPS];
+    __shared__ float wpart[AT_WARPS][AT_D];
+    __shared__ float wstat[AT_WARPS][2];
+    const int h = blockIdx.x, c = blockIdx.y, l = blockIdx.z, t = threadIdx.x;
+    const int lane = t & 31, wid = t >> 5, g8 = lane >> 2, c4 = lane & 3;
+    const int HD = H * AT_D;
+    const long long n4 = min(fill[2], pp.cap4);
+    const long long per = ((n4 + AT_CHUNKS - 1) / AT_CHUNKS + 15) / 16 * 16;      // whole tiles per chunk
+    const long long r0 = (long long)c * per, r1 = min(n4, r0 + per);
+    {
+        const __half qv = q[((size_t)l * H + h) * AT_D + t];
+        const int e = t & 7;
+        qs[t] = __half2float(qv);
+        qp[(t & ~7) | ((e & 3) * 2 + (e >> 2))] = qv;
+    }
+    __syncthreads();
+    const float rs = rsqrtf((float)AT_D);
+    const float qsum = block_sum(qs[t], red);
+    const int g = ng == 1 ? 0 : h;
+    // the query as B fragments: instruction j = 2 * word + u of a lane's 32 dimensions takes the pairs
+    // (e[2u], e[2u+4]) and (e[2u+1], e[2u+5]) of octet 4 * c4 + word; only column 0 (lanes 0..3) is not zero
+    uint32_t qf[8][2];
+    {
+        const uint32_t* qp32 = reinterpret_cast<const uint32_t*>(qp);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int oct = 4 * c4 + (j >> 1), u = j & 1;
+            qf[j][0] = g8 == 0 ? qp32[oct * 4 + 2 * u] : 0u;
+            qf[j][1] = g8 == 0 ? qp32[oct * 4 + 2 * u + 1] : 0u;
+        }
+    }
+    const long long t0 = r0 + 16 * wid;             // this warp's first tile
+    I4Addr ad;
+    ad.pitch = (size_t)(HD / 2);
+    ad.ng = (size_t)ng;
+    ad.k = pp.int4_codes + ((size_t)(2 * l) * pp.cap4 + (size_t)(t0 + g8)) * ad.pitch + (size_t)h * (AT_D / 2) + 16 * c4;
+    ad.v = pp.int4_codes + ((size_t)(2 * l + 1) * pp.cap4 + (size_t)(t0 + 2 * c4)) * ad.pitch + (size_t)h * (AT_D / 2) + 8 * g8;
+    ad.ks = reinterpret_cast<const uint32_t*>(pp.int4_sz) + ((size_t)(2 * l) * pp.cap4 + (size_t)(t0 + g8)) * ng + g;
+    ad.vs = reinterpret_cast<const uint32_t*>(pp.int4_sz) + ((size_t)(2 * l + 1) * pp.cap4 + (size_t)(t0 + g8)) * ng + g;
+    I4State st;
+#pragma unroll
+    for (int b = 0; b < 8; ++b) st.acc[b][0] = st.acc[b][1] = st.acc[b][2] = st.acc[b][3] = 0.0f;
+    st.m = -INFINITY;
+    st.den = st.zacc = 0.0f;
+    st.F = 4096.0f;                                 // the weights are scaled by a power of two before the binary16 split
+    constexpr long long STEP = 16 * AT_WARPS;
+    I4Tile xa, xb;                                  // two tiles in turn: one is consumed while the other is in flight
+    long long tile = t0;
+    if (tile < r1) {
+        i4_fetch(xa, ad, tile, t0, r1, g8, c4);
+        for (;;) {
+            i4_fetch(xb, ad, tile + STEP, t0, r1, g8, c4);
+            i4_tile(st, xa, qf, tile, r1, rs, qsum, g8, c4);
+            tile += STEP;
+            if (tile >= r1) break;
+            i4_fetch(xa, ad, tile + STEP, t0, r1, g8, c4);
+            i4_tile(st, xb, qf, tile, r1, rs, qsum, g8, c4);
+            tile += STEP;
+            if (tile >= r1) break;
+        }
+    }
+    // ---- this warp's result
+    const float den = warp_sum(st.den);
+    const float zs = warp_sum(st.zacc);
+    if (c4 == 0) {
+        const float invF = 1.0f / st.F;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            wpart[wid][16 * g8 + 2 * b] = (st.acc[b][0] + st.acc[b][1]) * invF + zs;
+            wpart[wid][16 * g8 + 2 * b + 1] = (st.acc[b][2] + st.acc[b][3]) * invF + zs;
+        }
+    }
+    if (lane == 0) {
+        wstat[wid][0] = st.m;
+        wstat[wid][1] = den;
+    }
+    __syncthreads();
+    float M = wstat[0][0];
+#pragma unroll
+    for (int k = 1; k < AT_WARPS; ++k) M = fmaxf(M, wstat[k][0]);
+    float sum = 0.0f, dsum = 0.0f;
+    if (M != -INFINITY) {
+#pragma unroll
+        for (int k = 0; k < AT_WARPS; ++k) {
+            const float e = wstat[k][0] == -INFINITY ? 0.0f : __expf(wstat[k][0] - M);
+            sum += e * wpart[k][t];
+            dsum += e * wstat[k][1];
+        }
+    }
+    float* rec = ws + (((size_t)l * H + h) * AT_RECS + AT_CHUNKS + c) * AT_REC;
+    rec[t] = sum;
+    if (t == 0) {
+        rec[AT_D] = M;
+        rec[AT_D + 1] = dsum;
+    }
+}
+
 // Merge the partial results of one (layer, head): out = sum_c e^(m_c - M) acc_c / sum_c e^(m_c - M) den_c.
 __global__ void __launch_bounds__(AT_D)
 k_attend_merge(const float* __restrict__ ws, int H, float* __restrict__ out) {
     const int h = blockIdx.x, l = blockIdx.y, t = threadIdx.x;
-    const float* rec = ws + ((size_t)l * H + h) * AT_CHUNKS * AT_REC;
+    const float* rec = ws + ((size_t)l * H + h) * AT_RECS * AT_REC;
     float M = -INFINITY;
-    for (int c = 0; c < AT_CHUNKS; ++c) M = fmaxf(M, rec[c * AT_REC + AT_D]);
+    for (int c = 0; c < AT_RECS; ++c) M = fmaxf(M, rec[c * AT_REC + AT_D]);
     float num = 0.0f, den = 0.0f;
     if (M != -INFINITY)
-        for (int c = 0; c < AT_CHUNKS; ++c) {
+        for (int c = 0; c < AT_RECS; ++c) {
             const float mc = rec[c * AT_REC + AT_D];
             if (mc == -INFINITY) continue;
             const float e = __expf(mc - M);
@@ -267,7 +559,7 @@ k_attend_merge(const float* __restrict__ ws, int H, float* __restrict__ out) {
 
 }  // namespace
 
-size_t sc_attend_workspace_bytes(int L, int H) { return (size_t)L * H * AT_CHUNKS * AT_REC * sizeof(float); }
+size_t sc_attend_workspace_bytes(int L, int H) { return (size_t)L * H * AT_RECS * AT_REC * sizeof(float); }
 
 int sc_attend(salicache_ctx* c, const void* d_q, const salicache_pools* pools, const int64_t* d_fill, float* d_out,
               cudaStream_t st) {
@@ -279,10 +571,12 @@ int sc_attend(salicache_ctx* c, const void* d_q, const salicache_pools* pools, c
     if (pp.cap16 >= (1ll << 28) || pp.cap8 >= (1ll << 28) || pp.cap4 >= (1ll << 28)) return SALICACHE_E_SHAPE;
     const int ng = p.group == AT_D ? p.heads : 1;
     dim3 grid(p.heads, AT_CHUNKS, p.L);
-    k_attend_partial<<<grid, AT_D, 0, st>>>((const __half*)d_q, pp, (const long long*)d_fill, p.heads, ng, c->attend_ws);
+    // FP16 and INT8 rows one row per thread; INT4 rows, the bulk of a compressed cache, on the matrix instructions
+    k_attend_partial<<<grid, AT_D, 0, st>>>((const __half*)d_q, pp, (const long long*)d_fill, p.heads, ng, 0, c->attend_ws);
+    k_attend_int4<<<grid, AT_D, 0, st>>>((const __half*)d_q, pp, (const long long*)d_fill, p.heads, ng, c->attend_ws);
     dim3 gm(p.heads, p.L);
     k_attend_merge<<<gm, AT_D, 0, st>>>(c->attend_ws, p.heads, d_out);
-    c->launches += 2;
+    c->launches += 3;
     SC_CHECK(cudaGetLastError());
     return SALICACHE_OK;
 }
