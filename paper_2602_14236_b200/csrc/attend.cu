@@ -295,62 +295,63 @@ __device__ __forceinline__ uint32_t nib_hi_pair(uint32_t t) { return hsub2u((t &
 
 // What one lane loads of a tile of 16 INT4 rows: the keys of rows g8 and g8 + 8 (32 dimensions at 32 * c4), the
 // values of rows 2 c4, 2 c4 + 1, 2 c4 + 8, 2 c4 + 9 (16 dimensions at 16 * g8) and the (scale, zero) pairs of
-// rows g8 and g8 + 8.
+// the one row whose softmax weight it computes: g8 + 8 * (c4 & 1).
 struct I4Tile {
     uint4 ka, kb;
     uint2 v0, v1, v2, v3;
-    uint32_t ksa, ksb, vsa, vsb;
+    uint32_t ks, vs;
 };
-// The lane's addresses of a tile: row 0 of its part of the chunk plus a running byte offset.
+// The lane's addresses in its warp's first tile.  PITCH (bytes per row of codes) and NG ((scale, zero) pairs per
+// row) are compile-time constants for the common shapes, so that the row offsets fold into the loads.
+template <int PITCH, int NG>
 struct I4Addr {
     const uint8_t* k;        // key codes of row g8
     const uint8_t* v;        // value codes of row 2 c4
-    const uint32_t* ks;      // key (scale, zero) of row g8
-    const uint32_t* vs;      // value (scale, zero) of row g8
-    size_t pitch;            // bytes per row of codes
-    size_t ng;               // (scale, zero) pairs per row
+    const uint32_t* ks;      // key (scale, zero) of the lane's own row
+    const uint32_t* vs;      // value (scale, zero) of the lane's own row
+    size_t pitch_rt, ng_rt;
+    __device__ __forceinline__ size_t pitch() const { return PITCH ? (size_t)PITCH : pitch_rt; }
+    __device__ __forceinline__ size_t ng() const { return NG ? (size_t)NG : ng_rt; }
 };
 // FULL: all 16 rows exist.  Otherwise rows at or beyond r1 read as zero codes and are not touched.
-template <bool FULL>
-__device__ __forceinline__ void i4_load(I4Tile& x, const I4Addr& a, long long tile, long long t0, long long r1, int g8, int c4) {
+template <bool FULL, int PITCH, int NG>
+__device__ __forceinline__ void i4_load(I4Tile& x, const I4Addr<PITCH, NG>& a, long long tile, long long t0, long long r1, int g8,
+                                        int c4) {
     const size_t d = (size_t)(tile - t0);
-    const uint8_t* k = a.k + d * a.pitch;
-    const uint8_t* v = a.v + d * a.pitch;
-    const uint32_t* ks = a.ks + d * a.ng;
-    const uint32_t* vs = a.vs + d * a.ng;
+    const size_t P = a.pitch();
+    const uint8_t* k = a.k + d * P;
+    const uint8_t* v = a.v + d * P;
+    const uint32_t* ks = a.ks + d * a.ng();
+    const uint32_t* vs = a.vs + d * a.ng();
     if (FULL) {
         x.ka = ld_stream16(k);
-        x.kb = ld_stream16(k + 8 * a.pitch);
+        x.kb = ld_stream16(k + 8 * P);
         x.v0 = ld_stream8(v);
-        x.v1 = ld_stream8(v + a.pitch);
-        x.v2 = ld_stream8(v + 8 * a.pitch);
-        x.v3 = ld_stream8(v + 9 * a.pitch);
-        x.ksa = __ldg(ks);
-        x.ksb = __ldg(ks + 8 * a.ng);
-        x.vsa = __ldg(vs);
-        x.vsb = __ldg(vs + 8 * a.ng);
+        x.v1 = ld_stream8(v + P);
+        x.v2 = ld_stream8(v + 8 * P);
+        x.v3 = ld_stream8(v + 9 * P);
+        x.ks = __ldg(ks);
+        x.vs = __ldg(vs);
     } else {
         x.ka = x.kb = make_uint4(0, 0, 0, 0);
         x.v0 = x.v1 = x.v2 = x.v3 = make_uint2(0, 0);
-        x.ksa = x.ksb = x.vsa = x.vsb = 0;
+        x.ks = x.vs = 0;
         const long long ra = tile + g8, rv = tile + 2 * c4;
-        if (ra < r1) {
-            x.ka = ld_stream16(k);
-            x.ksa = __ldg(ks);
-            x.vsa = __ldg(vs);
-        }
-        if (ra + 8 < r1) {
-            x.kb = ld_stream16(k + 8 * a.pitch);
-            x.ksb = __ldg(ks + 8 * a.ng);
-            x.vsb = __ldg(vs + 8 * a.ng);
+        if (ra < r1) x.ka = ld_stream16(k);
+        if (ra + 8 < r1) x.kb = ld_stream16(k + 8 * P);
+        if (ra + 8 * (c4 & 1) < r1) {
+            x.ks = __ldg(ks);
+            x.vs = __ldg(vs);
         }
         if (rv < r1) x.v0 = ld_stream8(v);
-        if (rv + 1 < r1) x.v1 = ld_stream8(v + a.pitch);
-        if (rv + 8 < r1) x.v2 = ld_stream8(v + 8 * a.pitch);
-        if (rv + 9 < r1) x.v3 = ld_stream8(v + 9 * a.pitch);
+        if (rv + 1 < r1) x.v1 = ld_stream8(v + P);
+        if (rv + 8 < r1) x.v2 = ld_stream8(v + 8 * P);
+        if (rv + 9 < r1) x.v3 = ld_stream8(v + 9 * P);
     }
 }
-__device__ __forceinline__ void i4_fetch(I4Tile& x, const I4Addr& a, long long tile, long long t0, long long r1, int g8, int c4) {
+template <int PITCH, int NG>
+__device__ __forceinline__ void i4_fetch(I4Tile& x, const I4Addr<PITCH, NG>& a, long long tile, long long t0, long long r1, int g8,
+                                         int c4) {
     if (tile + 16 <= r1) i4_load<true>(x, a, tile, t0, r1, g8, c4);
     else i4_load<false>(x, a, tile, t0, r1, g8, c4);      // loads nothing at all once tile >= r1
 }
@@ -364,8 +365,8 @@ struct I4State {
 
 __device__ __forceinline__ void i4_tile(I4State& st, const I4Tile& x, const uint32_t (&qf)[8][2], long long tile, long long r1,
                                         float rs, float qsum, int g8, int c4) {
-    // ---- scores of rows tile + g8 and tile + g8 + 8
-    const bool va = tile + g8 < r1, vb = tile + g8 + 8 < r1;
+    // ---- scores: the query sits in columns 0 and 2 of B, so that the lanes with c4 == 0 receive the products
+    // of rows g8 and g8 + 8 in column 0 and the lanes with c4 == 1 the same two in column 2
     float sc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
     {
         const uint32_t wa[4] = {x.ka.x, x.ka.y, x.ka.z, x.ka.w}, wb[4] = {x.kb.x, x.kb.y, x.kb.z, x.kb.w};
@@ -378,16 +379,15 @@ __device__ __forceinline__ void i4_tile(I4State& st, const I4Tile& x, const uint
             mma16816(sc, pa[2], pb[2], pa[3], pb[3], qf[2 * w4 + 1][0], qf[2 * w4 + 1][1]);
         }
     }
-    // column 0 (lanes with c4 == 0) holds the dot products of rows g8 (sc[0]) and g8 + 8 (sc[2])
-    const bool own = c4 == 0;
-    const float2 kza = w2f(x.ksa), kzb = w2f(x.ksb), vza = w2f(x.vsa), vzb = w2f(x.vsb);      // (scale, zero)
-    const float sa = own && va ? rs * (sc[0] * kza.x + qsum * kza.y) : -INFINITY;
-    const float sb = own && vb ? rs * (sc[2] * kzb.x + qsum * kzb.y) : -INFINITY;
+    // one row per lane: c4 == 0 takes row g8, c4 == 1 takes row g8 + 8; the other lanes have none
+    const bool own = c4 < 2 && tile + g8 + 8 * c4 < r1;
+    const float2 kz = w2f(x.ks), vz = w2f(x.vs);    // (scale, zero); both 0 for an absent row
+    const float s = own ? rs * ((c4 ? sc[2] : sc[0]) * kz.x + qsum * kz.y) : -INFINITY;
+    const float sv = own ? vz.x : 0.0f;
     // ---- online softmax of this warp.  The maximum rarely moves after the first tiles and the scale F
     // almost never: one vote decides whether the reductions and the rescaling of the sums are needed.
-    const float sm = fmaxf(sa, sb), sv = fmaxf(vza.x, vzb.x);       // scales of absent rows are 0
-    if (__any_sync(0xffffffffu, sm > st.m || sv * st.F >= 32768.0f)) {
-        const float m_new = fmaxf(st.m, warp_max(sm));
+    if (__any_sync(0xffffffffu, s > st.m || sv * st.F >= 32768.0f)) {
+        const float m_new = fmaxf(st.m, warp_max(s));
         const float corr = st.m == -INFINITY ? 0.0f : __expf(st.m - m_new);
         st.m = m_new;
         // keep weight * scale * F below 32768 (binary16): F only ever shrinks, by powers of two
@@ -404,22 +404,21 @@ __device__ __forceinline__ void i4_tile(I4State& st, const I4Tile& x, const uint
         st.den *= corr;
         st.zacc *= corr;
     }
-    const float pa_ = __expf(sa - st.m), pb_ = __expf(sb - st.m);      // 0 for rows that are not this lane's
-    st.den += pa_ + pb_;
-    st.zacc += pa_ * vza.y + pb_ * vzb.y;
-    // weights as a two-term binary16 split (high, low), packed per row
-    uint32_t packa, packb;
+    const float pr = __expf(s - st.m);              // 0 for a lane without a row
+    st.den += pr;
+    st.zacc += pr * vz.y;
+    // the weight as a two-term binary16 split (high, low)
+    uint32_t pack;
     {
-        const float wa_ = pa_ * vza.x * st.F, wb_ = pb_ * vzb.x * st.F;
-        const __half ha = __float2half_rn(wa_), hb = __float2half_rn(wb_);
-        const __half la = __float2half_rn(wa_ - __half2float(ha)), lb = __float2half_rn(wb_ - __half2float(hb));
-        packa = (uint32_t)__half_as_ushort(ha) | ((uint32_t)__half_as_ushort(la) << 16);
-        packb = (uint32_t)__half_as_ushort(hb) | ((uint32_t)__half_as_ushort(lb) << 16);
+        const float w = pr * sv * st.F;
+        const __half hi = __float2half_rn(w);
+        const __half lo = __float2half_rn(w - __half2float(hi));
+        pack = (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
     }
     // B fragment of the second product: column 0 = high halves, column 1 = low halves, k = tile rows as loaded.
-    // Row r of the tile was scored by lane 4 * (r % 8).
-    const uint32_t x1 = __shfl_sync(0xffffffffu, packa, 8 * c4), x2 = __shfl_sync(0xffffffffu, packa, 8 * c4 + 4);
-    const uint32_t y1 = __shfl_sync(0xffffffffu, packb, 8 * c4), y2 = __shfl_sync(0xffffffffu, packb, 8 * c4 + 4);
+    // Row r of the tile was weighted by lane 4 * (r % 8) + r / 8.
+    const uint32_t x1 = __shfl_sync(0xffffffffu, pack, 8 * c4), x2 = __shfl_sync(0xffffffffu, pack, 8 * c4 + 4);
+    const uint32_t y1 = __shfl_sync(0xffffffffu, pack, 8 * c4 + 1), y2 = __shfl_sync(0xffffffffu, pack, 8 * c4 + 5);
     const uint32_t psel = g8 == 0 ? 0x5410u : 0x7632u;
     const uint32_t b0 = g8 < 2 ? __byte_perm(x1, x2, psel) : 0u, b1 = g8 < 2 ? __byte_perm(y1, y2, psel) : 0u;
     // ---- values: instruction b takes byte b of the lane's 8 bytes of each row: dimensions 16 g8 + 2 b (A row g8)
@@ -436,6 +435,7 @@ __device__ __forceinline__ void i4_tile(I4State& st, const I4Tile& x, const uint
     }
 }
 
+template <int PITCH, int NG>
 __global__ void __launch_bounds__(AT_D)
 k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int ng,
               float* __restrict__ ws) {
@@ -461,25 +461,27 @@ k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restr
     const float qsum = block_sum(qs[t], red);
     const int g = ng == 1 ? 0 : h;
     // the query as B fragments: instruction j = 2 * word + u of a lane's 32 dimensions takes the pairs
-    // (e[2u], e[2u+4]) and (e[2u+1], e[2u+5]) of octet 4 * c4 + word; only column 0 (lanes 0..3) is not zero
+    // (e[2u], e[2u+4]) and (e[2u+1], e[2u+5]) of octet 4 * c4 + word; columns 0 and 2 (lanes 0..3 and 8..11)
     uint32_t qf[8][2];
     {
         const uint32_t* qp32 = reinterpret_cast<const uint32_t*>(qp);
+        const bool has = g8 == 0 || g8 == 2;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const int oct = 4 * c4 + (j >> 1), u = j & 1;
-            qf[j][0] = g8 == 0 ? qp32[oct * 4 + 2 * u] : 0u;
-            qf[j][1] = g8 == 0 ? qp32[oct * 4 + 2 * u + 1] : 0u;
+            qf[j][0] = has ? qp32[oct * 4 + 2 * u] : 0u;
+            qf[j][1] = has ? qp32[oct * 4 + 2 * u + 1] : 0u;
         }
     }
     const long long t0 = r0 + 16 * wid;             // this warp's first tile
-    I4Addr ad;
-    ad.pitch = (size_t)(HD / 2);
-    ad.ng = (size_t)ng;
-    ad.k = pp.int4_codes + ((size_t)(2 * l) * pp.cap4 + (size_t)(t0 + g8)) * ad.pitch + (size_t)h * (AT_D / 2) + 16 * c4;
-    ad.v = pp.int4_codes + ((size_t)(2 * l + 1) * pp.cap4 + (size_t)(t0 + 2 * c4)) * ad.pitch + (size_t)h * (AT_D / 2) + 8 * g8;
-    ad.ks = reinterpret_cast<const uint32_t*>(pp.int4_sz) + ((size_t)(2 * l) * pp.cap4 + (size_t)(t0 + g8)) * ng + g;
-    ad.vs = reinterpret_cast<const uint32_t*>(pp.int4_sz) + ((size_t)(2 * l + 1) * pp.cap4 + (size_t)(t0 + g8)) * ng + g;
+    I4Addr<PITCH, NG> ad;
+    ad.pitch_rt = (size_t)(HD / 2);
+    ad.ng_rt = (size_t)ng;
+    const size_t own_row = (size_t)(t0 + g8 + 8 * (c4 & 1));
+    ad.k = pp.int4_codes + ((size_t)(2 * l) * pp.cap4 + (size_t)(t0 + g8)) * ad.pitch() + (size_t)h * (AT_D / 2) + 16 * c4;
+    ad.v = pp.int4_codes + ((size_t)(2 * l + 1) * pp.cap4 + (size_t)(t0 + 2 * c4)) * ad.pitch() + (size_t)h * (AT_D / 2) + 8 * g8;
+    ad.ks = reinterpret_cast<const uint32_t*>(pp.int4_sz) + ((size_t)(2 * l) * pp.cap4 + own_row) * ad.ng() + g;
+    ad.vs = reinterpret_cast<const uint32_t*>(pp.int4_sz) + ((size_t)(2 * l + 1) * pp.cap4 + own_row) * ad.ng() + g;
     I4State st;
 #pragma unroll
     for (int b = 0; b < 8; ++b) st.acc[b][0] = st.acc[b][1] = st.acc[b][2] = st.acc[b][3] = 0.0f;
@@ -573,7 +575,11 @@ int sc_attend(salicache_ctx* c, const void* d_q, const salicache_pools* pools, c
     dim3 grid(p.heads, AT_CHUNKS, p.L);
     // FP16 and INT8 rows one row per thread; INT4 rows, the bulk of a compressed cache, on the matrix instructions
     k_attend_partial<<<grid, AT_D, 0, st>>>((const __half*)d_q, pp, (const long long*)d_fill, p.heads, ng, 0, c->attend_ws);
-    k_attend_int4<<<grid, AT_D, 0, st>>>((const __half*)d_q, pp, (const long long*)d_fill, p.heads, ng, c->attend_ws);
+    const __half* qh = (const __half*)d_q;
+    const long long* fl = (const long long*)d_fill;
+    if (p.heads == 32 && ng == 32) k_attend_int4<32 * AT_D / 2, 32><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, c->attend_ws);
+    else if (p.heads == 32 && ng == 1) k_attend_int4<32 * AT_D / 2, 1><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, c->attend_ws);
+    else k_attend_int4<0, 0><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, c->attend_ws);
     dim3 gm(p.heads, p.L);
     k_attend_merge<<<gm, AT_D, 0, st>>>(c->attend_ws, p.heads, d_out);
     c->launches += 3;
