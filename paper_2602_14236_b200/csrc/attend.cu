@@ -288,10 +288,34 @@ __device__ __forceinline__ float warp_sum(float v) {
     for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
 }
-// Low / high nibbles of bytes 0 and 2 as a binary16 pair.  The high nibble needs no shift: 64 (0x5400) has its
-// unit in the last place at 1/16, so a nibble in bits 4..7 of the mantissa adds exactly its value.
-__device__ __forceinline__ uint32_t nib_lo_pair(uint32_t t) { return hsub2u((t & 0x000f000fu) | 0x64006400u, 0x64006400u); }
-__device__ __forceinline__ uint32_t nib_hi_pair(uint32_t t) { return hsub2u((t & 0x00f000f0u) | 0x54005400u, 0x54005400u); }
+// (a & b) | c in one instruction.  The compiler splits the expression into two when b and c are both literals
+// (a logic instruction takes one immediate), so the masks and magic numbers below live in registers.
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+// Codes to binary16 pairs.  A nibble in bits 0..3 of each half is OR-ed into the mantissa of 1024 (0x6400, unit in
+// the last place 1), one in bits 4..7 into that of 64 (0x5400, unit 1/16): either adds exactly its value.
+struct NibConst {
+    uint32_t mask_lo, mask_hi, magic_lo, magic_hi;
+    __device__ __forceinline__ void init() {        // opaque to the compiler, so that they stay in registers
+        asm volatile("mov.b32 %0, 0x000f000f;" : "=r"(mask_lo));
+        asm volatile("mov.b32 %0, 0x00f000f0;" : "=r"(mask_hi));
+        asm volatile("mov.b32 %0, 0x64006400;" : "=r"(magic_lo));
+        asm volatile("mov.b32 %0, 0x54005400;" : "=r"(magic_hi));
+    }
+    __device__ __forceinline__ uint32_t lo(uint32_t t) const { return hsub2u(and_or(t, mask_lo, magic_lo), magic_lo); }
+    __device__ __forceinline__ uint32_t hi(uint32_t t) const { return hsub2u(and_or(t, mask_hi, magic_hi), magic_hi); }
+    // the four pairs (e0,e4) (e1,e5) (e2,e6) (e3,e7) of a word of 8 nibbles
+    __device__ __forceinline__ void word(uint32_t x, uint32_t out[4]) const {
+        const uint32_t y = x >> 8;
+        out[0] = lo(x);
+        out[1] = hi(x);
+        out[2] = lo(y);
+        out[3] = hi(y);
+    }
+};
 
 // What one lane loads of a tile of 16 INT4 rows: the keys of rows g8 and g8 + 8 (32 dimensions at 32 * c4), the
 // values of rows 2 c4, 2 c4 + 1, 2 c4 + 8, 2 c4 + 9 (16 dimensions at 16 * g8) and the (scale, zero) pairs of
@@ -363,8 +387,8 @@ struct I4State {
     float m, den, zacc, F;
 };
 
-__device__ __forceinline__ void i4_tile(I4State& st, const I4Tile& x, const uint32_t (&qf)[8][2], long long tile, long long r1,
-                                        float rs, float qsum, int g8, int c4) {
+__device__ __forceinline__ void i4_tile(I4State& st, const I4Tile& x, const uint32_t (&qf)[8][2], const NibConst& nc, long long tile,
+                                        long long r1, float rs, float qsum, int g8, int c4) {
     // ---- scores: the query sits in columns 0 and 2 of B, so that the lanes with c4 == 0 receive the products
     // of rows g8 and g8 + 8 in column 0 and the lanes with c4 == 1 the same two in column 2
     float sc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -373,8 +397,8 @@ __device__ __forceinline__ void i4_tile(I4State& st, const I4Tile& x, const uint
 #pragma unroll
         for (int w4 = 0; w4 < 4; ++w4) {
             uint32_t pa[4], pb[4];
-            nibbles_to_h2(wa[w4], pa);
-            nibbles_to_h2(wb[w4], pb);
+            nc.word(wa[w4], pa);
+            nc.word(wb[w4], pb);
             mma16816(sc, pa[0], pb[0], pa[1], pb[1], qf[2 * w4][0], qf[2 * w4][1]);
             mma16816(sc, pa[2], pb[2], pa[3], pb[3], qf[2 * w4 + 1][0], qf[2 * w4 + 1][1]);
         }
@@ -430,7 +454,7 @@ __device__ __forceinline__ void i4_tile(I4State& st, const I4Tile& x, const uint
             const uint32_t sel = (uint32_t)((b & 3) | ((b & 3) << 4) | ((4 + (b & 3)) << 8) | ((4 + (b & 3)) << 12));
             const uint32_t t1 = __byte_perm(w0[b >> 2], w1[b >> 2], sel);      // bytes (row 2 c4: b, -, row 2 c4 + 1: b, -)
             const uint32_t t2 = __byte_perm(w2[b >> 2], w3[b >> 2], sel);
-            mma16816(st.acc[b], nib_lo_pair(t1), nib_hi_pair(t1), nib_lo_pair(t2), nib_hi_pair(t2), b0, b1);
+            mma16816(st.acc[b], nc.lo(t1), nc.hi(t1), nc.lo(t2), nc.hi(t2), b0, b1);
         }
     }
 }
@@ -482,6 +506,8 @@ k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restr
     ad.v = pp.int4_codes + ((size_t)(2 * l + 1) * pp.cap4 + (size_t)(t0 + 2 * c4)) * ad.pitch() + (size_t)h * (AT_D / 2) + 8 * g8;
     ad.ks = reinterpret_cast<const uint32_t*>(pp.int4_sz) + ((size_t)(2 * l) * pp.cap4 + own_row) * ad.ng() + g;
     ad.vs = reinterpret_cast<const uint32_t*>(pp.int4_sz) + ((size_t)(2 * l + 1) * pp.cap4 + own_row) * ad.ng() + g;
+    NibConst nc;
+    nc.init();
     I4State st;
 #pragma unroll
     for (int b = 0; b < 8; ++b) st.acc[b][0] = st.acc[b][1] = st.acc[b][2] = st.acc[b][3] = 0.0f;
@@ -495,11 +521,11 @@ k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restr
         i4_fetch(xa, ad, tile, t0, r1, g8, c4);
         for (;;) {
             i4_fetch(xb, ad, tile + STEP, t0, r1, g8, c4);
-            i4_tile(st, xa, qf, tile, r1, rs, qsum, g8, c4);
+            i4_tile(st, xa, qf, nc, tile, r1, rs, qsum, g8, c4);
             tile += STEP;
             if (tile >= r1) break;
             i4_fetch(xa, ad, tile + STEP, t0, r1, g8, c4);
-            i4_tile(st, xb, qf, tile, r1, rs, qsum, g8, c4);
+            i4_tile(st, xb, qf, nc, tile, r1, rs, qsum, g8, c4);
             tile += STEP;
             if (tile >= r1) break;
         }
