@@ -9,6 +9,8 @@
 // no cross-lane reduction), the softmax statistics are kept online, and the values are accumulated four
 // dimensions per lane, one row per warp at a time.  Single precision throughout.
 #include <cuda_fp16.h>
+
+#include <algorithm>
 #include <math.h>
 
 #include "common.cuh"
@@ -105,8 +107,16 @@ k_attend_partial(const __half* __restrict__ q, AtPools pp, const long long* __re
     const long long n16 = min(fill[0], pp.cap16), n8 = min(fill[1], pp.cap8);
     const long long n4 = with_int4 ? min(fill[2], pp.cap4) : 0;      // the INT4 rows may be left to k_attend_int4
     const long long R = n16 + n8 + n4;
-    const long long per = (R + AT_CHUNKS - 1) / AT_CHUNKS;
+    const long long per = (R + gridDim.y - 1) / gridDim.y;      // the host sizes the grid's chunks by the pools' capacity
     const long long r0 = (long long)c * per, r1 = min(R, r0 + per);
+    if (r0 >= r1) {                                 // nothing in this chunk: a record the merge skips
+        if (t == 0) {
+            float* rec = ws + (((size_t)l * H + h) * AT_RECS + c) * AT_REC;
+            rec[AT_D] = -INFINITY;
+            rec[AT_D + 1] = 0.0f;
+        }
+        return;
+    }
     {
         const __half qv = q[((size_t)l * H + h) * AT_D + t];
         const int e = t & 7;
@@ -474,6 +484,14 @@ k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restr
     const long long n4 = min(fill[2], pp.cap4);
     const long long per = ((n4 + AT_CHUNKS - 1) / AT_CHUNKS + 15) / 16 * 16;      // whole tiles per chunk
     const long long r0 = (long long)c * per, r1 = min(n4, r0 + per);
+    if (r0 >= r1) {                                 // nothing in this chunk: a record the merge skips
+        if (t == 0) {
+            float* rec = ws + (((size_t)l * H + h) * AT_RECS + AT_CHUNKS + c) * AT_REC;
+            rec[AT_D] = -INFINITY;
+            rec[AT_D + 1] = 0.0f;
+        }
+        return;
+    }
     {
         const __half qv = q[((size_t)l * H + h) * AT_D + t];
         const int e = t & 7;
@@ -568,14 +586,15 @@ k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restr
 
 // Merge the partial results of one (layer, head): out = sum_c e^(m_c - M) acc_c / sum_c e^(m_c - M) den_c.
 __global__ void __launch_bounds__(AT_D)
-k_attend_merge(const float* __restrict__ ws, int H, float* __restrict__ out) {
+k_attend_merge(const float* __restrict__ ws, int H, int nch, float* __restrict__ out) {
     const int h = blockIdx.x, l = blockIdx.y, t = threadIdx.x;
     const float* rec = ws + ((size_t)l * H + h) * AT_RECS * AT_REC;
+    // records 0 .. nch-1 come from k_attend_partial, AT_CHUNKS .. AT_RECS-1 from k_attend_int4
     float M = -INFINITY;
-    for (int c = 0; c < AT_RECS; ++c) M = fmaxf(M, rec[c * AT_REC + AT_D]);
+    for (int c = 0; c < AT_RECS; c = (c == nch - 1 ? AT_CHUNKS : c + 1)) M = fmaxf(M, rec[c * AT_REC + AT_D]);
     float num = 0.0f, den = 0.0f;
     if (M != -INFINITY)
-        for (int c = 0; c < AT_RECS; ++c) {
+        for (int c = 0; c < AT_RECS; c = (c == nch - 1 ? AT_CHUNKS : c + 1)) {
             const float mc = rec[c * AT_REC + AT_D];
             if (mc == -INFINITY) continue;
             const float e = __expf(mc - M);
@@ -599,15 +618,18 @@ int sc_attend(salicache_ctx* c, const void* d_q, const salicache_pools* pools, c
     if (pp.cap16 >= (1ll << 28) || pp.cap8 >= (1ll << 28) || pp.cap4 >= (1ll << 28)) return SALICACHE_E_SHAPE;
     const int ng = p.group == AT_D ? p.heads : 1;
     dim3 grid(p.heads, AT_CHUNKS, p.L);
-    // FP16 and INT8 rows one row per thread; INT4 rows, the bulk of a compressed cache, on the matrix instructions
-    k_attend_partial<<<grid, AT_D, 0, st>>>((const __half*)d_q, pp, (const long long*)d_fill, p.heads, ng, 0, c->attend_ws);
+    // FP16 and INT8 rows one row per thread; INT4 rows, the bulk of a compressed cache, on the matrix instructions.
+    // The first kernel gets as many chunks as its two pools can fill with four tiles each, 64 at most.
+    const int nch = (int)std::min<long long>(AT_CHUNKS, std::max<long long>(1, (pp.cap16 + pp.cap8 + 4 * AT_D - 1) / (4 * AT_D)));
+    dim3 grid16(p.heads, nch, p.L);
+    k_attend_partial<<<grid16, AT_D, 0, st>>>((const __half*)d_q, pp, (const long long*)d_fill, p.heads, ng, 0, c->attend_ws);
     const __half* qh = (const __half*)d_q;
     const long long* fl = (const long long*)d_fill;
     if (p.heads == 32 && ng == 32) k_attend_int4<32 * AT_D / 2, 32><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, c->attend_ws);
     else if (p.heads == 32 && ng == 1) k_attend_int4<32 * AT_D / 2, 1><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, c->attend_ws);
     else k_attend_int4<0, 0><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, c->attend_ws);
     dim3 gm(p.heads, p.L);
-    k_attend_merge<<<gm, AT_D, 0, st>>>(c->attend_ws, p.heads, d_out);
+    k_attend_merge<<<gm, AT_D, 0, st>>>(c->attend_ws, p.heads, nch, d_out);
     c->launches += 3;
     SC_CHECK(cudaGetLastError());
     return SALICACHE_OK;
