@@ -587,20 +587,25 @@ k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restr
 // Merge the partial results of one (layer, head): out = sum_c e^(m_c - M) acc_c / sum_c e^(m_c - M) den_c.
 __global__ void __launch_bounds__(AT_D)
 k_attend_merge(const float* __restrict__ ws, int H, int nch, float* __restrict__ out) {
+    __shared__ float ew[AT_RECS];                   // e^(m_c - M), 0 for a record that is empty or was not written
+    __shared__ float red[AT_WARPS];
+    static_assert(AT_RECS == AT_D, "one record per thread in the statistics pass");
     const int h = blockIdx.x, l = blockIdx.y, t = threadIdx.x;
     const float* rec = ws + ((size_t)l * H + h) * AT_RECS * AT_REC;
     // records 0 .. nch-1 come from k_attend_partial, AT_CHUNKS .. AT_RECS-1 from k_attend_int4
-    float M = -INFINITY;
-    for (int c = 0; c < AT_RECS; c = (c == nch - 1 ? AT_CHUNKS : c + 1)) M = fmaxf(M, rec[c * AT_REC + AT_D]);
-    float num = 0.0f, den = 0.0f;
-    if (M != -INFINITY)
-        for (int c = 0; c < AT_RECS; c = (c == nch - 1 ? AT_CHUNKS : c + 1)) {
-            const float mc = rec[c * AT_REC + AT_D];
-            if (mc == -INFINITY) continue;
-            const float e = __expf(mc - M);
-            num += e * rec[c * AT_REC + t];
-            den += e * rec[c * AT_REC + AT_D + 1];
-        }
+    const bool written = t < nch || t >= AT_CHUNKS;
+    const float mc = written ? rec[t * AT_REC + AT_D] : -INFINITY;
+    const float dc = written ? rec[t * AT_REC + AT_D + 1] : 0.0f;
+    const float M = block_max(mc, red);
+    const float e = mc == -INFINITY ? 0.0f : __expf(mc - M);
+    ew[t] = e;
+    const float den = block_sum(e * dc, red);       // (its barriers also publish ew)
+    float num = 0.0f;
+#pragma unroll 8
+    for (int c = 0; c < AT_RECS; ++c) {
+        const float w = ew[c];
+        if (w != 0.0f) num += w * rec[c * AT_REC + t];
+    }
     out[((size_t)l * H + h) * AT_D + t] = den > 0.0f ? num / den : 0.0f;
 }
 
