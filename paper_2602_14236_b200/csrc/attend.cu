@@ -4,10 +4,11 @@
 //
 //   score_j = q_h . K^_{j,h} / sqrt(D),   p = softmax_j(score),   out_h = sum_j p_j V^_{j,h}
 //
-// Split over the rows (AT_CHUNKS partial results per layer and head, merged by a second kernel).  Within a
-// CTA the scores are computed one row per thread (the thread walks the head's 128 key elements of its row:
-// no cross-lane reduction), the softmax statistics are kept online, and the values are accumulated four
-// dimensions per lane, one row per warp at a time.  Single precision throughout.
+// Split over the rows: per layer and head up to AT_CHUNKS partial results of each of two kernels, merged by a
+// third.  k_attend_partial takes the FP16 and INT8 rows: scores one row per thread (the thread walks the
+// head's 128 key elements of its row: no cross-lane reduction), values four dimensions per lane, one row per
+// warp at a time.  k_attend_int4 takes the INT4 rows, the bulk of a compressed cache, 16 rows per warp at a
+// time through matrix instructions.  Online softmax and single precision accumulation in both.
 #include <cuda_fp16.h>
 
 #include <algorithm>

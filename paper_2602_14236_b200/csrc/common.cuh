@@ -48,7 +48,7 @@ struct salicache_ctx {
     uint8_t* base_frames;      // anyres only: [chunk+1][336*336*3]
     // select / pack scratch
     int64_t* row_prefix;       // [max_batch+1] stored rows before each frame of the batch
-    float* attend_ws;          // partial attention results [L][heads][64][head_dim + 2]
+    float* attend_ws;          // partial attention results [L][heads][128][head_dim + 2]
     int* d_status;             // deferred status word
     int sm_count;
     long long launches;        // kernels launched through this context so far
