@@ -17,8 +17,9 @@ pytestmark = pytest.mark.gpu
 ATOL, RTOL = 2e-5, 1e-4
 
 
-def _store(L, heads, T, background, group=128, seed=0, s_lo=0.0):
-    """Random scores -> decisions -> pools on both sides (the pools are bit-identical, checked elsewhere)."""
+def _store(L, heads, T, background, group=128, seed=0, s_lo=0.0, v_scale=1.0, keep=None):
+    """Random scores -> decisions -> pools on both sides (the pools are bit-identical, checked elsewhere).
+    `keep`, a dict, receives the dense K and the decisions."""
     import torch
     HD, n_tok = heads * 128, 576
     ctx = sc.Context(sc.salicache_default_params(max_batch=8, chunk_frames=4, L=L, heads=heads, group=group,
@@ -29,7 +30,9 @@ def _store(L, heads, T, background, group=128, seed=0, s_lo=0.0):
     counts = out["counts"].cpu().numpy()
     caps = tuple(int(c) + 3 for c in counts[:, [4, 3, 2]].sum(axis=0))
     K = rng.standard_normal((T, L, n_tok, HD)).astype(np.float16)
-    V = rng.standard_normal((T, L, n_tok, HD)).astype(np.float16)
+    V = (v_scale * rng.standard_normal((T, L, n_tok, HD))).astype(np.float16)
+    if keep is not None:
+        keep.update(K=K, decision=out["decision"].cpu().numpy())
     pools = sc.PoolSet(L, HD, *caps, G=group)
     sc.salicache_pack_kv(ctx, torch.from_numpy(K).cuda(), torch.from_numpy(V).cuda(), L * n_tok * HD, out["idx"],
                          out["counts"], out["row_offset"], T, pools.c)
@@ -44,7 +47,8 @@ def _store(L, heads, T, background, group=128, seed=0, s_lo=0.0):
     return ctx, pools, ref, out["fill"], rng
 
 
-def _check(ctx, pools, ref, fill, q):
+def _check(ctx, pools, ref, fill, q, scale=1.0):
+    """`scale`: magnitude of the values relative to 1; the absolute part of the tolerance grows with it."""
     import torch
     L, H, D = q.shape
     d_out = torch.full((L, H, D), 7.0, dtype=torch.float32, device="cuda")
@@ -54,7 +58,7 @@ def _check(ctx, pools, ref, fill, q):
     want = oracle.attend(q.view(np.uint16), ref, n)
     got = d_out.cpu().numpy().astype(np.float64)
     err = np.abs(got - want)
-    assert (err <= ATOL + RTOL * np.abs(want)).all(), f"worst {err.max():.3e} at |out| {np.abs(want).ravel()[err.argmax()]:.3e}"
+    assert (err <= ATOL * scale + RTOL * np.abs(want)).all(), f"worst {err.max():.3e} at |out| {np.abs(want).ravel()[err.argmax()]:.3e}"
     return got, want
 
 
@@ -99,3 +103,26 @@ def test_attention_at_the_benchmark_shape():
     ctx, pools, ref, fill, rng = _store(L=32, heads=32, T=2, background="int4", seed=9, s_lo=0.3)
     q = rng.standard_normal((32, 32, 128)).astype(np.float16)
     _check(ctx, pools, ref, fill, q)
+
+
+def test_attention_int4_rows_peaked_and_large_values():
+    """The INT4 kernel forms its value product from softmax weights split into two binary16 terms and scaled by a
+    power of two that shrinks when a row's value scale is large.  A query aligned with one INT4 row (that row takes
+    nearly all the weight, the others span many orders of magnitude) and values 300 times larger (value scales of
+    about 150, which force the smaller power of two) exercise both; 8 heads take the kernel's generic-shape build,
+    and 37 frames' worth of rows leave a ragged last tile."""
+    for heads, v_scale in ((32, 1.0), (32, 300.0), (8, 300.0)):
+        keep = {}
+        ctx, pools, ref, fill, rng = _store(L=2, heads=heads, T=2, background="int4", seed=11, s_lo=0.3, v_scale=v_scale,
+                                            keep=keep)
+        n4 = int(min(int(fill[2].item()), ref.cap4))
+        assert n4 > 64
+        if n4 % 16 == 0:                            # end in a ragged tile
+            fill = fill.clone()
+            fill[2] = n4 - 5
+        q = rng.standard_normal((2, heads, 128)).astype(np.float16)
+        _check(ctx, pools, ref, fill, q, scale=v_scale)
+        # aligned with the key of the first token stored as INT4 (frame 0)
+        tok = int(np.flatnonzero(keep["decision"][0] == sc.INT4)[0])
+        k_row = keep["K"][0, :, tok, :].reshape(2, heads, 128).astype(np.float32)
+        _check(ctx, pools, ref, fill, (3.0 * k_row).astype(np.float16), scale=v_scale)
