@@ -234,6 +234,27 @@ def select(dP, s, has_prev: bool, p: Params = Params()):
     return dec, idx, counts, int(red[0]), float(R[0])
 
 
+def select_anchored(frames: np.ndarray, s: np.ndarray, first_has_no_prev: bool, anchor: np.ndarray, p: Params = Params()):
+    """Anchor-frame mode: every token is compared (Eq. 5 read literally) with the patch its cache entry came from.
+    frames u8 [T][h][w][3], s f32 [T][n_tok], anchor u8 [h][w][3] (updated in place).
+    Returns dP f32 [T][n_tok], decision u8 [T][n_tok], idx i32 [T][3][n_tok], counts i32 [T][5], redundant u8 [T]."""
+    frames, s = _c(frames, np.uint8), _c(s, np.float32)
+    assert anchor.dtype == np.uint8 and anchor.flags["C_CONTIGUOUS"]
+    T, h, w, _ = frames.shape
+    n = (h // p.patch) * (w // p.patch)
+    assert s.shape == (T, n) and anchor.shape == (h, w, 3)
+    dP = np.empty((T, n), np.float32)
+    dec = np.empty((T, n), np.uint8)
+    idx = np.empty((T, 3, n), np.int32)
+    counts = np.empty((T, 5), np.int32)
+    red = np.zeros(T, np.uint8)
+    lib().oracle_select_anchored(_p(frames), _p(s), C.c_int(T), C.c_int(h), C.c_int(w), C.c_int(p.patch),
+                                 C.c_int(int(first_has_no_prev)), C.c_int(p.patch_reuse), C.c_float(p.tau_t),
+                                 C.c_float(p.theta_R), C.c_float(p.tau_high), C.c_float(p.tau_med), C.c_float(p.tau_low),
+                                 _p(anchor), _p(dP), _p(dec), _p(idx), _p(counts), _p(red))
+    return dP, dec, idx, counts, red
+
+
 def source_frames(decision: np.ndarray, first: int = 0, prev=None) -> np.ndarray:
     """decision u8 [T][n_tok] -> int32 [T][n_tok]: the frame whose entry each token uses (reuse chains resolved)."""
     decision = _c(decision, np.uint8)

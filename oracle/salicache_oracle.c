@@ -528,6 +528,53 @@ EXPORT void oracle_select(const float* dP, const float* s, int n_tok, int has_pr
 }
 
 /* ------------------------------------------------------------------------- */
+/* Anchor-frame mode of the temporal test (a variant: the paper compares        */
+/* consecutive frames, Sec. III-A, which lets a slow pan or a slow fade stay    */
+/* "static" forever because every single step is below tau_t).  Here token i of */
+/* frame t is compared with the patch its cache entry was computed from: the    */
+/* patch of the last frame in which token i was not REUSE (the frame Alg. 1's   */
+/* pointer chain resolves to).  `anchor` is that composite image, [h][w][3],     */
+/* read and updated in frame order:                                             */
+/*   dP[t][i]  = Eq. 5 read literally between anchor and frame t (RMS grey-level */
+/*               difference over patch i); 0 for a frame without predecessor;   */
+/*   decisions = Eq. 6 / Eq. 8 on (dP[t], s[t]) exactly as oracle_select;        */
+/*   anchor    <- frame t on every patch whose token is not REUSE.               */
+/* The flow score is not used in this mode: each token has its own reference     */
+/* frame, so it would need one flow field per (frame, anchor) pair.              */
+/* Frames depend on their predecessors' decisions: a scan, not a map.            */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_select_anchored(const uint8_t* frames, const float* s, int T, int h, int w, int patch,
+                                   int first_has_no_prev, int patch_reuse, float tau_t, float theta_R, float tau_high,
+                                   float tau_med, float tau_low, uint8_t* anchor, float* dP, uint8_t* decision,
+                                   int32_t* idx, int32_t* counts, uint8_t* frame_redundant) {
+    int gw = w / patch, n_tok = (h / patch) * gw;
+    size_t fb = (size_t)h * w * 3;
+    double* d = (double*)malloc((size_t)n_tok * sizeof(double));
+    for (int t = 0; t < T; ++t) {
+        const uint8_t* f = frames + (size_t)t * fb;
+        int has_prev = !(first_has_no_prev && t == 0);
+        float* dp = dP + (size_t)t * n_tok;
+        if (has_prev) {
+            oracle_diff_score(anchor, f, h, w, patch, d);
+            for (int i = 0; i < n_tok; ++i) dp[i] = (float)d[i];
+        } else {
+            for (int i = 0; i < n_tok; ++i) dp[i] = 0.0f;
+        }
+        uint8_t* dec = decision + (size_t)t * n_tok;
+        oracle_select(dp, s + (size_t)t * n_tok, n_tok, has_prev, patch_reuse, tau_t, theta_R, tau_high, tau_med, tau_low,
+                      dec, idx + (size_t)t * 3 * n_tok, counts + (size_t)t * 5, frame_redundant + t, NULL);
+        for (int i = 0; i < n_tok; ++i) {
+            if (dec[i] == 0) continue;
+            int py = i / gw, px = i % gw;
+            for (int y = py * patch; y < (py + 1) * patch; ++y)
+                memcpy(anchor + ((size_t)y * w + (size_t)px * patch) * 3, f + ((size_t)y * w + (size_t)px * patch) * 3,
+                       (size_t)patch * 3);
+        }
+    }
+    free(d);
+}
+
+/* ------------------------------------------------------------------------- */
 /* Source-frame table (Alg. 1 line 7: C[t] <- Pointer(C[t-1]); Fig. 3 counts    */
 /* reuse per patch).  src[t][i] = src[t-1][i] when token i of frame t is REUSE, */
 /* else t: every token names the frame whose entry it uses, chains resolved.   */
