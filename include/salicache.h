@@ -260,6 +260,31 @@ SALICACHE_API int salicache_saliency_noalloc(const salicache_params* p, const ui
                                              int32_t* d_status_or_null, void* cuda_stream);
 
 /*
+ * Temporal test and decisions in anchor-frame mode (a variant; the paper's test compares consecutive frames,
+ * Sec. III-A, under which a slow pan or fade whose every step stays below tau_t is reused forever).  Token i of
+ * frame b is compared with the patch its cache entry was computed from, i.e. patch i of the last frame in which
+ * token i was not SALICACHE_REUSE (the frame Alg. 1's pointers resolve to).  d_anchor holds that composite image.
+ * For b = 0 .. B-1 in order:
+ *   d_deltaP[b][i] = Eq. 5 read literally (as salicache_diff_score) between d_anchor and frame b; 0 for a first
+ *                    frame without predecessor;
+ *   decisions, index lists, counts, redundancy flag = salicache_select's rule (Eq. 6, Eq. 8) on that row;
+ *   d_anchor <- frame b on every patch whose token is not SALICACHE_REUSE;
+ * then row offsets and d_fill as salicache_select.  tau_t is a grey-level threshold here.  Each frame depends on
+ * the decisions of the one before: the frames of one call are processed in sequence by one cluster of CTAs.
+ *   d_frames  DEVICE u8 [B][H][W][3], 16-byte aligned;  d_s DEVICE f32 [B][N_tok] (salicache_saliency)
+ *   d_anchor  DEVICE u8 [H][W][3], 16-byte aligned, caller-owned, read and written: pass the same buffer to the
+ *             next call (first_has_no_prev = 0) to continue the video; its content is ignored, and replaced, when
+ *             first_has_no_prev != 0 (frame 0 then stores every token)
+ *   d_deltaP  DEVICE f32 [B][N_tok], written;  the remaining arguments as for salicache_select
+ * Contexts with an anyres token layout, a patch size other than 14 or more than 48 x 48 patches: E_PARAM.
+ * Errors: E_NULL, E_SHAPE (B < 0 or > max_batch), E_ALIGN, E_PARAM, E_CUDA.
+ */
+SALICACHE_API int salicache_select_anchored(salicache_ctx* ctx, const uint8_t* d_frames, const float* d_s, int B,
+                                            int first_has_no_prev, uint8_t* d_anchor, float* d_deltaP, uint8_t* d_decision,
+                                            int32_t* d_idx, int32_t* d_counts, uint8_t* d_frame_redundant,
+                                            int64_t* d_row_offset, int64_t* d_fill, void* cuda_stream);
+
+/*
  * Decode attention straight from the mixed-precision store (Eq. 2 with the just-in-time dequantisation of
  * Sec. III-C fused in): for every layer l and head h,
  *   score_j = q[l][h] . K^_j / sqrt(head_dim),  p = softmax_j(score),  out[l][h] = sum_j p_j V^_j,

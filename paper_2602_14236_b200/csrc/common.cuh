@@ -71,6 +71,10 @@ int sc_sources(salicache_ctx* c, const uint8_t* d_decision, int B, int first_fra
                cudaStream_t st);
 int sc_frame_redundancy(salicache_ctx* c, const float* d_deltaP, int B, int first_has_no_prev, uint8_t* d_frame_redundant,
                         cudaStream_t st);
+// anchor.cu
+int sc_select_anchored(salicache_ctx* c, const uint8_t* d_frames, const float* d_s, int B, int first_has_no_prev,
+                       uint8_t* d_anchor, float* d_deltaP, uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts,
+                       uint8_t* d_frame_redundant, int64_t* d_row_offset, int64_t* d_fill, cudaStream_t st);
 // attend.cu
 size_t sc_attend_workspace_bytes(int L, int H);
 int sc_attend(salicache_ctx* c, const void* d_q, const salicache_pools* pools, const int64_t* d_fill, float* d_out,
