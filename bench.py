@@ -368,6 +368,43 @@ def run_extras(sc, synth, ctx, wl, T, frames, dP, dev, peak, pools, fill, stored
                          "ms": round(ms, 3), "cache_bytes": int(stored_bytes), "l2": "cache larger than L2",
                          "algorithmic_GBps": round(stored_bytes / ms / 1e6, 1),
                          "frac_of_hbm_peak": round(stored_bytes / ms / 1e6 / peak, 4)}
+    # anchor-frame mode: the scan over the frames of this workload (Eq. 5 literal against the anchor image + decisions)
+    if wl.n_images == 1 and T > 1:
+        tau_grey = 3.0
+        ca = sc.Context(sc.salicache_default_params(H=wl.H, W=wl.W, max_batch=T, chunk_frames=2, L=1, tau_t=tau_grey,
+                                                    **synth.thresholds(wl.background)))
+        n = wl.n_tok
+        s_a = torch.zeros((T, n), dtype=torch.float32, device=dev)
+        sc.salicache_saliency(ca, frames, T, s_a)
+        anchor = torch.zeros((wl.H, wl.W, 3), dtype=torch.uint8, device=dev)
+        dP_a = torch.zeros((T, n), dtype=torch.float32, device=dev)
+        dec_a = torch.zeros((T, n), dtype=torch.uint8, device=dev)
+        idx_a = torch.zeros((T, 3, n), dtype=torch.int32, device=dev)
+        cnt_a = torch.zeros((T, 5), dtype=torch.int32, device=dev)
+        red_a = torch.zeros((T,), dtype=torch.uint8, device=dev)
+        off_a = torch.zeros((T, 3), dtype=torch.int64, device=dev)
+        fill_a = torch.zeros((3,), dtype=torch.int64, device=dev)
+
+        def anchored():
+            fill_a.zero_()
+            sc.salicache_select_anchored(ca, frames, s_a, T, True, anchor, dP_a, dec_a, idx_a, cnt_a, red_a, off_a, fill_a)
+
+        ms = timed(anchored, reps=5)
+        reuse_anchor = float(cnt_a[:, 0].sum().item()) / (T * n)
+        # the same threshold on consecutive frames, for the share of reused tokens
+        sc.salicache_diff_score(ca, frames[:-1], frames[1:], T - 1, dP_a[1:])
+        fill_a.zero_()
+        sc.salicache_select(ca, dP_a, s_a, T, True, dec_a, idx_a, cnt_a, red_a, off_a, fill_a)
+        torch.cuda.synchronize()
+        reuse_consecutive = float(cnt_a[:, 0].sum().item()) / (T * n)
+        out["select_anchored"] = {
+            "what": f"salicache_select_anchored over the {T} frames in sequence (each token scored against the patch its "
+                    f"entry came from, tau_t = {tau_grey} grey levels); one cluster of 8 CTAs, one frame per step",
+            "ms": round(ms, 3), "us_per_frame": round(1e3 * ms / T, 2), "frames_per_s": round(T / ms * 1e3, 1),
+            "l2": "flushed between repetitions",
+            "reused_tokens_percent": {"anchor_mode": round(100 * reuse_anchor, 2),
+                                      "consecutive_frames_same_threshold": round(100 * reuse_consecutive, 2)}}
+        ca.close()
     # Fig. 3 style breakdown: workload 2 frames under the four-tier rule
     wl2 = synth.WORKLOADS[2]
     p2 = sc.salicache_default_params(max_batch=wl2.T, chunk_frames=wl2.T, L=1, **synth.thresholds("four"))

@@ -22,7 +22,7 @@ namespace cg = cooperative_groups;
 namespace {
 
 constexpr int AN_CLUSTER = 8;       // CTAs per video
-constexpr int AN_THREADS = 256;
+constexpr int AN_THREADS = 1024;    // a step is a few dependent memory round trips: every thread gets two or three chunks
 constexpr int AN_WARPS = AN_THREADS / 32;
 constexpr int AN_MAX_OWN = 288;     // tokens one CTA may own: ceil(48 / 8) bands of up to 48 patches
 constexpr int AN_XCH = 6;           // shared per frame and CTA: static patches, then counts of REUSE PRUNE INT4 INT8 FP16
@@ -48,15 +48,16 @@ __device__ __forceinline__ uint32_t head_mask(int n, int w4) {
     return k >= 4 ? 0xffffffffu : (k <= 0 ? 0u : ((1u << (8 * k)) - 1u));
 }
 
+static_assert(AN_MAX_OWN <= AN_THREADS, "one owned token per thread");
+
 __global__ void __cluster_dims__(AN_CLUSTER, 1, 1) __launch_bounds__(AN_THREADS)
 k_select_anchored(AnchorArgs a) {
     cg::cluster_group cluster = cg::this_cluster();
-    __shared__ unsigned int acc[AN_MAX_OWN];        // squared differences per owned patch
+    __shared__ unsigned int acc[2][AN_MAX_OWN];     // squared differences per owned patch; the other half is cleared meanwhile
     __shared__ uint8_t dec_l[AN_MAX_OWN];           // this frame's decisions of the owned tokens
     __shared__ int xch[2][AN_CLUSTER][AN_XCH];      // by frame parity and source CTA; written by every CTA of the cluster
-    __shared__ int s_cnt[AN_XCH];
+    __shared__ int s_cnt[2][AN_XCH];
     __shared__ int s_warp[3][AN_WARPS];
-    __shared__ int s_base[3];
     const int rank = (int)cluster.block_rank(), tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int n_tok = a.gh * a.gw;
     const int nb = (a.gh + AN_CLUSTER - 1) / AN_CLUSTER;                // bands per CTA
@@ -65,16 +66,23 @@ k_select_anchored(AnchorArgs a) {
     const int row_bytes = a.W * 3, chunks = row_bytes / 16;             // W is a multiple of 16
     const int rows = (band1 - band0) * 14;
     const size_t fb = (size_t)a.H * row_bytes;
+    const bool owner = tid < n_own;                                     // thread tid owns token tok0 + tid
     uint8_t* anc = a.anchor + (size_t)band0 * 14 * row_bytes;           // plain loads and stores: this CTA rewrites it
+    // the index lists start as all -1; the frames' steps then write the entries that exist
+    for (size_t i = (size_t)rank * AN_THREADS + tid; i < (size_t)a.B * 3 * n_tok; i += (size_t)AN_CLUSTER * AN_THREADS) a.idx[i] = -1;
+    if (owner) acc[0][tid] = 0;
+    if (tid < AN_XCH) s_cnt[0][tid] = 0;
+    cluster.sync();                                 // orders the fill before any CTA's entries, and the shared arrays
     for (int t = 0; t < a.B; ++t) {
         const bool has_prev = !(a.first_has_no_prev && t == 0);
         const uint8_t* fr = a.frames + (size_t)t * fb + (size_t)band0 * 14 * row_bytes;
         const int par = t & 1;
+        // pull the next frame's bands into the L2 while this one is worked on; fetch this token's spatial score early
+        if (t + 1 < a.B)
+            for (int i = tid; i < (rows * row_bytes + 127) / 128; i += AN_THREADS)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(fr + fb + (size_t)i * 128));
+        const float sv = owner ? __ldg(a.s + (size_t)t * n_tok + tok0 + tid) : 0.0f;
         // ---- Eq. 5 read literally, against the anchor: exact integer sums per patch
-        for (int i = tid; i < n_own; i += AN_THREADS) acc[i] = 0;
-        if (tid < AN_XCH) s_cnt[tid] = 0;
-        if (tid < 3) s_base[tid] = 0;
-        __syncthreads();
         if (has_prev)
             for (int i = tid; i < rows * chunks; i += AN_THREADS) {
                 const int r = i / chunks, k = i - r * chunks;
@@ -93,39 +101,48 @@ k_select_anchored(AnchorArgs a) {
                     hi = __dp4a(dh, dh, hi);
                 }
                 const int pl = (r / 14) * a.gw + p0;
-                atomicAdd(&acc[pl], lo);
-                if (hi) atomicAdd(&acc[pl + 1], hi);
+                atomicAdd(&acc[par][pl], lo);
+                if (hi) atomicAdd(&acc[par][pl + 1], hi);
             }
         __syncthreads();
-        // ---- scores, the tier each owned token would get in a frame that is not redundant, local counts
-        int my[AN_XCH] = {0, 0, 0, 0, 0, 0};
-        for (int i = tid; i < n_own; i += AN_THREADS) {
-            const float d = has_prev ? (float)sqrt((double)acc[i] / (double)(3 * 14 * 14)) : 0.0f;
-            a.dP[(size_t)t * n_tok + tok0 + i] = d;
-            const bool is_static = has_prev && d < a.tau_t;
-            int code;
+        // ---- the score, the code the token would get in a frame that is not redundant, the CTA's counts
+        int code = -1;
+        bool is_static = false;
+        if (owner) {
+            const float d = has_prev ? (float)sqrt((double)acc[par][tid] / (double)(3 * 14 * 14)) : 0.0f;
+            a.dP[(size_t)t * n_tok + tok0 + tid] = d;
+            is_static = has_prev && d < a.tau_t;
             if (a.patch_reuse && is_static) code = SALICACHE_REUSE;
-            else {
-                const float sv = a.s[(size_t)t * n_tok + tok0 + i];
-                code = sv > a.tau_high ? SALICACHE_FP16 : (sv > a.tau_med ? SALICACHE_INT8 : (sv > a.tau_low ? SALICACHE_INT4 : SALICACHE_PRUNE));
-            }
-            dec_l[i] = (uint8_t)code;
-            my[0] += is_static ? 1 : 0;
-            my[1 + code]++;
+            else code = sv > a.tau_high ? SALICACHE_FP16 : (sv > a.tau_med ? SALICACHE_INT8 : (sv > a.tau_low ? SALICACHE_INT4 : SALICACHE_PRUNE));
+            acc[par ^ 1][tid] = 0;                                      // for the next frame
         }
-#pragma unroll
-        for (int c = 0; c < AN_XCH; ++c) {
-            int v = my[c];
-#pragma unroll
-            for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            if (lane == 0 && v) atomicAdd(&s_cnt[c], v);
+        if (tid < AN_XCH) s_cnt[par ^ 1][tid] = 0;
+        unsigned m3[3];                                                 // lanes of this warp with an FP16, INT8, INT4 code
+        {
+            const unsigned ms = __ballot_sync(0xffffffffu, is_static);
+            const unsigned m0 = __ballot_sync(0xffffffffu, code == SALICACHE_REUSE);
+            const unsigned m1 = __ballot_sync(0xffffffffu, code == SALICACHE_PRUNE);
+            m3[2] = __ballot_sync(0xffffffffu, code == SALICACHE_INT4);
+            m3[1] = __ballot_sync(0xffffffffu, code == SALICACHE_INT8);
+            m3[0] = __ballot_sync(0xffffffffu, code == SALICACHE_FP16);
+            if (lane == 0) {
+                s_warp[0][wid] = __popc(m3[0]);
+                s_warp[1][wid] = __popc(m3[1]);
+                s_warp[2][wid] = __popc(m3[2]);
+                if (ms) atomicAdd(&s_cnt[par][0], __popc(ms));
+                if (m0) atomicAdd(&s_cnt[par][1 + SALICACHE_REUSE], __popc(m0));
+                if (m1) atomicAdd(&s_cnt[par][1 + SALICACHE_PRUNE], __popc(m1));
+                if (m3[2]) atomicAdd(&s_cnt[par][1 + SALICACHE_INT4], __popc(m3[2]));
+                if (m3[1]) atomicAdd(&s_cnt[par][1 + SALICACHE_INT8], __popc(m3[1]));
+                if (m3[0]) atomicAdd(&s_cnt[par][1 + SALICACHE_FP16], __popc(m3[0]));
+            }
         }
         __syncthreads();
         // ---- every CTA of the cluster receives this CTA's six numbers
         if (tid < AN_CLUSTER * AN_XCH) {
             const int dst = tid / AN_XCH, c = tid - dst * AN_XCH;
             int* remote = cluster.map_shared_rank(&xch[par][rank][c], dst);
-            *remote = s_cnt[c];
+            *remote = s_cnt[par][c];
         }
         cluster.sync();
         int n_static = 0, before[3] = {0, 0, 0}, total[5] = {0, 0, 0, 0, 0};
@@ -142,55 +159,24 @@ k_select_anchored(AnchorArgs a) {
         // Eq. 6, as k_select computes it
         const float R = has_prev ? __fdiv_rn((float)n_static, (float)n_tok) : 0.0f;
         const bool redundant = has_prev && (R > a.theta_R);
-        if (redundant) {
-            total[SALICACHE_REUSE] = n_tok;
-            total[SALICACHE_PRUNE] = total[SALICACHE_INT4] = total[SALICACHE_INT8] = total[SALICACHE_FP16] = 0;
-        }
         // ---- decisions and the stable per-tier index lists (FP16, INT8, INT4) of the owned tokens
-        for (int base = 0; base < n_own; base += AN_THREADS) {
-            const int i = base + tid;
-            int d = -1;
-            if (i < n_own) {
-                d = redundant ? SALICACHE_REUSE : dec_l[i];
-                dec_l[i] = (uint8_t)d;
-                a.decision[(size_t)t * n_tok + tok0 + i] = (uint8_t)d;
-            }
-            unsigned m3[3];
-            m3[0] = __ballot_sync(0xffffffffu, d == SALICACHE_FP16);
-            m3[1] = __ballot_sync(0xffffffffu, d == SALICACHE_INT8);
-            m3[2] = __ballot_sync(0xffffffffu, d == SALICACHE_INT4);
-            if (lane == 0) {
-#pragma unroll
-                for (int q = 0; q < 3; ++q) s_warp[q][wid] = __popc(m3[q]);
-            }
-            __syncthreads();
+        if (owner) {
+            const int d = redundant ? SALICACHE_REUSE : code;
+            dec_l[tid] = (uint8_t)d;
+            a.decision[(size_t)t * n_tok + tok0 + tid] = (uint8_t)d;
             const int tier = d == SALICACHE_FP16 ? 0 : (d == SALICACHE_INT8 ? 1 : (d == SALICACHE_INT4 ? 2 : -1));
             if (tier >= 0) {
-                int pos = before[tier] + s_base[tier];
+                int pos = before[tier];
                 for (int k = 0; k < wid; ++k) pos += s_warp[tier][k];
                 pos += __popc(m3[tier] & ((1u << lane) - 1u));
-                a.idx[((size_t)t * 3 + tier) * n_tok + pos] = tok0 + i;
+                a.idx[((size_t)t * 3 + tier) * n_tok + pos] = tok0 + tid;
             }
-            __syncthreads();
-            if (tid < 3) {
-                int q = 0;
-                for (int k = 0; k < AN_WARPS; ++k) q += s_warp[tid][k];
-                s_base[tid] += q;
-            }
-            __syncthreads();
-        }
-        // the lists' tails are -1; the CTAs share the work
-        {
-            const int tot3[3] = {total[SALICACHE_FP16], total[SALICACHE_INT8], total[SALICACHE_INT4]};
-#pragma unroll
-            for (int q = 0; q < 3; ++q)
-                for (int i = tot3[q] + rank * AN_THREADS + tid; i < n_tok; i += AN_CLUSTER * AN_THREADS)
-                    a.idx[((size_t)t * 3 + q) * n_tok + i] = -1;
         }
         if (rank == 0) {
-            if (tid < 5) a.counts[(size_t)t * 5 + tid] = total[tid];
+            if (tid < 5) a.counts[(size_t)t * 5 + tid] = redundant ? (tid == SALICACHE_REUSE ? n_tok : 0) : total[tid];
             if (tid == 0) a.redundant[t] = redundant ? 1 : 0;
         }
+        __syncthreads();
         // ---- the anchor takes the pixels of every owned patch whose token is not REUSE
         if (!redundant)
             for (int i = tid; i < rows * chunks; i += AN_THREADS) {
