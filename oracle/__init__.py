@@ -234,6 +234,23 @@ def select(dP, s, has_prev: bool, p: Params = Params()):
     return dec, idx, counts, int(red[0]), float(R[0])
 
 
+def select_ranked(dP, s, has_prev: bool, shares_permille, p: Params = Params()):
+    """One frame, tiers by rank of s among the tokens that are not reused.  shares_permille = (FP16, INT8, INT4) shares
+    of those tokens in thousandths.  Returns decision u8, idx i32 [3][n_tok], counts i32 [5], redundant."""
+    s = _c(s, np.float32)
+    n = s.shape[0]
+    dP = _c(dP if dP is not None else np.zeros(n, np.float32), np.float32)
+    dec = np.empty(n, np.uint8)
+    idx = np.empty((3, n), np.int32)
+    counts = np.empty(5, np.int32)
+    red = np.zeros(1, np.uint8)
+    pm16, pm8, pm4 = (int(x) for x in shares_permille)
+    lib().oracle_select_ranked(_p(dP), _p(s), C.c_int(n), C.c_int(int(has_prev)), C.c_int(p.patch_reuse), C.c_float(p.tau_t),
+                               C.c_float(p.theta_R), C.c_int(pm16), C.c_int(pm8), C.c_int(pm4), _p(dec), _p(idx), _p(counts),
+                               _p(red))
+    return dec, idx, counts, int(red[0])
+
+
 def select_anchored(frames: np.ndarray, s: np.ndarray, first_has_no_prev: bool, anchor: np.ndarray, p: Params = Params()):
     """Anchor-frame mode: every token is compared (Eq. 5 read literally) with the patch its cache entry came from.
     frames u8 [T][h][w][3], s f32 [T][n_tok], anchor u8 [h][w][3] (updated in place).

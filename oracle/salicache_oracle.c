@@ -528,6 +528,68 @@ EXPORT void oracle_select(const float* dP, const float* s, int n_tok, int has_pr
 }
 
 /* ------------------------------------------------------------------------- */
+/* Adaptive tier thresholds (a variant: the paper's thresholds are fixed and it */
+/* names their adaptation to the content as future work, Sec. V).  Reading: the */
+/* temporal test is unchanged (Eq. 6, and patch reuse); among the tokens of a   */
+/* frame that are not reused, the tiers of Eq. 8 are given out by rank of s_i   */
+/* instead of by fixed thresholds, so that fixed shares of them are kept at     */
+/* each precision whatever the frame's saliency level: with n_live such tokens, */
+/*   q16 = (n_live * pm16 + 500) / 1000 (integer division), likewise q8, q4,     */
+/*   each clipped to what is left of n_live;                                     */
+/* the q16 most salient are FP16, the next q8 INT8, the next q4 INT4, the rest   */
+/* pruned.  Ties in s go to the lower token id.  The thresholds of Eq. 8 thus     */
+/* become order statistics of the frame's own scores.                            */
+/* ------------------------------------------------------------------------- */
+typedef struct { float s; int32_t i; } oracle_ranked_t;
+static int oracle_ranked_cmp(const void* a, const void* b) {
+    const oracle_ranked_t* x = (const oracle_ranked_t*)a;
+    const oracle_ranked_t* y = (const oracle_ranked_t*)b;
+    if (x->s > y->s) return -1;
+    if (x->s < y->s) return 1;
+    return x->i < y->i ? -1 : (x->i > y->i ? 1 : 0);
+}
+EXPORT void oracle_select_ranked(const float* dP, const float* s, int n_tok, int has_prev, int patch_reuse, float tau_t,
+                                 float theta_R, int pm16, int pm8, int pm4, uint8_t* decision, int32_t* idx,
+                                 int32_t* counts, uint8_t* frame_redundant) {
+    int n_static = 0;
+    if (has_prev)
+        for (int i = 0; i < n_tok; ++i) n_static += (dP[i] < tau_t);
+    float R = has_prev ? (float)n_static / (float)n_tok : 0.0f;
+    int redundant = has_prev && (R > theta_R);
+    oracle_ranked_t* live = (oracle_ranked_t*)malloc((size_t)n_tok * sizeof(oracle_ranked_t));
+    int n_live = 0;
+    for (int i = 0; i < n_tok; ++i) {
+        if (redundant || (patch_reuse && has_prev && dP[i] < tau_t)) decision[i] = 0;
+        else {
+            live[n_live].s = s[i];
+            live[n_live].i = i;
+            ++n_live;
+        }
+    }
+    qsort(live, (size_t)n_live, sizeof(oracle_ranked_t), oracle_ranked_cmp);
+    long left = n_live;
+    long q16 = ((long)n_live * pm16 + 500) / 1000; if (q16 > left) q16 = left; left -= q16;
+    long q8 = ((long)n_live * pm8 + 500) / 1000;   if (q8 > left) q8 = left;   left -= q8;
+    long q4 = ((long)n_live * pm4 + 500) / 1000;   if (q4 > left) q4 = left;
+    for (int r = 0; r < n_live; ++r)
+        decision[live[r].i] = r < q16 ? 4 : (r < q16 + q8 ? 3 : (r < q16 + q8 + q4 ? 2 : 1));
+    free(live);
+    for (int c = 0; c < 5; ++c) counts[c] = 0;
+    int n16 = 0, n8 = 0, n4 = 0;
+    for (int i = 0; i < n_tok; ++i) {
+        uint8_t d = decision[i];
+        counts[d]++;
+        if (d == 4) idx[0 * n_tok + n16++] = i;
+        else if (d == 3) idx[1 * n_tok + n8++] = i;
+        else if (d == 2) idx[2 * n_tok + n4++] = i;
+    }
+    for (int i = n16; i < n_tok; ++i) idx[0 * n_tok + i] = -1;
+    for (int i = n8; i < n_tok; ++i) idx[1 * n_tok + i] = -1;
+    for (int i = n4; i < n_tok; ++i) idx[2 * n_tok + i] = -1;
+    *frame_redundant = (uint8_t)redundant;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Anchor-frame mode of the temporal test (a variant: the paper compares        */
 /* consecutive frames, Sec. III-A, which lets a slow pan or a slow fade stay    */
 /* "static" forever because every single step is below tau_t).  Here token i of */
