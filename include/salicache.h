@@ -260,6 +260,22 @@ SALICACHE_API int salicache_saliency_noalloc(const salicache_params* p, const ui
                                              int32_t* d_status_or_null, void* cuda_stream);
 
 /*
+ * Decisions with adaptive tier thresholds (a variant; the paper's thresholds are fixed and Sec. V names their
+ * adaptation to the content as future work).  The temporal test is salicache_select's (Eq. 6, patch reuse).  Among
+ * the n_live tokens of a frame that are not reused, Eq. 8's tiers are given out by rank of s_i in fixed shares:
+ *   q16 = (n_live * share_fp16_permille + 500) / 1000 (integer division), likewise q8 and q4, each clipped to what
+ *   is left of n_live; the q16 most salient tokens are FP16, the next q8 INT8, the next q4 INT4, the rest PRUNE;
+ *   equal scores go to the lower token id first.
+ * tau_high, tau_med and tau_low of the context are not used.  All other arguments, outputs and errors as for
+ * salicache_select; shares outside [0, 1000]: E_PARAM; contexts with more than 3072 tokens per frame: E_PARAM.
+ */
+SALICACHE_API int salicache_select_ranked(salicache_ctx* ctx, const float* d_deltaP, const float* d_s, int B,
+                                          int first_has_no_prev, int share_fp16_permille, int share_int8_permille,
+                                          int share_int4_permille, uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts,
+                                          uint8_t* d_frame_redundant, int64_t* d_row_offset, int64_t* d_fill,
+                                          void* cuda_stream);
+
+/*
  * Temporal test and decisions in anchor-frame mode (a variant; the paper's test compares consecutive frames,
  * Sec. III-A, under which a slow pan or fade whose every step stays below tau_t is reused forever).  Token i of
  * frame b is compared with the patch its cache entry was computed from, i.e. patch i of the last frame in which

@@ -9,7 +9,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 LIB = os.path.join(_PKG, "libsalicache.so")
-SOURCES = ["api.cu", "flow.cu", "saliency.cu", "select.cu", "anchor.cu", "kv.cu", "attend.cu", "noalloc.cu"]
+SOURCES = ["api.cu", "flow.cu", "saliency.cu", "select.cu", "anchor.cu", "ranked.cu", "kv.cu", "attend.cu", "noalloc.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--fmad=true",
          "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-I", os.path.join(_ROOT, "include"), "-I", CSRC]
 

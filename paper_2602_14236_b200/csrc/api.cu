@@ -260,6 +260,21 @@ int salicache_select(salicache_ctx* c, const float* d_deltaP, const float* d_s, 
                      d_row_offset, d_fill, (cudaStream_t)cuda_stream);
 }
 
+int salicache_select_ranked(salicache_ctx* c, const float* d_deltaP, const float* d_s, int B, int first_has_no_prev,
+                            int share_fp16_permille, int share_int8_permille, int share_int4_permille, uint8_t* d_decision,
+                            int32_t* d_idx, int32_t* d_counts, uint8_t* d_frame_redundant, int64_t* d_row_offset,
+                            int64_t* d_fill, void* cuda_stream) {
+    if (!c || !d_s || !d_decision || !d_idx || !d_counts || !d_frame_redundant || !d_row_offset || !d_fill)
+        return SALICACHE_E_NULL;
+    if (B < 0 || B > c->p.max_batch) return SALICACHE_E_SHAPE;
+    if (share_fp16_permille < 0 || share_int8_permille < 0 || share_int4_permille < 0 || share_fp16_permille > 1000 ||
+        share_int8_permille > 1000 || share_int4_permille > 1000)
+        return SALICACHE_E_PARAM;
+    return sc_select_ranked(c, d_deltaP, d_s, B, first_has_no_prev, share_fp16_permille, share_int8_permille,
+                            share_int4_permille, d_decision, d_idx, d_counts, d_frame_redundant, d_row_offset, d_fill,
+                            (cudaStream_t)cuda_stream);
+}
+
 int salicache_select_anchored(salicache_ctx* c, const uint8_t* d_frames, const float* d_s, int B, int first_has_no_prev,
                               uint8_t* d_anchor, float* d_deltaP, uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts,
                               uint8_t* d_frame_redundant, int64_t* d_row_offset, int64_t* d_fill, void* cuda_stream) {
