@@ -429,6 +429,17 @@ def run_extras(sc, synth, ctx, wl, T, frames, dP, dev, peak, pools, fill, stored
     ng = wl2.HD // 128
     per_tok = wl2.HD * 2
     stored = c[4] * per_tok + c[3] * (wl2.HD + 2 * ng) + c[2] * (wl2.HD // 2 + 4 * ng)
+    # the adaptive rule on the same scores: shares of the stored-or-pruned tokens taken from the paper's Fig. 3
+    # (FP16 31.7, INT8 7.1, INT4 21.4, pruned 13.1 % of all patches = 432, 97, 292 per mille of those not skipped)
+    shares = (432, 97, 292)
+    fill2.zero_()
+    ms_ranked = timed(lambda: sc.salicache_select_ranked(c2, dP2, s2, wl2.T, True, shares, dec2, idx2, cnt2, red2, off2, fill2), reps=5)
+    cr = cnt2.sum(dim=0).cpu().numpy().astype(float)
+    out["adaptive_tiers_workload2"] = {
+        "what": "salicache_select_ranked on workload 2: tiers by rank of the spatial score, shares 432 / 97 / 292 per mille "
+                "of the tokens that are not reused (Fig. 3's proportions)",
+        "ms": round(ms_ranked, 4), "frames": wl2.T,
+        "percent": {k: round(100 * cr[i] / cr.sum(), 2) for k, i in (("reuse", 0), ("prune", 1), ("int4", 2), ("int8", 3), ("fp16", 4))}}
     out["four_tier_workload2"] = {
         "what": "workload 2 frames, four-tier rule (Eq. 8); paper Fig. 3: skipped 26.7, pruned 13.1, INT4 21.4, INT8 7.1, FP16 31.7 %",
         "percent": {k: round(100 * c[i] / tot, 2) for k, i in (("reuse", 0), ("prune", 1), ("int4", 2), ("int8", 3), ("fp16", 4))},
