@@ -391,6 +391,8 @@ __device__ __forceinline__ void i4_fetch(I4Tile& x, const I4Addr<PITCH, NG>& a, 
     else i4_load<false>(x, a, tile, t0, r1, g8, c4);      // loads nothing at all once tile >= r1
 }
 
+constexpr int I4_MIN_ROWS = 512;   // 8 tiles per warp
+
 // Running state of a warp: m is its maximum (the same in every lane); den and zacc are per-lane partial sums;
 // acc[b] holds, in the lanes with c4 == 0, dimensions 16 g8 + 2 b (.x high, .y low) and 16 g8 + 2 b + 1 (.z, .w).
 struct I4State {
@@ -483,7 +485,9 @@ k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restr
     const int lane = t & 31, wid = t >> 5, g8 = lane >> 2, c4 = lane & 3;
     const int HD = H * AT_D;
     const long long n4 = min(fill[2], pp.cap4);
-    const long long per = ((n4 + AT_CHUNKS - 1) / AT_CHUNKS + 15) / 16 * 16;      // whole tiles per chunk
+    // whole tiles per chunk, and at least I4_MIN_ROWS rows: a small cache is spread over fewer CTAs (the rest leave
+    // at once), so that the fixed cost of a CTA, staging the query and merging its warps, is paid less often
+    const long long per = max((long long)I4_MIN_ROWS, ((n4 + AT_CHUNKS - 1) / AT_CHUNKS + 15) / 16 * 16);
     const long long r0 = (long long)c * per, r1 = min(n4, r0 + per);
     if (r0 >= r1) {                                 // nothing in this chunk: a record the merge skips
         if (t == 0) {
