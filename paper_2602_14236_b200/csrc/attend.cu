@@ -391,8 +391,6 @@ __device__ __forceinline__ void i4_fetch(I4Tile& x, const I4Addr<PITCH, NG>& a, 
     else i4_load<false>(x, a, tile, t0, r1, g8, c4);      // loads nothing at all once tile >= r1
 }
 
-constexpr int I4_MIN_ROWS = 512;   // 8 tiles per warp
-
 // Running state of a warp: m is its maximum (the same in every lane); den and zacc are per-lane partial sums;
 // acc[b] holds, in the lanes with c4 == 0, dimensions 16 g8 + 2 b (.x high, .y low) and 16 g8 + 2 b + 1 (.z, .w).
 struct I4State {
@@ -474,7 +472,7 @@ __device__ __forceinline__ void i4_tile(I4State& st, const I4Tile& x, const uint
 
 template <int PITCH, int NG>
 __global__ void __launch_bounds__(AT_D)
-k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int ng,
+k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int ng, int min_rows,
               float* __restrict__ ws) {
     __shared__ __align__(16) float qs[AT_D];
     __shared__ __align__(16) __half qp[AT_D];       // every 8 elements ordered 0 4 1 5 2 6 3 7
@@ -485,9 +483,9 @@ k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restr
     const int lane = t & 31, wid = t >> 5, g8 = lane >> 2, c4 = lane & 3;
     const int HD = H * AT_D;
     const long long n4 = min(fill[2], pp.cap4);
-    // whole tiles per chunk, and at least I4_MIN_ROWS rows: a small cache is spread over fewer CTAs (the rest leave
-    // at once), so that the fixed cost of a CTA, staging the query and merging its warps, is paid less often
-    const long long per = max((long long)I4_MIN_ROWS, ((n4 + AT_CHUNKS - 1) / AT_CHUNKS + 15) / 16 * 16);
+    // whole tiles per chunk, and at least min_rows rows: a cache that is not huge is spread over fewer CTAs (the
+    // rest leave at once), so that the fixed cost of a CTA, staging the query and merging its warps, is paid less often
+    const long long per = max((long long)min_rows, ((n4 + AT_CHUNKS - 1) / AT_CHUNKS + 15) / 16 * 16);
     const long long r0 = (long long)c * per, r1 = min(n4, r0 + per);
     if (r0 >= r1) {                                 // nothing in this chunk: a record the merge skips
         if (t == 0) {
@@ -635,9 +633,12 @@ int sc_attend(salicache_ctx* c, const void* d_q, const salicache_pools* pools, c
     k_attend_partial<<<grid16, AT_D, 0, st>>>((const __half*)d_q, pp, (const long long*)d_fill, p.heads, ng, 0, c->attend_ws);
     const __half* qh = (const __half*)d_q;
     const long long* fl = (const long long*)d_fill;
-    if (p.heads == 32 && ng == 32) k_attend_int4<32 * AT_D / 2, 32><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, c->attend_ws);
-    else if (p.heads == 32 && ng == 1) k_attend_int4<32 * AT_D / 2, 1><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, c->attend_ws);
-    else k_attend_int4<0, 0><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, c->attend_ws);
+    // rows per chunk of the INT4 kernel: up to 4096 (64 tiles per warp) when there are many (layer, head) pairs to
+    // fill the GPU with, fewer when there are few
+    const int min_rows = (int)std::min<long long>(4096, std::max<long long>(256, 8ll * p.L * p.heads)) / 16 * 16;
+    if (p.heads == 32 && ng == 32) k_attend_int4<32 * AT_D / 2, 32><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, min_rows, c->attend_ws);
+    else if (p.heads == 32 && ng == 1) k_attend_int4<32 * AT_D / 2, 1><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, min_rows, c->attend_ws);
+    else k_attend_int4<0, 0><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, min_rows, c->attend_ws);
     dim3 gm(p.heads, p.L);
     k_attend_merge<<<gm, AT_D, 0, st>>>(c->attend_ws, p.heads, nch, d_out);
     c->launches += 3;
