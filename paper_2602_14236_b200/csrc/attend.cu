@@ -20,9 +20,12 @@ namespace {
 
 constexpr int AT_D = 128;           // head size = threads per CTA = quantisation group
 constexpr int AT_WARPS = AT_D / 32;
-constexpr int AT_CHUNKS = 64;       // partial results per (layer, head)
+constexpr int AT_CHUNKS = 64;       // partial results of the INT4 kernel per (layer, head)
+constexpr int AT_CH16 = 32;         // ... of the FP16 kernel (at most), and
+constexpr int AT_CH8 = 32;          // ... of the INT8 kernel
 constexpr int AT_REC = AT_D + 2;    // partial record: 128 sums, running maximum, running denominator
-constexpr int AT_RECS = 2 * AT_CHUNKS;   // records per (layer, head): AT_CHUNKS of each of the two partial kernels
+constexpr int AT_RECS = AT_CH16 + AT_CH8 + AT_CHUNKS;   // records per (layer, head): FP16, then INT8, then INT4 chunks
+constexpr int AT_REC8 = AT_CH16, AT_REC4 = AT_CH16 + AT_CH8;      // first record of the INT8 and of the INT4 kernel
 
 struct AtPools {
     const uint8_t* fp16_pool;
@@ -93,7 +96,7 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 
 __global__ void __launch_bounds__(AT_D)
 k_attend_partial(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int ng,
-                 int with_int4, float* __restrict__ ws) {
+                 int with_int8, int with_int4, float* __restrict__ ws) {
     __shared__ __align__(16) float qs[AT_D];        // the query as binary32 (for sum(q))
     __shared__ __align__(16) __half qn[AT_D];       // the query in natural order
     __shared__ __align__(16) __half qp[AT_D];       // the query with every 8 elements ordered 0 4 1 5 2 6 3 7 (INT4 pairs)
@@ -105,8 +108,9 @@ k_attend_partial(const __half* __restrict__ q, AtPools pp, const long long* __re
     const int h = blockIdx.x, c = blockIdx.y, l = blockIdx.z, t = threadIdx.x;
     const int lane = t & 31, wid = t >> 5;
     const int HD = H * AT_D;
-    const long long n16 = min(fill[0], pp.cap16), n8 = min(fill[1], pp.cap8);
-    const long long n4 = with_int4 ? min(fill[2], pp.cap4) : 0;      // the INT4 rows may be left to k_attend_int4
+    const long long n16 = min(fill[0], pp.cap16);
+    const long long n8 = with_int8 ? min(fill[1], pp.cap8) : 0;      // the INT8 rows may be left to k_attend_int8,
+    const long long n4 = with_int4 ? min(fill[2], pp.cap4) : 0;      // the INT4 rows to k_attend_int4
     const long long R = n16 + n8 + n4;
     const long long per = (R + gridDim.y - 1) / gridDim.y;      // the host sizes the grid's chunks by the pools' capacity
     const long long r0 = (long long)c * per, r1 = min(R, r0 + per);
@@ -489,7 +493,7 @@ k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restr
     const long long r0 = (long long)c * per, r1 = min(n4, r0 + per);
     if (r0 >= r1) {                                 // nothing in this chunk: a record the merge skips
         if (t == 0) {
-            float* rec = ws + (((size_t)l * H + h) * AT_RECS + AT_CHUNKS + c) * AT_REC;
+            float* rec = ws + (((size_t)l * H + h) * AT_RECS + AT_REC4 + c) * AT_REC;
             rec[AT_D] = -INFINITY;
             rec[AT_D + 1] = 0.0f;
         }
@@ -579,12 +583,241 @@ k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restr
             dsum += e * wstat[k][1];
         }
     }
-    float* rec = ws + (((size_t)l * H + h) * AT_RECS + AT_CHUNKS + c) * AT_REC;
+    float* rec = ws + (((size_t)l * H + h) * AT_RECS + AT_REC4 + c) * AT_REC;
     rec[t] = sum;
     if (t == 0) {
         rec[AT_D] = M;
         rec[AT_D + 1] = dsum;
     }
+}
+
+// ---- INT8 rows on the matrix instructions, the same plan as for INT4: scores = 16 key rows x 16 dimensions
+// times the query in columns 0 and 2; values = 16 dimensions x 16 value rows times the split weights.  A code
+// byte becomes binary16 by a byte permute with 0x64 above it (1024 + (code + 128) after flipping its sign bit)
+// and one subtraction of 1152.  Symmetric quantiser: no zero point.
+struct I8Tile {
+    uint4 ka0, ka1, kb0, kb1;      // keys of rows g8 and g8 + 8: dimensions 16 c4 .. + 15 and 64 + 16 c4 .. + 15
+    uint4 v0, v1, v2, v3;          // values of rows c4, c4 + 4, c4 + 8, c4 + 12: dimensions 16 g8 .. + 15
+    uint32_t ks, vs;               // binary16 scales of the row whose weight this lane computes: g8 + 8 * (c4 & 1)
+};
+struct I8Addr {
+    const uint8_t* k;
+    const uint8_t* v;
+    const uint16_t* ks;
+    const uint16_t* vs;
+    size_t pitch, ng;
+};
+__device__ __forceinline__ void i8_fetch(I8Tile& x, const I8Addr& a, long long tile, long long t0, long long r1, int g8, int c4) {
+    const size_t d = (size_t)(tile - t0), P = a.pitch;
+    const uint8_t* k = a.k + d * P;
+    const uint8_t* v = a.v + d * P;
+    const uint16_t* ks = a.ks + d * a.ng;
+    const uint16_t* vs = a.vs + d * a.ng;
+    if (tile + 16 <= r1) {
+        x.ka0 = ld_stream16(k);
+        x.ka1 = ld_stream16(k + 64);
+        x.kb0 = ld_stream16(k + 8 * P);
+        x.kb1 = ld_stream16(k + 8 * P + 64);
+        x.v0 = ld_stream16(v);
+        x.v1 = ld_stream16(v + 4 * P);
+        x.v2 = ld_stream16(v + 8 * P);
+        x.v3 = ld_stream16(v + 12 * P);
+        x.ks = __ldg(ks);
+        x.vs = __ldg(vs);
+    } else {                                        // rows at or beyond r1 read as zero codes and are not touched
+        const uint4 z = make_uint4(0, 0, 0, 0);
+        x.ka0 = x.ka1 = x.kb0 = x.kb1 = x.v0 = x.v1 = x.v2 = x.v3 = z;
+        x.ks = x.vs = 0;
+        const long long ra = tile + g8, rv = tile + c4;
+        if (ra < r1) { x.ka0 = ld_stream16(k); x.ka1 = ld_stream16(k + 64); }
+        if (ra + 8 < r1) { x.kb0 = ld_stream16(k + 8 * P); x.kb1 = ld_stream16(k + 8 * P + 64); }
+        if (ra + 8 * (c4 & 1) < r1) { x.ks = __ldg(ks); x.vs = __ldg(vs); }
+        if (rv < r1) x.v0 = ld_stream16(v);
+        if (rv + 4 < r1) x.v1 = ld_stream16(v + 4 * P);
+        if (rv + 8 < r1) x.v2 = ld_stream16(v + 8 * P);
+        if (rv + 12 < r1) x.v3 = ld_stream16(v + 12 * P);
+    }
+}
+struct ByteConst {
+    uint32_t hi64, magic;           // 0x64 in every byte; binary16 pair (1152, 1152)
+    __device__ __forceinline__ void init() {        // opaque to the compiler, so that they stay in registers
+        asm volatile("mov.b32 %0, 0x64646464;" : "=r"(hi64));
+        asm volatile("mov.b32 %0, 0x64806480;" : "=r"(magic));
+    }
+    // bytes i and j (0..3) of a word of sign-flipped codes as a binary16 pair
+    template <int I, int J>
+    __device__ __forceinline__ uint32_t pair(uint32_t u) const { return hsub2u(__byte_perm(u, hi64, 0x4040 | I | (J << 8)), magic); }
+};
+
+__device__ __forceinline__ void i8_tile(I4State& st, const I8Tile& x, const uint32_t (&qf)[8][2], const ByteConst& bc, long long tile,
+                                        long long r1, float rs, int g8, int c4) {
+    float sc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    {
+        const uint32_t wa[8] = {x.ka0.x, x.ka0.y, x.ka0.z, x.ka0.w, x.ka1.x, x.ka1.y, x.ka1.z, x.ka1.w};
+        const uint32_t wb[8] = {x.kb0.x, x.kb0.y, x.kb0.z, x.kb0.w, x.kb1.x, x.kb1.y, x.kb1.z, x.kb1.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t ua = wa[j] ^ 0x80808080u, ub = wb[j] ^ 0x80808080u;
+            mma16816(sc, bc.pair<0, 1>(ua), bc.pair<0, 1>(ub), bc.pair<2, 3>(ua), bc.pair<2, 3>(ub), qf[j][0], qf[j][1]);
+        }
+    }
+    // one row per lane: c4 == 0 takes row g8 (column 0), c4 == 1 takes row g8 + 8 (column 2)
+    const bool own = c4 < 2 && tile + g8 + 8 * c4 < r1;
+    const float s = own ? rs * (c4 ? sc[2] : sc[0]) * h2f((uint16_t)x.ks) : -INFINITY;
+    const float sv = own ? h2f((uint16_t)x.vs) : 0.0f;
+    if (__any_sync(0xffffffffu, s > st.m || sv * st.F >= 32768.0f)) {
+        const float m_new = fmaxf(st.m, warp_max(s));
+        const float corr = st.m == -INFINITY ? 0.0f : __expf(st.m - m_new);
+        st.m = m_new;
+        const float smax = warp_max(sv);
+        float Fn = st.F;
+        for (int k = 0; k < 40 && smax * Fn >= 32768.0f; ++k) Fn *= 0.5f;
+        const float rescale = corr * (Fn / st.F);
+        st.F = Fn;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) st.acc[b][i] *= rescale;
+        }
+        st.den *= corr;
+    }
+    const float pr = __expf(s - st.m);
+    st.den += pr;
+    uint32_t pack;
+    {
+        const float w = pr * sv * st.F;
+        const __half hi = __float2half_rn(w);
+        const __half lo = __float2half_rn(w - __half2float(hi));
+        pack = (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
+    }
+    // B fragment: column 0 = high halves, column 1 = low halves; k = tile rows c4, c4 + 4, c4 + 8, c4 + 12.
+    // Row r of the tile was weighted by lane 4 * (r % 8) + r / 8.
+    const uint32_t x1 = __shfl_sync(0xffffffffu, pack, 4 * c4), x2 = __shfl_sync(0xffffffffu, pack, 4 * c4 + 16);
+    const uint32_t y1 = __shfl_sync(0xffffffffu, pack, 4 * c4 + 1), y2 = __shfl_sync(0xffffffffu, pack, 4 * c4 + 17);
+    const uint32_t psel = g8 == 0 ? 0x5410u : 0x7632u;
+    const uint32_t b0 = g8 < 2 ? __byte_perm(x1, x2, psel) : 0u, b1 = g8 < 2 ? __byte_perm(y1, y2, psel) : 0u;
+    {
+        const uint32_t w0[4] = {x.v0.x, x.v0.y, x.v0.z, x.v0.w}, w1[4] = {x.v1.x, x.v1.y, x.v1.z, x.v1.w};
+        const uint32_t w2[4] = {x.v2.x, x.v2.y, x.v2.z, x.v2.w}, w3[4] = {x.v3.x, x.v3.y, x.v3.z, x.v3.w};
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            // bytes 2 b and 2 b + 1 (dimensions 16 g8 + 2 b, + 1) of two rows in one word: (r.d, r.d+1, r'.d, r'.d+1)
+            const uint32_t sel = (b & 1) ? 0x7632u : 0x5410u;
+            const uint32_t t1 = __byte_perm(w0[b >> 1], w1[b >> 1], sel) ^ 0x80808080u;
+            const uint32_t t2 = __byte_perm(w2[b >> 1], w3[b >> 1], sel) ^ 0x80808080u;
+            mma16816(st.acc[b], bc.pair<0, 2>(t1), bc.pair<1, 3>(t1), bc.pair<0, 2>(t2), bc.pair<1, 3>(t2), b0, b1);
+        }
+    }
+}
+
+// Merge the four warps of a CTA of the matrix-instruction kernels and write its partial record.
+__device__ __forceinline__ void mma_finish(const I4State& st, float (*wpart)[AT_D], float (*wstat)[2], float* rec, int g8, int c4) {
+    const int t = threadIdx.x, lane = t & 31, wid = t >> 5;
+    const float den = warp_sum(st.den);
+    const float zs = warp_sum(st.zacc);
+    if (c4 == 0) {
+        const float invF = 1.0f / st.F;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            wpart[wid][16 * g8 + 2 * b] = (st.acc[b][0] + st.acc[b][1]) * invF + zs;
+            wpart[wid][16 * g8 + 2 * b + 1] = (st.acc[b][2] + st.acc[b][3]) * invF + zs;
+        }
+    }
+    if (lane == 0) {
+        wstat[wid][0] = st.m;
+        wstat[wid][1] = den;
+    }
+    __syncthreads();
+    float M = wstat[0][0];
+#pragma unroll
+    for (int k = 1; k < AT_WARPS; ++k) M = fmaxf(M, wstat[k][0]);
+    float sum = 0.0f, dsum = 0.0f;
+    if (M != -INFINITY) {
+#pragma unroll
+        for (int k = 0; k < AT_WARPS; ++k) {
+            const float e = wstat[k][0] == -INFINITY ? 0.0f : __expf(wstat[k][0] - M);
+            sum += e * wpart[k][t];
+            dsum += e * wstat[k][1];
+        }
+    }
+    rec[t] = sum;
+    if (t == 0) {
+        rec[AT_D] = M;
+        rec[AT_D + 1] = dsum;
+    }
+}
+
+__global__ void __launch_bounds__(AT_D)
+k_attend_int8(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int ng, int min_rows,
+              float* __restrict__ ws) {
+    __shared__ __align__(16) __half qn[AT_D];
+    __shared__ float wpart[AT_WARPS][AT_D];
+    __shared__ float wstat[AT_WARPS][2];
+    const int h = blockIdx.x, c = blockIdx.y, l = blockIdx.z, t = threadIdx.x;
+    const int lane = t & 31, wid = t >> 5, g8 = lane >> 2, c4 = lane & 3;
+    const size_t HD = (size_t)H * AT_D;
+    const long long n8 = min(fill[1], pp.cap8);
+    const long long per = max((long long)min_rows, ((n8 + AT_CH8 - 1) / AT_CH8 + 15) / 16 * 16);
+    const long long r0 = (long long)c * per, r1 = min(n8, r0 + per);
+    float* rec = ws + (((size_t)l * H + h) * AT_RECS + AT_REC8 + c) * AT_REC;
+    if (r0 >= r1) {                                 // nothing in this chunk: a record the merge skips
+        if (t == 0) {
+            rec[AT_D] = -INFINITY;
+            rec[AT_D + 1] = 0.0f;
+        }
+        return;
+    }
+    qn[t] = q[((size_t)l * H + h) * AT_D + t];
+    __syncthreads();
+    const float rs = rsqrtf((float)AT_D);
+    const int g = ng == 1 ? 0 : h;
+    // the query as B fragments: instruction j takes dimensions base .. base + 3 of the lane's key bytes, base =
+    // 16 c4 + 4 j for j < 4 and 64 + 16 c4 + 4 (j - 4) after; columns 0 and 2 (lanes 0..3 and 8..11)
+    uint32_t qf[8][2];
+    {
+        const uint32_t* q32 = reinterpret_cast<const uint32_t*>(qn);
+        const bool has = g8 == 0 || g8 == 2;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int base = (j < 4 ? 16 * c4 + 4 * j : 64 + 16 * c4 + 4 * (j - 4)) / 2;
+            qf[j][0] = has ? q32[base] : 0u;
+            qf[j][1] = has ? q32[base + 1] : 0u;
+        }
+    }
+    const long long t0 = r0 + 16 * wid;             // this warp's first tile
+    I8Addr ad;
+    ad.pitch = HD;
+    ad.ng = (size_t)ng;
+    const size_t own_row = (size_t)(t0 + g8 + 8 * (c4 & 1));
+    ad.k = pp.int8_codes + ((size_t)(2 * l) * pp.cap8 + (size_t)(t0 + g8)) * HD + (size_t)h * AT_D + 16 * c4;
+    ad.v = pp.int8_codes + ((size_t)(2 * l + 1) * pp.cap8 + (size_t)(t0 + c4)) * HD + (size_t)h * AT_D + 16 * g8;
+    ad.ks = reinterpret_cast<const uint16_t*>(pp.int8_scale) + ((size_t)(2 * l) * pp.cap8 + own_row) * ng + g;
+    ad.vs = reinterpret_cast<const uint16_t*>(pp.int8_scale) + ((size_t)(2 * l + 1) * pp.cap8 + own_row) * ng + g;
+    ByteConst bc;
+    bc.init();
+    I4State st;
+#pragma unroll
+    for (int b = 0; b < 8; ++b) st.acc[b][0] = st.acc[b][1] = st.acc[b][2] = st.acc[b][3] = 0.0f;
+    st.m = -INFINITY;
+    st.den = st.zacc = 0.0f;
+    st.F = 4096.0f;
+    constexpr long long STEP = 16 * AT_WARPS;
+    I8Tile xa, xb;                                  // two tiles in turn: one is consumed while the other is in flight
+    long long tile = t0;
+    if (tile < r1) {
+        i8_fetch(xa, ad, tile, t0, r1, g8, c4);
+        for (;;) {
+            i8_fetch(xb, ad, tile + STEP, t0, r1, g8, c4);
+            i8_tile(st, xa, qf, bc, tile, r1, rs, g8, c4);
+            tile += STEP;
+            if (tile >= r1) break;
+            i8_fetch(xa, ad, tile + STEP, t0, r1, g8, c4);
+            i8_tile(st, xb, qf, bc, tile, r1, rs, g8, c4);
+            tile += STEP;
+            if (tile >= r1) break;
+        }
+    }
+    mma_finish(st, wpart, wstat, rec, g8, c4);
 }
 
 // Merge the partial results of one (layer, head): out = sum_c e^(m_c - M) acc_c / sum_c e^(m_c - M) den_c.
@@ -595,8 +828,8 @@ k_attend_merge(const float* __restrict__ ws, int H, int nch, float* __restrict__
     static_assert(AT_RECS == AT_D, "one record per thread in the statistics pass");
     const int h = blockIdx.x, l = blockIdx.y, t = threadIdx.x;
     const float* rec = ws + ((size_t)l * H + h) * AT_RECS * AT_REC;
-    // records 0 .. nch-1 come from k_attend_partial, AT_CHUNKS .. AT_RECS-1 from k_attend_int4
-    const bool written = t < nch || t >= AT_CHUNKS;
+    // records 0 .. nch-1 come from k_attend_partial, the rest from k_attend_int8 and k_attend_int4
+    const bool written = t < nch || t >= AT_REC8;
     const float mc = written ? rec[t * AT_REC + AT_D] : -INFINITY;
     const float dc = written ? rec[t * AT_REC + AT_D + 1] : 0.0f;
     const float M = block_max(mc, red);
@@ -626,22 +859,24 @@ int sc_attend(salicache_ctx* c, const void* d_q, const salicache_pools* pools, c
     if (pp.cap16 >= (1ll << 28) || pp.cap8 >= (1ll << 28) || pp.cap4 >= (1ll << 28)) return SALICACHE_E_SHAPE;
     const int ng = p.group == AT_D ? p.heads : 1;
     dim3 grid(p.heads, AT_CHUNKS, p.L);
-    // FP16 and INT8 rows one row per thread; INT4 rows, the bulk of a compressed cache, on the matrix instructions.
-    // The first kernel gets as many chunks as its two pools can fill with four tiles each, 64 at most.
-    const int nch = (int)std::min<long long>(AT_CHUNKS, std::max<long long>(1, (pp.cap16 + pp.cap8 + 4 * AT_D - 1) / (4 * AT_D)));
+    // FP16 rows one row per thread; INT8 and INT4 rows, the bulk of a compressed cache, on the matrix instructions.
+    // The first kernel gets as many chunks as its pool can fill with four tiles each, 32 at most.
+    const int nch = (int)std::min<long long>(AT_CH16, std::max<long long>(1, (pp.cap16 + 4 * AT_D - 1) / (4 * AT_D)));
     dim3 grid16(p.heads, nch, p.L);
-    k_attend_partial<<<grid16, AT_D, 0, st>>>((const __half*)d_q, pp, (const long long*)d_fill, p.heads, ng, 0, c->attend_ws);
+    k_attend_partial<<<grid16, AT_D, 0, st>>>((const __half*)d_q, pp, (const long long*)d_fill, p.heads, ng, 0, 0, c->attend_ws);
     const __half* qh = (const __half*)d_q;
     const long long* fl = (const long long*)d_fill;
     // rows per chunk of the INT4 kernel: up to 4096 (64 tiles per warp) when there are many (layer, head) pairs to
     // fill the GPU with, fewer when there are few
     const int min_rows = (int)std::min<long long>(4096, std::max<long long>(256, 8ll * p.L * p.heads)) / 16 * 16;
+    dim3 grid8(p.heads, AT_CH8, p.L);
+    k_attend_int8<<<grid8, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, min_rows, c->attend_ws);
     if (p.heads == 32 && ng == 32) k_attend_int4<32 * AT_D / 2, 32><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, min_rows, c->attend_ws);
     else if (p.heads == 32 && ng == 1) k_attend_int4<32 * AT_D / 2, 1><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, min_rows, c->attend_ws);
     else k_attend_int4<0, 0><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, min_rows, c->attend_ws);
     dim3 gm(p.heads, p.L);
     k_attend_merge<<<gm, AT_D, 0, st>>>(c->attend_ws, p.heads, nch, d_out);
-    c->launches += 3;
+    c->launches += 4;
     SC_CHECK(cudaGetLastError());
     return SALICACHE_OK;
 }
