@@ -368,6 +368,41 @@ def run_extras(sc, synth, ctx, wl, T, frames, dP, dev, peak, pools, fill, stored
                          "ms": round(ms, 3), "cache_bytes": int(stored_bytes), "l2": "cache larger than L2",
                          "algorithmic_GBps": round(stored_bytes / ms / 1e6, 1),
                          "frac_of_hbm_peak": round(stored_bytes / ms / 1e6 / peak, 4)}
+    # the same attention over a cache with an INT8 background (the other workloads' tier mix): 16 frames of random K/V,
+    # spatial scores uniform in [0.2, 0.6], so that about half the tokens are FP16 and half INT8
+    if wl.head_dim == 128 and wl.heads * 128 == wl.HD:
+        Tm = 16
+        g = torch.Generator(device=dev)
+        g.manual_seed(11)
+        cm = sc.Context(sc.salicache_default_params(max_batch=Tm, chunk_frames=2, L=wl.L, heads=wl.heads, **synth.thresholds("int8")))
+        Km = torch.randn((Tm, wl.L, 576, wl.HD), generator=g, device=dev, dtype=torch.float16)
+        Vm = torch.randn((Tm, wl.L, 576, wl.HD), generator=g, device=dev, dtype=torch.float16)
+        sm = (0.2 + 0.4 * torch.rand((Tm, 576), generator=g, device=dev)).float()
+        decm = torch.zeros((Tm, 576), dtype=torch.uint8, device=dev)
+        idxm = torch.zeros((Tm, 3, 576), dtype=torch.int32, device=dev)
+        cntm = torch.zeros((Tm, 5), dtype=torch.int32, device=dev)
+        redm = torch.zeros((Tm,), dtype=torch.uint8, device=dev)
+        offm = torch.zeros((Tm, 3), dtype=torch.int64, device=dev)
+        fillm = torch.zeros((3,), dtype=torch.int64, device=dev)
+        sc.salicache_select(cm, None, sm, Tm, False, decm, idxm, cntm, redm, offm, fillm)
+        cc = cntm.sum(dim=0).cpu().numpy()
+        pm = sc.PoolSet(wl.L, wl.HD, int(cc[4]) + 1, int(cc[3]) + 1, int(cc[2]) + 1, device=dev)
+        sc.salicache_pack_kv(cm, Km, Vm, wl.L * 576 * wl.HD, idxm, cntm, offm, Tm, pm.c)
+        torch.cuda.synchronize()
+        del Km, Vm
+        ngm = wl.HD // 128
+        bytes_m = 2 * wl.L * (int(cc[4]) * wl.HD * 2 + int(cc[3]) * (wl.HD + 2 * ngm) + int(cc[2]) * (wl.HD // 2 + 4 * ngm))
+        g.manual_seed(7)
+        qm = torch.randn((wl.L, wl.heads, 128), generator=g, device=dev, dtype=torch.float32).to(torch.float16)
+        om = torch.zeros((wl.L, wl.heads, 128), dtype=torch.float32, device=dev)
+        ms = timed(lambda: sc.salicache_attend(cm, qm, pm.c, fillm, om), reps=5)
+        out["attend_int8_background"] = {
+            "what": "salicache_attend over a 16-frame cache with an INT8 background (random K/V)",
+            "rows": {"fp16": int(cc[4]), "int8": int(cc[3]), "int4": int(cc[2])}, "ms": round(ms, 3), "cache_bytes": int(bytes_m),
+            "l2": "cache larger than L2", "algorithmic_GBps": round(bytes_m / ms / 1e6, 1),
+            "frac_of_hbm_peak": round(bytes_m / ms / 1e6 / peak, 4)}
+        del pm
+        cm.close()
     # anchor-frame mode: the scan over the frames of this workload (Eq. 5 literal against the anchor image + decisions)
     if wl.n_images == 1 and T > 1:
         tau_grey = 3.0

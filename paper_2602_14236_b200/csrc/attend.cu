@@ -4,11 +4,11 @@
 //
 //   score_j = q_h . K^_{j,h} / sqrt(D),   p = softmax_j(score),   out_h = sum_j p_j V^_{j,h}
 //
-// Split over the rows: per layer and head up to AT_CHUNKS partial results of each of two kernels, merged by a
-// third.  k_attend_partial takes the FP16 and INT8 rows: scores one row per thread (the thread walks the
-// head's 128 key elements of its row: no cross-lane reduction), values four dimensions per lane, one row per
-// warp at a time.  k_attend_int4 takes the INT4 rows, the bulk of a compressed cache, 16 rows per warp at a
-// time through matrix instructions.  Online softmax and single precision accumulation in both.
+// Split over the rows: per layer and head a few dozen partial results of each of three kernels, merged by a
+// fourth.  k_attend_partial takes the FP16 rows: scores one row per thread (the thread walks the head's 128
+// key elements of its row: no cross-lane reduction), values four dimensions per lane, one row per warp at a
+// time.  k_attend_int8 and k_attend_int4 take the quantised rows, the bulk of a compressed cache, 16 rows per
+// warp at a time through matrix instructions.  Online softmax and single precision accumulation in all.
 #include <cuda_fp16.h>
 
 #include <algorithm>
