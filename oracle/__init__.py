@@ -384,6 +384,21 @@ def attend(q16: np.ndarray, pools: "Pools", n_rows) -> np.ndarray:
     return out
 
 
+def attend_gqa(q16: np.ndarray, pools: "Pools", n_rows, q_per_kv: int) -> np.ndarray:
+    """Grouped-query decode attention: query head hq uses the rows of key/value head hq // q_per_kv.
+    q16: fp16 bits [L][H * q_per_kv][D], H the pools' heads.  Returns float64 of the same shape."""
+    q16 = _c(q16, np.uint16)
+    L, HQ, D = q16.shape
+    assert HQ % q_per_kv == 0 and (HQ // q_per_kv) * D == pools.HD
+    out = np.empty((L, HQ, D), np.float64)
+    n16, n8, n4 = (int(x) for x in n_rows)
+    lib().oracle_attend_gqa(_p(q16), C.c_int(L), C.c_int(HQ // q_per_kv), C.c_int(q_per_kv), C.c_int(D), C.c_int(pools.G),
+                            _p(pools.fp16_pool), C.c_int64(pools.cap16), C.c_int64(n16), _p(pools.int8_codes),
+                            _p(pools.int8_scale), C.c_int64(pools.cap8), C.c_int64(n8), _p(pools.int4_codes),
+                            _p(pools.int4_sz), C.c_int64(pools.cap4), C.c_int64(n4), _p(out))
+    return out
+
+
 def stored_bytes(counts_all: np.ndarray, L: int, HD: int, G: int, n_tok: int) -> int:
     """Bytes the mixed-precision store holds for frames with the given per-code counts [T][5]
     (Eq. 3 applied per tier, plus all metadata: scales/zeros, index lists, decision bytes,

@@ -927,3 +927,48 @@ EXPORT void oracle_attend(const uint16_t* q, int L, int H, int D, int G, const u
             free(sc);
         }
 }
+
+/* Grouped-query form (the paper's evaluation model, LLaVA-1.6 Mistral-7B, has 8 key/value heads serving 32 query   */
+/* heads, Sec. IV-A): query head hq attends to the rows of key/value head hq / q_per_kv; everything else as above.   */
+/* q, out: [L][H * q_per_kv][D].                                                                                     */
+EXPORT void oracle_attend_gqa(const uint16_t* q, int L, int H, int q_per_kv, int D, int G, const uint16_t* fp16_pool,
+                              int64_t cap16, int64_t n16, const int8_t* int8_codes, const uint16_t* int8_scale, int64_t cap8,
+                              int64_t n8, const uint8_t* int4_codes, const uint16_t* int4_sz, int64_t cap4, int64_t n4,
+                              double* out) {
+    int HD = H * D, HQ = H * q_per_kv;
+    int64_t caps[3] = {cap16, cap8, cap4}, ns[3] = {n16, n8, n4};
+    int64_t R = n16 + n8 + n4;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int l = 0; l < L; ++l)
+        for (int hq = 0; hq < HQ; ++hq) {
+            int h = hq / q_per_kv;
+            const uint16_t* qv = q + ((size_t)l * HQ + hq) * D;
+            double* o = out + ((size_t)l * HQ + hq) * D;
+            for (int d = 0; d < D; ++d) o[d] = 0.0;
+            if (R == 0) continue;
+            double* sc = (double*)malloc((size_t)R * sizeof(double));
+            double mx = -INFINITY;
+            int64_t j = 0;
+            for (int t = 0; t < 3; ++t)
+                for (int64_t r = 0; r < ns[t]; ++r, ++j) {
+                    size_t prow = (size_t)(2 * l) * caps[t] + r;
+                    double dot = 0.0;
+                    for (int d = 0; d < D; ++d)
+                        dot += (double)oracle_half_to_float(qv[d]) *
+                               pool_value(t, prow, h, d, HD, D, G, fp16_pool, int8_codes, int8_scale, int4_codes, int4_sz);
+                    sc[j] = dot / sqrt((double)D);
+                    if (sc[j] > mx) mx = sc[j];
+                }
+            double den = 0.0;
+            for (j = 0; j < R; ++j) { sc[j] = exp(sc[j] - mx); den += sc[j]; }
+            j = 0;
+            for (int t = 0; t < 3; ++t)
+                for (int64_t r = 0; r < ns[t]; ++r, ++j) {
+                    size_t prow = (size_t)(2 * l + 1) * caps[t] + r;
+                    double p = sc[j] / den;
+                    for (int d = 0; d < D; ++d)
+                        o[d] += p * pool_value(t, prow, h, d, HD, D, G, fp16_pool, int8_codes, int8_scale, int4_codes, int4_sz);
+                }
+            free(sc);
+        }
+}

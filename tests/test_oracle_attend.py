@@ -86,3 +86,29 @@ def test_empty_store_row_order_and_query_scale():
     from scipy.special import softmax
     sc = np.einsum("lhd,ljhd->lhj", q.astype(np.float64), dense[:, 0]) / np.sqrt(D)
     assert np.allclose(part, np.einsum("lhj,ljhd->lhd", softmax(sc, axis=-1), dense[:, 1]), rtol=1e-12, atol=1e-13)
+
+
+def test_grouped_query_attention_against_library_softmax_and_the_one_query_per_head_routine():
+    """Query head hq reads key/value head hq // q_per_kv.  Pinned by the textbook expression with library routines on
+    the dequantised cache, by q_per_kv = 1 (the plain routine), and by feeding the plain routine the queries of one
+    slot of every group (it must return that slot's rows of the grouped result)."""
+    from scipy.special import softmax
+    rng = np.random.default_rng(4)
+    L, H, D, G = 2, 3, 128, 4
+    pools, n = _filled_pools(rng, L, H, D)
+    q = rng.standard_normal((L, H * G, D)).astype(np.float16)
+    got = oracle.attend_gqa(q.view(np.uint16), pools, n, G)
+    dense = _dense(pools, n, L, H, D)                                            # [L][2][rows][H][D]
+    kv = np.repeat(dense, G, axis=3)                                             # key/value head of every query head
+    scores = np.einsum("lhd,ljhd->lhj", q.astype(np.float64), kv[:, 0]) / np.sqrt(D)
+    want = np.einsum("lhj,ljhd->lhd", softmax(scores, axis=-1), kv[:, 1])
+    assert np.allclose(got, want, rtol=1e-12, atol=1e-13)
+    for slot in range(G):
+        plain = oracle.attend(np.ascontiguousarray(q[:, slot::G]).view(np.uint16), pools, n)
+        assert np.array_equal(plain, got[:, slot::G])
+    q1 = rng.standard_normal((L, H, D)).astype(np.float16)
+    assert np.array_equal(oracle.attend_gqa(q1.view(np.uint16), pools, n, 1), oracle.attend(q1.view(np.uint16), pools, n))
+    # a transposed head mapping (hq % H instead of hq // q_per_kv) would fail the slot test above; check it does differ
+    wrong = np.einsum("lhj,ljhd->lhd", softmax(np.einsum("lhd,ljhd->lhj", q.astype(np.float64), np.tile(dense, (1, 1, 1, G, 1))[:, 0]) / np.sqrt(D), axis=-1),
+                      np.tile(dense, (1, 1, 1, G, 1))[:, 1])
+    assert not np.allclose(got, wrong, rtol=1e-6, atol=1e-8)
