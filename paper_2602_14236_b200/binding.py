@@ -50,7 +50,7 @@ EXPORTS = [
     "salicache_tokens_per_frame", "salicache_launch_count", "salicache_flow_score", "salicache_saliency", "salicache_select",
     "salicache_pack_kv", "salicache_unpack_kv", "salicache_poll_status", "salicache_saliency_noalloc",
     "salicache_frame_redundancy", "salicache_source_frames", "salicache_diff_score", "salicache_attend",
-    "salicache_select_anchored", "salicache_select_ranked",
+    "salicache_select_anchored", "salicache_select_ranked", "salicache_attend_gqa",
 ]
 
 _lib = None
@@ -88,6 +88,7 @@ def lib():
         _lib.salicache_unpack_kv.argtypes = [vp, C.POINTER(Pools), vp, vp, vp, vp, i32, i32, vp, vp, i64, vp]
         _lib.salicache_poll_status.argtypes = [vp, vp]
         _lib.salicache_attend.argtypes = [vp, vp, C.POINTER(Pools), vp, vp, vp]
+        _lib.salicache_attend_gqa.argtypes = [vp, vp, i32, C.POINTER(Pools), vp, vp, vp]
         _lib.salicache_saliency_noalloc.argtypes = [C.POINTER(Params), vp, i32, vp, vp, vp]
     return _lib
 
@@ -221,6 +222,11 @@ def salicache_unpack_kv(ctx: Context, pools: Pools, d_idx, d_counts, d_decision,
 def salicache_attend(ctx: Context, d_q, pools: Pools, d_fill, d_out, stream=None):
     _check(lib().salicache_attend(ctx.handle, _ptr(d_q), C.byref(pools), _ptr(d_fill), _ptr(d_out), _stream(stream)),
            "salicache_attend")
+
+
+def salicache_attend_gqa(ctx: Context, d_q, q_per_kv: int, pools: Pools, d_fill, d_out, stream=None):
+    _check(lib().salicache_attend_gqa(ctx.handle, _ptr(d_q), int(q_per_kv), C.byref(pools), _ptr(d_fill), _ptr(d_out),
+                                      _stream(stream)), "salicache_attend_gqa")
 
 
 def salicache_poll_status(ctx: Context, stream=None) -> int:

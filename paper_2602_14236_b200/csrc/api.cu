@@ -340,7 +340,16 @@ int salicache_attend(salicache_ctx* c, const void* d_q, const salicache_pools* p
     int rc = check_pools(pools);
     if (rc != SALICACHE_OK) return rc;
     if (!aligned16(d_q) || !aligned16(d_out)) return SALICACHE_E_ALIGN;
-    return sc_attend(c, d_q, pools, d_fill, d_out, (cudaStream_t)cuda_stream);
+    return sc_attend(c, d_q, 1, pools, d_fill, d_out, (cudaStream_t)cuda_stream);
+}
+
+int salicache_attend_gqa(salicache_ctx* c, const void* d_q, int q_per_kv, const salicache_pools* pools, const int64_t* d_fill,
+                         float* d_out, void* cuda_stream) {
+    if (!c || !d_q || !d_fill || !d_out) return SALICACHE_E_NULL;
+    int rc = check_pools(pools);
+    if (rc != SALICACHE_OK) return rc;
+    if (!aligned16(d_q) || !aligned16(d_out)) return SALICACHE_E_ALIGN;
+    return sc_attend(c, d_q, q_per_kv, pools, d_fill, d_out, (cudaStream_t)cuda_stream);
 }
 
 int salicache_poll_status(salicache_ctx* c, void* cuda_stream) {

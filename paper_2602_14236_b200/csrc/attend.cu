@@ -95,7 +95,7 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 }
 
 __global__ void __launch_bounds__(AT_D)
-k_attend_partial(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int ng,
+k_attend_partial(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int gq, int ng,
                  int with_int8, int with_int4, float* __restrict__ ws) {
     __shared__ __align__(16) float qs[AT_D];        // the query as binary32 (for sum(q))
     __shared__ __align__(16) __half qn[AT_D];       // the query in natural order
@@ -105,7 +105,8 @@ k_attend_partial(const __half* __restrict__ q, AtPools pp, const long long* __re
     __shared__ float red[AT_WARPS];
     __shared__ float part[AT_WARPS][AT_D];
     // heads vary fastest over the grid: the CTAs that read the 32 slices of one row run at about the same time
-    const int h = blockIdx.x, c = blockIdx.y, l = blockIdx.z, t = threadIdx.x;
+    const int hq = blockIdx.x, c = blockIdx.y, l = blockIdx.z, t = threadIdx.x;
+    const int h = hq / gq, Hq = H * gq;          // query head hq reads key/value head h
     const int lane = t & 31, wid = t >> 5;
     const int HD = H * AT_D;
     const long long n16 = min(fill[0], pp.cap16);
@@ -116,14 +117,14 @@ k_attend_partial(const __half* __restrict__ q, AtPools pp, const long long* __re
     const long long r0 = (long long)c * per, r1 = min(R, r0 + per);
     if (r0 >= r1) {                                 // nothing in this chunk: a record the merge skips
         if (t == 0) {
-            float* rec = ws + (((size_t)l * H + h) * AT_RECS + c) * AT_REC;
+            float* rec = ws + (((size_t)l * Hq + hq) * AT_RECS + c) * AT_REC;
             rec[AT_D] = -INFINITY;
             rec[AT_D + 1] = 0.0f;
         }
         return;
     }
     {
-        const __half qv = q[((size_t)l * H + h) * AT_D + t];
+        const __half qv = q[((size_t)l * Hq + hq) * AT_D + t];
         const int e = t & 7;
         qs[t] = __half2float(qv);
         qn[t] = qv;
@@ -256,7 +257,7 @@ k_attend_partial(const __half* __restrict__ q, AtPools pp, const long long* __re
 #pragma unroll
     for (int k = 0; k < 4; ++k) part[wid][4 * lane + k] = acc[k] + zacc;
     __syncthreads();
-    float* rec = ws + (((size_t)l * H + h) * AT_RECS + c) * AT_REC;
+    float* rec = ws + (((size_t)l * Hq + hq) * AT_RECS + c) * AT_REC;
     float sum = 0.0f;
 #pragma unroll
     for (int k = 0; k < AT_WARPS; ++k) sum += part[k][t];
@@ -476,14 +477,15 @@ __device__ __forceinline__ void i4_tile(I4State& st, const I4Tile& x, const uint
 
 template <int PITCH, int NG>
 __global__ void __launch_bounds__(AT_D)
-k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int ng, int min_rows,
+k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int gq, int ng, int min_rows,
               float* __restrict__ ws) {
     __shared__ __align__(16) float qs[AT_D];
     __shared__ __align__(16) __half qp[AT_D];       // every 8 elements ordered 0 4 1 5 2 6 3 7
     __shared__ float red[AT_WARPS];
     __shared__ float wpart[AT_WARPS][AT_D];
     __shared__ float wstat[AT_WARPS][2];
-    const int h = blockIdx.x, c = blockIdx.y, l = blockIdx.z, t = threadIdx.x;
+    const int hq = blockIdx.x, c = blockIdx.y, l = blockIdx.z, t = threadIdx.x;
+    const int h = hq / gq, Hq = H * gq;          // query head hq reads key/value head h
     const int lane = t & 31, wid = t >> 5, g8 = lane >> 2, c4 = lane & 3;
     const int HD = H * AT_D;
     const long long n4 = min(fill[2], pp.cap4);
@@ -493,14 +495,14 @@ k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restr
     const long long r0 = (long long)c * per, r1 = min(n4, r0 + per);
     if (r0 >= r1) {                                 // nothing in this chunk: a record the merge skips
         if (t == 0) {
-            float* rec = ws + (((size_t)l * H + h) * AT_RECS + AT_REC4 + c) * AT_REC;
+            float* rec = ws + (((size_t)l * Hq + hq) * AT_RECS + AT_REC4 + c) * AT_REC;
             rec[AT_D] = -INFINITY;
             rec[AT_D + 1] = 0.0f;
         }
         return;
     }
     {
-        const __half qv = q[((size_t)l * H + h) * AT_D + t];
+        const __half qv = q[((size_t)l * Hq + hq) * AT_D + t];
         const int e = t & 7;
         qs[t] = __half2float(qv);
         qp[(t & ~7) | ((e & 3) * 2 + (e >> 2))] = qv;
@@ -583,7 +585,7 @@ k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restr
             dsum += e * wstat[k][1];
         }
     }
-    float* rec = ws + (((size_t)l * H + h) * AT_RECS + AT_REC4 + c) * AT_REC;
+    float* rec = ws + (((size_t)l * Hq + hq) * AT_RECS + AT_REC4 + c) * AT_REC;
     rec[t] = sum;
     if (t == 0) {
         rec[AT_D] = M;
@@ -748,18 +750,19 @@ __device__ __forceinline__ void mma_finish(const I4State& st, float (*wpart)[AT_
 }
 
 __global__ void __launch_bounds__(AT_D)
-k_attend_int8(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int ng, int min_rows,
+k_attend_int8(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int gq, int ng, int min_rows,
               float* __restrict__ ws) {
     __shared__ __align__(16) __half qn[AT_D];
     __shared__ float wpart[AT_WARPS][AT_D];
     __shared__ float wstat[AT_WARPS][2];
-    const int h = blockIdx.x, c = blockIdx.y, l = blockIdx.z, t = threadIdx.x;
+    const int hq = blockIdx.x, c = blockIdx.y, l = blockIdx.z, t = threadIdx.x;
+    const int h = hq / gq, Hq = H * gq;          // query head hq reads key/value head h
     const int lane = t & 31, wid = t >> 5, g8 = lane >> 2, c4 = lane & 3;
     const size_t HD = (size_t)H * AT_D;
     const long long n8 = min(fill[1], pp.cap8);
     const long long per = max((long long)min_rows, ((n8 + AT_CH8 - 1) / AT_CH8 + 15) / 16 * 16);
     const long long r0 = (long long)c * per, r1 = min(n8, r0 + per);
-    float* rec = ws + (((size_t)l * H + h) * AT_RECS + AT_REC8 + c) * AT_REC;
+    float* rec = ws + (((size_t)l * Hq + hq) * AT_RECS + AT_REC8 + c) * AT_REC;
     if (r0 >= r1) {                                 // nothing in this chunk: a record the merge skips
         if (t == 0) {
             rec[AT_D] = -INFINITY;
@@ -767,7 +770,7 @@ k_attend_int8(const __half* __restrict__ q, AtPools pp, const long long* __restr
         }
         return;
     }
-    qn[t] = q[((size_t)l * H + h) * AT_D + t];
+    qn[t] = q[((size_t)l * Hq + hq) * AT_D + t];
     __syncthreads();
     const float rs = rsqrtf((float)AT_D);
     const int g = ng == 1 ? 0 : h;
@@ -847,35 +850,40 @@ k_attend_merge(const float* __restrict__ ws, int H, int nch, float* __restrict__
 
 }  // namespace
 
-size_t sc_attend_workspace_bytes(int L, int H) { return (size_t)L * H * AT_RECS * AT_REC * sizeof(float); }
+// The workspace holds the partial records of up to max(H, 64) query heads per layer: grouped-query attention has
+// more query heads than key/value heads.
+static int attend_max_query_heads(int H) { return H > 64 ? H : 64; }
+size_t sc_attend_workspace_bytes(int L, int H) { return (size_t)L * attend_max_query_heads(H) * AT_RECS * AT_REC * sizeof(float); }
 
-int sc_attend(salicache_ctx* c, const void* d_q, const salicache_pools* pools, const int64_t* d_fill, float* d_out,
+int sc_attend(salicache_ctx* c, const void* d_q, int q_per_kv, const salicache_pools* pools, const int64_t* d_fill, float* d_out,
               cudaStream_t st) {
     const salicache_params& p = c->p;
     if (p.head_dim != AT_D || (p.group != AT_D && p.group != p.heads * p.head_dim)) return SALICACHE_E_PARAM;
+    if (q_per_kv < 1 || (long long)p.heads * q_per_kv > attend_max_query_heads(p.heads)) return SALICACHE_E_SHAPE;
     AtPools pp{(const uint8_t*)pools->fp16_pool, (const uint8_t*)pools->int8_codes, (const uint8_t*)pools->int8_scale,
                (const uint8_t*)pools->int4_codes, (const uint8_t*)pools->int4_sz, pools->cap_fp16, pools->cap_int8,
                pools->cap_int4};
     if (pp.cap16 >= (1ll << 28) || pp.cap8 >= (1ll << 28) || pp.cap4 >= (1ll << 28)) return SALICACHE_E_SHAPE;
     const int ng = p.group == AT_D ? p.heads : 1;
-    dim3 grid(p.heads, AT_CHUNKS, p.L);
+    const int gq = q_per_kv, Hq = p.heads * gq;     // query heads; query head hq reads key/value head hq / gq
+    dim3 grid(Hq, AT_CHUNKS, p.L);
     // FP16 rows one row per thread; INT8 and INT4 rows, the bulk of a compressed cache, on the matrix instructions.
     // The first kernel gets as many chunks as its pool can fill with four tiles each, 32 at most.
     const int nch = (int)std::min<long long>(AT_CH16, std::max<long long>(1, (pp.cap16 + 4 * AT_D - 1) / (4 * AT_D)));
-    dim3 grid16(p.heads, nch, p.L);
-    k_attend_partial<<<grid16, AT_D, 0, st>>>((const __half*)d_q, pp, (const long long*)d_fill, p.heads, ng, 0, 0, c->attend_ws);
+    dim3 grid16(Hq, nch, p.L);
     const __half* qh = (const __half*)d_q;
     const long long* fl = (const long long*)d_fill;
-    // rows per chunk of the INT4 kernel: up to 4096 (64 tiles per warp) when there are many (layer, head) pairs to
-    // fill the GPU with, fewer when there are few
-    const int min_rows = (int)std::min<long long>(4096, std::max<long long>(256, 8ll * p.L * p.heads)) / 16 * 16;
-    dim3 grid8(p.heads, AT_CH8, p.L);
-    k_attend_int8<<<grid8, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, min_rows, c->attend_ws);
-    if (p.heads == 32 && ng == 32) k_attend_int4<32 * AT_D / 2, 32><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, min_rows, c->attend_ws);
-    else if (p.heads == 32 && ng == 1) k_attend_int4<32 * AT_D / 2, 1><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, min_rows, c->attend_ws);
-    else k_attend_int4<0, 0><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, ng, min_rows, c->attend_ws);
-    dim3 gm(p.heads, p.L);
-    k_attend_merge<<<gm, AT_D, 0, st>>>(c->attend_ws, p.heads, nch, d_out);
+    k_attend_partial<<<grid16, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, 0, 0, c->attend_ws);
+    // rows per chunk of the quantised kernels: up to 4096 (64 tiles per warp) when there are many (layer, head) pairs
+    // to fill the GPU with, fewer when there are few
+    const int min_rows = (int)std::min<long long>(4096, std::max<long long>(256, 8ll * p.L * Hq)) / 16 * 16;
+    dim3 grid8(Hq, AT_CH8, p.L);
+    k_attend_int8<<<grid8, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
+    if (p.heads == 32 && ng == 32) k_attend_int4<32 * AT_D / 2, 32><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
+    else if (p.heads == 32 && ng == 1) k_attend_int4<32 * AT_D / 2, 1><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
+    else k_attend_int4<0, 0><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
+    dim3 gm(Hq, p.L);
+    k_attend_merge<<<gm, AT_D, 0, st>>>(c->attend_ws, Hq, nch, d_out);
     c->launches += 4;
     SC_CHECK(cudaGetLastError());
     return SALICACHE_OK;

@@ -48,7 +48,7 @@ struct salicache_ctx {
     uint8_t* base_frames;      // anyres only: [chunk+1][336*336*3]
     // select / pack scratch
     int64_t* row_prefix;       // [max_batch+1] stored rows before each frame of the batch
-    float* attend_ws;          // partial attention results [L][heads][128][head_dim + 2]
+    float* attend_ws;          // partial attention results [L][max(heads, 64)][128][head_dim + 2]
     int* d_status;             // deferred status word
     int sm_count;
     long long launches;        // kernels launched through this context so far
@@ -81,7 +81,7 @@ int sc_select_anchored(salicache_ctx* c, const uint8_t* d_frames, const float* d
                        uint8_t* d_frame_redundant, int64_t* d_row_offset, int64_t* d_fill, cudaStream_t st);
 // attend.cu
 size_t sc_attend_workspace_bytes(int L, int H);
-int sc_attend(salicache_ctx* c, const void* d_q, const salicache_pools* pools, const int64_t* d_fill, float* d_out,
+int sc_attend(salicache_ctx* c, const void* d_q, int q_per_kv, const salicache_pools* pools, const int64_t* d_fill, float* d_out,
               cudaStream_t st);
 // kv.cu
 int sc_pack(salicache_ctx* c, const void* d_K, const void* d_V, int64_t frame_stride, const int32_t* d_idx,

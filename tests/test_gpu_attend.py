@@ -126,3 +126,32 @@ def test_attention_int4_rows_peaked_and_large_values():
         tok = int(np.flatnonzero(keep["decision"][0] == sc.INT4)[0])
         k_row = keep["K"][0, :, tok, :].reshape(2, heads, 128).astype(np.float32)
         _check(ctx, pools, ref, fill, (3.0 * k_row).astype(np.float16), scale=v_scale)
+
+
+@pytest.mark.parametrize("heads,q_per_kv,background", [(8, 4, "four"), (8, 4, "int4"), (32, 2, "int8")])
+def test_grouped_query_attention_matches_the_oracle(heads, q_per_kv, background):
+    """The paper's evaluation model has 8 key/value heads for 32 query heads: query head hq reads key/value head
+    hq // q_per_kv.  Also 32 key/value heads with two queries each (64 query heads, the most the workspace holds)."""
+    import torch
+    ctx, pools, ref, fill, rng = _store(L=2, heads=heads, T=2, background=background, seed=21)
+    q = rng.standard_normal((2, heads * q_per_kv, 128)).astype(np.float16)
+    d_out = torch.full((2, heads * q_per_kv, 128), 7.0, dtype=torch.float32, device="cuda")
+    sc.salicache_attend_gqa(ctx, torch.from_numpy(q).cuda(), q_per_kv, pools.c, fill, d_out)
+    torch.cuda.synchronize()
+    n = np.minimum(fill.cpu().numpy(), [ref.cap16, ref.cap8, ref.cap4])
+    want = oracle.attend_gqa(q.view(np.uint16), ref, n, q_per_kv)
+    err = np.abs(d_out.cpu().numpy().astype(np.float64) - want)
+    assert (err <= ATOL + RTOL * np.abs(want)).all(), f"worst {err.max():.3e}"
+    # one query per key/value head is the plain call; too many query heads are refused
+    lib = sc.lib()
+    import ctypes
+    qd, od = torch.from_numpy(q).cuda(), d_out
+    assert lib.salicache_attend_gqa(ctx.handle, qd.data_ptr(), 0, ctypes.byref(pools.c), fill.data_ptr(), od.data_ptr(), None) == sc.E_SHAPE
+    assert lib.salicache_attend_gqa(ctx.handle, qd.data_ptr(), 65, ctypes.byref(pools.c), fill.data_ptr(), od.data_ptr(), None) == sc.E_SHAPE
+    q1 = np.ascontiguousarray(q[:, ::q_per_kv])
+    a = torch.zeros((2, heads, 128), dtype=torch.float32, device="cuda")
+    b = torch.zeros_like(a)
+    sc.salicache_attend_gqa(ctx, torch.from_numpy(q1).cuda(), 1, pools.c, fill, a)
+    sc.salicache_attend(ctx, torch.from_numpy(q1).cuda(), pools.c, fill, b)
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
