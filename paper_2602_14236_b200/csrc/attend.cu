@@ -593,6 +593,257 @@ k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restr
     }
 }
 
+// ---- INT4 rows, grouped queries: the 2 to 4 query heads that share a key/value head are the columns of the
+// matrix instructions, so the codes of a tile are expanded once for all of them.  Query j sits in column 2 j of
+// the score product; lane (g8, c4) therefore finds the products of query c4 with rows g8 and g8 + 8 in its own
+// accumulator, and keeps that query's softmax statistics (shared by the 8 lanes with the same c4).  In the value
+// product the weights of query j fill columns 2 j (high halves) and 2 j + 1 (low halves), so every lane's
+// accumulators belong to query c4: dimensions 16 g8 + 2 b and 16 g8 + 2 b + 1.
+constexpr int GQ_MAX = 4;
+
+struct G4Tile {
+    uint4 ka, kb;                  // keys of rows g8 and g8 + 8: 32 dimensions at 32 * c4
+    uint2 v0, v1, v2, v3;          // values of rows 2 c4, 2 c4 + 1, 2 c4 + 8, 2 c4 + 9: 16 dimensions at 16 * g8
+    uint32_t ksa, ksb, vsa, vsb;   // (scale, zero) of the keys and values of rows g8 and g8 + 8
+};
+struct G4Addr {
+    const uint8_t* k;
+    const uint8_t* v;
+    const uint32_t* ks;
+    const uint32_t* vs;
+    size_t pitch, ng;
+};
+__device__ __forceinline__ void g4_fetch(G4Tile& x, const G4Addr& a, long long tile, long long t0, long long r1, int g8, int c4) {
+    const size_t d = (size_t)(tile - t0), P = a.pitch;
+    const uint8_t* k = a.k + d * P;
+    const uint8_t* v = a.v + d * P;
+    const uint32_t* ks = a.ks + d * a.ng;
+    const uint32_t* vs = a.vs + d * a.ng;
+    if (tile + 16 <= r1) {
+        x.ka = ld_stream16(k);
+        x.kb = ld_stream16(k + 8 * P);
+        x.v0 = ld_stream8(v);
+        x.v1 = ld_stream8(v + P);
+        x.v2 = ld_stream8(v + 8 * P);
+        x.v3 = ld_stream8(v + 9 * P);
+        x.ksa = __ldg(ks);
+        x.ksb = __ldg(ks + 8 * a.ng);
+        x.vsa = __ldg(vs);
+        x.vsb = __ldg(vs + 8 * a.ng);
+    } else {                                        // rows at or beyond r1 read as zero codes and are not touched
+        x.ka = x.kb = make_uint4(0, 0, 0, 0);
+        x.v0 = x.v1 = x.v2 = x.v3 = make_uint2(0, 0);
+        x.ksa = x.ksb = x.vsa = x.vsb = 0;
+        const long long ra = tile + g8, rv = tile + 2 * c4;
+        if (ra < r1) { x.ka = ld_stream16(k); x.ksa = __ldg(ks); x.vsa = __ldg(vs); }
+        if (ra + 8 < r1) { x.kb = ld_stream16(k + 8 * P); x.ksb = __ldg(ks + 8 * a.ng); x.vsb = __ldg(vs + 8 * a.ng); }
+        if (rv < r1) x.v0 = ld_stream8(v);
+        if (rv + 1 < r1) x.v1 = ld_stream8(v + P);
+        if (rv + 8 < r1) x.v2 = ld_stream8(v + 8 * P);
+        if (rv + 9 < r1) x.v3 = ld_stream8(v + 9 * P);
+    }
+}
+// max / sum over the 8 lanes that share c4 (one query)
+__device__ __forceinline__ float group_max(float v) {
+#pragma unroll
+    for (int o = 16; o >= 4; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float group_sum(float v) {
+#pragma unroll
+    for (int o = 16; o >= 4; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ void g4_tile(I4State& st, const G4Tile& x, const uint32_t (&qf)[8][2], const NibConst& nc, long long tile,
+                                        long long r1, float rs, float qsum, int g8, int c4) {
+    float sc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    {
+        const uint32_t wa[4] = {x.ka.x, x.ka.y, x.ka.z, x.ka.w}, wb[4] = {x.kb.x, x.kb.y, x.kb.z, x.kb.w};
+#pragma unroll
+        for (int w4 = 0; w4 < 4; ++w4) {
+            uint32_t pa[4], pb[4];
+            nc.word(wa[w4], pa);
+            nc.word(wb[w4], pb);
+            mma16816(sc, pa[0], pb[0], pa[1], pb[1], qf[2 * w4][0], qf[2 * w4][1]);
+            mma16816(sc, pa[2], pb[2], pa[3], pb[3], qf[2 * w4 + 1][0], qf[2 * w4 + 1][1]);
+        }
+    }
+    // this lane: query c4 against rows g8 (sc[0]) and g8 + 8 (sc[2])
+    const bool va = tile + g8 < r1, vb = tile + g8 + 8 < r1;
+    const float2 kza = w2f(x.ksa), kzb = w2f(x.ksb), vza = w2f(x.vsa), vzb = w2f(x.vsb);
+    const float sa = va ? rs * (sc[0] * kza.x + qsum * kza.y) : -INFINITY;
+    const float sb = vb ? rs * (sc[2] * kzb.x + qsum * kzb.y) : -INFINITY;
+    const float sm = fmaxf(sa, sb), sv = fmaxf(va ? vza.x : 0.0f, vb ? vzb.x : 0.0f);
+    if (__any_sync(0xffffffffu, sm > st.m || sv * st.F >= 32768.0f)) {
+        const float m_new = fmaxf(st.m, group_max(sm));                 // of this lane's query
+        const float corr = st.m == -INFINITY ? 0.0f : __expf(st.m - m_new);
+        st.m = m_new;
+        const float smax = warp_max(sv);                                // F is shared by the whole warp
+        float Fn = st.F;
+        for (int k = 0; k < 40 && smax * Fn >= 32768.0f; ++k) Fn *= 0.5f;
+        const float rescale = corr * (Fn / st.F);
+        st.F = Fn;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) st.acc[b][i] *= rescale;
+        }
+        st.den *= corr;
+        st.zacc *= corr;
+    }
+    const float pa_ = __expf(sa - st.m), pb_ = __expf(sb - st.m);
+    st.den += pa_ + pb_;
+    st.zacc += pa_ * vza.y + pb_ * vzb.y;
+    uint32_t packa, packb;                          // weights of (row g8, query c4) and (row g8 + 8, query c4): high | low
+    {
+        const float wa_ = pa_ * vza.x * st.F, wb_ = pb_ * vzb.x * st.F;
+        const __half ha = __float2half_rn(wa_), hb = __float2half_rn(wb_);
+        const __half la = __float2half_rn(wa_ - __half2float(ha)), lb = __float2half_rn(wb_ - __half2float(hb));
+        packa = (uint32_t)__half_as_ushort(ha) | ((uint32_t)__half_as_ushort(la) << 16);
+        packb = (uint32_t)__half_as_ushort(hb) | ((uint32_t)__half_as_ushort(lb) << 16);
+    }
+    // B fragment of the value product: this lane supplies column g8 = high (even) or low (odd) halves of query g8 / 2,
+    // for the rows 2 c4, 2 c4 + 1 (b0) and 2 c4 + 8, 2 c4 + 9 (b1); the weight of (row r, query j) is in lane 4 (r % 8) + j
+    const int la = 8 * c4 + (g8 >> 1);
+    const uint32_t x1 = __shfl_sync(0xffffffffu, packa, la), x2 = __shfl_sync(0xffffffffu, packa, la + 4);
+    const uint32_t y1 = __shfl_sync(0xffffffffu, packb, la), y2 = __shfl_sync(0xffffffffu, packb, la + 4);
+    const uint32_t psel = (g8 & 1) ? 0x7632u : 0x5410u;
+    const uint32_t b0 = __byte_perm(x1, x2, psel), b1 = __byte_perm(y1, y2, psel);
+    {
+        const uint32_t w0[2] = {x.v0.x, x.v0.y}, w1[2] = {x.v1.x, x.v1.y}, w2[2] = {x.v2.x, x.v2.y}, w3[2] = {x.v3.x, x.v3.y};
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            const uint32_t sel = (uint32_t)((b & 3) | ((b & 3) << 4) | ((4 + (b & 3)) << 8) | ((4 + (b & 3)) << 12));
+            const uint32_t t1 = __byte_perm(w0[b >> 2], w1[b >> 2], sel);      // bytes (row 2 c4: b, -, row 2 c4 + 1: b, -)
+            const uint32_t t2 = __byte_perm(w2[b >> 2], w3[b >> 2], sel);
+            mma16816(st.acc[b], nc.lo(t1), nc.hi(t1), nc.lo(t2), nc.hi(t2), b0, b1);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(AT_D)
+k_attend_int4_gqa(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int gq, int ng, int min_rows,
+                  float* __restrict__ ws) {
+    __shared__ __align__(16) __half qp[GQ_MAX][AT_D];       // per query, every 8 elements ordered 0 4 1 5 2 6 3 7
+    __shared__ float qsum_s[GQ_MAX];
+    __shared__ float wpart[AT_WARPS][GQ_MAX][AT_D];
+    __shared__ float wstat[AT_WARPS][GQ_MAX][2];
+    const int h = blockIdx.x, c = blockIdx.y, l = blockIdx.z, t = threadIdx.x;
+    const int lane = t & 31, wid = t >> 5, g8 = lane >> 2, c4 = lane & 3;
+    const int Hq = H * gq;
+    const size_t HD2 = (size_t)H * (AT_D / 2);
+    const long long n4 = min(fill[2], pp.cap4);
+    const long long per = max((long long)min_rows, ((n4 + AT_CHUNKS - 1) / AT_CHUNKS + 15) / 16 * 16);
+    const long long r0 = (long long)c * per, r1 = min(n4, r0 + per);
+    float* rec0 = ws + (((size_t)l * Hq + (size_t)h * gq) * AT_RECS + AT_REC4 + c) * AT_REC;      // of the group's first query
+    if (r0 >= r1) {                                 // nothing in this chunk: records the merge skips
+        if (t < gq) {
+            float* rec = rec0 + (size_t)t * AT_RECS * AT_REC;
+            rec[AT_D] = -INFINITY;
+            rec[AT_D + 1] = 0.0f;
+        }
+        return;
+    }
+    // warp w stages query w of the group and sums it
+    if (wid < GQ_MAX) {
+        float part = 0.0f;
+#pragma unroll
+        for (int k = 0; k < AT_D / 32; ++k) {
+            const int e = lane + 32 * k;
+            const __half qv = wid < gq ? q[((size_t)l * Hq + (size_t)h * gq + wid) * AT_D + e] : __float2half(0.0f);
+            const int e8 = e & 7;
+            qp[wid][(e & ~7) | ((e8 & 3) * 2 + (e8 >> 2))] = qv;
+            part += __half2float(qv);
+        }
+        part = warp_sum(part);
+        if (lane == 0) qsum_s[wid] = part;
+    }
+    __syncthreads();
+    const float rs = rsqrtf((float)AT_D);
+    const float qsum = qsum_s[c4];                  // this lane's query
+    const int g = ng == 1 ? 0 : h;
+    // B fragments of the score product: the lanes with g8 = 2 j hold query j (column 2 j), the others zeros
+    uint32_t qf[8][2];
+    {
+        const uint32_t* qp32 = reinterpret_cast<const uint32_t*>(qp[(g8 >> 1) & (GQ_MAX - 1)]);
+        const bool has = (g8 & 1) == 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int oct = 4 * c4 + (j >> 1), u = j & 1;
+            qf[j][0] = has ? qp32[oct * 4 + 2 * u] : 0u;
+            qf[j][1] = has ? qp32[oct * 4 + 2 * u + 1] : 0u;
+        }
+    }
+    const long long t0 = r0 + 16 * wid;             // this warp's first tile
+    G4Addr ad;
+    ad.pitch = HD2;
+    ad.ng = (size_t)ng;
+    ad.k = pp.int4_codes + ((size_t)(2 * l) * pp.cap4 + (size_t)(t0 + g8)) * HD2 + (size_t)h * (AT_D / 2) + 16 * c4;
+    ad.v = pp.int4_codes + ((size_t)(2 * l + 1) * pp.cap4 + (size_t)(t0 + 2 * c4)) * HD2 + (size_t)h * (AT_D / 2) + 8 * g8;
+    ad.ks = reinterpret_cast<const uint32_t*>(pp.int4_sz) + ((size_t)(2 * l) * pp.cap4 + (size_t)(t0 + g8)) * ng + g;
+    ad.vs = reinterpret_cast<const uint32_t*>(pp.int4_sz) + ((size_t)(2 * l + 1) * pp.cap4 + (size_t)(t0 + g8)) * ng + g;
+    NibConst nc;
+    nc.init();
+    I4State st;
+#pragma unroll
+    for (int b = 0; b < 8; ++b) st.acc[b][0] = st.acc[b][1] = st.acc[b][2] = st.acc[b][3] = 0.0f;
+    st.m = -INFINITY;
+    st.den = st.zacc = 0.0f;
+    st.F = 4096.0f;
+    constexpr long long STEP = 16 * AT_WARPS;
+    G4Tile xa, xb;                                  // two tiles in turn: one is consumed while the other is in flight
+    long long tile = t0;
+    if (tile < r1) {
+        g4_fetch(xa, ad, tile, t0, r1, g8, c4);
+        for (;;) {
+            g4_fetch(xb, ad, tile + STEP, t0, r1, g8, c4);
+            g4_tile(st, xa, qf, nc, tile, r1, rs, qsum, g8, c4);
+            tile += STEP;
+            if (tile >= r1) break;
+            g4_fetch(xa, ad, tile + STEP, t0, r1, g8, c4);
+            g4_tile(st, xb, qf, nc, tile, r1, rs, qsum, g8, c4);
+            tile += STEP;
+            if (tile >= r1) break;
+        }
+    }
+    // ---- this warp's results, one per query
+    {
+        const float den = group_sum(st.den), zs = group_sum(st.zacc);
+        const float invF = 1.0f / st.F;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            wpart[wid][c4][16 * g8 + 2 * b] = (st.acc[b][0] + st.acc[b][1]) * invF + zs;
+            wpart[wid][c4][16 * g8 + 2 * b + 1] = (st.acc[b][2] + st.acc[b][3]) * invF + zs;
+        }
+        if (g8 == 0) {
+            wstat[wid][c4][0] = st.m;
+            wstat[wid][c4][1] = den;
+        }
+    }
+    __syncthreads();
+    for (int j = 0; j < gq; ++j) {
+        float M = wstat[0][j][0];
+#pragma unroll
+        for (int k = 1; k < AT_WARPS; ++k) M = fmaxf(M, wstat[k][j][0]);
+        float sum = 0.0f, dsum = 0.0f;
+        if (M != -INFINITY) {
+#pragma unroll
+            for (int k = 0; k < AT_WARPS; ++k) {
+                const float e = wstat[k][j][0] == -INFINITY ? 0.0f : __expf(wstat[k][j][0] - M);
+                sum += e * wpart[k][j][t];
+                dsum += e * wstat[k][j][1];
+            }
+        }
+        float* rec = rec0 + (size_t)j * AT_RECS * AT_REC;
+        rec[t] = sum;
+        if (t == 0) {
+            rec[AT_D] = M;
+            rec[AT_D + 1] = dsum;
+        }
+    }
+}
+
 // ---- INT8 rows on the matrix instructions, the same plan as for INT4: scores = 16 key rows x 16 dimensions
 // times the query in columns 0 and 2; values = 16 dimensions x 16 value rows times the split weights.  A code
 // byte becomes binary16 by a byte permute with 0x64 above it (1024 + (code + 128) after flipping its sign bit)
@@ -879,7 +1130,10 @@ int sc_attend(salicache_ctx* c, const void* d_q, int q_per_kv, const salicache_p
     const int min_rows = (int)std::min<long long>(4096, std::max<long long>(256, 8ll * p.L * Hq)) / 16 * 16;
     dim3 grid8(Hq, AT_CH8, p.L);
     k_attend_int8<<<grid8, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
-    if (p.heads == 32 && ng == 32) k_attend_int4<32 * AT_D / 2, 32><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
+    if (gq > 1 && gq <= GQ_MAX) {                   // the queries of a group share the expansion of the codes
+        dim3 gridg(p.heads, AT_CHUNKS, p.L);
+        k_attend_int4_gqa<<<gridg, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
+    } else if (p.heads == 32 && ng == 32) k_attend_int4<32 * AT_D / 2, 32><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
     else if (p.heads == 32 && ng == 1) k_attend_int4<32 * AT_D / 2, 1><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
     else k_attend_int4<0, 0><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
     dim3 gm(Hq, p.L);
