@@ -963,6 +963,206 @@ __device__ __forceinline__ void i8_tile(I4State& st, const I8Tile& x, const uint
     }
 }
 
+// ---- INT8 rows, grouped queries: as k_attend_int4_gqa, with the byte expansion of k_attend_int8.
+struct G8Tile {
+    uint4 ka0, ka1, kb0, kb1;      // keys of rows g8 and g8 + 8: dimensions 16 c4 .. + 15 and 64 + 16 c4 .. + 15
+    uint4 v0, v1, v2, v3;          // values of rows c4, c4 + 4, c4 + 8, c4 + 12: dimensions 16 g8 .. + 15
+    uint32_t ksa, ksb, vsa, vsb;   // binary16 scales of the keys and values of rows g8 and g8 + 8
+};
+__device__ __forceinline__ void g8_fetch(G8Tile& x, const I8Addr& a, long long tile, long long t0, long long r1, int g8, int c4) {
+    const size_t d = (size_t)(tile - t0), P = a.pitch;
+    const uint8_t* k = a.k + d * P;
+    const uint8_t* v = a.v + d * P;
+    const uint16_t* ks = a.ks + d * a.ng;
+    const uint16_t* vs = a.vs + d * a.ng;
+    const uint4 z = make_uint4(0, 0, 0, 0);
+    const long long ra = tile + g8, rv = tile + c4;
+    const bool full = tile + 16 <= r1;
+    const bool pa = full || ra < r1, pb = full || ra + 8 < r1;
+    x.ka0 = pa ? ld_stream16(k) : z;
+    x.ka1 = pa ? ld_stream16(k + 64) : z;
+    x.kb0 = pb ? ld_stream16(k + 8 * P) : z;
+    x.kb1 = pb ? ld_stream16(k + 8 * P + 64) : z;
+    x.v0 = full || rv < r1 ? ld_stream16(v) : z;
+    x.v1 = full || rv + 4 < r1 ? ld_stream16(v + 4 * P) : z;
+    x.v2 = full || rv + 8 < r1 ? ld_stream16(v + 8 * P) : z;
+    x.v3 = full || rv + 12 < r1 ? ld_stream16(v + 12 * P) : z;
+    x.ksa = pa ? (uint32_t)__ldg(ks) : 0u;
+    x.vsa = pa ? (uint32_t)__ldg(vs) : 0u;
+    x.ksb = pb ? (uint32_t)__ldg(ks + 8 * a.ng) : 0u;
+    x.vsb = pb ? (uint32_t)__ldg(vs + 8 * a.ng) : 0u;
+}
+
+__device__ __forceinline__ void g8_tile(I4State& st, const G8Tile& x, const uint32_t (&qf)[8][2], const ByteConst& bc, long long tile,
+                                        long long r1, float rs, int g8, int c4) {
+    float sc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    {
+        const uint32_t wa[8] = {x.ka0.x, x.ka0.y, x.ka0.z, x.ka0.w, x.ka1.x, x.ka1.y, x.ka1.z, x.ka1.w};
+        const uint32_t wb[8] = {x.kb0.x, x.kb0.y, x.kb0.z, x.kb0.w, x.kb1.x, x.kb1.y, x.kb1.z, x.kb1.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t ua = wa[j] ^ 0x80808080u, ub = wb[j] ^ 0x80808080u;
+            mma16816(sc, bc.pair<0, 1>(ua), bc.pair<0, 1>(ub), bc.pair<2, 3>(ua), bc.pair<2, 3>(ub), qf[j][0], qf[j][1]);
+        }
+    }
+    // this lane: query c4 against rows g8 (sc[0]) and g8 + 8 (sc[2])
+    const bool va = tile + g8 < r1, vb = tile + g8 + 8 < r1;
+    const float sa = va ? rs * sc[0] * h2f((uint16_t)x.ksa) : -INFINITY;
+    const float sb = vb ? rs * sc[2] * h2f((uint16_t)x.ksb) : -INFINITY;
+    const float sva = va ? h2f((uint16_t)x.vsa) : 0.0f, svb = vb ? h2f((uint16_t)x.vsb) : 0.0f;
+    const float sm = fmaxf(sa, sb), sv = fmaxf(sva, svb);
+    if (__any_sync(0xffffffffu, sm > st.m || sv * st.F >= 32768.0f)) {
+        const float m_new = fmaxf(st.m, group_max(sm));
+        const float corr = st.m == -INFINITY ? 0.0f : __expf(st.m - m_new);
+        st.m = m_new;
+        const float smax = warp_max(sv);
+        float Fn = st.F;
+        for (int k = 0; k < 40 && smax * Fn >= 32768.0f; ++k) Fn *= 0.5f;
+        const float rescale = corr * (Fn / st.F);
+        st.F = Fn;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) st.acc[b][i] *= rescale;
+        }
+        st.den *= corr;
+    }
+    const float pa_ = __expf(sa - st.m), pb_ = __expf(sb - st.m);
+    st.den += pa_ + pb_;
+    uint32_t packa, packb;
+    {
+        const float wa_ = pa_ * sva * st.F, wb_ = pb_ * svb * st.F;
+        const __half ha = __float2half_rn(wa_), hb = __float2half_rn(wb_);
+        const __half la = __float2half_rn(wa_ - __half2float(ha)), lb = __float2half_rn(wb_ - __half2float(hb));
+        packa = (uint32_t)__half_as_ushort(ha) | ((uint32_t)__half_as_ushort(la) << 16);
+        packb = (uint32_t)__half_as_ushort(hb) | ((uint32_t)__half_as_ushort(lb) << 16);
+    }
+    // column g8 of the value product = high (even) or low (odd) halves of query g8 / 2; k = rows c4, c4 + 4 (b0) and
+    // c4 + 8, c4 + 12 (b1); the weight of (row r, query j) is in lane 4 (r % 8) + j, in packa for r < 8, else packb
+    const int la = 4 * c4 + (g8 >> 1);
+    const uint32_t x1 = __shfl_sync(0xffffffffu, packa, la), x2 = __shfl_sync(0xffffffffu, packa, la + 16);
+    const uint32_t y1 = __shfl_sync(0xffffffffu, packb, la), y2 = __shfl_sync(0xffffffffu, packb, la + 16);
+    const uint32_t psel = (g8 & 1) ? 0x7632u : 0x5410u;
+    const uint32_t b0 = __byte_perm(x1, x2, psel), b1 = __byte_perm(y1, y2, psel);
+    {
+        const uint32_t w0[4] = {x.v0.x, x.v0.y, x.v0.z, x.v0.w}, w1[4] = {x.v1.x, x.v1.y, x.v1.z, x.v1.w};
+        const uint32_t w2[4] = {x.v2.x, x.v2.y, x.v2.z, x.v2.w}, w3[4] = {x.v3.x, x.v3.y, x.v3.z, x.v3.w};
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            const uint32_t sel = (b & 1) ? 0x7632u : 0x5410u;
+            const uint32_t t1 = __byte_perm(w0[b >> 1], w1[b >> 1], sel) ^ 0x80808080u;
+            const uint32_t t2 = __byte_perm(w2[b >> 1], w3[b >> 1], sel) ^ 0x80808080u;
+            mma16816(st.acc[b], bc.pair<0, 2>(t1), bc.pair<1, 3>(t1), bc.pair<0, 2>(t2), bc.pair<1, 3>(t2), b0, b1);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(AT_D)
+k_attend_int8_gqa(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int gq, int ng, int min_rows,
+                  float* __restrict__ ws) {
+    __shared__ __align__(16) __half qn[GQ_MAX][AT_D];
+    __shared__ float wpart[AT_WARPS][GQ_MAX][AT_D];
+    __shared__ float wstat[AT_WARPS][GQ_MAX][2];
+    const int h = blockIdx.x, c = blockIdx.y, l = blockIdx.z, t = threadIdx.x;
+    const int lane = t & 31, wid = t >> 5, g8 = lane >> 2, c4 = lane & 3;
+    const int Hq = H * gq;
+    const size_t HD = (size_t)H * AT_D;
+    const long long n8 = min(fill[1], pp.cap8);
+    const long long per = max((long long)min_rows, ((n8 + AT_CH8 - 1) / AT_CH8 + 15) / 16 * 16);
+    const long long r0 = (long long)c * per, r1 = min(n8, r0 + per);
+    float* rec0 = ws + (((size_t)l * Hq + (size_t)h * gq) * AT_RECS + AT_REC8 + c) * AT_REC;      // of the group's first query
+    if (r0 >= r1) {
+        if (t < gq) {
+            float* rec = rec0 + (size_t)t * AT_RECS * AT_REC;
+            rec[AT_D] = -INFINITY;
+            rec[AT_D + 1] = 0.0f;
+        }
+        return;
+    }
+#pragma unroll
+    for (int j = 0; j < GQ_MAX; ++j) qn[j][t] = j < gq ? q[((size_t)l * Hq + (size_t)h * gq + j) * AT_D + t] : __float2half(0.0f);
+    __syncthreads();
+    const float rs = rsqrtf((float)AT_D);
+    const int g = ng == 1 ? 0 : h;
+    uint32_t qf[8][2];                              // the lanes with g8 = 2 j hold query j (column 2 j)
+    {
+        const uint32_t* q32 = reinterpret_cast<const uint32_t*>(qn[(g8 >> 1) & (GQ_MAX - 1)]);
+        const bool has = (g8 & 1) == 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int base = (j < 4 ? 16 * c4 + 4 * j : 64 + 16 * c4 + 4 * (j - 4)) / 2;
+            qf[j][0] = has ? q32[base] : 0u;
+            qf[j][1] = has ? q32[base + 1] : 0u;
+        }
+    }
+    const long long t0 = r0 + 16 * wid;
+    I8Addr ad;
+    ad.pitch = HD;
+    ad.ng = (size_t)ng;
+    ad.k = pp.int8_codes + ((size_t)(2 * l) * pp.cap8 + (size_t)(t0 + g8)) * HD + (size_t)h * AT_D + 16 * c4;
+    ad.v = pp.int8_codes + ((size_t)(2 * l + 1) * pp.cap8 + (size_t)(t0 + c4)) * HD + (size_t)h * AT_D + 16 * g8;
+    ad.ks = reinterpret_cast<const uint16_t*>(pp.int8_scale) + ((size_t)(2 * l) * pp.cap8 + (size_t)(t0 + g8)) * ng + g;
+    ad.vs = reinterpret_cast<const uint16_t*>(pp.int8_scale) + ((size_t)(2 * l + 1) * pp.cap8 + (size_t)(t0 + g8)) * ng + g;
+    ByteConst bc;
+    bc.init();
+    I4State st;
+#pragma unroll
+    for (int b = 0; b < 8; ++b) st.acc[b][0] = st.acc[b][1] = st.acc[b][2] = st.acc[b][3] = 0.0f;
+    st.m = -INFINITY;
+    st.den = st.zacc = 0.0f;
+    st.F = 4096.0f;
+    constexpr long long STEP = 16 * AT_WARPS;
+    G8Tile xa, xb;
+    long long tile = t0;
+    if (tile < r1) {
+        g8_fetch(xa, ad, tile, t0, r1, g8, c4);
+        for (;;) {
+            g8_fetch(xb, ad, tile + STEP, t0, r1, g8, c4);
+            g8_tile(st, xa, qf, bc, tile, r1, rs, g8, c4);
+            tile += STEP;
+            if (tile >= r1) break;
+            g8_fetch(xa, ad, tile + STEP, t0, r1, g8, c4);
+            g8_tile(st, xb, qf, bc, tile, r1, rs, g8, c4);
+            tile += STEP;
+            if (tile >= r1) break;
+        }
+    }
+    {
+        const float den = group_sum(st.den);
+        const float invF = 1.0f / st.F;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            wpart[wid][c4][16 * g8 + 2 * b] = (st.acc[b][0] + st.acc[b][1]) * invF;
+            wpart[wid][c4][16 * g8 + 2 * b + 1] = (st.acc[b][2] + st.acc[b][3]) * invF;
+        }
+        if (g8 == 0) {
+            wstat[wid][c4][0] = st.m;
+            wstat[wid][c4][1] = den;
+        }
+    }
+    __syncthreads();
+    for (int j = 0; j < gq; ++j) {
+        float M = wstat[0][j][0];
+#pragma unroll
+        for (int k = 1; k < AT_WARPS; ++k) M = fmaxf(M, wstat[k][j][0]);
+        float sum = 0.0f, dsum = 0.0f;
+        if (M != -INFINITY) {
+#pragma unroll
+            for (int k = 0; k < AT_WARPS; ++k) {
+                const float e = wstat[k][j][0] == -INFINITY ? 0.0f : __expf(wstat[k][j][0] - M);
+                sum += e * wpart[k][j][t];
+                dsum += e * wstat[k][j][1];
+            }
+        }
+        float* rec = rec0 + (size_t)j * AT_RECS * AT_REC;
+        rec[t] = sum;
+        if (t == 0) {
+            rec[AT_D] = M;
+            rec[AT_D + 1] = dsum;
+        }
+    }
+}
+
 // Merge the four warps of a CTA of the matrix-instruction kernels and write its partial record.
 __device__ __forceinline__ void mma_finish(const I4State& st, float (*wpart)[AT_D], float (*wstat)[2], float* rec, int g8, int c4) {
     const int t = threadIdx.x, lane = t & 31, wid = t >> 5;
@@ -1128,8 +1328,13 @@ int sc_attend(salicache_ctx* c, const void* d_q, int q_per_kv, const salicache_p
     // rows per chunk of the quantised kernels: up to 4096 (64 tiles per warp) when there are many (layer, head) pairs
     // to fill the GPU with, fewer when there are few
     const int min_rows = (int)std::min<long long>(4096, std::max<long long>(256, 8ll * p.L * Hq)) / 16 * 16;
-    dim3 grid8(Hq, AT_CH8, p.L);
-    k_attend_int8<<<grid8, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
+    if (gq > 1 && gq <= GQ_MAX) {                   // the queries of a group share the expansion of the codes
+        dim3 grid8g(p.heads, AT_CH8, p.L);
+        k_attend_int8_gqa<<<grid8g, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
+    } else {
+        dim3 grid8(Hq, AT_CH8, p.L);
+        k_attend_int8<<<grid8, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
+    }
     if (gq > 1 && gq <= GQ_MAX) {                   // the queries of a group share the expansion of the codes
         dim3 gridg(p.heads, AT_CHUNKS, p.L);
         k_attend_int4_gqa<<<gridg, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
