@@ -1163,6 +1163,161 @@ k_attend_int8_gqa(const __half* __restrict__ q, AtPools pp, const long long* __r
     }
 }
 
+// ---- FP16 rows, grouped queries: the rows need no expansion, so a tile is 16 loads of 16 bytes per lane, two
+// byte permutes per value operand and 16 matrix instructions for up to 4 queries.  One query per key/value
+// head keeps the scalar kernel above (k_attend_partial), which already runs close to the memory bandwidth.
+struct G16Tile {
+    uint4 ka[4], kb[4];            // keys of rows g8 and g8 + 8: dimensions 32 c4 .. + 31
+    uint4 v[4][2];                 // values of rows c4, c4 + 4, c4 + 8, c4 + 12: dimensions 16 g8 .. + 15
+};
+__device__ __forceinline__ void g16_fetch(G16Tile& x, const uint8_t* k, const uint8_t* v, size_t P, long long tile, long long r1,
+                                          int g8, int c4) {
+    const uint4 z = make_uint4(0, 0, 0, 0);
+    const bool full = tile + 16 <= r1;
+    const long long ra = tile + g8, rv = tile + c4;
+    const bool pa = full || ra < r1, pb = full || ra + 8 < r1;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        x.ka[i] = pa ? ld_stream16(k + 16 * i) : z;
+        x.kb[i] = pb ? ld_stream16(k + 8 * P + 16 * i) : z;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const bool pv = full || rv + 4 * j < r1;
+        x.v[j][0] = pv ? ld_stream16(v + 4 * j * P) : z;
+        x.v[j][1] = pv ? ld_stream16(v + 4 * j * P + 16) : z;
+    }
+}
+
+__global__ void __launch_bounds__(AT_D)
+k_attend_fp16_gqa(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int gq, int min_rows,
+                  float* __restrict__ ws) {
+    __shared__ __align__(16) __half qn[GQ_MAX][AT_D];
+    __shared__ float wpart[AT_WARPS][GQ_MAX][AT_D];
+    __shared__ float wstat[AT_WARPS][GQ_MAX][2];
+    const int h = blockIdx.x, c = blockIdx.y, l = blockIdx.z, t = threadIdx.x;
+    const int lane = t & 31, wid = t >> 5, g8 = lane >> 2, c4 = lane & 3;
+    const int Hq = H * gq;
+    const size_t P = (size_t)H * AT_D * 2;          // bytes per row
+    const long long n16 = min(fill[0], pp.cap16);
+    const long long per = max((long long)min_rows, ((n16 + gridDim.y - 1) / gridDim.y + 15) / 16 * 16);
+    const long long r0 = (long long)c * per, r1 = min(n16, r0 + per);
+    float* rec0 = ws + (((size_t)l * Hq + (size_t)h * gq) * AT_RECS + c) * AT_REC;       // of the group's first query
+    if (r0 >= r1) {
+        if (t < gq) {
+            float* rec = rec0 + (size_t)t * AT_RECS * AT_REC;
+            rec[AT_D] = -INFINITY;
+            rec[AT_D + 1] = 0.0f;
+        }
+        return;
+    }
+#pragma unroll
+    for (int j = 0; j < GQ_MAX; ++j) qn[j][t] = j < gq ? q[((size_t)l * Hq + (size_t)h * gq + j) * AT_D + t] : __float2half(0.0f);
+    __syncthreads();
+    const float rs = rsqrtf((float)AT_D);
+    uint32_t qf[8][2];                              // the lanes with g8 = 2 j hold query j (column 2 j)
+    {
+        const uint32_t* q32 = reinterpret_cast<const uint32_t*>(qn[(g8 >> 1) & (GQ_MAX - 1)]);
+        const bool has = (g8 & 1) == 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            qf[j][0] = has ? q32[16 * c4 + 2 * j] : 0u;               // dimensions 32 c4 + 4 j, + 1
+            qf[j][1] = has ? q32[16 * c4 + 2 * j + 1] : 0u;           //            32 c4 + 4 j + 2, + 3
+        }
+    }
+    const long long t0 = r0 + 16 * wid;
+    const uint8_t* kbase = pp.fp16_pool + ((size_t)(2 * l) * pp.cap16 + (size_t)(t0 + g8)) * P + (size_t)h * AT_D * 2 + 64 * c4;
+    const uint8_t* vbase = pp.fp16_pool + ((size_t)(2 * l + 1) * pp.cap16 + (size_t)(t0 + c4)) * P + (size_t)h * AT_D * 2 + 32 * g8;
+    float acc[8][4];
+#pragma unroll
+    for (int b = 0; b < 8; ++b) acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.0f;
+    float m = -INFINITY, den = 0.0f;
+    constexpr float F = 4096.0f;                    // the weights are scaled by a power of two before the binary16 split
+    constexpr long long STEP = 16 * AT_WARPS;
+    for (long long tile = t0; tile < r1; tile += STEP) {
+        G16Tile x;
+        g16_fetch(x, kbase + (size_t)(tile - t0) * P, vbase + (size_t)(tile - t0) * P, P, tile, r1, g8, c4);
+        float sc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            mma16816(sc, x.ka[i].x, x.kb[i].x, x.ka[i].y, x.kb[i].y, qf[2 * i][0], qf[2 * i][1]);
+            mma16816(sc, x.ka[i].z, x.kb[i].z, x.ka[i].w, x.kb[i].w, qf[2 * i + 1][0], qf[2 * i + 1][1]);
+        }
+        // this lane: query c4 against rows g8 (sc[0]) and g8 + 8 (sc[2])
+        const float sa = tile + g8 < r1 ? rs * sc[0] : -INFINITY;
+        const float sb = tile + g8 + 8 < r1 ? rs * sc[2] : -INFINITY;
+        const float sm = fmaxf(sa, sb);
+        if (__any_sync(0xffffffffu, sm > m)) {
+            const float m_new = fmaxf(m, group_max(sm));
+            const float corr = m == -INFINITY ? 0.0f : __expf(m - m_new);
+            m = m_new;
+#pragma unroll
+            for (int b = 0; b < 8; ++b) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[b][i] *= corr;
+            }
+            den *= corr;
+        }
+        const float pa_ = __expf(sa - m), pb_ = __expf(sb - m);
+        den += pa_ + pb_;
+        uint32_t packa, packb;
+        {
+            const float wa_ = pa_ * F, wb_ = pb_ * F;
+            const __half ha = __float2half_rn(wa_), hb = __float2half_rn(wb_);
+            const __half la = __float2half_rn(wa_ - __half2float(ha)), lb = __float2half_rn(wb_ - __half2float(hb));
+            packa = (uint32_t)__half_as_ushort(ha) | ((uint32_t)__half_as_ushort(la) << 16);
+            packb = (uint32_t)__half_as_ushort(hb) | ((uint32_t)__half_as_ushort(lb) << 16);
+        }
+        const int la = 4 * c4 + (g8 >> 1);
+        const uint32_t x1 = __shfl_sync(0xffffffffu, packa, la), x2 = __shfl_sync(0xffffffffu, packa, la + 16);
+        const uint32_t y1 = __shfl_sync(0xffffffffu, packb, la), y2 = __shfl_sync(0xffffffffu, packb, la + 16);
+        const uint32_t psel = (g8 & 1) ? 0x7632u : 0x5410u;
+        const uint32_t b0 = __byte_perm(x1, x2, psel), b1 = __byte_perm(y1, y2, psel);
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            // word b of a row's 32 bytes holds dimensions 16 g8 + 2 b and + 1: pair the same dimension of two rows
+            const uint32_t w0 = b < 4 ? (&x.v[0][0].x)[b] : (&x.v[0][1].x)[b - 4], w1 = b < 4 ? (&x.v[1][0].x)[b] : (&x.v[1][1].x)[b - 4];
+            const uint32_t w2 = b < 4 ? (&x.v[2][0].x)[b] : (&x.v[2][1].x)[b - 4], w3 = b < 4 ? (&x.v[3][0].x)[b] : (&x.v[3][1].x)[b - 4];
+            mma16816(acc[b], __byte_perm(w0, w1, 0x5410), __byte_perm(w0, w1, 0x7632), __byte_perm(w2, w3, 0x5410),
+                     __byte_perm(w2, w3, 0x7632), b0, b1);
+        }
+    }
+    {
+        const float dsum = group_sum(den);
+        constexpr float invF = 1.0f / F;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            wpart[wid][c4][16 * g8 + 2 * b] = (acc[b][0] + acc[b][1]) * invF;
+            wpart[wid][c4][16 * g8 + 2 * b + 1] = (acc[b][2] + acc[b][3]) * invF;
+        }
+        if (g8 == 0) {
+            wstat[wid][c4][0] = m;
+            wstat[wid][c4][1] = dsum;
+        }
+    }
+    __syncthreads();
+    for (int j = 0; j < gq; ++j) {
+        float M = wstat[0][j][0];
+#pragma unroll
+        for (int k = 1; k < AT_WARPS; ++k) M = fmaxf(M, wstat[k][j][0]);
+        float sum = 0.0f, dsum = 0.0f;
+        if (M != -INFINITY) {
+#pragma unroll
+            for (int k = 0; k < AT_WARPS; ++k) {
+                const float e = wstat[k][j][0] == -INFINITY ? 0.0f : __expf(wstat[k][j][0] - M);
+                sum += e * wpart[k][j][t];
+                dsum += e * wstat[k][j][1];
+            }
+        }
+        float* rec = rec0 + (size_t)j * AT_RECS * AT_REC;
+        rec[t] = sum;
+        if (t == 0) {
+            rec[AT_D] = M;
+            rec[AT_D + 1] = dsum;
+        }
+    }
+}
+
 // Merge the four warps of a CTA of the matrix-instruction kernels and write its partial record.
 __device__ __forceinline__ void mma_finish(const I4State& st, float (*wpart)[AT_D], float (*wstat)[2], float* rec, int g8, int c4) {
     const int t = threadIdx.x, lane = t & 31, wid = t >> 5;
@@ -1324,7 +1479,13 @@ int sc_attend(salicache_ctx* c, const void* d_q, int q_per_kv, const salicache_p
     dim3 grid16(Hq, nch, p.L);
     const __half* qh = (const __half*)d_q;
     const long long* fl = (const long long*)d_fill;
-    k_attend_partial<<<grid16, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, 0, 0, c->attend_ws);
+    if (gq > 1 && gq <= GQ_MAX) {
+        dim3 grid16g(p.heads, nch, p.L);
+        const int min_rows16 = (int)std::min<long long>(1024, std::max<long long>(64, 2ll * p.L * p.heads)) / 16 * 16;
+        k_attend_fp16_gqa<<<grid16g, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, min_rows16, c->attend_ws);
+    } else {
+        k_attend_partial<<<grid16, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, 0, 0, c->attend_ws);
+    }
     // rows per chunk of the quantised kernels: up to 4096 (64 tiles per warp) when there are many (layer, head) pairs
     // to fill the GPU with, fewer when there are few
     const int min_rows = (int)std::min<long long>(4096, std::max<long long>(256, 8ll * p.L * Hq)) / 16 * 16;
