@@ -1479,7 +1479,7 @@ int sc_attend(salicache_ctx* c, const void* d_q, int q_per_kv, const salicache_p
     dim3 grid16(Hq, nch, p.L);
     const __half* qh = (const __half*)d_q;
     const long long* fl = (const long long*)d_fill;
-    if (gq > 1 && gq <= GQ_MAX) {
+    if (gq <= GQ_MAX) {
         dim3 grid16g(p.heads, nch, p.L);
         const int min_rows16 = (int)std::min<long long>(1024, std::max<long long>(64, 2ll * p.L * p.heads)) / 16 * 16;
         k_attend_fp16_gqa<<<grid16g, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, min_rows16, c->attend_ws);
