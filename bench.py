@@ -403,6 +403,41 @@ def run_extras(sc, synth, ctx, wl, T, frames, dP, dev, peak, pools, fill, stored
             "frac_of_hbm_peak": round(bytes_m / ms / 1e6 / peak, 4)}
         del pm
         cm.close()
+    # grouped-query attention at the shape of the paper's evaluation model (8 key/value heads, 4 queries each, 32 layers)
+    # over a four-tier cache of 128 frames of random K/V
+    if True:
+        Tg, Hg, gq = 128, 8, 4
+        HDg = Hg * 128
+        g = torch.Generator(device=dev)
+        g.manual_seed(13)
+        cg = sc.Context(sc.salicache_default_params(max_batch=Tg, chunk_frames=2, L=32, heads=Hg, **synth.thresholds("four")))
+        Kg = torch.randn((Tg, 32, 576, HDg), generator=g, device=dev, dtype=torch.float16)
+        Vg = torch.randn((Tg, 32, 576, HDg), generator=g, device=dev, dtype=torch.float16)
+        sg = (0.2 + 0.4 * torch.rand((Tg, 576), generator=g, device=dev)).float()
+        decg = torch.zeros((Tg, 576), dtype=torch.uint8, device=dev)
+        idxg = torch.zeros((Tg, 3, 576), dtype=torch.int32, device=dev)
+        cntg = torch.zeros((Tg, 5), dtype=torch.int32, device=dev)
+        redg = torch.zeros((Tg,), dtype=torch.uint8, device=dev)
+        offg = torch.zeros((Tg, 3), dtype=torch.int64, device=dev)
+        fillg = torch.zeros((3,), dtype=torch.int64, device=dev)
+        sc.salicache_select(cg, None, sg, Tg, False, decg, idxg, cntg, redg, offg, fillg)
+        cc = cntg.sum(dim=0).cpu().numpy()
+        pg = sc.PoolSet(32, HDg, int(cc[4]) + 1, int(cc[3]) + 1, int(cc[2]) + 1, device=dev)
+        sc.salicache_pack_kv(cg, Kg, Vg, 32 * 576 * HDg, idxg, cntg, offg, Tg, pg.c)
+        torch.cuda.synchronize()
+        del Kg, Vg
+        bytes_g = 2 * 32 * (int(cc[4]) * HDg * 2 + int(cc[3]) * (HDg + 2 * Hg) + int(cc[2]) * (HDg // 2 + 4 * Hg))
+        qg = torch.randn((32, Hg * gq, 128), generator=g, device=dev, dtype=torch.float32).to(torch.float16)
+        og = torch.zeros((32, Hg * gq, 128), dtype=torch.float32, device=dev)
+        ms = timed(lambda: sc.salicache_attend_gqa(cg, qg, gq, pg.c, fillg, og), reps=5)
+        out["attend_gqa_8x4"] = {
+            "what": "salicache_attend_gqa: 32 query heads over 8 key/value heads (the paper's Mistral-7B shape), 32 layers, "
+                    "four-tier cache of 128 frames of random K/V",
+            "rows": {"fp16": int(cc[4]), "int8": int(cc[3]), "int4": int(cc[2])}, "ms": round(ms, 3), "cache_bytes": int(bytes_g),
+            "l2": "cache larger than L2", "algorithmic_GBps": round(bytes_g / ms / 1e6, 1),
+            "frac_of_hbm_peak": round(bytes_g / ms / 1e6 / peak, 4)}
+        del pg
+        cg.close()
     # anchor-frame mode: the scan over the frames of this workload (Eq. 5 literal against the anchor image + decisions)
     if wl.n_images == 1 and T > 1:
         tau_grey = 3.0

@@ -321,9 +321,9 @@ SALICACHE_API int salicache_attend(salicache_ctx* ctx, const void* d_q, const sa
  * heads that serve 32 query heads, Sec. IV-A): query head hq, 0 <= hq < heads * q_per_kv, attends to the rows of
  * key/value head hq / q_per_kv of the store (heads = the context's heads, the store's key/value heads).
  *   d_q, d_out   DEVICE f16 / f32 [L][heads * q_per_kv][head_dim], 16-byte aligned
- * q_per_kv = 1 is salicache_attend.  q_per_kv < 1 or heads * q_per_kv > max(heads, 64): E_SHAPE.  Each query head
- * reads its key/value head's rows itself; the heads of a group run side by side, so the rows come from the L2
- * for all but the first.  Other arguments and errors as for salicache_attend.
+ * q_per_kv = 1 is salicache_attend.  q_per_kv < 1 or heads * q_per_kv > max(heads, 64): E_SHAPE.  Up to 4 queries
+ * per key/value head share one pass over its rows (the store is read once for the whole group); with more, every
+ * query head reads the rows itself.  Other arguments and errors as for salicache_attend.
  */
 SALICACHE_API int salicache_attend_gqa(salicache_ctx* ctx, const void* d_q, int q_per_kv, const salicache_pools* pools,
                                        const int64_t* d_fill, float* d_out, void* cuda_stream);

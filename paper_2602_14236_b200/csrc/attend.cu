@@ -4,11 +4,12 @@
 //
 //   score_j = q_h . K^_{j,h} / sqrt(D),   p = softmax_j(score),   out_h = sum_j p_j V^_{j,h}
 //
-// Split over the rows: per layer and head a few dozen partial results of each of three kernels, merged by a
-// fourth.  k_attend_partial takes the FP16 rows: scores one row per thread (the thread walks the head's 128
-// key elements of its row: no cross-lane reduction), values four dimensions per lane, one row per warp at a
-// time.  k_attend_int8 and k_attend_int4 take the quantised rows, the bulk of a compressed cache, 16 rows per
-// warp at a time through matrix instructions.  Online softmax and single precision accumulation in all.
+// Split over the rows: per layer and head a few dozen partial results of each of three kernels (one per tier),
+// merged by a fourth.  All three walk 16 rows per warp at a time through matrix instructions: the FP16 rows as
+// they are, the INT8 and INT4 rows after expanding the codes to binary16 in registers; with grouped queries the
+// 2 to 4 query heads of a key/value head are the columns of those instructions.  k_attend_partial, scalar code
+// with one row per thread, remains for more than 4 queries per key/value head.  Online softmax and single
+// precision accumulation in all.
 #include <cuda_fp16.h>
 
 #include <algorithm>
