@@ -128,10 +128,11 @@ def test_attention_int4_rows_peaked_and_large_values():
         _check(ctx, pools, ref, fill, (3.0 * k_row).astype(np.float16), scale=v_scale)
 
 
-@pytest.mark.parametrize("heads,q_per_kv,background", [(8, 4, "four"), (8, 4, "int4"), (32, 2, "int8")])
+@pytest.mark.parametrize("heads,q_per_kv,background", [(8, 4, "four"), (8, 4, "int4"), (32, 2, "int8"), (8, 3, "int8"), (8, 8, "four")])
 def test_grouped_query_attention_matches_the_oracle(heads, q_per_kv, background):
     """The paper's evaluation model has 8 key/value heads for 32 query heads: query head hq reads key/value head
-    hq // q_per_kv.  Also 32 key/value heads with two queries each (64 query heads, the most the workspace holds)."""
+    hq // q_per_kv.  Also 32 key/value heads with two queries each (64 query heads, the most the workspace holds), a group
+    of three, and a group of eight (more than the matrix-instruction kernels take: every query head reads for itself)."""
     import torch
     ctx, pools, ref, fill, rng = _store(L=2, heads=heads, T=2, background=background, seed=21)
     q = rng.standard_normal((2, heads * q_per_kv, 128)).astype(np.float16)
