@@ -322,8 +322,8 @@ SALICACHE_API int salicache_attend(salicache_ctx* ctx, const void* d_q, const sa
  * key/value head hq / q_per_kv of the store (heads = the context's heads, the store's key/value heads).
  *   d_q, d_out   DEVICE f16 / f32 [L][heads * q_per_kv][head_dim], 16-byte aligned
  * q_per_kv = 1 is salicache_attend.  q_per_kv < 1 or heads * q_per_kv > max(heads, 64): E_SHAPE.  Up to 4 queries
- * per key/value head share one pass over its rows (the store is read once for the whole group); with more, every
- * query head reads the rows itself.  Other arguments and errors as for salicache_attend.
+ * per key/value head share one pass over its rows (the store is read once for the whole group); larger groups take
+ * one pass per 4 queries.  Other arguments and errors as for salicache_attend.
  */
 SALICACHE_API int salicache_attend_gqa(salicache_ctx* ctx, const void* d_q, int q_per_kv, const salicache_pools* pools,
                                        const int64_t* d_fill, float* d_out, void* cuda_stream);

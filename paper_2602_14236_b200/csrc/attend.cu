@@ -6,10 +6,9 @@
 //
 // Split over the rows: per layer and head a few dozen partial results of each of three kernels (one per tier),
 // merged by a fourth.  All three walk 16 rows per warp at a time through matrix instructions: the FP16 rows as
-// they are, the INT8 and INT4 rows after expanding the codes to binary16 in registers; with grouped queries the
-// 2 to 4 query heads of a key/value head are the columns of those instructions.  k_attend_partial, scalar code
-// with one row per thread, remains for more than 4 queries per key/value head.  Online softmax and single
-// precision accumulation in all.
+// they are, the INT8 and INT4 rows after expanding the codes to binary16 in registers; with grouped queries up to
+// 4 query heads of a key/value head are the columns of those instructions.  Online softmax and single precision
+// accumulation in all.
 #include <cuda_fp16.h>
 
 #include <algorithm>
@@ -40,38 +39,10 @@ struct AtPools {
 __device__ __forceinline__ float h2f(uint16_t b) { return __half2float(__ushort_as_half(b)); }
 __device__ __forceinline__ float2 w2f(uint32_t w) { return __half22float2(*reinterpret_cast<const __half2*>(&w)); }
 
-// c + a.lo * b.lo + a.hi * b.hi with a, b pairs of binary16: the mixed-precision multiply-add forms each
-// product exactly and rounds the sum once to binary32.
-__device__ __forceinline__ float dot2(uint32_t a, uint32_t b, float c) {
-    float d;
-    asm("{ .reg .b16 al, ah, bl, bh; .reg .f32 t; mov.b32 {al, ah}, %1; mov.b32 {bl, bh}, %2;\n\t"
-        "fma.rn.f32.f16 t, al, bl, %3; fma.rn.f32.f16 %0, ah, bh, t; }"
-        : "=f"(d)
-        : "r"(a), "r"(b), "f"(c));
-    return d;
-}
 __device__ __forceinline__ uint32_t hsub2u(uint32_t a, uint32_t b) {
     __half2 r = __hsub2(*reinterpret_cast<const __half2*>(&a), *reinterpret_cast<const __half2*>(&b));
     return *reinterpret_cast<const uint32_t*>(&r);
 }
-// Codes to binary16 without integer-to-float conversions: OR the code into the mantissa of 1024 (binary16
-// 0x6400, unit in the last place 1) and subtract 1024 again; both steps are exact.
-// Four INT4 code pairs of a word of 8 nibbles e0..e7: (e0,e4) (e1,e5) (e2,e6) (e3,e7).
-__device__ __forceinline__ void nibbles_to_h2(uint32_t x, uint32_t out[4]) {
-#pragma unroll
-    for (int k = 0; k < 4; k += 2) {
-        const uint32_t y = x >> (4 * k);
-        out[k] = hsub2u((y & 0x000f000fu) | 0x64006400u, 0x64006400u);
-        out[k + 1] = hsub2u((y & 0x00f000f0u) | 0x54005400u, 0x54005400u);      // 64 + nibble: unit in the last place 1/16
-    }
-}
-// Two INT8 code pairs of a word of 4 bytes b0..b3: (b0,b1) (b2,b3).  The bytes are biased by 128 first.
-__device__ __forceinline__ void bytes_to_h2(uint32_t w, uint32_t out[2]) {
-    const uint32_t u = w ^ 0x80808080u;
-    out[0] = hsub2u(__byte_perm(u, 0x64646464u, 0x4140), 0x64806480u);
-    out[1] = hsub2u(__byte_perm(u, 0x64646464u, 0x4342), 0x64806480u);
-}
-
 __device__ __forceinline__ float block_max(float v, float* red) {
 #pragma unroll
     for (int o = 16; o; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
@@ -93,180 +64,6 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
     for (int k = 0; k < AT_WARPS; ++k) r += red[k];      // fixed order: deterministic
     __syncthreads();
     return r;
-}
-
-__global__ void __launch_bounds__(AT_D)
-k_attend_partial(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int gq, int ng,
-                 int with_int8, int with_int4, float* __restrict__ ws) {
-    __shared__ __align__(16) float qs[AT_D];        // the query as binary32 (for sum(q))
-    __shared__ __align__(16) __half qn[AT_D];       // the query in natural order
-    __shared__ __align__(16) __half qp[AT_D];       // the query with every 8 elements ordered 0 4 1 5 2 6 3 7 (INT4 pairs)
-    __shared__ float4 rowrec[AT_D];                 // per row of the tile: weight * value scale, weight * value zero,
-                                                    // pool row (as an integer)
-    __shared__ float red[AT_WARPS];
-    __shared__ float part[AT_WARPS][AT_D];
-    // heads vary fastest over the grid: the CTAs that read the 32 slices of one row run at about the same time
-    const int hq = blockIdx.x, c = blockIdx.y, l = blockIdx.z, t = threadIdx.x;
-    const int h = hq / gq, Hq = H * gq;          // query head hq reads key/value head h
-    const int lane = t & 31, wid = t >> 5;
-    const int HD = H * AT_D;
-    const long long n16 = min(fill[0], pp.cap16);
-    const long long n8 = with_int8 ? min(fill[1], pp.cap8) : 0;      // the INT8 rows may be left to k_attend_int8,
-    const long long n4 = with_int4 ? min(fill[2], pp.cap4) : 0;      // the INT4 rows to k_attend_int4
-    const long long R = n16 + n8 + n4;
-    const long long per = (R + gridDim.y - 1) / gridDim.y;      // the host sizes the grid's chunks by the pools' capacity
-    const long long r0 = (long long)c * per, r1 = min(R, r0 + per);
-    if (r0 >= r1) {                                 // nothing in this chunk: a record the merge skips
-        if (t == 0) {
-            float* rec = ws + (((size_t)l * Hq + hq) * AT_RECS + c) * AT_REC;
-            rec[AT_D] = -INFINITY;
-            rec[AT_D + 1] = 0.0f;
-        }
-        return;
-    }
-    {
-        const __half qv = q[((size_t)l * Hq + hq) * AT_D + t];
-        const int e = t & 7;
-        qs[t] = __half2float(qv);
-        qn[t] = qv;
-        qp[(t & ~7) | ((e & 3) * 2 + (e >> 2))] = qv;      // element e of its octet goes to slot 2 (e mod 4) + e div 4
-    }
-    __syncthreads();
-    const float rs = rsqrtf((float)AT_D);
-    float qsum = block_sum(qs[t], red);             // the INT4 zero point adds z * sum(q) to a score
-    const int g = ng == 1 ? 0 : h;                  // group of this head's elements in a row's scale array
-    float m = -INFINITY, den = 0.0f;
-    float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-    float zacc = 0.0f;                              // sum of p * zero over this warp's INT4 rows: the same for every dimension
-    // this lane's slice of the head's values in row 0 of each pool's V plane of layer l
-    const uint8_t* vbase16 = pp.fp16_pool + (((size_t)(2 * l + 1) * pp.cap16) * HD + (size_t)h * AT_D) * 2 + lane * 8;
-    const uint8_t* vbase8 = pp.int8_codes + ((size_t)(2 * l + 1) * pp.cap8) * HD + (size_t)h * AT_D + lane * 4;
-    const uint8_t* vbase4 = pp.int4_codes + ((size_t)(2 * l + 1) * pp.cap4) * (HD / 2) + (size_t)h * (AT_D / 2) + lane * 2;
-    const uint4* qn4 = reinterpret_cast<const uint4*>(qn);
-    const uint4* qp4 = reinterpret_cast<const uint4*>(qp);
-    for (long long tile = r0; tile < r1; tile += AT_D) {
-        const long long r = tile + t;
-        float s = -INFINITY;
-        int vrow = 0;
-        float vsc = 1.0f, vzr = 0.0f;               // scale and zero of the row's VALUE slice (its key has its own)
-        if (r < r1) {
-            float dot = 0.0f;
-            if (r < n16) {
-                const size_t prow = (size_t)(2 * l) * pp.cap16 + r;
-                const uint4* kp = reinterpret_cast<const uint4*>(pp.fp16_pool + (prow * HD + (size_t)h * AT_D) * 2);
-                vrow = (int)r;
-#pragma unroll 4
-                for (int i = 0; i < AT_D / 8; ++i) {
-                    const uint4 w = __ldg(kp + i), qq = qn4[i];
-                    dot = dot2(w.x, qq.x, dot);
-                    dot = dot2(w.y, qq.y, dot);
-                    dot = dot2(w.z, qq.z, dot);
-                    dot = dot2(w.w, qq.w, dot);
-                }
-                s = dot * rs;
-            } else if (r < n16 + n8) {
-                const long long row = r - n16;
-                const size_t prow = (size_t)(2 * l) * pp.cap8 + row;
-                const uint4* kp = reinterpret_cast<const uint4*>(pp.int8_codes + prow * HD + (size_t)h * AT_D);
-                vrow = (int)row;
-                vsc = h2f(reinterpret_cast<const uint16_t*>(pp.int8_scale)[((size_t)(2 * l + 1) * pp.cap8 + row) * ng + g]);
-#pragma unroll 2
-                for (int i = 0; i < AT_D / 16; ++i) {
-                    const uint4 w = __ldg(kp + i);
-                    const uint4 qa = qn4[2 * i], qb = qn4[2 * i + 1];
-                    uint32_t c[2];
-                    bytes_to_h2(w.x, c); dot = dot2(c[0], qa.x, dot); dot = dot2(c[1], qa.y, dot);
-                    bytes_to_h2(w.y, c); dot = dot2(c[0], qa.z, dot); dot = dot2(c[1], qa.w, dot);
-                    bytes_to_h2(w.z, c); dot = dot2(c[0], qb.x, dot); dot = dot2(c[1], qb.y, dot);
-                    bytes_to_h2(w.w, c); dot = dot2(c[0], qb.z, dot); dot = dot2(c[1], qb.w, dot);
-                }
-                s = dot * (rs * h2f(reinterpret_cast<const uint16_t*>(pp.int8_scale)[prow * ng + g]));
-            } else {
-                const long long row = r - n16 - n8;
-                const size_t prow = (size_t)(2 * l) * pp.cap4 + row;
-                const uint4* kp = reinterpret_cast<const uint4*>(pp.int4_codes + prow * (HD / 2) + (size_t)h * (AT_D / 2));
-                float d4[4] = {0.0f, 0.0f, 0.0f, 0.0f};      // four partial sums: shorter dependency chains
-                vrow = (int)row;
-                {
-                    const uint32_t vz = reinterpret_cast<const uint32_t*>(pp.int4_sz)[((size_t)(2 * l + 1) * pp.cap4 + row) * ng + g];
-                    vsc = h2f((uint16_t)(vz & 0xffff));
-                    vzr = h2f((uint16_t)(vz >> 16));
-                }
-#pragma unroll 2
-                for (int i = 0; i < AT_D / 32; ++i) {
-                    const uint4 w = __ldg(kp + i);
-                    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const uint4 qq = qp4[4 * i + k];
-                        uint32_t c[4];
-                        nibbles_to_h2(ww[k], c);
-                        d4[0] = dot2(c[0], qq.x, d4[0]);
-                        d4[1] = dot2(c[1], qq.y, d4[1]);
-                        d4[2] = dot2(c[2], qq.z, d4[2]);
-                        d4[3] = dot2(c[3], qq.w, d4[3]);
-                    }
-                }
-                dot = (d4[0] + d4[1]) + (d4[2] + d4[3]);
-                const uint32_t sz = reinterpret_cast<const uint32_t*>(pp.int4_sz)[prow * ng + g];
-                s = rs * (dot * h2f((uint16_t)(sz & 0xffff)) + qsum * h2f((uint16_t)(sz >> 16)));
-            }
-        }
-        // online softmax: new running maximum, rescale what has been accumulated so far
-        const float mt = block_max(s, red);
-        const float m_new = fmaxf(m, mt);
-        const float corr = m == -INFINITY ? 0.0f : __expf(m - m_new);
-        const float p = r < r1 ? __expf(s - m_new) : 0.0f;
-        rowrec[t] = make_float4(p * vsc, p * vzr, __int_as_float(vrow), 0.0f);
-        den = den * corr + block_sum(p, red);       // (its barriers also publish rowrec)
-        m = m_new;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) acc[k] *= corr;
-        zacc *= corr;
-        // values: warp w takes the tile's rows w, w + 4, ...; a lane owns dimensions 4 * lane .. 4 * lane + 3
-        const int n_tile = (int)min((long long)AT_D, r1 - tile);
-        // the rows of a tile are ordered by tier (FP16, INT8, INT4): three loops without a per-row branch
-        const int e16 = (int)max(0ll, min((long long)n_tile, n16 - tile));
-        const int e8 = (int)max(0ll, min((long long)n_tile, n16 + n8 - tile));
-        int rr = wid;
-        for (; rr < e16; rr += AT_WARPS) {
-            const float4 rec = rowrec[rr];
-            const uint2 w = __ldg(reinterpret_cast<const uint2*>(vbase16 + (size_t)__float_as_int(rec.z) * ((size_t)HD * 2)));
-            const float2 a = w2f(w.x), b = w2f(w.y);
-            acc[0] += rec.x * a.x; acc[1] += rec.x * a.y; acc[2] += rec.x * b.x; acc[3] += rec.x * b.y;
-        }
-        for (; rr < e8; rr += AT_WARPS) {
-            const float4 rec = rowrec[rr];
-            const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(vbase8 + (size_t)__float_as_int(rec.z) * (size_t)HD));
-            uint32_t cw[2];
-            bytes_to_h2(w, cw);
-            const float2 a = w2f(cw[0]), b = w2f(cw[1]);
-            acc[0] += rec.x * a.x; acc[1] += rec.x * a.y; acc[2] += rec.x * b.x; acc[3] += rec.x * b.y;
-        }
-#pragma unroll 4
-        for (; rr < n_tile; rr += AT_WARPS) {
-            const float4 rec = rowrec[rr];
-            const uint32_t w = __ldg(reinterpret_cast<const uint16_t*>(vbase4 + (size_t)__float_as_int(rec.z) * (size_t)(HD / 2)));
-            const uint32_t y = __byte_perm(w, 0u, 0x4140);      // bytes (e1 e0) 0 (e3 e2) 0: pairs (e0,e2), (e1,e3) by one mask
-            const float2 a = w2f(hsub2u((y & 0x000f000fu) | 0x64006400u, 0x64006400u));
-            const float2 b = w2f(hsub2u(((y >> 4) & 0x000f000fu) | 0x64006400u, 0x64006400u));
-            acc[0] += rec.x * a.x; acc[1] += rec.x * b.x; acc[2] += rec.x * a.y; acc[3] += rec.x * b.y;
-            zacc += rec.y;
-        }
-        __syncthreads();                            // rowrec is rewritten by the next tile
-    }
-#pragma unroll
-    for (int k = 0; k < 4; ++k) part[wid][4 * lane + k] = acc[k] + zacc;
-    __syncthreads();
-    float* rec = ws + (((size_t)l * Hq + hq) * AT_RECS + c) * AT_REC;
-    float sum = 0.0f;
-#pragma unroll
-    for (int k = 0; k < AT_WARPS; ++k) sum += part[k][t];
-    rec[t] = sum;
-    if (t == 0) {
-        rec[AT_D] = m;
-        rec[AT_D + 1] = den;
-    }
 }
 
 // ---- INT4 rows on the tensor cores.  A single query is a matrix-vector product, but forming it with
@@ -594,8 +391,9 @@ k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restr
     }
 }
 
-// ---- INT4 rows, grouped queries: the 2 to 4 query heads that share a key/value head are the columns of the
-// matrix instructions, so the codes of a tile are expanded once for all of them.  Query j sits in column 2 j of
+// ---- INT4 rows, grouped queries: up to 4 of the query heads that share a key/value head (queries q0 .. q0 + gqn - 1
+// of each group; larger groups take several launches) are the columns of the matrix instructions, so the codes of a
+// tile are expanded once for all of them.  Query j sits in column 2 j of
 // the score product; lane (g8, c4) therefore finds the products of query c4 with rows g8 and g8 + 8 in its own
 // accumulator, and keeps that query's softmax statistics (shared by the 8 lanes with the same c4).  In the value
 // product the weights of query j fill columns 2 j (high halves) and 2 j + 1 (low halves), so every lane's
@@ -724,7 +522,8 @@ __device__ __forceinline__ void g4_tile(I4State& st, const G4Tile& x, const uint
 }
 
 __global__ void __launch_bounds__(AT_D)
-k_attend_int4_gqa(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int gq, int ng, int min_rows,
+k_attend_int4_gqa(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int gq, int q0, int gqn, int ng,
+                  int min_rows,
                   float* __restrict__ ws) {
     __shared__ __align__(16) __half qp[GQ_MAX][AT_D];       // per query, every 8 elements ordered 0 4 1 5 2 6 3 7
     __shared__ float qsum_s[GQ_MAX];
@@ -737,9 +536,9 @@ k_attend_int4_gqa(const __half* __restrict__ q, AtPools pp, const long long* __r
     const long long n4 = min(fill[2], pp.cap4);
     const long long per = max((long long)min_rows, ((n4 + AT_CHUNKS - 1) / AT_CHUNKS + 15) / 16 * 16);
     const long long r0 = (long long)c * per, r1 = min(n4, r0 + per);
-    float* rec0 = ws + (((size_t)l * Hq + (size_t)h * gq) * AT_RECS + AT_REC4 + c) * AT_REC;      // of the group's first query
+    float* rec0 = ws + (((size_t)l * Hq + (size_t)h * gq + q0) * AT_RECS + AT_REC4 + c) * AT_REC;      // of the group's first query
     if (r0 >= r1) {                                 // nothing in this chunk: records the merge skips
-        if (t < gq) {
+        if (t < gqn) {
             float* rec = rec0 + (size_t)t * AT_RECS * AT_REC;
             rec[AT_D] = -INFINITY;
             rec[AT_D + 1] = 0.0f;
@@ -752,7 +551,7 @@ k_attend_int4_gqa(const __half* __restrict__ q, AtPools pp, const long long* __r
 #pragma unroll
         for (int k = 0; k < AT_D / 32; ++k) {
             const int e = lane + 32 * k;
-            const __half qv = wid < gq ? q[((size_t)l * Hq + (size_t)h * gq + wid) * AT_D + e] : __float2half(0.0f);
+            const __half qv = wid < gqn ? q[((size_t)l * Hq + (size_t)h * gq + q0 + wid) * AT_D + e] : __float2half(0.0f);
             const int e8 = e & 7;
             qp[wid][(e & ~7) | ((e8 & 3) * 2 + (e8 >> 2))] = qv;
             part += __half2float(qv);
@@ -823,7 +622,7 @@ k_attend_int4_gqa(const __half* __restrict__ q, AtPools pp, const long long* __r
         }
     }
     __syncthreads();
-    for (int j = 0; j < gq; ++j) {
+    for (int j = 0; j < gqn; ++j) {
         float M = wstat[0][j][0];
 #pragma unroll
         for (int k = 1; k < AT_WARPS; ++k) M = fmaxf(M, wstat[k][j][0]);
@@ -1059,7 +858,8 @@ __device__ __forceinline__ void g8_tile(I4State& st, const G8Tile& x, const uint
 }
 
 __global__ void __launch_bounds__(AT_D)
-k_attend_int8_gqa(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int gq, int ng, int min_rows,
+k_attend_int8_gqa(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int gq, int q0, int gqn, int ng,
+                  int min_rows,
                   float* __restrict__ ws) {
     __shared__ __align__(16) __half qn[GQ_MAX][AT_D];
     __shared__ float wpart[AT_WARPS][GQ_MAX][AT_D];
@@ -1071,9 +871,9 @@ k_attend_int8_gqa(const __half* __restrict__ q, AtPools pp, const long long* __r
     const long long n8 = min(fill[1], pp.cap8);
     const long long per = max((long long)min_rows, ((n8 + AT_CH8 - 1) / AT_CH8 + 15) / 16 * 16);
     const long long r0 = (long long)c * per, r1 = min(n8, r0 + per);
-    float* rec0 = ws + (((size_t)l * Hq + (size_t)h * gq) * AT_RECS + AT_REC8 + c) * AT_REC;      // of the group's first query
+    float* rec0 = ws + (((size_t)l * Hq + (size_t)h * gq + q0) * AT_RECS + AT_REC8 + c) * AT_REC;      // of the group's first query
     if (r0 >= r1) {
-        if (t < gq) {
+        if (t < gqn) {
             float* rec = rec0 + (size_t)t * AT_RECS * AT_REC;
             rec[AT_D] = -INFINITY;
             rec[AT_D + 1] = 0.0f;
@@ -1081,7 +881,7 @@ k_attend_int8_gqa(const __half* __restrict__ q, AtPools pp, const long long* __r
         return;
     }
 #pragma unroll
-    for (int j = 0; j < GQ_MAX; ++j) qn[j][t] = j < gq ? q[((size_t)l * Hq + (size_t)h * gq + j) * AT_D + t] : __float2half(0.0f);
+    for (int j = 0; j < GQ_MAX; ++j) qn[j][t] = j < gqn ? q[((size_t)l * Hq + (size_t)h * gq + q0 + j) * AT_D + t] : __float2half(0.0f);
     __syncthreads();
     const float rs = rsqrtf((float)AT_D);
     const int g = ng == 1 ? 0 : h;
@@ -1142,7 +942,7 @@ k_attend_int8_gqa(const __half* __restrict__ q, AtPools pp, const long long* __r
         }
     }
     __syncthreads();
-    for (int j = 0; j < gq; ++j) {
+    for (int j = 0; j < gqn; ++j) {
         float M = wstat[0][j][0];
 #pragma unroll
         for (int k = 1; k < AT_WARPS; ++k) M = fmaxf(M, wstat[k][j][0]);
@@ -1191,7 +991,8 @@ __device__ __forceinline__ void g16_fetch(G16Tile& x, const uint8_t* k, const ui
 }
 
 __global__ void __launch_bounds__(AT_D)
-k_attend_fp16_gqa(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int gq, int min_rows,
+k_attend_fp16_gqa(const __half* __restrict__ q, AtPools pp, const long long* __restrict__ fill, int H, int gq, int q0, int gqn,
+                  int min_rows,
                   float* __restrict__ ws) {
     __shared__ __align__(16) __half qn[GQ_MAX][AT_D];
     __shared__ float wpart[AT_WARPS][GQ_MAX][AT_D];
@@ -1203,9 +1004,9 @@ k_attend_fp16_gqa(const __half* __restrict__ q, AtPools pp, const long long* __r
     const long long n16 = min(fill[0], pp.cap16);
     const long long per = max((long long)min_rows, ((n16 + gridDim.y - 1) / gridDim.y + 15) / 16 * 16);
     const long long r0 = (long long)c * per, r1 = min(n16, r0 + per);
-    float* rec0 = ws + (((size_t)l * Hq + (size_t)h * gq) * AT_RECS + c) * AT_REC;       // of the group's first query
+    float* rec0 = ws + (((size_t)l * Hq + (size_t)h * gq + q0) * AT_RECS + c) * AT_REC;       // of the group's first query
     if (r0 >= r1) {
-        if (t < gq) {
+        if (t < gqn) {
             float* rec = rec0 + (size_t)t * AT_RECS * AT_REC;
             rec[AT_D] = -INFINITY;
             rec[AT_D + 1] = 0.0f;
@@ -1213,7 +1014,7 @@ k_attend_fp16_gqa(const __half* __restrict__ q, AtPools pp, const long long* __r
         return;
     }
 #pragma unroll
-    for (int j = 0; j < GQ_MAX; ++j) qn[j][t] = j < gq ? q[((size_t)l * Hq + (size_t)h * gq + j) * AT_D + t] : __float2half(0.0f);
+    for (int j = 0; j < GQ_MAX; ++j) qn[j][t] = j < gqn ? q[((size_t)l * Hq + (size_t)h * gq + q0 + j) * AT_D + t] : __float2half(0.0f);
     __syncthreads();
     const float rs = rsqrtf((float)AT_D);
     uint32_t qf[8][2];                              // the lanes with g8 = 2 j hold query j (column 2 j)
@@ -1297,7 +1098,7 @@ k_attend_fp16_gqa(const __half* __restrict__ q, AtPools pp, const long long* __r
         }
     }
     __syncthreads();
-    for (int j = 0; j < gq; ++j) {
+    for (int j = 0; j < gqn; ++j) {
         float M = wstat[0][j][0];
 #pragma unroll
         for (int k = 1; k < AT_WARPS; ++k) M = fmaxf(M, wstat[k][j][0]);
@@ -1473,39 +1274,37 @@ int sc_attend(salicache_ctx* c, const void* d_q, int q_per_kv, const salicache_p
     if (pp.cap16 >= (1ll << 28) || pp.cap8 >= (1ll << 28) || pp.cap4 >= (1ll << 28)) return SALICACHE_E_SHAPE;
     const int ng = p.group == AT_D ? p.heads : 1;
     const int gq = q_per_kv, Hq = p.heads * gq;     // query heads; query head hq reads key/value head hq / gq
-    dim3 grid(Hq, AT_CHUNKS, p.L);
-    // FP16 rows one row per thread; INT8 and INT4 rows, the bulk of a compressed cache, on the matrix instructions.
-    // The first kernel gets as many chunks as its pool can fill with four tiles each, 32 at most.
-    const int nch = (int)std::min<long long>(AT_CH16, std::max<long long>(1, (pp.cap16 + 4 * AT_D - 1) / (4 * AT_D)));
-    dim3 grid16(Hq, nch, p.L);
     const __half* qh = (const __half*)d_q;
     const long long* fl = (const long long*)d_fill;
-    if (gq <= GQ_MAX) {
-        dim3 grid16g(p.heads, nch, p.L);
-        const int min_rows16 = (int)std::min<long long>(1024, std::max<long long>(64, 2ll * p.L * p.heads)) / 16 * 16;
-        k_attend_fp16_gqa<<<grid16g, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, min_rows16, c->attend_ws);
-    } else {
-        k_attend_partial<<<grid16, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, 0, 0, c->attend_ws);
-    }
-    // rows per chunk of the quantised kernels: up to 4096 (64 tiles per warp) when there are many (layer, head) pairs
-    // to fill the GPU with, fewer when there are few
+    // chunks of the FP16 kernel: as many as its pool can fill with four tiles each, 32 at most
+    const int nch = (int)std::min<long long>(AT_CH16, std::max<long long>(1, (pp.cap16 + 4 * AT_D - 1) / (4 * AT_D)));
+    // rows per chunk: up to 4096 of the quantised tiers, 1024 of FP16 (64 tiles per warp) when there are many (layer,
+    // head) pairs to fill the GPU with, fewer when there are few
     const int min_rows = (int)std::min<long long>(4096, std::max<long long>(256, 8ll * p.L * Hq)) / 16 * 16;
-    if (gq > 1 && gq <= GQ_MAX) {                   // the queries of a group share the expansion of the codes
-        dim3 grid8g(p.heads, AT_CH8, p.L);
-        k_attend_int8_gqa<<<grid8g, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
+    const int min_rows16 = (int)std::min<long long>(1024, std::max<long long>(64, 2ll * p.L * p.heads)) / 16 * 16;
+    int launches = 0;
+    if (gq == 1) {
+        // one query per head: the FP16 kernel with a single column; INT8 and INT4 with a softmax row per lane
+        k_attend_fp16_gqa<<<dim3(p.heads, nch, p.L), AT_D, 0, st>>>(qh, pp, fl, p.heads, 1, 0, 1, min_rows16, c->attend_ws);
+        k_attend_int8<<<dim3(p.heads, AT_CH8, p.L), AT_D, 0, st>>>(qh, pp, fl, p.heads, 1, ng, min_rows, c->attend_ws);
+        dim3 grid(p.heads, AT_CHUNKS, p.L);
+        if (p.heads == 32 && ng == 32) k_attend_int4<32 * AT_D / 2, 32><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, 1, ng, min_rows, c->attend_ws);
+        else if (p.heads == 32 && ng == 1) k_attend_int4<32 * AT_D / 2, 1><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, 1, ng, min_rows, c->attend_ws);
+        else k_attend_int4<0, 0><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, 1, ng, min_rows, c->attend_ws);
+        launches = 3;
     } else {
-        dim3 grid8(Hq, AT_CH8, p.L);
-        k_attend_int8<<<grid8, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
+        // grouped queries: up to GQ_MAX queries of every key/value head per launch share one pass over its rows
+        for (int q0 = 0; q0 < gq; q0 += GQ_MAX) {
+            const int gqn = std::min(GQ_MAX, gq - q0);
+            k_attend_fp16_gqa<<<dim3(p.heads, nch, p.L), AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, q0, gqn, min_rows16, c->attend_ws);
+            k_attend_int8_gqa<<<dim3(p.heads, AT_CH8, p.L), AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, q0, gqn, ng, min_rows, c->attend_ws);
+            k_attend_int4_gqa<<<dim3(p.heads, AT_CHUNKS, p.L), AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, q0, gqn, ng, min_rows, c->attend_ws);
+            launches += 3;
+        }
     }
-    if (gq > 1 && gq <= GQ_MAX) {                   // the queries of a group share the expansion of the codes
-        dim3 gridg(p.heads, AT_CHUNKS, p.L);
-        k_attend_int4_gqa<<<gridg, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
-    } else if (p.heads == 32 && ng == 32) k_attend_int4<32 * AT_D / 2, 32><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
-    else if (p.heads == 32 && ng == 1) k_attend_int4<32 * AT_D / 2, 1><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
-    else k_attend_int4<0, 0><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, ng, min_rows, c->attend_ws);
     dim3 gm(Hq, p.L);
     k_attend_merge<<<gm, AT_D, 0, st>>>(c->attend_ws, Hq, nch, d_out);
-    c->launches += 4;
+    c->launches += launches + 1;
     SC_CHECK(cudaGetLastError());
     return SALICACHE_OK;
 }

@@ -132,7 +132,7 @@ def test_attention_int4_rows_peaked_and_large_values():
 def test_grouped_query_attention_matches_the_oracle(heads, q_per_kv, background):
     """The paper's evaluation model has 8 key/value heads for 32 query heads: query head hq reads key/value head
     hq // q_per_kv.  Also 32 key/value heads with two queries each (64 query heads, the most the workspace holds), a group
-    of three, and a group of eight (more than the matrix-instruction kernels take: every query head reads for itself)."""
+    of three, and a group of eight (two passes of four)."""
     import torch
     ctx, pools, ref, fill, rng = _store(L=2, heads=heads, T=2, background=background, seed=21)
     q = rng.standard_normal((2, heads * q_per_kv, 128)).astype(np.float16)
