@@ -289,7 +289,7 @@ k_attend_int4(const __half* __restrict__ q, AtPools pp, const long long* __restr
     const long long n4 = min(fill[2], pp.cap4);
     // whole tiles per chunk, and at least min_rows rows: a cache that is not huge is spread over fewer CTAs (the
     // rest leave at once), so that the fixed cost of a CTA, staging the query and merging its warps, is paid less often
-    const long long per = max((long long)min_rows, ((n4 + AT_CHUNKS - 1) / AT_CHUNKS + 15) / 16 * 16);
+    const long long per = max((long long)min_rows, ((n4 + gridDim.y - 1) / gridDim.y + 15) / 16 * 16);
     const long long r0 = (long long)c * per, r1 = min(n4, r0 + per);
     if (r0 >= r1) {                                 // nothing in this chunk: a record the merge skips
         if (t == 0) {
@@ -534,7 +534,7 @@ k_attend_int4_gqa(const __half* __restrict__ q, AtPools pp, const long long* __r
     const int Hq = H * gq;
     const size_t HD2 = (size_t)H * (AT_D / 2);
     const long long n4 = min(fill[2], pp.cap4);
-    const long long per = max((long long)min_rows, ((n4 + AT_CHUNKS - 1) / AT_CHUNKS + 15) / 16 * 16);
+    const long long per = max((long long)min_rows, ((n4 + gridDim.y - 1) / gridDim.y + 15) / 16 * 16);
     const long long r0 = (long long)c * per, r1 = min(n4, r0 + per);
     float* rec0 = ws + (((size_t)l * Hq + (size_t)h * gq + q0) * AT_RECS + AT_REC4 + c) * AT_REC;      // of the group's first query
     if (r0 >= r1) {                                 // nothing in this chunk: records the merge skips
@@ -869,7 +869,7 @@ k_attend_int8_gqa(const __half* __restrict__ q, AtPools pp, const long long* __r
     const int Hq = H * gq;
     const size_t HD = (size_t)H * AT_D;
     const long long n8 = min(fill[1], pp.cap8);
-    const long long per = max((long long)min_rows, ((n8 + AT_CH8 - 1) / AT_CH8 + 15) / 16 * 16);
+    const long long per = max((long long)min_rows, ((n8 + gridDim.y - 1) / gridDim.y + 15) / 16 * 16);
     const long long r0 = (long long)c * per, r1 = min(n8, r0 + per);
     float* rec0 = ws + (((size_t)l * Hq + (size_t)h * gq + q0) * AT_RECS + AT_REC8 + c) * AT_REC;      // of the group's first query
     if (r0 >= r1) {
@@ -1168,7 +1168,7 @@ k_attend_int8(const __half* __restrict__ q, AtPools pp, const long long* __restr
     const int lane = t & 31, wid = t >> 5, g8 = lane >> 2, c4 = lane & 3;
     const size_t HD = (size_t)H * AT_D;
     const long long n8 = min(fill[1], pp.cap8);
-    const long long per = max((long long)min_rows, ((n8 + AT_CH8 - 1) / AT_CH8 + 15) / 16 * 16);
+    const long long per = max((long long)min_rows, ((n8 + gridDim.y - 1) / gridDim.y + 15) / 16 * 16);
     const long long r0 = (long long)c * per, r1 = min(n8, r0 + per);
     float* rec = ws + (((size_t)l * Hq + hq) * AT_RECS + AT_REC8 + c) * AT_REC;
     if (r0 >= r1) {                                 // nothing in this chunk: a record the merge skips
@@ -1233,14 +1233,14 @@ k_attend_int8(const __half* __restrict__ q, AtPools pp, const long long* __restr
 
 // Merge the partial results of one (layer, head): out = sum_c e^(m_c - M) acc_c / sum_c e^(m_c - M) den_c.
 __global__ void __launch_bounds__(AT_D)
-k_attend_merge(const float* __restrict__ ws, int H, int nch, float* __restrict__ out) {
+k_attend_merge(const float* __restrict__ ws, int H, int nch16, int nch8, int nch4, float* __restrict__ out) {
     __shared__ float ew[AT_RECS];                   // e^(m_c - M), 0 for a record that is empty or was not written
     __shared__ float red[AT_WARPS];
     static_assert(AT_RECS == AT_D, "one record per thread in the statistics pass");
     const int h = blockIdx.x, l = blockIdx.y, t = threadIdx.x;
     const float* rec = ws + ((size_t)l * H + h) * AT_RECS * AT_REC;
-    // records 0 .. nch-1 come from k_attend_partial, the rest from k_attend_int8 and k_attend_int4
-    const bool written = t < nch || t >= AT_REC8;
+    // the first nch16, nch8, nch4 records of the FP16, INT8, INT4 ranges were written by this call's kernels
+    const bool written = t < nch16 || (t >= AT_REC8 && t < AT_REC8 + nch8) || (t >= AT_REC4 && t < AT_REC4 + nch4);
     const float mc = written ? rec[t * AT_REC + AT_D] : -INFINITY;
     const float dc = written ? rec[t * AT_REC + AT_D + 1] : 0.0f;
     const float M = block_max(mc, red);
@@ -1282,12 +1282,15 @@ int sc_attend(salicache_ctx* c, const void* d_q, int q_per_kv, const salicache_p
     // head) pairs to fill the GPU with, fewer when there are few
     const int min_rows = (int)std::min<long long>(4096, std::max<long long>(256, 8ll * p.L * Hq)) / 16 * 16;
     const int min_rows16 = (int)std::min<long long>(1024, std::max<long long>(64, 2ll * p.L * p.heads)) / 16 * 16;
+    // chunks of the quantised kernels: no more than their pools can fill with min_rows rows each
+    const int nch8 = (int)std::min<long long>(AT_CH8, std::max<long long>(1, (pp.cap8 + min_rows - 1) / min_rows));
+    const int nch4 = (int)std::min<long long>(AT_CHUNKS, std::max<long long>(1, (pp.cap4 + min_rows - 1) / min_rows));
     int launches = 0;
     if (gq == 1) {
         // one query per head: the FP16 kernel with a single column; INT8 and INT4 with a softmax row per lane
         k_attend_fp16_gqa<<<dim3(p.heads, nch, p.L), AT_D, 0, st>>>(qh, pp, fl, p.heads, 1, 0, 1, min_rows16, c->attend_ws);
-        k_attend_int8<<<dim3(p.heads, AT_CH8, p.L), AT_D, 0, st>>>(qh, pp, fl, p.heads, 1, ng, min_rows, c->attend_ws);
-        dim3 grid(p.heads, AT_CHUNKS, p.L);
+        k_attend_int8<<<dim3(p.heads, nch8, p.L), AT_D, 0, st>>>(qh, pp, fl, p.heads, 1, ng, min_rows, c->attend_ws);
+        dim3 grid(p.heads, nch4, p.L);
         if (p.heads == 32 && ng == 32) k_attend_int4<32 * AT_D / 2, 32><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, 1, ng, min_rows, c->attend_ws);
         else if (p.heads == 32 && ng == 1) k_attend_int4<32 * AT_D / 2, 1><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, 1, ng, min_rows, c->attend_ws);
         else k_attend_int4<0, 0><<<grid, AT_D, 0, st>>>(qh, pp, fl, p.heads, 1, ng, min_rows, c->attend_ws);
@@ -1297,13 +1300,13 @@ int sc_attend(salicache_ctx* c, const void* d_q, int q_per_kv, const salicache_p
         for (int q0 = 0; q0 < gq; q0 += GQ_MAX) {
             const int gqn = std::min(GQ_MAX, gq - q0);
             k_attend_fp16_gqa<<<dim3(p.heads, nch, p.L), AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, q0, gqn, min_rows16, c->attend_ws);
-            k_attend_int8_gqa<<<dim3(p.heads, AT_CH8, p.L), AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, q0, gqn, ng, min_rows, c->attend_ws);
-            k_attend_int4_gqa<<<dim3(p.heads, AT_CHUNKS, p.L), AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, q0, gqn, ng, min_rows, c->attend_ws);
+            k_attend_int8_gqa<<<dim3(p.heads, nch8, p.L), AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, q0, gqn, ng, min_rows, c->attend_ws);
+            k_attend_int4_gqa<<<dim3(p.heads, nch4, p.L), AT_D, 0, st>>>(qh, pp, fl, p.heads, gq, q0, gqn, ng, min_rows, c->attend_ws);
             launches += 3;
         }
     }
     dim3 gm(Hq, p.L);
-    k_attend_merge<<<gm, AT_D, 0, st>>>(c->attend_ws, Hq, nch, d_out);
+    k_attend_merge<<<gm, AT_D, 0, st>>>(c->attend_ws, Hq, nch, nch8, nch4, d_out);
     c->launches += launches + 1;
     SC_CHECK(cudaGetLastError());
     return SALICACHE_OK;
