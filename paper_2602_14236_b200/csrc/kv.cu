@@ -366,9 +366,12 @@ k_unpack(__half* __restrict__ K, __half* __restrict__ V, KvGeom g, const int32_t
                 uint32_t o[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    int qa = (int)(int8_t)((w[k >> 1] >> (16 * (k & 1))) & 255);
-                    int qb = (int)(int8_t)((w[k >> 1] >> (16 * (k & 1) + 8)) & 255);
-                    o[k] = as_u32(__floats2half2_rn(__fmul_rn((float)qa, s), __fmul_rn((float)qb, s)));
+                    // code -> float without the conversion unit: the sign-flipped byte under the exponent of 2^23 is
+                    // 8388608 + code + 128 exactly; one subtraction gives the code
+                    const uint32_t u = w[k >> 1] ^ 0x80808080u;
+                    const float qa = __uint_as_float(__byte_perm(u, 0x4b000000u, (k & 1) ? 0x7652 : 0x7650)) - 8388736.0f;
+                    const float qb = __uint_as_float(__byte_perm(u, 0x4b000000u, (k & 1) ? 0x7653 : 0x7651)) - 8388736.0f;
+                    o[k] = as_u32(__floats2half2_rn(__fmul_rn(qa, s), __fmul_rn(qb, s)));
                 }
                 st_stream(dst + i * 32, make_uint4(o[0], o[1], o[2], o[3]));
             }
@@ -389,7 +392,9 @@ k_unpack(__half* __restrict__ K, __half* __restrict__ V, KvGeom g, const int32_t
                 uint32_t o[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    float qa = (float)((c[i] >> (8 * k)) & 15), qb = (float)((c[i] >> (8 * k + 4)) & 15);
+                    // code -> float without the conversion unit: the nibble under the exponent of 2^23 is 8388608 + code
+                    const float qa = __uint_as_float(((c[i] >> (8 * k)) & 15u) | 0x4b000000u) - 8388608.0f;
+                    const float qb = __uint_as_float(((c[i] >> (8 * k + 4)) & 15u) | 0x4b000000u) - 8388608.0f;
                     o[k] = as_u32(__floats2half2_rn(__fadd_rn(__fmul_rn(qa, s), z), __fadd_rn(__fmul_rn(qb, s), z)));
                 }
                 st_stream(dst + i * 32, make_uint4(o[0], o[1], o[2], o[3]));
