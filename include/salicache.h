@@ -301,6 +301,20 @@ SALICACHE_API int salicache_select_anchored(salicache_ctx* ctx, const uint8_t* d
                                             int64_t* d_row_offset, int64_t* d_fill, void* cuda_stream);
 
 /*
+ * salicache_select_anchored for n_videos independent videos of B frames each in one launch (one cluster of CTAs per
+ * video, so that a GPU works on many streams at once; a single video occupies 8 of its SMs).  Every array has a
+ * leading video dimension: d_frames [n_videos][B][H][W][3], d_s and d_deltaP [n_videos][B][N_tok], d_anchor
+ * [n_videos][H][W][3], d_decision [n_videos][B][N_tok], d_idx [n_videos][B][3][N_tok], d_counts [n_videos][B][5],
+ * d_frame_redundant [n_videos][B], d_row_offset [n_videos][B][3], d_fill [n_videos][3] (each video fills pools of its
+ * own); first_has_no_prev applies to every video.  n_videos < 0 or > 4096: E_SHAPE; otherwise as salicache_select_anchored.
+ */
+SALICACHE_API int salicache_select_anchored_batch(salicache_ctx* ctx, const uint8_t* d_frames, const float* d_s, int n_videos,
+                                                  int B, int first_has_no_prev, uint8_t* d_anchor, float* d_deltaP,
+                                                  uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts,
+                                                  uint8_t* d_frame_redundant, int64_t* d_row_offset, int64_t* d_fill,
+                                                  void* cuda_stream);
+
+/*
  * Decode attention straight from the mixed-precision store (Eq. 2 with the just-in-time dequantisation of
  * Sec. III-C fused in): for every layer l and head h,
  *   score_j = q[l][h] . K^_j / sqrt(head_dim),  p = softmax_j(score),  out[l][h] = sum_j p_j V^_j,

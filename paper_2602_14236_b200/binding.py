@@ -50,7 +50,7 @@ EXPORTS = [
     "salicache_tokens_per_frame", "salicache_launch_count", "salicache_flow_score", "salicache_saliency", "salicache_select",
     "salicache_pack_kv", "salicache_unpack_kv", "salicache_poll_status", "salicache_saliency_noalloc",
     "salicache_frame_redundancy", "salicache_source_frames", "salicache_diff_score", "salicache_attend",
-    "salicache_select_anchored", "salicache_select_ranked", "salicache_attend_gqa",
+    "salicache_select_anchored", "salicache_select_ranked", "salicache_attend_gqa", "salicache_select_anchored_batch",
 ]
 
 _lib = None
@@ -83,6 +83,7 @@ def lib():
         _lib.salicache_source_frames.argtypes = [vp, vp, i32, i32, vp, vp, vp]
         _lib.salicache_select.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         _lib.salicache_select_ranked.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        _lib.salicache_select_anchored_batch.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         _lib.salicache_select_anchored.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         _lib.salicache_pack_kv.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, C.POINTER(Pools), vp]
         _lib.salicache_unpack_kv.argtypes = [vp, C.POINTER(Pools), vp, vp, vp, vp, i32, i32, vp, vp, i64, vp]
@@ -204,6 +205,14 @@ def salicache_select_anchored(ctx: Context, d_frames, d_s, B: int, first_has_no_
                                            _ptr(d_deltaP), _ptr(d_decision), _ptr(d_idx), _ptr(d_counts),
                                            _ptr(d_frame_redundant), _ptr(d_row_offset), _ptr(d_fill), _stream(stream)),
            "salicache_select_anchored")
+
+
+def salicache_select_anchored_batch(ctx: Context, d_frames, d_s, n_videos: int, B: int, first_has_no_prev: bool, d_anchor, d_deltaP,
+                                    d_decision, d_idx, d_counts, d_frame_redundant, d_row_offset, d_fill, stream=None):
+    _check(lib().salicache_select_anchored_batch(ctx.handle, _ptr(d_frames), _ptr(d_s), n_videos, B, int(first_has_no_prev),
+                                                 _ptr(d_anchor), _ptr(d_deltaP), _ptr(d_decision), _ptr(d_idx), _ptr(d_counts),
+                                                 _ptr(d_frame_redundant), _ptr(d_row_offset), _ptr(d_fill), _stream(stream)),
+           "salicache_select_anchored_batch")
 
 
 def salicache_pack_kv(ctx: Context, d_K, d_V, frame_stride: int, d_idx, d_counts, d_row_offset, B: int, pools: Pools,

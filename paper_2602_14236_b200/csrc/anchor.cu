@@ -12,7 +12,8 @@
 // tokens are contiguous in token order); what a step has to share, the number of static patches (Eq. 6) and
 // the per-tier counts that place each CTA's tokens in the index lists, crosses the cluster through distributed
 // shared memory, one cluster barrier per frame.  A CTA reads and writes only its own bands of the anchor image,
-// so the image needs no synchronisation beyond the CTA's own barrier.
+// so the image needs no synchronisation beyond the CTA's own barrier.  Several videos are several clusters of one
+// launch; they share nothing.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -60,6 +61,20 @@ k_select_anchored(AnchorArgs a) {
     __shared__ int s_warp[3][AN_WARPS];
     const int rank = (int)cluster.block_rank(), tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int n_tok = a.gh * a.gw;
+    {   // one cluster per video: every array has a leading video dimension
+        const size_t vid = blockIdx.x / AN_CLUSTER, vb = vid * (size_t)a.B;
+        const size_t frame = (size_t)a.H * a.W * 3;
+        a.frames += vb * frame;
+        a.s += vb * n_tok;
+        a.anchor += vid * frame;
+        a.dP += vb * n_tok;
+        a.decision += vb * n_tok;
+        a.idx += vb * 3 * n_tok;
+        a.counts += vb * 5;
+        a.redundant += vb;
+        a.row_offset += vb * 3;
+        a.fill += vid * 3;
+    }
     const int nb = (a.gh + AN_CLUSTER - 1) / AN_CLUSTER;                // bands per CTA
     const int band0 = min(a.gh, rank * nb), band1 = min(a.gh, band0 + nb);
     const int tok0 = band0 * a.gw, n_own = (band1 - band0) * a.gw;
@@ -221,16 +236,16 @@ k_select_anchored(AnchorArgs a) {
 
 }  // namespace
 
-int sc_select_anchored(salicache_ctx* c, const uint8_t* d_frames, const float* d_s, int B, int first_has_no_prev,
+int sc_select_anchored(salicache_ctx* c, const uint8_t* d_frames, const float* d_s, int n_videos, int B, int first_has_no_prev,
                        uint8_t* d_anchor, float* d_deltaP, uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts,
                        uint8_t* d_frame_redundant, int64_t* d_row_offset, int64_t* d_fill, cudaStream_t st) {
     const salicache_params& p = c->p;
     const PlaneGeom& g = c->plane[0];
     if (c->n_planes != 1 || g.layout != 0 || p.patch != 14 || g.gh > 48 || g.gw > 48) return SALICACHE_E_PARAM;
-    if (B == 0) return SALICACHE_OK;
+    if (B == 0 || n_videos == 0) return SALICACHE_OK;
     AnchorArgs a{d_frames, d_s, d_anchor, d_deltaP, d_decision, d_idx, d_counts, d_frame_redundant, d_row_offset, d_fill,
                  B, g.H, g.W, g.gh, g.gw, first_has_no_prev, p.patch_reuse, p.tau_t, p.theta_R, p.tau_high, p.tau_med, p.tau_low};
-    k_select_anchored<<<AN_CLUSTER, AN_THREADS, 0, st>>>(a);
+    k_select_anchored<<<AN_CLUSTER * n_videos, AN_THREADS, 0, st>>>(a);
     c->launches++;
     SC_CHECK(cudaGetLastError());
     return SALICACHE_OK;

@@ -283,7 +283,20 @@ int salicache_select_anchored(salicache_ctx* c, const uint8_t* d_frames, const f
         return SALICACHE_E_NULL;
     if (B < 0 || B > c->p.max_batch) return SALICACHE_E_SHAPE;
     if (!aligned16(d_frames) || !aligned16(d_anchor)) return SALICACHE_E_ALIGN;
-    return sc_select_anchored(c, d_frames, d_s, B, first_has_no_prev, d_anchor, d_deltaP, d_decision, d_idx, d_counts,
+    return sc_select_anchored(c, d_frames, d_s, 1, B, first_has_no_prev, d_anchor, d_deltaP, d_decision, d_idx, d_counts,
+                              d_frame_redundant, d_row_offset, d_fill, (cudaStream_t)cuda_stream);
+}
+
+int salicache_select_anchored_batch(salicache_ctx* c, const uint8_t* d_frames, const float* d_s, int n_videos, int B,
+                                    int first_has_no_prev, uint8_t* d_anchor, float* d_deltaP, uint8_t* d_decision,
+                                    int32_t* d_idx, int32_t* d_counts, uint8_t* d_frame_redundant, int64_t* d_row_offset,
+                                    int64_t* d_fill, void* cuda_stream) {
+    if (!c || !d_frames || !d_s || !d_anchor || !d_deltaP || !d_decision || !d_idx || !d_counts || !d_frame_redundant ||
+        !d_row_offset || !d_fill)
+        return SALICACHE_E_NULL;
+    if (B < 0 || B > c->p.max_batch || n_videos < 0 || n_videos > 4096) return SALICACHE_E_SHAPE;
+    if (!aligned16(d_frames) || !aligned16(d_anchor)) return SALICACHE_E_ALIGN;
+    return sc_select_anchored(c, d_frames, d_s, n_videos, B, first_has_no_prev, d_anchor, d_deltaP, d_decision, d_idx, d_counts,
                               d_frame_redundant, d_row_offset, d_fill, (cudaStream_t)cuda_stream);
 }
 

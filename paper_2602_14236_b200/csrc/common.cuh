@@ -76,7 +76,7 @@ int sc_select_ranked(salicache_ctx* c, const float* d_deltaP, const float* d_s, 
                      int pm8, int pm4, uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts, uint8_t* d_frame_redundant,
                      int64_t* d_row_offset, int64_t* d_fill, cudaStream_t st);
 // anchor.cu
-int sc_select_anchored(salicache_ctx* c, const uint8_t* d_frames, const float* d_s, int B, int first_has_no_prev,
+int sc_select_anchored(salicache_ctx* c, const uint8_t* d_frames, const float* d_s, int n_videos, int B, int first_has_no_prev,
                        uint8_t* d_anchor, float* d_deltaP, uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts,
                        uint8_t* d_frame_redundant, int64_t* d_row_offset, int64_t* d_fill, cudaStream_t st);
 // attend.cu

@@ -131,3 +131,38 @@ def test_anchored_mode_argument_checks():
     wl = synth.WORKLOADS[4]
     anyres = sc.Context(sc.salicache_default_params(H=wl.H, W=wl.W, n_images=wl.n_images, max_batch=4, chunk_frames=2, L=1))
     assert lib.salicache_select_anchored(*args(anyres, anchor.data_ptr(), 1)) == sc.E_PARAM
+
+
+def test_several_videos_in_one_launch_match_one_video_at_a_time():
+    """Five videos of different content, one cluster each, against the oracle video by video; the videos keep their own
+    anchor images and fills."""
+    import torch
+    H = W = 336
+    V, T = 5, 9
+    rng = np.random.default_rng(77)
+    frames = np.stack([_video(rng, T, H, W, p_move=0.2 + 0.15 * v) for v in range(V)])
+    kw = dict(synth.thresholds("four"), tau_t=2.5, theta_R=0.8)
+    ctx = sc.Context(sc.salicache_default_params(max_batch=16, chunk_frames=2, L=1, **kw))
+    n = ctx.n_tok
+    s = rng.uniform(0.15, 0.6, (V, T, n)).astype(np.float32)
+    p = gu.oracle_params(ctx.params)
+    fill0 = np.arange(3 * V, dtype=np.int64).reshape(V, 3)
+    d = dict(
+        dP=torch.full((V, T, n), -1.0, dtype=torch.float32, device="cuda"),
+        decision=torch.full((V, T, n), 255, dtype=torch.uint8, device="cuda"),
+        idx=torch.full((V, T, 3, n), -7, dtype=torch.int32, device="cuda"),
+        counts=torch.full((V, T, 5), -1, dtype=torch.int32, device="cuda"),
+        redundant=torch.full((V, T), 255, dtype=torch.uint8, device="cuda"),
+        row_offset=torch.full((V, T, 3), -1, dtype=torch.int64, device="cuda"),
+        fill=torch.from_numpy(fill0.copy()).cuda(),
+    )
+    anchors = torch.zeros((V, H, W, 3), dtype=torch.uint8, device="cuda")
+    sc.salicache_select_anchored_batch(ctx, torch.from_numpy(frames).cuda(), torch.from_numpy(s).cuda(), V, T, True, anchors, d["dP"],
+                                       d["decision"], d["idx"], d["counts"], d["redundant"], d["row_offset"], d["fill"])
+    torch.cuda.synchronize()
+    got = {k: v.cpu().numpy() for k, v in d.items()}
+    for v in range(V):
+        a = np.zeros((H, W, 3), np.uint8)
+        ref = oracle.select_anchored(frames[v], s[v], True, a, p)
+        _compare({k: x[v] for k, x in got.items()}, ref, fill0=tuple(fill0[v]))
+        assert np.array_equal(anchors[v].cpu().numpy(), a)
