@@ -474,6 +474,27 @@ def run_extras(sc, synth, ctx, wl, T, frames, dP, dev, peak, pools, fill, stored
             "l2": "flushed between repetitions",
             "reused_tokens_percent": {"anchor_mode": round(100 * reuse_anchor, 2),
                                       "consecutive_frames_same_threshold": round(100 * reuse_consecutive, 2)}}
+        # eighteen such videos at once: one cluster of 8 CTAs each, 144 of the 148 SMs
+        NV = 18
+        fr_v = frames.unsqueeze(0).expand(NV, *frames.shape).contiguous()
+        s_v = s_a.unsqueeze(0).expand(NV, T, n).contiguous()
+        anchor_v = torch.zeros((NV, wl.H, wl.W, 3), dtype=torch.uint8, device=dev)
+        dP_v = torch.zeros((NV, T, n), dtype=torch.float32, device=dev)
+        dec_v = torch.zeros((NV, T, n), dtype=torch.uint8, device=dev)
+        idx_v = torch.zeros((NV, T, 3, n), dtype=torch.int32, device=dev)
+        cnt_v = torch.zeros((NV, T, 5), dtype=torch.int32, device=dev)
+        red_v = torch.zeros((NV, T), dtype=torch.uint8, device=dev)
+        off_v = torch.zeros((NV, T, 3), dtype=torch.int64, device=dev)
+        fill_v = torch.zeros((NV, 3), dtype=torch.int64, device=dev)
+
+        def anchored_batch():
+            fill_v.zero_()
+            sc.salicache_select_anchored_batch(ca, fr_v, s_v, NV, T, True, anchor_v, dP_v, dec_v, idx_v, cnt_v, red_v, off_v, fill_v)
+
+        ms_v = timed(anchored_batch, reps=3)
+        out["select_anchored"]["batch"] = {"videos": NV, "ms": round(ms_v, 3), "frames_per_s": round(NV * T / ms_v * 1e3, 1),
+                                           "algorithmic_GBps": round(NV * T * 2 * wl.H * wl.W * 3 / ms_v / 1e6, 1)}
+        del fr_v, s_v, anchor_v, dP_v, dec_v, idx_v
         ca.close()
     # Fig. 3 style breakdown: workload 2 frames under the four-tier rule
     wl2 = synth.WORKLOADS[2]
