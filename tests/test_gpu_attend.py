@@ -128,13 +128,14 @@ def test_attention_int4_rows_peaked_and_large_values():
         _check(ctx, pools, ref, fill, (3.0 * k_row).astype(np.float16), scale=v_scale)
 
 
-@pytest.mark.parametrize("heads,q_per_kv,background", [(8, 4, "four"), (8, 4, "int4"), (32, 2, "int8"), (8, 3, "int8"), (8, 8, "four")])
-def test_grouped_query_attention_matches_the_oracle(heads, q_per_kv, background):
+@pytest.mark.parametrize("heads,q_per_kv,background,group", [(8, 4, "four", 128), (8, 4, "int4", 128), (32, 2, "int8", 128),
+                                                             (8, 3, "int8", 128), (8, 8, "four", 128), (8, 4, "four", 1024)])
+def test_grouped_query_attention_matches_the_oracle(heads, q_per_kv, background, group):
     """The paper's evaluation model has 8 key/value heads for 32 query heads: query head hq reads key/value head
     hq // q_per_kv.  Also 32 key/value heads with two queries each (64 query heads, the most the workspace holds), a group
-    of three, and a group of eight (two passes of four)."""
+    of three, a group of eight (two passes of four), and whole-row quantisation groups."""
     import torch
-    ctx, pools, ref, fill, rng = _store(L=2, heads=heads, T=2, background=background, seed=21)
+    ctx, pools, ref, fill, rng = _store(L=2, heads=heads, T=2, background=background, group=group, seed=21)
     q = rng.standard_normal((2, heads * q_per_kv, 128)).astype(np.float16)
     d_out = torch.full((2, heads * q_per_kv, 128), 7.0, dtype=torch.float32, device="cuda")
     sc.salicache_attend_gqa(ctx, torch.from_numpy(q).cuda(), q_per_kv, pools.c, fill, d_out)
