@@ -1,7 +1,7 @@
 """CPU oracle of the Sali-Cache pre-attention filter and K/V store (test infrastructure).
 
 Thin ctypes binding over ``salicache_oracle.c``: argument marshalling only, all of
-the arithmetic is in the C file.  Only tests, the smoke check and the benchmark's
+the arithmetic (the accounting of Eq. 3 included) is in the C file.  Only tests, the smoke check and the benchmark's
 CPU-baseline leg may import this package; the CUDA library never does.
 """
 from __future__ import annotations
@@ -403,14 +403,34 @@ def stored_bytes(counts_all: np.ndarray, L: int, HD: int, G: int, n_tok: int) ->
     """Bytes the mixed-precision store holds for frames with the given per-code counts [T][5]
     (Eq. 3 applied per tier, plus all metadata: scales/zeros, index lists, decision bytes,
     an 8-byte pointer-table entry and three 8-byte row offsets per frame)."""
-    counts_all = np.asarray(counts_all, np.int64).reshape(-1, 5)
-    ng = HD // G
-    n4, n8, n16 = counts_all[:, 2].sum(), counts_all[:, 3].sum(), counts_all[:, 4].sum()
-    payload = L * 2 * (n16 * HD * 2 + n8 * (HD + 2 * ng) + n4 * (HD // 2 + 4 * ng))
-    meta = counts_all.shape[0] * (n_tok + 8 + 24 + 20) + 4 * (n4 + n8 + n16)
-    return int(payload + meta)
+    c = _c(np.asarray(counts_all).reshape(-1, 5), np.int64)
+    f = lib().oracle_stored_bytes
+    f.restype = C.c_int64
+    return int(f(_p(c), C.c_int64(c.shape[0]), C.c_int(L), C.c_int(HD), C.c_int(G), C.c_int(n_tok)))
 
 
 def raw_bytes(T: int, L: int, HD: int, n_tok: int) -> int:
     """Eq. 3 for T frames of n_tok tokens, fp16, K and V."""
-    return 2 * L * T * n_tok * HD * 2
+    f = lib().oracle_raw_bytes
+    f.restype = C.c_int64
+    return int(f(C.c_int64(T), C.c_int(L), C.c_int(HD), C.c_int(n_tok)))
+
+
+def anyres_tokens(full: np.ndarray, base: np.ndarray, tg: int = 24) -> np.ndarray:
+    """Per-patch values of the whole frame ((2 tg)^2, row-major) and of the base image (tg^2) in token order:
+    base, tile (0,0), (0,1), (1,0), (1,1), each row-major."""
+    full, base = _c(full, np.float64).ravel(), _c(base, np.float64).ravel()
+    assert full.size == 4 * tg * tg and base.size == tg * tg
+    out = np.empty(5 * tg * tg, np.float64)
+    lib().oracle_anyres_tokens(_p(full), _p(base), C.c_int(tg), _p(out))
+    return out
+
+
+def row_offsets(counts_all: np.ndarray, fill=None):
+    """First pool row of every frame per tier (FP16, INT8, INT4) for per-code counts [T][5], continuing from
+    the running fill [3].  Returns (off int64 [T][3], fill after the last frame int64 [3])."""
+    c = _c(np.asarray(counts_all).reshape(-1, 5), np.int32)
+    fill = np.zeros(3, np.int64) if fill is None else _c(fill, np.int64).copy()
+    off = np.empty((c.shape[0], 3), np.int64)
+    lib().oracle_row_offsets(_p(c), C.c_int(c.shape[0]), _p(fill), _p(off))
+    return off, fill

@@ -972,3 +972,59 @@ EXPORT void oracle_attend_gqa(const uint16_t* q, int L, int H, int q_per_kv, int
             free(sc);
         }
 }
+
+/* ------------------------------------------------------------------------- */
+/* Token order of a dynamic-resolution frame (Sec. II-A mentions the encoding  */
+/* only; reading): a frame of 2x2 tiles of tg x tg patches plus one base image */
+/* of tg x tg patches has (1 + 4) tg^2 tokens: the base image first, then tile */
+/* (0,0), (0,1), (1,0), (1,1), each row-major.  full = per-patch values on the */
+/* (2 tg) x (2 tg) grid of the whole frame (row-major), base = on the base     */
+/* image's grid.                                                               */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_anyres_tokens(const double* full, const double* base, int tg, double* out) {
+    int k = 0;
+    for (int i = 0; i < tg * tg; ++i) out[k++] = base[i];
+    for (int r = 0; r < 2; ++r)
+        for (int c = 0; c < 2; ++c)
+            for (int y = 0; y < tg; ++y)
+                for (int x = 0; x < tg; ++x) out[k++] = full[(size_t)(r * tg + y) * (2 * tg) + (c * tg + x)];
+}
+
+/* ------------------------------------------------------------------------- */
+/* Pool rows of a run of frames (the store step of Alg. 1, line 16): frame t's */
+/* rows of a tier follow those of the frames before it, so its first row is    */
+/* the running fill of that tier; the fill then grows by the frame's count.    */
+/* counts [T][5] by code; off [T][3] and fill [3] in the order FP16, INT8,     */
+/* INT4.  Offsets are absolute: a ring pool takes them modulo its capacity.    */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_row_offsets(const int32_t* counts, int T, int64_t* fill, int64_t* off) {
+    const int code[3] = {4, 3, 2};
+    for (int t = 0; t < T; ++t)
+        for (int k = 0; k < 3; ++k) {
+            off[(size_t)t * 3 + k] = fill[k];
+            fill[k] += counts[(size_t)t * 5 + code[k]];
+        }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Memory accounting (Eq. 3: M = 2 n_l L d sizeof(dtype), applied per tier).   */
+/* raw: T frames of n_tok tokens, K and V, L layers, HD = heads x head_dim     */
+/* fp16 elements per token.  stored: the pools' payload for the per-code       */
+/* counts [T][5] (FP16 rows 2 HD bytes, INT8 rows HD + 2 HD/G, INT4 rows       */
+/* HD/2 + 4 HD/G per layer and tensor) plus the metadata kept per frame (one   */
+/* decision byte per token, an 8-byte pointer-table entry, three 8-byte row    */
+/* offsets, five 4-byte counts) and a 4-byte index-list entry per stored token.*/
+/* ------------------------------------------------------------------------- */
+EXPORT int64_t oracle_raw_bytes(int64_t T, int L, int HD, int n_tok) { return 2 * (int64_t)L * T * n_tok * HD * 2; }
+
+EXPORT int64_t oracle_stored_bytes(const int64_t* counts, int64_t T, int L, int HD, int G, int n_tok) {
+    int64_t n4 = 0, n8 = 0, n16 = 0, ng = HD / G;
+    for (int64_t t = 0; t < T; ++t) {
+        n4 += counts[t * 5 + 2];
+        n8 += counts[t * 5 + 3];
+        n16 += counts[t * 5 + 4];
+    }
+    int64_t payload = (int64_t)L * 2 * (n16 * HD * 2 + n8 * (HD + 2 * ng) + n4 * (HD / 2 + 4 * ng));
+    int64_t meta = T * ((int64_t)n_tok + 8 + 24 + 20) + 4 * (n4 + n8 + n16);
+    return payload + meta;
+}

@@ -61,7 +61,7 @@ def lib():
     global _lib
     if _lib is None:
         path = _build.LIB
-        if os.path.exists(os.path.join(_build.CSRC, "api.cu")) and os.path.exists("/usr/local/cuda/bin/nvcc"):
+        if os.path.exists(os.path.join(_build.CSRC, "api.cu")) and _build.nvcc_path() is not None:
             path = _build.build()
         if not os.path.exists(path):
             raise ImportError(f"{path} is missing: build it with `python -m paper_2602_14236_b200.build`; "

@@ -22,10 +22,21 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
+def nvcc_path():
+    """The compiler to use: $NVCC, else nvcc on PATH, else the default CUDA location; None when there is none."""
+    import shutil
+    for cand in (os.environ.get("NVCC"), shutil.which("nvcc"), "/usr/local/cuda/bin/nvcc"):
+        if cand and os.path.exists(cand):
+            return cand
+    return None
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
-    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    nvcc = nvcc_path()
+    if nvcc is None:
+        raise RuntimeError("nvcc not found (set $NVCC)")
     objs = []
     bdir = os.path.join(_PKG, "_build")
     os.makedirs(bdir, exist_ok=True)

@@ -139,7 +139,8 @@ int salicache_create(salicache_ctx** out, const salicache_params* p) {
     }
     int st = SALICACHE_OK;
     if (cudaMemcpy(c->lut, lut, sizeof(lut), cudaMemcpyHostToDevice) != cudaSuccess ||
-        cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess)
+        cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess ||
+        cudaDeviceSynchronize() != cudaSuccess)      // the table and the zeroed scratch are in place before any stream uses them
         st = SALICACHE_E_CUDA;
     if (st == SALICACHE_OK) st = sc_flow_init();
     if (st == SALICACHE_OK) st = sc_saliency_init(p->H, words);

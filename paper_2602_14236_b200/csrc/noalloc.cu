@@ -51,6 +51,9 @@ int setup_device(int dev, unsigned char** base) {
         lut[i] = v <= 0.04045 ? v / 12.92 : pow((v + 0.055) / 1.055, 2.4);
     }
     if (cudaMemcpy(ptr + NA_LUT_OFF, lut, sizeof(lut), cudaMemcpyHostToDevice) != cudaSuccess) return SALICACHE_E_CUDA;
+    // a copy from pageable memory may return before the table has landed, and only the legacy default stream is
+    // ordered behind it: wait here, so that the caller's stream (any stream) sees the table
+    if (cudaDeviceSynchronize() != cudaSuccess) return SALICACHE_E_CUDA;
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SALICACHE_E_CUDA;
     g_sm_count[dev] = sms;

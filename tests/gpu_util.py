@@ -78,9 +78,7 @@ def oracle_select_all(dP: np.ndarray, s: np.ndarray, p: oracle.Params, first_has
     for t in range(T):
         has_prev = dP is not None and not (first_has_no_prev and t == 0)
         dec[t], idx[t], counts[t], red[t], _ = oracle.select(dP[t] if dP is not None else None, s[t], has_prev, p)
-    off = np.zeros((T, 3), np.int64)
-    per = counts[:, [oracle.FP16, oracle.INT8, oracle.INT4]].astype(np.int64)
-    off[1:] = np.cumsum(per, axis=0)[:-1]
+    off, _ = oracle.row_offsets(counts)
     return dec, idx, counts, red, off
 
 

@@ -18,7 +18,7 @@ ATOL, RTOL = 2e-5, 1e-4
 
 
 def _store(L, heads, T, background, group=128, seed=0, s_lo=0.0, v_scale=1.0, keep=None):
-    """Random scores -> decisions -> pools on both sides (the pools are bit-identical, checked elsewhere).
+    """Random scores -> decisions -> pools on both sides, each by its own store; the pools are compared here.
     `keep`, a dict, receives the dense K and the decisions."""
     import torch
     HD, n_tok = heads * 128, 576
@@ -37,13 +37,20 @@ def _store(L, heads, T, background, group=128, seed=0, s_lo=0.0, v_scale=1.0, ke
     sc.salicache_pack_kv(ctx, torch.from_numpy(K).cuda(), torch.from_numpy(V).cuda(), L * n_tok * HD, out["idx"],
                          out["counts"], out["row_offset"], T, pools.c)
     torch.cuda.synchronize()
+    # the oracle's pools are filled by the oracle's own store from the same K/V and decisions; the device's pools
+    # must equal them byte for byte before either side attends
     ref = oracle.Pools(L, HD, group, *caps)
+    h_idx, h_counts, h_off = (out[k].cpu().numpy() for k in ("idx", "counts", "row_offset"))
+    want_off, want_fill = oracle.row_offsets(h_counts)
+    assert np.array_equal(h_off, want_off) and np.array_equal(out["fill"].cpu().numpy(), want_fill)
+    for t in range(T):
+        assert oracle.pack_frame(K[t].view(np.uint16), V[t].view(np.uint16), h_idx[t], h_counts[t], h_off[t], ref) == 0
     g = lambda t: t.cpu().numpy()
-    ref.fp16_pool[:] = g(pools.fp16_pool).view(np.uint16)
-    ref.int8_codes[:] = g(pools.int8_codes)
-    ref.int8_scale[:] = g(pools.int8_scale).view(np.uint16)
-    ref.int4_codes[:] = g(pools.int4_codes)
-    ref.int4_sz[:] = g(pools.int4_sz).view(np.uint16)
+    assert np.array_equal(g(pools.fp16_pool).view(np.uint16), ref.fp16_pool)
+    assert np.array_equal(g(pools.int8_codes), ref.int8_codes)
+    assert np.array_equal(g(pools.int8_scale).view(np.uint16), ref.int8_scale)
+    assert np.array_equal(g(pools.int4_codes), ref.int4_codes)
+    assert np.array_equal(g(pools.int4_sz).view(np.uint16), ref.int4_sz)
     return ctx, pools, ref, out["fill"], rng
 
 

@@ -1,6 +1,6 @@
 """GPU parity on the workloads' own shapes: the anyres layout of workload 4, the streamed segments of
-workload 5 with a ring budget, and workload 3 at the full K/V shape (32 layers) in the launch
-configuration the benchmark times (8-frame store launches)."""
+workload 5 with a ring budget, and workload 3 at the full K/V shape (32 layers): an 8-frame store launch
+checked on every pool byte, and the 40-frame store launch the benchmark times checked on sampled slabs."""
 import numpy as np
 import pytest
 
@@ -14,13 +14,8 @@ pytestmark = pytest.mark.gpu
 
 
 def _anyres_tokens(full48: np.ndarray, base24: np.ndarray) -> np.ndarray:
-    """Token order of the anyres layout: base image, then tiles (0,0) (0,1) (1,0) (1,1), each 24x24 row-major."""
-    g = full48.reshape(48, 48)
-    parts = [base24.reshape(-1)]
-    for r in range(2):
-        for c in range(2):
-            parts.append(g[24 * r:24 * r + 24, 24 * c:24 * c + 24].reshape(-1))
-    return np.concatenate(parts)
+    """Per-patch values of the whole frame and of the base image in the token order of the anyres layout."""
+    return oracle.anyres_tokens(full48, base24)
 
 
 def test_anyres_scores_follow_the_token_layout_and_match_the_oracle():
@@ -120,8 +115,8 @@ def test_ring_budget_frame_by_frame_matches_the_oracle_ring():
     assert np.array_equal(pools.fp16_pool.cpu().numpy().view(np.uint16), ref.fp16_pool)
 
 
-def test_workload_3_full_shape_in_the_benchmark_launch_configuration():
-    """32 layers x 32 heads x 128, eight frames per store launch, around the pan -> hold transition."""
+def test_workload_3_full_shape_every_pool_byte():
+    """32 layers x 32 heads x 128, one store launch of eight frames around the pan -> hold transition."""
     import torch
     wl = synth.WORKLOADS[3]
     T, L, n_tok, HD = 8, wl.L, wl.n_tok, wl.HD
@@ -175,6 +170,61 @@ def test_workload_3_full_shape_in_the_benchmark_launch_configuration():
     assert np.array_equal(pools.int4_codes.cpu().numpy(), ref.int4_codes)
     assert np.array_equal(pools.int4_sz.cpu().numpy().view(np.uint16), ref.int4_sz)
     assert np.array_equal(pools.fp16_pool.cpu().numpy().view(np.uint16), ref.fp16_pool)
+
+def test_workload_3_store_launch_of_40_frames_as_the_benchmark_times_it():
+    """The benchmark stores 40 frames per launch at 32 layers: 40 panning frames of workload 3, every token INT4 or
+    FP16, 40 x 576 x 64 = 1.47 million token rows in one launch.  Decisions and row offsets are compared whole; the
+    pools on sampled (frame, layer) slabs, K and V, against the oracle's store of the same slab."""
+    import torch
+    wl = synth.WORKLOADS[3]
+    T, L, n_tok, HD = 40, wl.L, wl.n_tok, wl.HD
+    fr = synth.frames(3, T=T + 1, t0=79)                        # pairs (79, 80) .. (118, 119): the 3 px/frame pan
+    ctx = sc.Context(sc.salicache_default_params(max_batch=T, chunk_frames=T, L=L, **synth.thresholds(wl.background)))
+    d_fr = torch.from_numpy(fr).cuda()
+    dP = torch.zeros((T, n_tok), dtype=torch.float32, device="cuda")
+    s = torch.zeros((T, n_tok), dtype=torch.float32, device="cuda")
+    red = torch.zeros((T,), dtype=torch.uint8, device="cuda")
+    dec = torch.zeros((T, n_tok), dtype=torch.uint8, device="cuda")
+    idx = torch.zeros((T, 3, n_tok), dtype=torch.int32, device="cuda")
+    counts = torch.zeros((T, 5), dtype=torch.int32, device="cuda")
+    off = torch.zeros((T, 3), dtype=torch.int64, device="cuda")
+    fill = torch.zeros((3,), dtype=torch.int64, device="cuda")
+    sc.salicache_flow_score(ctx, d_fr[:-1], d_fr[1:], T, dP)
+    sc.salicache_frame_redundancy(ctx, dP, T, False, red)
+    sc.salicache_saliency(ctx, d_fr[1:], T, s, red)
+    sc.salicache_select(ctx, dP, s, T, False, dec, idx, counts, red, off, fill)
+    K = torch.empty((T, L, n_tok, HD), dtype=torch.float16, device="cuda")
+    V = torch.empty_like(K)
+    for t in range(T):
+        k, v = synth.kv_torch(3, t, "cuda")
+        K[t].copy_(k)
+        V[t].copy_(v)
+    del k, v
+    h_counts, h_idx, h_off = counts.cpu().numpy(), idx.cpu().numpy(), off.cpu().numpy()
+    tot = h_counts[:, [4, 3, 2]].sum(axis=0)
+    assert tot.sum() * 2 * L > 1_400_000                        # (nearly) every token of every frame is stored
+    pools = sc.PoolSet(L, HD, int(tot[0]) + 1, 1, int(tot[2]) + 1)
+    sc.salicache_pack_kv(ctx, K, V, L * n_tok * HD, idx, counts, off, T, pools.c)
+    torch.cuda.synchronize()
+    assert sc.salicache_poll_status(ctx) == 0
+    p = gu.oracle_params(ctx.params)
+    h_dP, h_s, h_red = dP.cpu().numpy(), s.cpu().numpy(), red.cpu().numpy()
+    for t in range(T):
+        d, i, c, r, _ = oracle.select(h_dP[t], h_s[t], True, p)
+        assert r == h_red[t] and np.array_equal(c, h_counts[t]) and np.array_equal(i, h_idx[t])
+    want_off, want_fill = oracle.row_offsets(h_counts)
+    assert np.array_equal(h_off, want_off) and np.array_equal(fill.cpu().numpy(), want_fill)
+    for t, l in ((0, 0), (0, 31), (13, 17), (27, 5), (39, 0), (39, 31)):
+        ref = oracle.Pools(1, HD, 128, int(tot[0]) + 1, 1, int(tot[2]) + 1)
+        hK = K[t, l:l + 1].cpu().numpy().view(np.uint16)
+        hV = V[t, l:l + 1].cpu().numpy().view(np.uint16)
+        assert oracle.pack_frame(hK, hV, h_idx[t], h_counts[t], h_off[t], ref) == 0
+        n16, n4 = int(h_counts[t, 4]), int(h_counts[t, 2])
+        r16, r4 = slice(int(h_off[t, 0]), int(h_off[t, 0]) + n16), slice(int(h_off[t, 2]), int(h_off[t, 2]) + n4)
+        assert n4 > 300
+        assert np.array_equal(pools.int4_codes[l, :, r4].cpu().numpy(), ref.int4_codes[0, :, r4]), (t, l)
+        assert np.array_equal(pools.int4_sz[l, :, r4].cpu().numpy().view(np.uint16), ref.int4_sz[0, :, r4]), (t, l)
+        assert np.array_equal(pools.fp16_pool[l, :, r16].cpu().numpy().view(np.uint16), ref.fp16_pool[0, :, r16]), (t, l)
 
 
 def test_literal_eq5_difference_score_matches_the_oracle():

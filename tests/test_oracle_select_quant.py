@@ -240,9 +240,103 @@ def test_pack_layout_and_unpack_roundtrip(ring):
             assert not Ko[:, i].any()
         elif dec[i] == REUSE:
             assert np.all(Ko[:, i] == 0x7E00)
-        elif dec[i] == INT8 or (dec[i] == INT4 and not (ring and i == idx[2, 0])):
-            tol = 0.05 if dec[i] == INT8 else 0.4
-            assert np.max(np.abs(Kof[:, i] - Kf[:, i])) < tol
+    # quantised rows, bit for bit: every group of every row of both tensors is the group dequantiser applied to
+    # the codes and the scale / zero found at the pool row that this test locates itself, (off + j) mod cap
+    for kv, (out, src) in enumerate(((Ko, K), (Vo, V))):
+        for l in range(L):
+            for j in range(counts[INT8]):
+                tok, row = idx[1, j], 1 + j
+                for g in range(HD // G):
+                    want = oracle.dequant_int8_group(pools.int8_codes[l, kv, row, g * G:(g + 1) * G], int(pools.int8_scale[l, kv, row, g]))
+                    assert np.array_equal(out[l, tok, g * G:(g + 1) * G], want)
+            for j in range(counts[INT4]):
+                tok, row = idx[2, j], (j % caps[2]) if ring else j
+                if ring and j + caps[2] < counts[INT4]:
+                    continue                                  # this row was overwritten by a later row of the same frame
+                for g in range(HD // G):
+                    want = oracle.dequant_int4_group(pools.int4_codes[l, kv, row, g * G // 2:(g + 1) * G // 2],
+                                                     int(pools.int4_sz[l, kv, row, g, 0]), int(pools.int4_sz[l, kv, row, g, 1]))
+                    assert np.array_equal(out[l, tok, g * G:(g + 1) * G], want)
+                    x = src[l, tok, g * G:(g + 1) * G].view(np.float16).astype(np.float64)
+                    sc = float(np.array(pools.int4_sz[l, kv, row, g, 0], np.uint16).view(np.float16))
+                    assert np.max(np.abs(want.view(np.float16).astype(np.float64) - x)) <= sc * (0.5 + 2.0 ** -9) + 2.0 ** -10 * np.abs(x).max()
+
+
+def test_unpack_uses_the_scale_of_its_own_group_and_plane():
+    """Groups, layers and tensors with very different ranges: a scale taken from the wrong group, layer or tensor
+    would be off by a factor of 2 or more, far outside the quantiser's error bound."""
+    L, n_tok, HD, G = 3, 16, 512, 128
+    rng = np.random.default_rng(21)
+    K = rng.standard_normal((L, n_tok, HD))
+    V = rng.standard_normal((L, n_tok, HD))
+    for l in range(L):
+        for g in range(HD // G):
+            K[l, :, g * G:(g + 1) * G] *= 2.0 ** (g + 4 * l - 6)
+            V[l, :, g * G:(g + 1) * G] *= 2.0 ** (3 - g - 2 * l)
+    K, V = K.astype(np.float16).view(np.uint16), V.astype(np.float16).view(np.uint16)
+    dec = (np.arange(n_tok) % 3 + 2).astype(np.uint8)             # INT4, INT8, FP16 in turn
+    idx = np.full((3, n_tok), -1, np.int32)
+    counts = np.zeros(5, np.int32)
+    for tier, code in enumerate((FP16, INT8, INT4)):
+        toks = np.nonzero(dec == code)[0]
+        idx[tier, :len(toks)] = toks
+        counts[code] = len(toks)
+    pools = oracle.Pools(L, HD, G, 8, 8, 8)
+    off = np.zeros(3, np.int64)
+    assert oracle.pack_frame(K, V, idx, counts, off, pools) == 0
+    Ko, Vo = np.zeros_like(K), np.zeros_like(V)
+    assert oracle.unpack_frame(n_tok, idx, counts, dec, off, pools, False, Ko, Vo) == 0
+    for out, src in ((Ko, K), (Vo, V)):
+        x = src.view(np.float16).astype(np.float64).reshape(L, n_tok, HD // G, G)
+        y = out.view(np.float16).astype(np.float64).reshape(L, n_tok, HD // G, G)
+        rng_ = x.max(axis=-1) - x.min(axis=-1)
+        amax = np.abs(x).max(axis=-1)
+        err = np.abs(y - x).max(axis=-1)
+        is8, is4 = (dec == INT8)[None, :, None], (dec == INT4)[None, :, None]
+        assert np.all(err[np.broadcast_to(is8, err.shape)] <= (amax / 127 * 0.5 * (1 + 2.0 ** -8) + amax * 2.0 ** -10)[np.broadcast_to(is8, err.shape)])
+        assert np.all(err[np.broadcast_to(is4, err.shape)] <= (rng_ / 15 * 0.5 * (1 + 2.0 ** -8) + amax * 2.0 ** -10)[np.broadcast_to(is4, err.shape)])
+        assert np.array_equal(out[:, dec == FP16], src[:, dec == FP16])
+
+
+def test_anyres_token_order_on_hand_written_grids():
+    """Base image first, then tiles (0,0), (0,1), (1,0), (1,1), each row-major."""
+    assert oracle.anyres_tokens([1, 2, 3, 4], [9], tg=1).tolist() == [9, 1, 2, 3, 4]
+    full = np.arange(16).reshape(4, 4)          # rows 0 1 2 3 / 4 5 6 7 / 8 9 10 11 / 12 13 14 15
+    want = [100, 101, 102, 103, 0, 1, 4, 5, 2, 3, 6, 7, 8, 9, 12, 13, 10, 11, 14, 15]
+    assert oracle.anyres_tokens(full, [100, 101, 102, 103], tg=2).tolist() == want
+    # the frame of workload 4: token 576 is the top-left patch of the frame, 576 + 24 starts its second patch row,
+    # 2 * 576 is patch (0, 24), 3 * 576 is patch (24, 0), the last token is patch (47, 47)
+    full = np.arange(48 * 48)
+    t = oracle.anyres_tokens(full, -np.arange(576) - 1)
+    assert t[0] == -1 and t[575] == -576
+    assert (t[576], t[576 + 24], t[2 * 576], t[3 * 576], t[-1]) == (0, 48, 24, 24 * 48, 48 * 48 - 1)
+    assert sorted(t[576:].tolist()) == list(range(48 * 48))
+
+
+def test_row_offsets_are_the_exclusive_scan_of_the_tier_counts():
+    rng = np.random.default_rng(4)
+    counts = rng.integers(0, 50, (9, 5)).astype(np.int32)
+    fill0 = np.array([7, 0, 123456789012], np.int64)
+    off, fill = oracle.row_offsets(counts, fill0)
+    for k, code in enumerate((FP16, INT8, INT4)):
+        acc = int(fill0[k])
+        for t in range(9):                      # brute force: every frame starts where the earlier ones end
+            assert off[t, k] == acc
+            acc += int(counts[t, code])
+        assert fill[k] == acc
+    # stored with these offsets, the frames' rows tile the pool without gap or overlap
+    L, n_tok, HD, G = 1, 24, 256, 128
+    frames = [_frame_case(L, n_tok, HD, G, seed=s) for s in (1, 2, 3)]
+    cs = np.stack([f[4] for f in frames])
+    off, fill = oracle.row_offsets(cs)
+    pools = oracle.Pools(L, HD, G, *[int(x) for x in fill])
+    pools.int8_scale[:] = 0xFFFF
+    pools.int4_sz[:] = 0xFFFF
+    for (K, V, dec, idx, counts), o in zip(frames, off):
+        assert oracle.pack_frame(K, V, idx, counts, o, pools) == 0
+    assert not (pools.int8_scale == 0xFFFF).any() and not (pools.int4_sz == 0xFFFF).any()      # every row written
+    K2 = frames[2][0]
+    assert np.array_equal(pools.fp16_pool[0, 0, off[2, 0]], K2[0, frames[2][3][0, 0]])
 
 
 def test_pack_without_ring_reports_overflow_and_drops_the_rows():

@@ -4,7 +4,8 @@ The allocation-free entry point serves hosts that cannot call cudaMalloc while t
 pool owns the GPU, or they sit under an allocator lock), so it keeps its scratch in a fixed array
 inside the library that every call on the device shares and that remembers the previous call.  The
 test therefore makes two calls in a row on different inputs and checks each against the
-context-based entry point: leftovers of the first call must not leak into the second.  This file
+context-based entry point and against the CPU oracle: leftovers of the first call must not leak
+into the second.  This file
 sorts after the other test files on purpose, so a run that stops at the first failure has already
 finished them."""
 import ctypes
@@ -12,6 +13,7 @@ import ctypes
 import numpy as np
 import pytest
 
+import oracle
 from paper_2602_14236_b200 import binding as sc
 from paper_2602_14236_b200 import synth
 
@@ -34,15 +36,21 @@ def test_two_calls_in_a_row_match_the_context_entry_point():
     busy = torch.from_numpy(synth.frames(2, T=sc.NOALLOC_MAX_FRAMES)).cuda()        # sprites: many edges
     calm = torch.from_numpy(synth.frames(3, T=3, t0=200)).cuda()                      # fewer frames, other content
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    side = torch.cuda.Stream()            # not the default stream: the one-time set-up must be visible to any stream
+    torch.cuda.synchronize()
     for frames in (busy, calm):
         B = frames.shape[0]
         s = torch.full((B, 576), -1.0, dtype=torch.float32, device="cuda")
-        sc.salicache_saliency_noalloc(params, frames, B, s, status)
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            sc.salicache_saliency_noalloc(params, frames, B, s, status)
         torch.cuda.synchronize()
         got = s.cpu().numpy()
         ref = _reference(params, frames)
         assert np.all(np.abs(got - ref) <= 1e-6 + 1e-4 * np.abs(ref))      # the tolerance of the score tests
         assert np.array_equal(got, ref)                                     # same kernels: same bits
+        want = oracle.saliency(frames.cpu().numpy())                        # and both are the oracle's score
+        assert np.all(np.abs(got - want) <= 1e-6 + 1e-4 * np.abs(want))
     assert int(status.item()) == 0
 
 
