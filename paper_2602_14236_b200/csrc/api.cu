@@ -108,9 +108,9 @@ int salicache_create(salicache_ctx** out, const salicache_params* p) {
     for (int l = 0; l < 3 && ok; ++l) {
         size_t Pl = P0 >> (2 * l);
         ok = ok && cudaMalloc(&c->pyr[l], slots * Pl * sizeof(float)) == cudaSuccess;
-        // zeroed, with a pad of one row + 2 behind the last plane: the flow kernels read (and multiply by zero)
-        // the tap after the last column / row
-        const size_t cbytes = (slots * 5 * Pl + (size_t)(p->W >> l) + 2) * sizeof(float);
+        // 16-byte records then one plane, each zeroed and followed by a pad of one row + 2: the flow kernels read
+        // (and multiply by zero) the tap after the last column / row
+        const size_t cbytes = (slots * 5 * Pl + 5 * ((size_t)(p->W >> l) + 2)) * sizeof(float);
         ok = ok && cudaMalloc(&c->coef[l], cbytes) == cudaSuccess;
         ok = ok && cudaMemset(c->coef[l], 0, cbytes) == cudaSuccess;
     }

@@ -36,7 +36,7 @@ struct salicache_ctx {
     PlaneGeom plane[2];
     // flow scratch (sized for the largest plane)
     float* pyr[3];             // [chunk+1][h_l*w_l]
-    float* coef[3];            // [2*chunk][5][h_l*w_l] expansion planes
+    float* coef[3];            // expansion coefficients: float4 [2*chunk][h_l*w_l] + pad, then float [2*chunk][h_l*w_l] + pad
     float* gh_a;               // [chunk][5][H*W] normal-equation terms, ping
     float* gh_b;               //                                         pong
     float* flow_a;             // [chunk][2][H*W] displacement carried between levels

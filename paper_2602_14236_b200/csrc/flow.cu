@@ -1,15 +1,16 @@
 // Temporal branch (Sec. III-A, Eq. 5): gray pyramid, polynomial expansion, coarse-to-fine
 // displacement updates and the per-patch RMS flow magnitude.
 //
-// Precision: the box sums, the 2x2 solve, sampling positions and the patch reduction are double (the
-// determinant cancels); pyramid levels are exact in float; expansion coefficients and the per-pixel
-// normal-equation terms (G, h) are stored as float, and the terms are formed in float from them.  The
-// effect on dP stays two orders of magnitude below the 1e-4 relative tolerance on every workload.
+// Precision: pyramid levels are exact in float; the expansion runs in double and its coefficients are
+// stored as float; the per-pixel normal-equation terms (G, h), their 15x15 window sums and the 2x2 solve
+// run in float, the sums without any subtraction and the solve with compensated products; sampling
+// positions are exact; the patch reduction is double.  The effect on dP stays more than an order of
+// magnitude below the 1e-4 relative tolerance on every workload.
 //
-// One displacement update = box sums of (G, h) over the 15x15 window + a 2x2 solve.  k_flow_update does
-// that on a 28x14 tile with separable sliding-window sums (columns from registers, rows from shared
-// memory) and, fused behind the solve, the (G, h) of the NEXT update at the same pixels (which needs no
-// halo), or the patch scores after the last update.
+// One displacement update = window sums of (G, h) + a 2x2 solve.  k_flow_update does that on a 56x28
+// (or 28x28) tile with separable sums (columns from registers, rows from shared memory) and, fused
+// behind the solve, the (G, h) of the NEXT update at the same pixels (which needs no halo), or the patch
+// scores after the last update.
 #include <math.h>
 
 #include "common.cuh"
@@ -68,7 +69,8 @@ struct PolyW {
     double inv_mu2, inv_mu2sq, inv_den, mu2;
 };
 
-// ---- polynomial expansion, 5x5: planes r2 r3 r4 r5 r6 (b_x, b_y, A_xx, A_yy, 2 A_xy), stored as float.
+// ---- polynomial expansion, 5x5: r2 r3 r4 r5 r6 = (b_x, b_y, A_xx, A_yy, 2 A_xy), stored as float in the form the
+// displacement updates read: (r2, r3, r4, r5) / 2 as one 16-byte record per pixel and r6 / 4 in a plane of its own.
 // Separable, in double: a 32x32 tile grown by 2 is staged in shared memory, each grown row gets its three
 // horizontal moment sums (weights g, g*b, g*b^2), and each thread then walks down a column of 8 pixels
 // with the five rows of sums it needs in registers.
@@ -77,7 +79,8 @@ constexpr int PEW = PX + 2 * PH, PEH = PY + 2 * PH;
 constexpr int PRUN = 8;                          // pixels per thread in the vertical pass
 
 __global__ void __launch_bounds__(256)
-k_poly_exp(const float* __restrict__ img, int h, int w, int n_frames, PolyW pw, float* __restrict__ coef) {
+k_poly_exp(const float* __restrict__ img, int h, int w, int n_frames, PolyW pw, float4* __restrict__ cq,
+           float* __restrict__ cr) {
     __shared__ double tile[PEH][PEW + 1];
     __shared__ double hm[3][PEH][PX];
     const int f = blockIdx.z, x0 = blockIdx.x * PX, y0 = blockIdx.y * PY;
@@ -134,83 +137,74 @@ k_poly_exp(const float* __restrict__ img, int h, int w, int n_frames, PolyW pw, 
                 }
                 const int y = y0 + oy0 + k;
                 if (y < h) {
-                    float* c = coef + (size_t)f * 5 * P + (size_t)y * w + x;
-                    c[0 * P] = (float)(m10 * pw.inv_mu2);
-                    c[1 * P] = (float)(m01 * pw.inv_mu2);
-                    c[2 * P] = (float)((m20 - pw.mu2 * m00) * pw.inv_den);
-                    c[3 * P] = (float)((m02 - pw.mu2 * m00) * pw.inv_den);
-                    c[4 * P] = (float)(m11 * pw.inv_mu2sq);
+                    const size_t o = (size_t)f * P + (size_t)y * w + x;
+                    cq[o] = make_float4((float)(0.5 * (m10 * pw.inv_mu2)), (float)(0.5 * (m01 * pw.inv_mu2)),
+                                        (float)(0.5 * ((m20 - pw.mu2 * m00) * pw.inv_den)),
+                                        (float)(0.5 * ((m02 - pw.mu2 * m00) * pw.inv_den)));
+                    cr[o] = (float)(0.25 * (m11 * pw.inv_mu2sq));
                 }
             }
         }
     }
 }
 
-// Bilinear corner set of a clamped continuous position (the coarse-to-fine transfer samples at multiples of
-// 1/4, which single precision holds exactly).
-struct Bilin {
-    int i00, i01, i10, i11;
-    float fx, fy;
+// Expansion coefficients of one frame at one level, as the displacement updates read them:
+//   q[p] = (b_x, b_y, A_xx, A_yy) / 2 as one 16-byte record per pixel,  r[p] = A_xy / 2.
+// Halving is exact, so (A1 + A2)/2 and -(b2 - b1)/2 become plain sums and differences of stored values.
+struct CoefView {
+    const float4* __restrict__ q;
+    const float* __restrict__ r;
 };
-__device__ __forceinline__ Bilin bilin_at(float y, float x, int h, int w) {
-    x = fminf(fmaxf(x, 0.0f), (float)(w - 1));
-    y = fminf(fmaxf(y, 0.0f), (float)(h - 1));
-    int x0 = (int)floorf(x), y0 = (int)floorf(y);
-    int x1 = min(x0 + 1, w - 1), y1 = min(y0 + 1, h - 1);
-    Bilin b;
-    b.fx = x - x0;
-    b.fy = y - y0;
-    b.i00 = y0 * w + x0;
-    b.i01 = y0 * w + x1;
-    b.i10 = y1 * w + x0;
-    b.i11 = y1 * w + x1;
-    return b;
+
+__device__ __forceinline__ float lerp2(float a, float b, float c, float d, float gx, float fx, float gy, float fy) {
+    const float top = a * gx + b * fx;
+    const float bot = c * gx + d * fx;
+    return top * gy + bot * fy;
 }
-__device__ __forceinline__ float bilin_fetch(const float* __restrict__ p, const Bilin& b) {
-    float top = p[b.i00] * (1.0f - b.fx) + p[b.i01] * b.fx;
-    float bot = p[b.i10] * (1.0f - b.fx) + p[b.i11] * b.fx;
-    return top * (1.0f - b.fy) + bot * b.fy;
+
+// floor(v) as a float and as an int without the conversion unit, for |v| < 2^22: adding 1.5 * 2^23 rounds to the
+// nearest integer, whose value sits in the low mantissa bits; one compare steps down where that rounded up.
+__device__ __forceinline__ void floor_fi(float v, float& f, int& i) {
+    const float t = v + 12582912.0f;
+    float r = t - 12582912.0f;
+    int k = __float_as_int(t) - 0x4B400000;
+    if (r > v) { r -= 1.0f; k -= 1; }
+    f = r;
+    i = k;
 }
 
 // Normal-equation terms of one pixel for the prior (du, dv): G = A^T A (g11 g12 g22), hv = A^T db,
 //   A = (A1(x) + A2(x~))/2,  db = -(b2(x~) - b1(x))/2 + A d~,  x~ = clamp(x + d~), bilinear fetch.
-// The sampling position is exact: floor and fraction of d~ are taken in the precision d~ comes in and the
-// integer part is added to the pixel index (x + d~ in single precision would move the sample by up to
-// 2e-5 px at x ~ 300); the interpolation and the products run in single precision on the
-// single-precision coefficients, whose rounding already bounds what they can deliver.
+// The sampling position is exact: the displacement is clamped to [-x, w-1-x] (integers, exact in single
+// precision), its floor and fraction are taken on the displacement itself and the integer part is added to the
+// pixel index (x + d~ in single precision would move the sample by up to 2e-5 px at x ~ 300); the interpolation
+// and the products run in single precision on the single-precision coefficients, whose rounding already bounds
+// what they can deliver.  xlo = -x, xhi = w-1-x, ylo = -y, yhi = h-1-y as floats.
 // The four taps are read at i, i+1, i+w, i+w+1 without clamping the far ones: where the position is
 // clamped to the last column or row the fraction is zero, so the far tap is multiplied by zero, and it
-// is a finite number (the next row, the next plane, or the zeroed pad behind the last plane).
-template <typename R>
-__device__ __forceinline__ void normal_terms(const float* __restrict__ c1, const float* __restrict__ c2, size_t P,
-                                             int h, int w, int y, int x, R du, R dv, float out[5]) {
-    const int p = y * w + x;
-    const R fdu = floor(du), fdv = floor(dv);
-    int x0 = x + (int)fdu, y0 = y + (int)fdv;
-    float fx = (float)(du - fdu), fy = (float)(dv - fdv);
-    if (x0 < 0) { x0 = 0; fx = 0.0f; }
-    if (x0 >= w - 1) { x0 = w - 1; fx = 0.0f; }
-    if (y0 < 0) { y0 = 0; fy = 0.0f; }
-    if (y0 >= h - 1) { y0 = h - 1; fy = 0.0f; }
+// is a finite number (the next row, the next frame's plane, or the zeroed pad behind the last plane).
+__device__ __forceinline__ void normal_terms(const CoefView& c1, const CoefView& c2, int w, int p, float xlo, float xhi,
+                                             float ylo, float yhi, float du, float dv, float out[5]) {
+    const float su = fminf(fmaxf(du, xlo), xhi), sv = fminf(fmaxf(dv, ylo), yhi);
+    float fdu, fdv;
+    int iu, iv;
+    floor_fi(su, fdu, iu);
+    floor_fi(sv, fdv, iv);
+    const float fx = su - fdu, fy = sv - fdv;
     const float gx = 1.0f - fx, gy = 1.0f - fy;
-    const float* q = c2 + (y0 * w + x0);
-    const float* a = c1 + p;
-    float v[5], u[5];
-#pragma unroll
-    for (int c = 0; c < 5; ++c) {
-        const float top = q[0] * gx + q[1] * fx;
-        const float bot = q[w] * gx + q[w + 1] * fx;
-        v[c] = top * gy + bot * fy;
-        u[c] = a[0];
-        q += P;
-        a += P;
-    }
-    const float duf = (float)du, dvf = (float)dv;
-    const float axx = 0.5f * (u[2] + v[2]);
-    const float ayy = 0.5f * (u[3] + v[3]);
-    const float axy = 0.5f * (0.5f * u[4] + 0.5f * v[4]);
-    const float dbx = -0.5f * (v[0] - u[0]) + (axx * duf + axy * dvf);
-    const float dby = -0.5f * (v[1] - u[1]) + (axy * duf + ayy * dvf);
+    const int i0 = p + iv * w + iu;
+    const float4 a = __ldg(c2.q + i0), b = __ldg(c2.q + i0 + 1), c = __ldg(c2.q + i0 + w), d = __ldg(c2.q + i0 + w + 1);
+    const float ra = __ldg(c2.r + i0), rb = __ldg(c2.r + i0 + 1), rc = __ldg(c2.r + i0 + w), rd = __ldg(c2.r + i0 + w + 1);
+    const float4 u = __ldg(c1.q + p);
+    const float ur = __ldg(c1.r + p);
+    const float vbx = lerp2(a.x, b.x, c.x, d.x, gx, fx, gy, fy);
+    const float vby = lerp2(a.y, b.y, c.y, d.y, gx, fx, gy, fy);
+    const float vxx = lerp2(a.z, b.z, c.z, d.z, gx, fx, gy, fy);
+    const float vyy = lerp2(a.w, b.w, c.w, d.w, gx, fx, gy, fy);
+    const float vxy = lerp2(ra, rb, rc, rd, gx, fx, gy, fy);
+    const float axx = u.z + vxx, ayy = u.w + vyy, axy = ur + vxy;
+    const float dbx = (u.x - vbx) + (axx * du + axy * dv);
+    const float dby = (u.y - vby) + (axy * du + ayy * dv);
     out[0] = axx * axx + axy * axy;
     out[1] = axx * axy + axy * ayy;
     out[2] = axy * axy + ayy * ayy;
@@ -228,105 +222,132 @@ __device__ __forceinline__ float det2(float a, float b, float c, float d) {
 }
 
 // ---- (G, h) of the first update of a level.  Prior: zero at the coarsest level, else the coarser
-// level's field carried over as d = 2 * bilinear(d_coarse) at ((x+1/2)/2 - 1/2, (y+1/2)/2 - 1/2).
+// level's field carried over as d = 2 * bilinear(d_coarse) at ((x+1/2)/2 - 1/2, (y+1/2)/2 - 1/2), clamped to the
+// coarse image.  For a fine coordinate x that position is x/2 - 1/4: left tap (x-1) >> 1 with weight 3/4 of the
+// right tap for even x and 1/4 for odd x; at x = 0 and at the last fine pixel the clamp puts it on the tap itself.
+__device__ __forceinline__ void coarse_tap(int x, int nc, int& i0, int& i1, float& f) {
+    i0 = (x - 1) >> 1;
+    f = (x & 1) ? 0.25f : 0.75f;
+    if (x == 0) { i0 = 0; f = 0.0f; }
+    i1 = i0 + 1;
+    if (i1 > nc - 1) { i1 = nc - 1; f = 0.0f; }      // x = 2 nc - 1: position nc - 3/4, clamped to nc - 1
+}
+
 __global__ void __launch_bounds__(256)
-k_flow_gh(const float* __restrict__ coef1, const float* __restrict__ coef2, size_t coef_stride, int h, int w,
-          const float* __restrict__ d_coarse, size_t flow_stride, float* __restrict__ gh, size_t gh_stride,
-          int n_pairs) {
-    const size_t P = (size_t)h * w;
+k_flow_gh(const float4* __restrict__ q1, const float* __restrict__ r1, const float4* __restrict__ q2,
+          const float* __restrict__ r2, int h, int w, unsigned w_inv, const float* __restrict__ d_coarse, size_t flow_stride,
+          float* __restrict__ gh, size_t gh_stride, int n_pairs) {
+    const int P = h * w;
     const int f = blockIdx.y, r = blockIdx.x * blockDim.x + threadIdx.x;        // grid: (pixels of the level, pairs)
-    if (r >= (int)P || f >= n_pairs) return;
-    const int y = r / w, x = r % w;
+    if (r >= P || f >= n_pairs) return;
+    const int y = (int)__umulhi((unsigned)r, w_inv), x = r - y * w;             // w_inv = ceil(2^32 / w): exact for r < 2^32 / w
+    const CoefView c1{q1 + (size_t)f * P, r1 + (size_t)f * P}, c2{q2 + (size_t)f * P, r2 + (size_t)f * P};
     float du = 0.0f, dv = 0.0f;
     if (d_coarse) {
-        const int hc = h / 2, wc = w / 2;
-        Bilin b = bilin_at((y + 0.5f) * 0.5f - 0.5f, (x + 0.5f) * 0.5f - 0.5f, hc, wc);
-        const float* c = d_coarse + (size_t)f * flow_stride;
-        du = 2.0f * bilin_fetch(c, b);
-        dv = 2.0f * bilin_fetch(c + (size_t)hc * wc, b);
+        const int hc = h >> 1, wc = w >> 1;
+        int x0, x1, y0, y1;
+        float fx, fy;
+        coarse_tap(x, wc, x0, x1, fx);
+        coarse_tap(y, hc, y0, y1, fy);
+        const float* cu = d_coarse + (size_t)f * flow_stride;
+        const float* cv = cu + hc * wc;
+        const int i00 = y0 * wc + x0, i01 = y0 * wc + x1, i10 = y1 * wc + x0, i11 = y1 * wc + x1;
+        const float gx = 1.0f - fx, gy = 1.0f - fy;
+        du = 2.0f * lerp2(__ldg(cu + i00), __ldg(cu + i01), __ldg(cu + i10), __ldg(cu + i11), gx, fx, gy, fy);
+        dv = 2.0f * lerp2(__ldg(cv + i00), __ldg(cv + i01), __ldg(cv + i10), __ldg(cv + i11), gx, fx, gy, fy);
     }
     float t[5];
-    normal_terms(coef1 + (size_t)f * coef_stride, coef2 + (size_t)f * coef_stride, P, h, w, y, x, du, dv, t);
+    normal_terms(c1, c2, w, r, (float)-x, (float)(w - 1 - x), (float)-y, (float)(h - 1 - y), du, dv, t);
     float* o = gh + (size_t)f * gh_stride + r;
 #pragma unroll
     for (int c = 0; c < 5; ++c) o[c * P] = t[c];
 }
 
-// ---- one displacement update on a tile of TW x 14 pixels (TW / 14 patches side by side).
-//   phase 1  one thread per (term, pair of columns of the tile grown by 8 columns each side): 28 8-byte
-//            loads down the columns, the 15-row sums of the 14 tile rows by a sliding window in double
-//            -> shared memory
-//   phase 2  one thread per (row, run of RUN columns): 15-column sums of the row sums, 2x2 solve -> d in
-//            shared memory
+// ---- one displacement update on a tile of TW x 28 pixels (TW / 14 x 2 patches).
+//   phase 1  one thread per (term, pair of columns of the tile grown by 8 columns each side): 42 8-byte
+//            loads down the columns in three blocks of 14 rows; the 15-row sums of the 28 tile rows are a
+//            suffix sum of one block plus a prefix sum of the next (no subtraction) -> shared memory
+//   phase 2  one thread per (row, run of RUN columns): 15-column sums of the row sums the same way,
+//            2x2 solve -> d in shared memory
 //   phase 3  one thread per pixel: the (G, h) of the NEXT update at d (no halo needed), and / or d itself,
 //            and / or the patch scores after the last update
 // The window covers the in-image part only: terms outside the image count as zero.
-constexpr int TH = 14;             // tile height = 1 patch
+constexpr int TH = 28;             // tile height = 2 patches
 constexpr int BR = 7;              // window radius (window 15)
-constexpr int ER = TH + 2 * BR;    // 28 rows loaded
+constexpr int BLK = 2 * BR;        // rows per block of the suffix / prefix scheme
 constexpr int UPD_THREADS = 224;
 constexpr int EMIT_NEXT = 1, EMIT_D = 2, EMIT_DP = 4, EMIT_D64 = 8;
 
 template <int TW>
 struct UpdGeom {
-    static constexpr int RUN = 4;                      // pixels per phase-2 thread
+    static constexpr int RUN = TW % 8 == 0 ? 8 : 4;    // pixels per phase-2 thread
     static constexpr int EW = TW + 16;                 // columns loaded: x0 - 8 .. x0 + TW + 7 (8-byte aligned pairs)
     static constexpr int S = EW % 8 == 4 ? EW : EW + 4; // row stride in floats, = 4 (mod 8): the 16-byte loads of 8
                                                        // consecutive rows fall on distinct banks
     static constexpr int NQ = 2 * BR + RUN + 2;        // row sums read per run, starting one column early (16-byte aligned)
-    static_assert(TW % 14 == 0 && RUN == 4 && S % 8 == 4 && NQ % 4 == 0 && 5 * (EW / 2) <= UPD_THREADS &&
-                      16 * (TW / RUN) <= UPD_THREADS, "tile geometry");
+    static constexpr int DPITCH = TW + 1;              // (du, dv) row pitch: odd, spreads phase 2's stores over the banks
+    static_assert(TW % 14 == 0 && (RUN == 4 || RUN == 8) && S % 8 == 4 && NQ % 4 == 0 && 5 * (EW / 2) <= UPD_THREADS &&
+                      TH * (TW / RUN) <= UPD_THREADS && UPD_THREADS % TW == 0,
+                  "tile geometry");
 };
 
 template <int TW, int FLAGS>
 __global__ void __launch_bounds__(UPD_THREADS, 4)
-k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, double eps,
-              const float* __restrict__ coef1, const float* __restrict__ coef2, size_t coef_stride,
+k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, float eps, const float4* __restrict__ q1,
+              const float* __restrict__ r1, const float4* __restrict__ q2, const float* __restrict__ r2,
               float* __restrict__ gh_out, float* __restrict__ d_out, double* __restrict__ d_out64, size_t flow_stride,
               float* __restrict__ dP, PlaneGeom g) {
     using G = UpdGeom<TW>;
-    constexpr int RUN = G::RUN, EW = G::EW, S = G::S, NQ = G::NQ;
-    constexpr int DSM_DOUBLES = (TH * (TW + 1) + 1) / 2 * 2 > UPD_THREADS + TW ? (TH * (TW + 1) + 1) / 2 * 2 : UPD_THREADS + TW + 2;
-    extern __shared__ __align__(16) double upd_smem[];
-    float2 (*dsm)[TW + 1] = reinterpret_cast<float2 (*)[TW + 1]>(upd_smem);            // [TH] (du, dv); the odd row pitch
-                                                                                       // spreads phase 2's stores over the banks
-    float (*vs)[TH][S] = reinterpret_cast<float (*)[TH][S]>(upd_smem + DSM_DOUBLES);   // [5] 15-row sums
+    constexpr int RUN = G::RUN, EW = G::EW, S = G::S, NQ = G::NQ, DPITCH = G::DPITCH;
+    extern __shared__ __align__(16) float upd_smem[];
+    float (*vs)[TH][S] = reinterpret_cast<float (*)[TH][S]>(upd_smem);                       // [5] 15-row sums
+    float2 (*dsm)[DPITCH] = reinterpret_cast<float2 (*)[DPITCH]>(upd_smem + 5 * TH * S);     // [TH] (du, dv)
     const int f = blockIdx.z;
     const int x0 = blockIdx.x * TW, y0 = blockIdx.y * TH;
-    const size_t P = (size_t)h * w;
+    const int P = h * w;
     const int t = threadIdx.x;
     if (t < 5 * (EW / 2)) {
         const int c = t / (EW / 2), cp = t - c * (EW / 2);
         const int x = x0 - 8 + 2 * cp;                  // even, and w is even: the pair is inside or outside together
         const bool xin = x >= 0 && x < w;
-        const float* src = gh_in + (size_t)f * gh_stride + (size_t)c * P + (xin ? x : 0);
-        float2 v[ER];
+        const float* src = gh_in + (size_t)f * gh_stride + c * P + (xin ? x : 0) + (y0 - BR) * w;
+        // rows y0 - 7 + r, r in [0, 42): those inside the image are r in [r_lo, r_hi)
+        const unsigned r_lo = y0 >= BR ? 0u : (unsigned)(BR - y0);
+        const unsigned r_n = (xin ? (unsigned)min(TH + 2 * BR, h - y0 + BR) : r_lo) - r_lo;
+        auto load = [&](int r) {
+            return ((unsigned)r - r_lo < r_n) ? __ldg(reinterpret_cast<const float2*>(src + r * w)) : make_float2(0.0f, 0.0f);
+        };
+        float2 a[BLK], b[BLK];
 #pragma unroll
-        for (int r = 0; r < ER; ++r) {
-            const int y = y0 - BR + r;
-            v[r] = (xin && y >= 0 && y < h) ? __ldg(reinterpret_cast<const float2*>(src + (size_t)y * w))
-                                            : make_float2(0.0f, 0.0f);
-        }
-        // 15-row sums in single precision without any subtraction (a sliding window would leave the rounding
-        // residue of a strong edge in the flat region behind it): rows 0..13 become suffix sums, rows 14..27
-        // prefix sums, and window r = rows r .. r+14 is suffix[r] + prefix[r+14].  At most 14 roundings per sum.
+        for (int r = 0; r < BLK; ++r) a[r] = load(r);
 #pragma unroll
-        for (int r = TH - 2; r >= 0; --r) {
-            v[r].x += v[r + 1].x;
-            v[r].y += v[r + 1].y;
-        }
+        for (int r = 0; r < BLK; ++r) b[r] = load(BLK + r);
+        // window of tile row r = rows r .. r+14 = (suffix of the block it starts in) + (prefix of the next block):
+        // at most 14 roundings per sum and no subtraction (a sliding window would leave the rounding residue of a
+        // strong edge in the flat region behind it)
 #pragma unroll
-        for (int r = TH + 1; r < ER; ++r) {
-            v[r].x += v[r - 1].x;
-            v[r].y += v[r - 1].y;
-        }
+        for (int r = BLK - 2; r >= 0; --r) { a[r].x += a[r + 1].x; a[r].y += a[r + 1].y; }
         float2* dst = reinterpret_cast<float2*>(&vs[c][0][2 * cp]);
+        float2 pre = make_float2(0.0f, 0.0f);
 #pragma unroll
-        for (int r = 0; r < TH; ++r) dst[r * (S / 2)] = make_float2(v[r].x + v[r + TH].x, v[r].y + v[r + TH].y);
+        for (int r = 0; r < BLK; ++r) {
+            pre.x += b[r].x; pre.y += b[r].y;
+            dst[r * (S / 2)] = make_float2(a[r].x + pre.x, a[r].y + pre.y);
+        }
+#pragma unroll
+        for (int r = 0; r < BLK; ++r) a[r] = load(2 * BLK + r);
+#pragma unroll
+        for (int r = BLK - 2; r >= 0; --r) { b[r].x += b[r + 1].x; b[r].y += b[r + 1].y; }
+        pre = make_float2(0.0f, 0.0f);
+#pragma unroll
+        for (int r = 0; r < BLK; ++r) {
+            pre.x += a[r].x; pre.y += a[r].y;
+            dst[(BLK + r) * (S / 2)] = make_float2(b[r].x + pre.x, b[r].y + pre.y);
+        }
     }
     __syncthreads();
-    if ((t & 15) < TH && (t >> 4) < TW / RUN) {
-        const int row = t & 15, run = t >> 4;      // a quarter warp reads 8 rows of one run: conflict-free 16-byte loads
+    if (t < TH * (TW / RUN)) {
+        const int row = t % TH, run = t / TH;      // a quarter warp reads 8 rows of one run: conflict-free 16-byte loads
         const int col0 = RUN * run;                // output columns col0 .. col0+RUN-1; their windows start at col0 + 1
         float s[5][RUN];
 #pragma unroll
@@ -341,17 +362,18 @@ k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, d
                 q[4 * i + 2] = pr.z;
                 q[4 * i + 3] = pr.w;
             }
-            // windows q[k+1 .. k+15], k = 0..3, again without subtraction: suffix sums ending at q[15],
+            // windows q[k+1 .. k+15], k = 0..RUN-1, again without subtraction: suffix sums ending at q[15],
             // prefix sums starting at q[16]
             float suf = q[RUN];
 #pragma unroll
             for (int i = RUN + 1; i <= 2 * BR + 1; ++i) suf += q[i];
-            float pre = 0.0f;
+            s[c][RUN - 1] = suf;
 #pragma unroll
-            for (int k = RUN - 1; k >= 0; --k) {      // suf = q[k+1] + ... + q[15]
-                if (k < RUN - 1) suf += q[k + 1];
+            for (int k = RUN - 2; k >= 0; --k) {      // suf = q[k+1] + ... + q[15]
+                suf += q[k + 1];
                 s[c][k] = suf;
             }
+            float pre = 0.0f;
 #pragma unroll
             for (int k = 1; k < RUN; ++k) {            // pre = q[16] + ... + q[15+k]
                 pre += q[2 * BR + 1 + k];
@@ -362,22 +384,25 @@ k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, d
 #pragma unroll
         for (int k = 0; k < RUN; ++k) {
             const float g11 = s[0][k], g12 = s[1][k], g22 = s[2][k], h1 = s[3][k], h2 = s[4][k];
-            const float inv = __frcp_rn(det2(g11, g12, g12, g22) + (float)eps);
+            const float inv = __frcp_rn(det2(g11, g12, g12, g22) + eps);
             dsm[row][col0 + k] = make_float2(det2(g22, g12, h2, h1) * inv, det2(g11, g12, h1, h2) * inv);
         }
     }
     __syncthreads();
-    // UPD_THREADS is a multiple of TW: a thread keeps its column, hence its patch, over its pixels
-    static_assert(UPD_THREADS % TW == 0, "a thread stays in one column");
-    double acc = 0.0;
-    constexpr int PER = (TH * TW + UPD_THREADS - 1) / UPD_THREADS;
+    // UPD_THREADS is a multiple of TW: a thread keeps its column, hence its patch column, over its pixels
+    constexpr int PER = (TH * TW + UPD_THREADS - 1) / UPD_THREADS, RSTEP = UPD_THREADS / TW;
+    const int ox = t % TW, oyb = t / TW;
+    const int x = x0 + ox;
+    const CoefView c1{q1 + (size_t)f * P, r1 + (size_t)f * P}, c2{q2 + (size_t)f * P, r2 + (size_t)f * P};
+    double acc_up = 0.0, acc_lo = 0.0;                 // upper / lower patch of the tile
+    const float xlo = (float)-x, xhi = (float)(w - 1 - x);
+    float ylo = (float)-(y0 + oyb), yhi = (float)(h - 1 - y0 - oyb);
+    int p = (y0 + oyb) * w + x;
 #pragma unroll
-    for (int j = 0; j < PER; ++j) {
-        const int i = t + j * UPD_THREADS;
-        if (i >= TH * TW) break;
-        const int oy = i / TW, ox = i - oy * TW;
+    for (int j = 0; j < PER; ++j, p += RSTEP * w, ylo -= (float)RSTEP, yhi -= (float)RSTEP) {
+        const int oy = oyb + j * RSTEP;
+        if ((TH * TW) % UPD_THREADS != 0 && oy >= TH) break;
         const float2 d = dsm[oy][ox];
-        const int y = y0 + oy, x = x0 + ox, p = y * w + x;
         if (FLAGS & EMIT_D) {
             float* o = d_out + (size_t)f * flow_stride;
             o[p] = d.x;
@@ -390,41 +415,46 @@ k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, d
         }
         if (FLAGS & EMIT_NEXT) {
             float tm[5];
-            normal_terms(coef1 + (size_t)f * coef_stride, coef2 + (size_t)f * coef_stride, P, h, w, y, x, d.x, d.y, tm);
+            normal_terms(c1, c2, w, p, xlo, xhi, ylo, yhi, d.x, d.y, tm);
             float* o = gh_out + (size_t)f * gh_stride + p;
 #pragma unroll
             for (int c = 0; c < 5; ++c) o[c * P] = tm[c];
         }
-        if (FLAGS & EMIT_DP) acc += (double)d.x * (double)d.x + (double)d.y * (double)d.y;
+        if (FLAGS & EMIT_DP) {
+            const double m = (double)d.x * (double)d.x + (double)d.y * (double)d.y;
+            if (oy < 14) acc_up += m; else acc_lo += m;
+        }
     }
     if (FLAGS & EMIT_DP) {     // Eq. 5 (flow reading): dP_i = sqrt(mean over the patch of u^2 + v^2)
-        double* part = upd_smem;                   // (du, dv) are no longer needed once every thread is here
+        double* part = reinterpret_cast<double*>(upd_smem);     // the row sums are no longer needed
+        part[t] = acc_up;                                       // t = oyb * TW + ox
+        part[UPD_THREADS + t] = acc_lo;
         __syncthreads();
-        part[t] = acc;
-        __syncthreads();
-        if (t < TW) {                              // column totals, then 14 columns per patch: fixed order, deterministic
-            double col = 0.0;
-#pragma unroll
-            for (int k = 0; k < UPD_THREADS / TW; ++k) col += part[t + k * TW];
-            part[UPD_THREADS + t] = col;
-        }
-        __syncthreads();
-        if (t < TW / 14) {
+        if (t < 2 * TW) {                          // column totals, then 14 columns per patch: fixed order, deterministic
+            const int half = t / TW, col = t - half * TW;
             double tot = 0.0;
 #pragma unroll
-            for (int q = 0; q < 14; ++q) tot += part[UPD_THREADS + 14 * t + q];
-            const int py = blockIdx.y, px = blockIdx.x * (TW / 14) + t;
-            dP[(size_t)f * g.n_tok + patch_token(g, py, px)] = (float)sqrt(tot / (double)(TH * 14));
+            for (int k = 0; k < RSTEP; ++k) tot += part[half * UPD_THREADS + k * TW + col];
+            part[2 * UPD_THREADS + t] = tot;
+        }
+        __syncthreads();
+        if (t < 2 * (TW / 14)) {
+            const int half = t / (TW / 14), pc = t - half * (TW / 14);
+            double tot = 0.0;
+#pragma unroll
+            for (int q = 0; q < 14; ++q) tot += part[2 * UPD_THREADS + half * TW + 14 * pc + q];
+            const int py = 2 * blockIdx.y + half, px = blockIdx.x * (TW / 14) + pc;
+            dP[(size_t)f * g.n_tok + patch_token(g, py, px)] = (float)sqrt(tot / 196.0);
         }
     }
 }
 
 template <int TW>
 constexpr size_t upd_smem_bytes() {
-    // (du, dv) as float2, reused as UPD_THREADS + TW doubles by the patch reduction; then the row sums
-    constexpr size_t d = (TH * (TW + 1) + 1) / 2 * 2 > UPD_THREADS + TW ? (TH * (TW + 1) + 1) / 2 * 2 : UPD_THREADS + TW + 2;
-    return d * sizeof(double) + (size_t)5 * TH * UpdGeom<TW>::S * sizeof(float);
+    // the row sums (reused as 2 * UPD_THREADS + 2 * TW doubles by the patch reduction), then (du, dv) as float2
+    return (size_t)5 * TH * UpdGeom<TW>::S * sizeof(float) + (size_t)TH * UpdGeom<TW>::DPITCH * sizeof(float2);
 }
+static_assert((2 * UPD_THREADS + 2 * 56) * sizeof(double) <= 5 * TH * UpdGeom<28>::S * sizeof(float), "patch reduction fits");
 
 template <int TW>
 int init_update() {
@@ -434,14 +464,18 @@ int init_update() {
     return SALICACHE_OK;
 }
 
+struct UpdArgs {
+    const float* gin; size_t gstride; int h, w; float eps;
+    const float4 *q1; const float* r1; const float4* q2; const float* r2;
+    float* gout; float* dout; double* dout64; size_t fstride; float* dP;
+};
+
 template <int TW>
-void launch_update(dim3 grid, cudaStream_t st, int flags, const float* gin, size_t gstride, int h, int w, double eps,
-                   const float* c1, const float* c2, size_t cstride, float* gout, float* dout, double* dout64,
-                   size_t fstride, float* dP, const PlaneGeom& g) {
+void launch_update(dim3 grid, cudaStream_t st, int flags, const UpdArgs& a, const PlaneGeom& g) {
 #define SC_UPD(F)                                                                                                   \
     case F:                                                                                                         \
-        k_flow_update<TW, F><<<grid, UPD_THREADS, upd_smem_bytes<TW>(), st>>>(gin, gstride, h, w, eps, c1, c2,     \
-                                                                               cstride, gout, dout, dout64, fstride, dP, g); \
+        k_flow_update<TW, F><<<grid, UPD_THREADS, upd_smem_bytes<TW>(), st>>>(a.gin, a.gstride, a.h, a.w, a.eps, a.q1, a.r1, \
+                                                                               a.q2, a.r2, a.gout, a.dout, a.dout64, a.fstride, a.dP, g); \
         break;
     switch (flags) {
         SC_UPD(EMIT_NEXT)
@@ -548,33 +582,43 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
         for (int l = 1; l < 3; ++l)
             k_pyr_down<<<dim3(blocks_for((long long)hs[l] * ws[l], T), nf), T, 0, st>>>(c->pyr[l - 1], hs[l - 1], ws[l - 1], nf,
                                                                                         c->pyr[l]);
-        for (int l = 0; l < 3; ++l) {
+        const size_t slots = (size_t)2 * c->chunk;
+        float4* cq[3];
+        float* cr[3];
+        for (int l = 0; l < 3; ++l) {      // the records, a pad of one row + 2, then the A_xy plane (and its pad)
+            cq[l] = reinterpret_cast<float4*>(c->coef[l]);
+            cr[l] = c->coef[l] + 4 * (slots * hs[l] * ws[l] + ws[l] + 2);
             dim3 gp((ws[l] + PX - 1) / PX, (hs[l] + PY - 1) / PY, nf);
-            k_poly_exp<<<gp, 256, 0, st>>>(c->pyr[l], hs[l], ws[l], nf, pw, c->coef[l]);
+            k_poly_exp<<<gp, 256, 0, st>>>(c->pyr[l], hs[l], ws[l], nf, pw, cq[l], cr[l]);
         }
         c->launches += 5;
-        const size_t fstride = 2 * P0, gstride = 5 * P0;
+        // Coarse to fine: first terms, then the updates, each launch over all pairs of the pass.  (Sub-batches sized
+        // for the L2 cache were measured and are slower: the kernels are bound by issue slots and load latency, not
+        // by DRAM, and small launches add ramp-up and tail time.)
+        const size_t fstride = 2 * P0;
         float* d_lvl[2] = {c->flow_a, c->flow_b};
         const float* coarse = nullptr;
         for (int l = 2; l >= 0; --l) {
             const size_t Pl = (size_t)hs[l] * ws[l];
-            const size_t cstride = 5 * Pl;
+            const size_t gstride = 5 * Pl;
             float* dl = d_lvl[l & 1];
             const int tw = ws[l] % 56 == 0 ? 56 : 28;
-            {
-                const int z0 = 0, nz = nb;
-                const float* c1 = c->coef[l] + (size_t)z0 * cstride;
-                const float* c2 = c1 + (sequence ? cstride : (size_t)nb * cstride);
-                float* gin = c->gh_a + (size_t)z0 * gstride;
-                float* gout = c->gh_b + (size_t)z0 * gstride;
+            const size_t second = sequence ? Pl : (size_t)nb * Pl;      // the pair's second frame, in pixels
+            const int sub = nb;
+            for (int z0 = 0; z0 < nb; z0 += sub) {
+                const int nz = nb - z0 < sub ? nb - z0 : sub;
+                const float4* q1 = cq[l] + (size_t)z0 * Pl;
+                const float* r1 = cr[l] + (size_t)z0 * Pl;
+                float* gin = c->gh_a;
+                float* gout = c->gh_b;
                 k_flow_gh<<<dim3(blocks_for((long long)Pl, 256), nz), 256, 0, st>>>(
-                    c1, c2, cstride, hs[l], ws[l], coarse ? coarse + (size_t)z0 * fstride : nullptr, fstride, gin, gstride, nz);
+                    q1, r1, q1 + second, r1 + second, hs[l], ws[l], (unsigned)((0x100000000ull + ws[l] - 1) / ws[l]), coarse ? coarse + (size_t)z0 * fstride : nullptr, fstride,
+                    gin, gstride, nz);
                 c->launches++;
                 dim3 grid(ws[l] / tw, hs[l] / TH, nz);
                 for (int it = 0; it < p.iters; ++it) {
                     const bool last = it == p.iters - 1;
                     int flags = last ? 0 : EMIT_NEXT;
-                    float* dout = dl + (size_t)z0 * fstride;
                     double* dout64 = nullptr;
                     if (last && l > 0) flags |= EMIT_D;
                     if (last && l == 0) {      // the field goes to the caller's buffer if there is one
@@ -584,13 +628,10 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
                             dout64 = d_flow_or_null + (size_t)(b0 + z0) * fstride;
                         }
                     }
-                    float* dp = d_deltaP + (size_t)(b0 + z0) * g.n_tok;
-                    if (tw == 56)
-                        launch_update<56>(grid, st, flags, gin, gstride, hs[l], ws[l], p.eps_det, c1, c2, cstride, gout, dout,
-                                          dout64, fstride, dp, g);
-                    else
-                        launch_update<28>(grid, st, flags, gin, gstride, hs[l], ws[l], p.eps_det, c1, c2, cstride, gout, dout,
-                                          dout64, fstride, dp, g);
+                    UpdArgs a{gin, gstride, hs[l], ws[l], (float)p.eps_det, q1, r1, q1 + second, r1 + second,
+                              gout, dl + (size_t)z0 * fstride, dout64, fstride, d_deltaP + (size_t)(b0 + z0) * g.n_tok};
+                    if (tw == 56) launch_update<56>(grid, st, flags, a, g);
+                    else launch_update<28>(grid, st, flags, a, g);
                     c->launches++;
                     float* t = gin; gin = gout; gout = t;
                 }
