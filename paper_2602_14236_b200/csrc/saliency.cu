@@ -31,39 +31,56 @@ __global__ void k_box_down2(const uint8_t* __restrict__ src, int H, int W, int n
 // ---- Canny up to the double threshold.  Tile 32x32, halo 4 (blur 2 + Sobel 1 + NMS 1).
 // Writes two bit planes (bit i of word wx = pixel 32*wx + i): kept = NMS-kept with m >= lo^2,
 // strong = kept with m >= hi^2.
+// The frame's bytes are staged with 16-byte loads (a row of W pixels is 3 W bytes, a multiple of 16), gray is
+// derived once from the staged bytes, and the 5x5 binomial blur runs as two passes of five taps: its integer sum
+// is the same whichever way it is bracketed.
 constexpr int CT = 32;
 constexpr int CG = CT + 8;   // gray tile
 constexpr int CB = CT + 4;   // blur tile
 constexpr int CM = CT + 2;   // magnitude tile
+constexpr int CRAW = 9;      // 16-byte chunks staged per row: 40 pixels = 120 bytes starting up to 12 bytes into a chunk
 
 __global__ void __launch_bounds__(256)
 k_canny_classify(const uint8_t* __restrict__ frames, size_t frame_bytes, int h, int w, int words, int lo2, int hi2,
                  uint32_t* __restrict__ bits_kept, uint32_t* __restrict__ bits_strong, const uint8_t* __restrict__ skip) {
+    __shared__ uint4 sraw[CG][CRAW];
     __shared__ uint8_t sg[CG][CG];
+    __shared__ uint16_t sh[CG][CB];      // horizontal pass of the blur, at most 16 * 255
     __shared__ uint8_t sb[CB][CB];
     __shared__ int smag[CM][CM];
     const int f = blockIdx.z, x0 = blockIdx.x * CT, y0 = blockIdx.y * CT;
     if (skip && skip[f]) return;
     const uint8_t* fr = frames + (size_t)f * frame_bytes;
-    for (int i = threadIdx.x; i < CG * CG; i += blockDim.x) {
-        int ry = i / CG, rx = i % CG;
-        sg[ry][rx] = (uint8_t)gray_at(fr, w, clampi(y0 - 4 + ry, 0, h - 1), clampi(x0 - 4 + rx, 0, w - 1));
+    const int row_bytes = 3 * w;
+    // bytes of the clamped columns x0-4 .. x0+35: from the chunk that holds the first one
+    const int xa = x0 >= 4 ? x0 - 4 : 0;
+    const int byte0 = (3 * xa) & ~15;
+    for (int i = threadIdx.x; i < CG * CRAW; i += blockDim.x) {
+        const int ry = i / CRAW, ch = i - ry * CRAW;
+        const int y = clampi(y0 - 4 + ry, 0, h - 1);
+        const int off = byte0 + 16 * ch;
+        if (off < row_bytes) sraw[ry][ch] = __ldg(reinterpret_cast<const uint4*>(fr + (size_t)y * row_bytes + off));
     }
     __syncthreads();
-    // blur at the clamped position, so that the Sobel taps read Bl(clamp(y), clamp(x))
+    for (int i = threadIdx.x; i < CG * CG; i += blockDim.x) {
+        const int ry = i / CG, rx = i - ry * CG;
+        const int x = clampi(x0 - 4 + rx, 0, w - 1);
+        const uint8_t* p = reinterpret_cast<const uint8_t*>(&sraw[ry][0]) + (3 * x - byte0);
+        sg[ry][rx] = (uint8_t)((77 * p[0] + 150 * p[1] + 29 * p[2] + 128) >> 8);
+    }
+    __syncthreads();
+    // blur at the clamped position, so that the Sobel taps read Bl(clamp(y), clamp(x)): column map first
+    for (int i = threadIdx.x; i < CG * CB; i += blockDim.x) {
+        const int gy = i / CB, rx = i - gy * CB;
+        const int gx0 = clampi(x0 - 2 + rx, 0, w - 1) - (x0 - 4);
+        const uint8_t* g = &sg[gy][gx0];
+        sh[gy][rx] = (uint16_t)(g[-2] + 4 * g[-1] + 6 * g[0] + 4 * g[1] + g[2]);
+    }
+    __syncthreads();
     for (int i = threadIdx.x; i < CB * CB; i += blockDim.x) {
-        int ry = i / CB, rx = i % CB;
-        int yc = clampi(y0 - 2 + ry, 0, h - 1), xc = clampi(x0 - 2 + rx, 0, w - 1);
-        int gy0 = yc - (y0 - 4), gx0 = xc - (x0 - 4);
-        const int k[5] = {1, 4, 6, 4, 1};
-        int acc = 0;
-#pragma unroll
-        for (int a = -2; a <= 2; ++a) {
-            int ra = 0;
-#pragma unroll
-            for (int b = -2; b <= 2; ++b) ra += k[b + 2] * sg[gy0 + a][gx0 + b];
-            acc += k[a + 2] * ra;
-        }
+        const int ry = i / CB, rx = i - ry * CB;
+        const int gy0 = clampi(y0 - 2 + ry, 0, h - 1) - (y0 - 4);
+        const int acc = sh[gy0 - 2][rx] + 4 * sh[gy0 - 1][rx] + 6 * sh[gy0][rx] + 4 * sh[gy0 + 1][rx] + sh[gy0 + 2][rx];
         sb[ry][rx] = (uint8_t)((acc + 128) >> 8);
     }
     __syncthreads();
@@ -192,21 +209,26 @@ __device__ __forceinline__ void rgb_to_lab(const double* __restrict__ lut, int R
 
 // ---- colour branch + blend + patch mean.  One CTA per 2x2 patches (28x28 pixels), halo 3.
 // Variances are taken about the LAB value of the tile's first pixel (variance is shift invariant),
-// which keeps flat regions exactly zero and small contrasts accurate; the sums of x and x^2 stay in
-// double because mean(x^2) - mean(x)^2 cancels.
-//   phase 1  LAB of the 34x34 grown tile -> shared memory
-//   then per channel (its row sums alone occupy shared memory, which keeps four CTAs on an SM):
-//   phase 2  one thread per (row, run of 4 columns): 7-column sums of x and x^2
-//   phase 3  one thread per (column, run of 4 rows): 7-row sums, variance added to the pixel's total
+// which keeps flat regions exactly zero and small contrasts accurate; the window sums stay in double
+// because mean(x^2) - mean(x)^2 cancels.  With x = (dL, da, db) the sum of the three variances is
+//   V = W[|x|^2] / n - (W[dL]^2 + W[da]^2 + W[db]^2) / n^2,    W[.] = 7x7 window sum,
+// so four planes are summed, not six.
+//   stage    the tile's bytes by 16-byte loads and the sRGB table into shared memory; warp 0 converts the
+//            tile's first pixel (the shift)
+//   convert  LAB of the 34x34 grown tile, minus the shift, and |x|^2 -> shared memory
+//   then per plane (its row sums alone occupy shared memory, which keeps four CTAs on an SM):
+//   phase 2  one thread per (row, run of 4 columns): 7-column sums
+//   phase 3  one thread per (column, run of 4 rows): 7-row sums
 //   last     C, blend with the edge bit, patch partial sums
 // Window sums of a run share their terms: the middle four once, then suffix sums to the left and prefix
 // sums to the right (11 additions for 4 windows).
 constexpr int ST = 28;
 constexpr int SR = 3;
 constexpr int SE = ST + 2 * SR;   // 34
-constexpr int SLP = SE + 2;       // lab row pitch (even: 16-byte loads of column pairs)
+constexpr int SLP = SE + 2;       // row pitch of the planes (even: 16-byte loads of column pairs)
 constexpr int CRUN = 4;
 constexpr int CNQ = 2 * SR + CRUN;   // 10 values feed 4 windows
+constexpr int SRAW = 8;           // 16-byte chunks staged per row: 34 pixels = 102 bytes starting up to 15 bytes into a chunk
 
 // w[k] = q[k] + ... + q[k+6], k = 0..3
 __device__ __forceinline__ void window4(const double q[CNQ], double w[CRUN]) {
@@ -219,74 +241,92 @@ __device__ __forceinline__ void window4(const double q[CNQ], double w[CRUN]) {
     w[3] = mid + p9;
 }
 
-__global__ void __launch_bounds__(256)
+struct ColorSmem {
+    double plane[4][SE][SLP];     // dL, da, db, |x|^2
+    double hs[SE][ST];            // 7-column sums of one plane
+    double lut[256];
+    uint4 raw[SE][SRAW];
+    double shift[3];
+    double psum[8][4];
+};
+
+__global__ void __launch_bounds__(256, 4)
 k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom g, int patch,
               const double* __restrict__ lut, const uint32_t* __restrict__ bits_edge, int words, double inv_sigma,
               double w_edge, double w_color, float* __restrict__ s_out, const uint8_t* __restrict__ skip) {
-    extern __shared__ __align__(16) double cs[];
-    double (*lab)[SE][SLP] = reinterpret_cast<double (*)[SE][SLP]>(cs);                              // [3]
-    double2 (*hs)[ST] = reinterpret_cast<double2 (*)[ST]>(cs + 3 * SE * SLP);                        // [SE] (sum x, sum x^2) of one channel
-    __shared__ double psum[8][4];
+    extern __shared__ __align__(16) unsigned char cs_raw[];
+    ColorSmem& sm = *reinterpret_cast<ColorSmem*>(cs_raw);
     const int f = blockIdx.z, x0 = blockIdx.x * ST, y0 = blockIdx.y * ST;
     if (skip && skip[f]) return;
     const int h = g.H, w = g.W;
     const uint8_t* fr = frames + (size_t)f * frame_bytes;
-    double L0, a0, b0;
-    {
-        const uint8_t* p = fr + ((size_t)y0 * w + x0) * 3;
-        rgb_to_lab(lut, p[0], p[1], p[2], L0, a0, b0);
+    const int row_bytes = 3 * w;
+    const int xa = x0 >= SR ? x0 - SR : 0;
+    const int byte0 = (3 * xa) & ~15;
+    sm.lut[threadIdx.x] = __ldg(lut + threadIdx.x);
+    for (int i = threadIdx.x; i < SE * SRAW; i += blockDim.x) {
+        const int ry = i / SRAW, ch = i - ry * SRAW;
+        const int y = clampi(y0 - SR + ry, 0, h - 1);
+        const int off = byte0 + 16 * ch;
+        if (off < row_bytes) sm.raw[ry][ch] = __ldg(reinterpret_cast<const uint4*>(fr + (size_t)y * row_bytes + off));
     }
-    for (int i = threadIdx.x; i < SE * SE; i += blockDim.x) {
-        int ry = i / SE, rx = i % SE;
-        const uint8_t* p = fr + ((size_t)clampi(y0 - SR + ry, 0, h - 1) * w + clampi(x0 - SR + rx, 0, w - 1)) * 3;
-        double L, a, b;
-        rgb_to_lab(lut, p[0], p[1], p[2], L, a, b);
-        lab[0][ry][rx] = L - L0;
-        lab[1][ry][rx] = a - a0;
-        lab[2][ry][rx] = b - b0;
+    if (threadIdx.x >= 224) {          // the last warp: the shift, straight from global memory
+        const uint8_t* p = fr + ((size_t)y0 * w + x0) * 3;
+        double L0, a0, b0;
+        rgb_to_lab(lut, p[0], p[1], p[2], L0, a0, b0);
+        if (threadIdx.x == 224) { sm.shift[0] = L0; sm.shift[1] = a0; sm.shift[2] = b0; }
+    }
+    __syncthreads();
+    {
+        const double L0 = sm.shift[0], a0 = sm.shift[1], b0 = sm.shift[2];
+        for (int i = threadIdx.x; i < SE * SE; i += blockDim.x) {
+            const int ry = i / SE, rx = i - ry * SE;
+            const int x = clampi(x0 - SR + rx, 0, w - 1);
+            const uint8_t* p = reinterpret_cast<const uint8_t*>(&sm.raw[ry][0]) + (3 * x - byte0);
+            double L, a, b;
+            rgb_to_lab(sm.lut, p[0], p[1], p[2], L, a, b);
+            L -= L0; a -= a0; b -= b0;
+            sm.plane[0][ry][rx] = L;
+            sm.plane[1][ry][rx] = a;
+            sm.plane[2][ry][rx] = b;
+            sm.plane[3][ry][rx] = L * L + a * a + b * b;
+        }
     }
     __syncthreads();
     const double inv_n = 1.0 / (double)((2 * SR + 1) * (2 * SR + 1));
     double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;   // the four patches of the tile
     const bool owner = threadIdx.x < ST * (ST / CRUN);          // phase 3: (column, run of 4 rows)
     const int ox = threadIdx.x % ST, oy0 = CRUN * (threadIdx.x / ST);
-    double V[CRUN] = {0.0, 0.0, 0.0, 0.0};
-    for (int c = 0; c < 3; ++c) {                               // one channel's row sums in shared memory at a time
+    double M[CRUN] = {0.0, 0.0, 0.0, 0.0}, S2[CRUN] = {0.0, 0.0, 0.0, 0.0};
+    for (int c = 0; c < 4; ++c) {                               // one plane's row sums in shared memory at a time
         for (int i = threadIdx.x; i < SE * (ST / CRUN); i += blockDim.x) {
             const int run = i % (ST / CRUN), ry = i / (ST / CRUN);
             const int cx = CRUN * run;                          // windows cx .. cx+3 read columns cx .. cx+9 of the grown tile
-            const double2* src = reinterpret_cast<const double2*>(&lab[c][ry][cx]);
-            double q[CNQ], q2[CNQ];
+            const double2* src = reinterpret_cast<const double2*>(&sm.plane[c][ry][cx]);
+            double q[CNQ];
 #pragma unroll
             for (int k = 0; k < CNQ / 2; ++k) {
                 double2 v = src[k];
                 q[2 * k] = v.x;
                 q[2 * k + 1] = v.y;
             }
-#pragma unroll
-            for (int k = 0; k < CNQ; ++k) q2[k] = q[k] * q[k];
-            double w1[CRUN], w2[CRUN];
+            double w1[CRUN];
             window4(q, w1);
-            window4(q2, w2);
-#pragma unroll
-            for (int k = 0; k < CRUN; ++k) hs[ry][cx + k] = make_double2(w1[k], w2[k]);
+            double2* dst = reinterpret_cast<double2*>(&sm.hs[ry][cx]);
+            dst[0] = make_double2(w1[0], w1[1]);
+            dst[1] = make_double2(w1[2], w1[3]);
         }
         __syncthreads();
         if (owner) {
-            double q[CNQ], q2[CNQ];
+            double q[CNQ];
 #pragma unroll
-            for (int k = 0; k < CNQ; ++k) {
-                double2 v = hs[oy0 + k][ox];
-                q[k] = v.x;
-                q2[k] = v.y;
-            }
-            double w1[CRUN], w2[CRUN];
+            for (int k = 0; k < CNQ; ++k) q[k] = sm.hs[oy0 + k][ox];
+            double w1[CRUN];
             window4(q, w1);
-            window4(q2, w2);
 #pragma unroll
             for (int k = 0; k < CRUN; ++k) {
-                double mean = w1[k] * inv_n;
-                V[k] += w2[k] * inv_n - mean * mean;
+                if (c < 3) M[k] += w1[k] * w1[k];
+                else S2[k] = w1[k];
             }
         }
         __syncthreads();
@@ -296,7 +336,8 @@ k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom 
 #pragma unroll
         for (int k = 0; k < CRUN; ++k) {
             const int oy = oy0 + k, y = y0 + oy;
-            double C = sqrt(fmax(V[k], 0.0)) * inv_sigma;
+            const double V = S2[k] * inv_n - M[k] * (inv_n * inv_n);
+            double C = sqrt(fmax(V, 0.0)) * inv_sigma;
             C = fmin(C, 1.0);
             uint32_t e = (bits_edge[((size_t)f * h + y) * words + (x >> 5)] >> (x & 31)) & 1u;
             double S = w_edge * (double)e + w_color * C;
@@ -316,13 +357,13 @@ k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom 
         acc3 += __shfl_xor_sync(0xffffffffu, acc3, o);
     }
     if ((threadIdx.x & 31) == 0) {
-        double* ps = psum[threadIdx.x >> 5];
+        double* ps = sm.psum[threadIdx.x >> 5];
         ps[0] = acc0; ps[1] = acc1; ps[2] = acc2; ps[3] = acc3;
     }
     __syncthreads();
     if (threadIdx.x < 4) {
         double tot = 0.0;
-        for (int wp = 0; wp < 8; ++wp) tot += psum[wp][threadIdx.x];      // fixed order: deterministic
+        for (int wp = 0; wp < 8; ++wp) tot += sm.psum[wp][threadIdx.x];      // fixed order: deterministic
         int py = blockIdx.y * 2 + threadIdx.x / 2, px = blockIdx.x * 2 + threadIdx.x % 2;
         s_out[(size_t)f * g.n_tok + patch_token(g, py, px)] = (float)(tot / (double)(patch * patch));
     }
@@ -332,7 +373,7 @@ inline unsigned blocks_for(long long n, int threads) { return (unsigned)((n + th
 
 }  // namespace
 
-static size_t color_smem() { return (size_t)(3 * SE * SLP + 2 * SE * ST) * sizeof(double); }
+static size_t color_smem() { return sizeof(ColorSmem); }
 
 int sc_saliency_init(int max_h, int max_words) {
     SC_CHECK(cudaFuncSetAttribute(k_color_patch, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)color_smem()));
