@@ -86,6 +86,12 @@ typedef struct salicache_params {
     int32_t L, heads, head_dim;   /* layers, heads, head size; heads*head_dim = row length HD        */
     int32_t group;           /* elements per quantisation group: 128 (one head), or heads*head_dim    */
                              /* (one scale, and zero, per token row)                                  */
+    /* colour term, frame-adaptive reading of Sec. IV-B's "adaptive thresholding based on the local   */
+    /* color variance" (a variant; 0 = the fixed sigma_ref above)                                     */
+    int32_t color_norm;      /* 1: C = min(1, sqrt(V) / (color_kappa * sigma_frame)) with             */
+                             /* sigma_frame = max(sqrt(mean over the image of V), color_sigma_min)    */
+    double  color_kappa;     /* 1.0                                                                   */
+    double  color_sigma_min; /* 0.5 (LAB units): an image without contrast stays without saliency     */
 } salicache_params;
 
 /* Fills *p with the defaults listed above for a 336x336, L=32, 32x128 configuration. */
@@ -235,7 +241,8 @@ SALICACHE_API int salicache_unpack_kv(salicache_ctx* ctx, const salicache_pools*
  * cudaMalloc / cudaFree and no allocating library routine.
  *
  *   p           HOST pointer; the fields read are H, W, patch, n_images, canny_lo, canny_hi,
- *               var_radius, sigma_ref, w_edge, w_color, hyst_max_iters.  n_images must be 1 and
+ *               var_radius, sigma_ref, w_edge, w_color, hyst_max_iters, color_norm.  n_images must
+ *               be 1, color_norm 0 (the frame-adaptive colour term needs a context's scratch) and
  *               H, W at most SALICACHE_NOALLOC_MAX_SIDE (multiples of 112 as for a context).
  *   d_frames    DEVICE, u8 [B][H][W][3], 16-byte aligned, caller-owned
  *   B           0 .. SALICACHE_NOALLOC_MAX_FRAMES; larger batches are rejected with E_SHAPE and

@@ -77,6 +77,9 @@ class Params:
     tau_med: float = 0.36
     tau_low: float = 0.25
     patch_reuse: int = 1
+    color_norm: int = 0          # 0: fixed sigma_ref; 1: frame-adaptive (kappa x the frame's RMS local contrast)
+    color_kappa: float = 1.0
+    color_sigma_min: float = 0.5
 
 
 def num_threads() -> int:
@@ -198,20 +201,57 @@ def color_contrast(rgb: np.ndarray, radius: int = 3, sigma_ref: float = 16.0) ->
     return out
 
 
+def color_variance(rgb: np.ndarray, radius: int = 3) -> np.ndarray:
+    """V [h][w]: summed population variance of L, a, b in the (2 radius + 1)^2 window."""
+    rgb = _c(rgb, np.uint8)
+    h, w, _ = rgb.shape
+    out = np.empty((h, w), np.float64)
+    lib().oracle_color_variance(_p(rgb), C.c_int(h), C.c_int(w), C.c_int(radius), _p(out))
+    return out
+
+
+def color_normalise_global(V: np.ndarray, kappa: float = 1.0, sigma_min: float = 0.5) -> np.ndarray:
+    """Frame-adaptive colour term from a V map: min(1, sqrt(V) / (kappa max(sqrt(mean V), sigma_min)))."""
+    V = _c(V, np.float64)
+    out = np.empty(V.shape, np.float64)
+    lib().oracle_color_normalise_global(_p(V), C.c_size_t(V.size), C.c_double(kappa), C.c_double(sigma_min), _p(out))
+    return out
+
+
+def color_contrast_global(rgb: np.ndarray, radius: int = 3, kappa: float = 1.0, sigma_min: float = 0.5) -> np.ndarray:
+    rgb = _c(rgb, np.uint8)
+    h, w, _ = rgb.shape
+    out = np.empty((h, w), np.float64)
+    lib().oracle_color_contrast_global(_p(rgb), C.c_int(h), C.c_int(w), C.c_int(radius), C.c_double(kappa),
+                                       C.c_double(sigma_min), _p(out))
+    return out
+
+
 def saliency(frames: np.ndarray, p: Params = Params(), want_map: bool = False):
-    """frames: [B][h][w][3] uint8 (or one frame).  Returns s [B][n_patches] float64."""
+    """frames: [B][h][w][3] uint8 (or one frame).  Returns s [B][n_patches] float64.
+    p.color_norm = 1 selects the frame-adaptive colour term (p.color_kappa in place of p.sigma_ref)."""
     frames = _c(frames, np.uint8)
-    if frames.ndim == 3:
-        h, w, _ = frames.shape
-        s = np.empty(((h // p.patch) * (w // p.patch),), np.float64)
-        S = np.empty((h, w), np.float64) if want_map else None
-        lib().oracle_saliency(_p(frames), C.c_int(h), C.c_int(w), C.c_int(p.patch), C.c_int(p.canny_lo),
-                              C.c_int(p.canny_hi), C.c_int(p.var_radius), C.c_double(p.sigma_ref),
-                              C.c_double(p.w_edge), C.c_double(p.w_color), _p(s),
-                              _p(S) if want_map else C.c_void_p(None))
-        return (s, S) if want_map else s
+    one = frames.ndim == 3
+    if one:
+        frames = frames[None]
     B, h, w, _ = frames.shape
+    def one_frame(b, s_b, S_b):
+        head = (_p(frames[b]), C.c_int(h), C.c_int(w), C.c_int(p.patch), C.c_int(p.canny_lo), C.c_int(p.canny_hi),
+                C.c_int(p.var_radius))
+        tail = (C.c_double(p.w_edge), C.c_double(p.w_color), _p(s_b), _p(S_b) if S_b is not None else C.c_void_p(None))
+        if p.color_norm:
+            lib().oracle_saliency_global(*head, C.c_double(p.color_kappa), C.c_double(p.color_sigma_min), *tail)
+        else:
+            lib().oracle_saliency(*head, C.c_double(p.sigma_ref), *tail)
+
     s = np.empty((B, (h // p.patch) * (w // p.patch)), np.float64)
+    if one or want_map or p.color_norm:
+        S = np.empty((B, h, w), np.float64) if want_map else None
+        for b in range(B):
+            one_frame(b, s[b], S[b] if want_map else None)
+        if one:
+            return (s[0], S[0]) if want_map else s[0]
+        return (s, S) if want_map else s
     lib().oracle_saliency_batch(_p(frames), C.c_int(B), C.c_int(h), C.c_int(w), C.c_int(p.patch),
                                 C.c_int(p.canny_lo), C.c_int(p.canny_hi), C.c_int(p.var_radius),
                                 C.c_double(p.sigma_ref), C.c_double(p.w_edge), C.c_double(p.w_color), _p(s))

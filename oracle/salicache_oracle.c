@@ -418,14 +418,15 @@ EXPORT void oracle_rgb_to_lab(const uint8_t* rgb, int n, double* lab) {
 /* variance").  Reading: V = sum over L, a, b of the population variance in    */
 /* the (2r+1)^2 clamp-to-edge window; C = min(1, sqrt(V)/sigma_ref).           */
 /* ------------------------------------------------------------------------- */
-EXPORT void oracle_color_contrast(const uint8_t* rgb, int h, int w, int radius, double sigma_ref, double* C) {
+/* V alone: the summed population variance of L, a, b in the window, per pixel. */
+EXPORT void oracle_color_variance(const uint8_t* rgb, int h, int w, int radius, double* V) {
     size_t P = (size_t)h * w;
     double* lab = (double*)malloc(3 * P * sizeof(double));
     oracle_rgb_to_lab(rgb, (int)P, lab);
     int n = (2 * radius + 1) * (2 * radius + 1);
     for (int y = 0; y < h; ++y)
         for (int x = 0; x < w; ++x) {
-            double V = 0.0;
+            double v = 0.0;
             for (int c = 0; c < 3; ++c) {
                 double mean = 0.0;
                 for (int dy = -radius; dy <= radius; ++dy)
@@ -438,12 +439,53 @@ EXPORT void oracle_color_contrast(const uint8_t* rgb, int h, int w, int radius, 
                         double dv = lab[3 * ((size_t)clampi(y + dy, 0, h - 1) * w + clampi(x + dx, 0, w - 1)) + c] - mean;
                         var += dv * dv;
                     }
-                V += var / n;
+                v += var / n;
             }
-            double c01 = sqrt(V) / sigma_ref;
-            C[(size_t)y * w + x] = c01 < 1.0 ? c01 : 1.0;
+            V[(size_t)y * w + x] = v;
         }
     free(lab);
+}
+
+EXPORT void oracle_color_contrast(const uint8_t* rgb, int h, int w, int radius, double sigma_ref, double* C) {
+    size_t P = (size_t)h * w;
+    oracle_color_variance(rgb, h, w, radius, C);
+    for (size_t i = 0; i < P; ++i) {
+        double c01 = sqrt(C[i]) / sigma_ref;
+        C[i] = c01 < 1.0 ? c01 : 1.0;
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Colour branch, frame-adaptive reading of "adaptive thresholding based on    */
+/* the local color variance" (Sec. IV-B): the local contrast sqrt(V) is        */
+/* measured against the frame's own contrast level instead of a fixed          */
+/* sigma_ref:                                                                  */
+/*   sigma_frame = max( sqrt( mean over the frame of V ), sigma_min ),         */
+/*   C = min(1, sqrt(V) / (kappa * sigma_frame)),                              */
+/* so a dim or low-contrast frame keeps the same share of salient pixels as a  */
+/* vivid one.  sigma_min (LAB units) keeps a frame without any contrast from   */
+/* having its rounding noise promoted to saliency; with sigma_min = 0 a frame  */
+/* whose V vanishes everywhere gets C = 0.  The normalisation is a function of */
+/* the V map alone.                                                            */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_color_normalise_global(const double* V, size_t n, double kappa, double sigma_min, double* C) {
+    double sum = 0.0;
+    for (size_t i = 0; i < n; ++i) sum += V[i];
+    double sigma = sqrt(sum / (double)n);
+    if (sigma < sigma_min) sigma = sigma_min;
+    for (size_t i = 0; i < n; ++i) {
+        double c01 = sigma > 0.0 ? sqrt(V[i]) / (kappa * sigma) : 0.0;
+        C[i] = c01 < 1.0 ? c01 : 1.0;
+    }
+}
+
+EXPORT void oracle_color_contrast_global(const uint8_t* rgb, int h, int w, int radius, double kappa, double sigma_min,
+                                         double* C) {
+    size_t P = (size_t)h * w;
+    double* V = (double*)malloc(P * sizeof(double));
+    oracle_color_variance(rgb, h, w, radius, V);
+    oracle_color_normalise_global(V, P, kappa, sigma_min, C);
+    free(V);
 }
 
 /* ------------------------------------------------------------------------- */
@@ -451,15 +493,17 @@ EXPORT void oracle_color_contrast(const uint8_t* rgb, int h, int w, int radius, 
 /*   S = clamp(w_edge E + w_color C, 0, 1),  s_i = mean over patch i of S.      */
 /* S_or_null receives the per-pixel map.                                       */
 /* ------------------------------------------------------------------------- */
-EXPORT void oracle_saliency(const uint8_t* rgb, int h, int w, int patch, int lo, int hi, int radius,
-                            double sigma_ref, double w_edge, double w_color, double* s, double* S_or_null) {
+static void saliency_impl(const uint8_t* rgb, int h, int w, int patch, int lo, int hi, int radius, int global_norm,
+                          double sigma_ref_or_kappa, double sigma_min, double w_edge, double w_color, double* s,
+                          double* S_or_null) {
     size_t P = (size_t)h * w;
     uint8_t* g = (uint8_t*)malloc(P);
     uint8_t* E = (uint8_t*)malloc(P);
     double* C = (double*)malloc(P * sizeof(double));
     oracle_gray(rgb, h, w, g);
     oracle_canny(g, h, w, lo, hi, E, NULL);
-    oracle_color_contrast(rgb, h, w, radius, sigma_ref, C);
+    if (global_norm) oracle_color_contrast_global(rgb, h, w, radius, sigma_ref_or_kappa, sigma_min, C);
+    else oracle_color_contrast(rgb, h, w, radius, sigma_ref_or_kappa, C);
     int gh = h / patch, gw = w / patch;
     for (size_t i = 0; i < P; ++i) {
         double v = w_edge * E[i] + w_color * C[i];
@@ -474,6 +518,18 @@ EXPORT void oracle_saliency(const uint8_t* rgb, int h, int w, int patch, int lo,
         }
     if (S_or_null) memcpy(S_or_null, C, P * sizeof(double));
     free(C); free(E); free(g);
+}
+
+EXPORT void oracle_saliency(const uint8_t* rgb, int h, int w, int patch, int lo, int hi, int radius,
+                            double sigma_ref, double w_edge, double w_color, double* s, double* S_or_null) {
+    saliency_impl(rgb, h, w, patch, lo, hi, radius, 0, sigma_ref, 0.0, w_edge, w_color, s, S_or_null);
+}
+
+/* The same with the frame-adaptive colour term (kappa and sigma_min in place of sigma_ref). */
+EXPORT void oracle_saliency_global(const uint8_t* rgb, int h, int w, int patch, int lo, int hi, int radius,
+                                   double kappa, double sigma_min, double w_edge, double w_color, double* s,
+                                   double* S_or_null) {
+    saliency_impl(rgb, h, w, patch, lo, hi, radius, 1, kappa, sigma_min, w_edge, w_color, s, S_or_null);
 }
 
 EXPORT void oracle_saliency_batch(const uint8_t* frames, int B, int h, int w, int patch, int lo, int hi, int radius,

@@ -34,6 +34,7 @@ class Params(C.Structure):
         ("tau_t", C.c_float), ("theta_R", C.c_float), ("tau_high", C.c_float), ("tau_med", C.c_float),
         ("tau_low", C.c_float), ("patch_reuse", C.c_int32),
         ("L", C.c_int32), ("heads", C.c_int32), ("head_dim", C.c_int32), ("group", C.c_int32),
+        ("color_norm", C.c_int32), ("color_kappa", C.c_double), ("color_sigma_min", C.c_double),
     ]
 
 

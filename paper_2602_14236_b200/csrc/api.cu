@@ -26,6 +26,8 @@ void free_scratch(salicache_ctx* c) {
     if (c->bits_kept) cudaFree(c->bits_kept);
     if (c->bits_edge) cudaFree(c->bits_edge);
     if (c->lut) cudaFree(c->lut);
+    if (c->sqrt_v) cudaFree(c->sqrt_v);
+    if (c->v_part) cudaFree(c->v_part);
     if (c->base_frames) cudaFree(c->base_frames);
     if (c->row_prefix) cudaFree(c->row_prefix);
     if (c->attend_ws) cudaFree(c->attend_ws);
@@ -46,6 +48,7 @@ int salicache_default_params(salicache_params* p) {
     p->tau_t = 0.5f; p->theta_R = 0.90f; p->tau_high = 0.40f; p->tau_med = 0.36f; p->tau_low = 0.25f;
     p->patch_reuse = 1;
     p->L = 32; p->heads = 32; p->head_dim = 128; p->group = 128;
+    p->color_norm = 0; p->color_kappa = 1.0; p->color_sigma_min = 0.5;
     return SALICACHE_OK;
 }
 
@@ -70,7 +73,8 @@ int salicache_create(salicache_ctx** out, const salicache_params* p) {
     if (p->pyr_levels != 3 || p->poly_n != 5 || p->win != 15 || p->var_radius != 3 || p->patch != 14 ||
         (p->group != 128 && p->group != p->heads * p->head_dim) || p->iters < 1 || p->iters > 64 || !(p->poly_sigma > 0) || !(p->sigma_ref > 0) ||
         p->canny_lo < 0 || p->canny_hi < p->canny_lo || p->canny_hi > 1442 || p->hyst_max_iters < 1 ||
-        (p->n_images != 1 && p->n_images != 5) || p->L < 1 || p->heads < 1 || p->head_dim < 1)
+        (p->n_images != 1 && p->n_images != 5) || p->L < 1 || p->heads < 1 || p->head_dim < 1 ||
+        (p->color_norm != 0 && p->color_norm != 1) || (p->color_norm == 1 && (!(p->color_kappa > 0) || !(p->color_sigma_min >= 0))))
         return SALICACHE_E_PARAM;
     const int HD = p->heads * p->head_dim;
     if (!sc_kv_supported_hd(HD)) return SALICACHE_E_PARAM;
@@ -121,6 +125,10 @@ int salicache_create(salicache_ctx** out, const salicache_params* p) {
     ok = ok && cudaMalloc(&c->bits_kept, (size_t)c->chunk * p->H * words * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->bits_edge, (size_t)c->chunk * p->H * words * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->lut, 256 * sizeof(double)) == cudaSuccess;
+    if (p->color_norm == 1) {
+        ok = ok && cudaMalloc(&c->sqrt_v, (size_t)c->chunk * P0 * sizeof(float)) == cudaSuccess;
+        ok = ok && cudaMalloc(&c->v_part, (size_t)c->chunk * (p->H / 28) * (p->W / 28) * sizeof(double)) == cudaSuccess;
+    }
     ok = ok && cudaMalloc(&c->row_prefix, ((size_t)p->max_batch + 1) * sizeof(int64_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_status, sizeof(int)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->attend_ws, sc_attend_workspace_bytes(p->L, p->heads)) == cudaSuccess;

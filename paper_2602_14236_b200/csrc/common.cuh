@@ -45,6 +45,8 @@ struct salicache_ctx {
     uint32_t* bits_kept;       // [chunk][H][Ww]  NMS-kept weak or strong pixels
     uint32_t* bits_edge;       // [chunk][H][Ww]  strong pixels, grown to the edge map E
     double* lut;               // 256 entries sRGB -> linear
+    float* sqrt_v;             // frame-adaptive colour term only: [chunk][H*W] local contrast sqrt(V)
+    double* v_part;            //                                  [chunk][tiles] per-tile sums of V
     uint8_t* base_frames;      // anyres only: [chunk+1][336*336*3]
     // select / pack scratch
     int64_t* row_prefix;       // [max_batch+1] stored rows before each frame of the batch

@@ -68,7 +68,7 @@ extern "C" int salicache_saliency_noalloc(const salicache_params* p, const uint8
                                           int32_t* d_status_or_null, void* cuda_stream) {
     if (!p || !d_frames || !d_s) return SALICACHE_E_NULL;
     if (p->var_radius != 3 || p->patch != 14 || !(p->sigma_ref > 0) || p->canny_lo < 0 || p->canny_hi < p->canny_lo ||
-        p->canny_hi > 1442 || p->hyst_max_iters < 1 || p->n_images != 1)
+        p->canny_hi > 1442 || p->hyst_max_iters < 1 || p->n_images != 1 || p->color_norm != 0)
         return SALICACHE_E_PARAM;
     if (p->H <= 0 || p->W <= 0 || p->H % 112 != 0 || p->W % 112 != 0) return SALICACHE_E_SHAPE;
     if (p->H > NA_MAX_SIDE || p->W > NA_MAX_SIDE || B < 0 || B > NA_MAX_FRAMES) return SALICACHE_E_SHAPE;

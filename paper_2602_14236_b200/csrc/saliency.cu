@@ -250,10 +250,15 @@ struct ColorSmem {
     double psum[8][4];
 };
 
+// ADAPTIVE = false: C = min(1, sqrt(V) * inv_sigma), blended and reduced to the patch scores here.
+// ADAPTIVE = true:  the frame-adaptive colour term needs the image's mean V first: this kernel leaves sqrt(V) per
+//                   pixel in `sqrt_v` and the tile's sum of V in `v_part`; k_color_adaptive finishes.
+template <bool ADAPTIVE>
 __global__ void __launch_bounds__(256, 4)
 k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom g, int patch,
               const double* __restrict__ lut, const uint32_t* __restrict__ bits_edge, int words, double inv_sigma,
-              double w_edge, double w_color, float* __restrict__ s_out, const uint8_t* __restrict__ skip) {
+              double w_edge, double w_color, float* __restrict__ s_out, const uint8_t* __restrict__ skip,
+              float* __restrict__ sqrt_v, double* __restrict__ v_part) {
     extern __shared__ __align__(16) unsigned char cs_raw[];
     ColorSmem& sm = *reinterpret_cast<ColorSmem*>(cs_raw);
     const int f = blockIdx.z, x0 = blockIdx.x * ST, y0 = blockIdx.y * ST;
@@ -336,8 +341,13 @@ k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom 
 #pragma unroll
         for (int k = 0; k < CRUN; ++k) {
             const int oy = oy0 + k, y = y0 + oy;
-            const double V = S2[k] * inv_n - M[k] * (inv_n * inv_n);
-            double C = sqrt(fmax(V, 0.0)) * inv_sigma;
+            const double V = fmax(S2[k] * inv_n - M[k] * (inv_n * inv_n), 0.0);
+            if (ADAPTIVE) {
+                sqrt_v[((size_t)f * h + y) * w + x] = (float)sqrt(V);
+                acc0 += V;
+                continue;
+            }
+            double C = sqrt(V) * inv_sigma;
             C = fmin(C, 1.0);
             uint32_t e = (bits_edge[((size_t)f * h + y) * words + (x >> 5)] >> (x & 31)) & 1u;
             double S = w_edge * (double)e + w_color * C;
@@ -361,9 +371,74 @@ k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom 
         ps[0] = acc0; ps[1] = acc1; ps[2] = acc2; ps[3] = acc3;
     }
     __syncthreads();
+    if (ADAPTIVE) {
+        if (threadIdx.x == 0) {
+            double tot = 0.0;
+            for (int wp = 0; wp < 8; ++wp) tot += sm.psum[wp][0];                 // fixed order: deterministic
+            v_part[((size_t)f * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x] = tot;
+        }
+        return;
+    }
     if (threadIdx.x < 4) {
         double tot = 0.0;
         for (int wp = 0; wp < 8; ++wp) tot += sm.psum[wp][threadIdx.x];      // fixed order: deterministic
+        int py = blockIdx.y * 2 + threadIdx.x / 2, px = blockIdx.x * 2 + threadIdx.x % 2;
+        s_out[(size_t)f * g.n_tok + patch_token(g, py, px)] = (float)(tot / (double)(patch * patch));
+    }
+}
+
+// ---- frame-adaptive colour term, second pass.  One CTA per 2x2 patches: the image's mean V from the tile sums
+// (every CTA adds them in the same fixed order), sigma = max(sqrt(mean V), sigma_min), then
+// C = min(1, sqrt(V) / (kappa sigma)), the blend with the edge bit and the patch means.
+__global__ void __launch_bounds__(256)
+k_color_adaptive(const float* __restrict__ sqrt_v, const double* __restrict__ v_part, PlaneGeom g, int patch,
+                 const uint32_t* __restrict__ bits_edge, int words, double kappa, double sigma_min, double w_edge,
+                 double w_color, float* __restrict__ s_out, const uint8_t* __restrict__ skip) {
+    __shared__ double red[256];
+    __shared__ double psum[8][4];
+    const int f = blockIdx.z, x0 = blockIdx.x * ST, y0 = blockIdx.y * ST;
+    if (skip && skip[f]) return;
+    const int h = g.H, w = g.W, n_tiles = gridDim.x * gridDim.y;
+    double part = 0.0;
+    for (int i = threadIdx.x; i < n_tiles; i += 256) part += v_part[(size_t)f * n_tiles + i];
+    red[threadIdx.x] = part;
+    __syncthreads();
+    for (int o = 128; o; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    double sigma = sqrt(red[0] / ((double)h * (double)w));
+    sigma = fmax(sigma, sigma_min);
+    const double inv = sigma > 0.0 ? 1.0 / (kappa * sigma) : 0.0;
+    double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;
+    for (int i = threadIdx.x; i < ST * ST; i += 256) {
+        const int oy = i / ST, ox = i - oy * ST;
+        const int y = y0 + oy, x = x0 + ox;
+        const double C = fmin((double)sqrt_v[((size_t)f * h + y) * w + x] * inv, 1.0);
+        const uint32_t e = (bits_edge[((size_t)f * h + y) * words + (x >> 5)] >> (x & 31)) & 1u;
+        double S = w_edge * (double)e + w_color * C;
+        S = fmin(fmax(S, 0.0), 1.0);
+        const bool lower = oy >= patch, right = ox >= patch;
+        acc0 += (!lower && !right) ? S : 0.0;
+        acc1 += (!lower && right) ? S : 0.0;
+        acc2 += (lower && !right) ? S : 0.0;
+        acc3 += (lower && right) ? S : 0.0;
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+        acc0 += __shfl_xor_sync(0xffffffffu, acc0, o);
+        acc1 += __shfl_xor_sync(0xffffffffu, acc1, o);
+        acc2 += __shfl_xor_sync(0xffffffffu, acc2, o);
+        acc3 += __shfl_xor_sync(0xffffffffu, acc3, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        double* ps = psum[threadIdx.x >> 5];
+        ps[0] = acc0; ps[1] = acc1; ps[2] = acc2; ps[3] = acc3;
+    }
+    __syncthreads();
+    if (threadIdx.x < 4) {
+        double tot = 0.0;
+        for (int wp = 0; wp < 8; ++wp) tot += psum[wp][threadIdx.x];
         int py = blockIdx.y * 2 + threadIdx.x / 2, px = blockIdx.x * 2 + threadIdx.x % 2;
         s_out[(size_t)f * g.n_tok + patch_token(g, py, px)] = (float)(tot / (double)(patch * patch));
     }
@@ -376,7 +451,8 @@ inline unsigned blocks_for(long long n, int threads) { return (unsigned)((n + th
 static size_t color_smem() { return sizeof(ColorSmem); }
 
 int sc_saliency_init(int max_h, int max_words) {
-    SC_CHECK(cudaFuncSetAttribute(k_color_patch, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)color_smem()));
+    SC_CHECK(cudaFuncSetAttribute(k_color_patch<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)color_smem()));
+    SC_CHECK(cudaFuncSetAttribute(k_color_patch<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)color_smem()));
     size_t smem = (size_t)2 * max_h * max_words * sizeof(uint32_t);
     if (smem > 227 * 1024) return SALICACHE_E_SHAPE;
     // always the full opt-in limit: the attribute belongs to the function, not to a context, so a
@@ -405,8 +481,17 @@ int sc_saliency(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_frames, s
         size_t smem = (size_t)2 * g.H * words * sizeof(uint32_t);
         k_hysteresis<<<nb, 1024, smem, st>>>(c->bits_kept, c->bits_edge, g.H, words, p.hyst_max_iters, c->d_status, skip);
         dim3 gs(g.W / ST, g.H / ST, nb);
-        k_color_patch<<<gs, 256, color_smem(), st>>>(fr, frame_bytes, g, p.patch, c->lut, c->bits_edge, words, 1.0 / p.sigma_ref,
-                                          p.w_edge, p.w_color, d_s + (size_t)b0 * g.n_tok, skip);
+        float* s_dst = d_s + (size_t)b0 * g.n_tok;
+        if (p.color_norm == 0) {
+            k_color_patch<false><<<gs, 256, color_smem(), st>>>(fr, frame_bytes, g, p.patch, c->lut, c->bits_edge, words,
+                                                                1.0 / p.sigma_ref, p.w_edge, p.w_color, s_dst, skip, nullptr, nullptr);
+        } else {
+            k_color_patch<true><<<gs, 256, color_smem(), st>>>(fr, frame_bytes, g, p.patch, c->lut, c->bits_edge, words, 0.0,
+                                                               p.w_edge, p.w_color, s_dst, skip, c->sqrt_v, c->v_part);
+            k_color_adaptive<<<gs, 256, 0, st>>>(c->sqrt_v, c->v_part, g, p.patch, c->bits_edge, words, p.color_kappa,
+                                                 p.color_sigma_min, p.w_edge, p.w_color, s_dst, skip);
+            c->launches++;
+        }
         c->launches += 3;
     }
     SC_CHECK(cudaGetLastError());

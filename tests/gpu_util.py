@@ -19,7 +19,8 @@ def oracle_params(p: sc.Params) -> oracle.Params:
                          iters=p.iters, eps_det=p.eps_det, canny_lo=p.canny_lo, canny_hi=p.canny_hi,
                          var_radius=p.var_radius, sigma_ref=p.sigma_ref, w_edge=p.w_edge, w_color=p.w_color,
                          tau_t=p.tau_t, theta_R=p.theta_R, tau_high=p.tau_high, tau_med=p.tau_med,
-                         tau_low=p.tau_low, patch_reuse=p.patch_reuse)
+                         tau_low=p.tau_low, patch_reuse=p.patch_reuse, color_norm=p.color_norm,
+                         color_kappa=p.color_kappa, color_sigma_min=p.color_sigma_min)
 
 
 def assert_scores_close(gpu: np.ndarray, ref: np.ndarray, what: str):

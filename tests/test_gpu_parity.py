@@ -79,6 +79,32 @@ def test_saliency_other_weights_clamp_per_pixel():
     gu.assert_scores_close(s, oracle.saliency(fr, gu.oracle_params(ctx.params)), "s (clamped blend)")
 
 
+def test_saliency_with_the_frame_adaptive_colour_term_matches_the_oracle():
+    """The colour term measured against the frame's own contrast level (a second pass over the image): vivid frames,
+    a nearly flat frame whose contrast lies under sigma_min, an entirely flat frame, and the anyres layout, where the
+    frame and its base image are each normalised by their own statistic."""
+    for kw in (dict(color_kappa=1.0), dict(color_kappa=1.7, w_edge=0.8, w_color=0.6)):
+        ctx = _ctx(color_norm=1, **kw)
+        p = gu.oracle_params(ctx.params)
+        fr = np.concatenate([synth.frames(2, T=2), synth.frames(1, T=2, t0=2)])
+        dim = (118 + (fr[0].astype(np.int32) - 118) // 64).astype(np.uint8)          # grey levels 116..119 only
+        flat = np.full_like(fr[0], 90)
+        fr = np.concatenate([fr, dim[None], flat[None]])
+        _, s = gu.gpu_scores(ctx, fr)
+        want = oracle.saliency(fr, p)
+        gu.assert_scores_close(s, want, "s, frame-adaptive colour term")
+        assert want[:4].max() > 0.3 and not s[5].any()
+        assert not np.allclose(want[:4], oracle.saliency(fr[:4]), atol=1e-3)          # it is not the fixed reading
+    ctx = sc.Context(sc.salicache_default_params(H=672, W=672, n_images=5, max_batch=2, chunk_frames=2, L=1, color_norm=1))
+    p = gu.oracle_params(ctx.params)
+    fr = synth.frames(4, T=2, t0=29)
+    _, s = gu.gpu_scores(ctx, fr)
+    base = np.stack([oracle.box_down2(f) for f in fr])
+    rs_full, rs_base = oracle.saliency(fr, p), oracle.saliency(base, p)
+    want = np.stack([oracle.anyres_tokens(rs_full[t], rs_base[t]) for t in range(2)])
+    gu.assert_scores_close(s, want, "s anyres, frame-adaptive colour term")
+
+
 def test_small_frame_and_single_frame_batches():
     ctx = _ctx(H=112, W=112)
     fr = synth.frames(1, T=3)[:, 100:212, 60:172].copy()

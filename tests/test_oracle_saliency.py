@@ -217,3 +217,75 @@ def test_saliency_batch_matches_single_frames():
     s = oracle.saliency(fr)
     for b in range(2):
         assert np.array_equal(s[b], oracle.saliency(fr[b]))
+
+
+# ----------------------------------------------------------------------------- frame-adaptive colour term
+def test_color_variance_is_what_the_fixed_reading_normalises():
+    fr = synth.frames(2, T=1)[0][40:110, 30:120]
+    V = oracle.color_variance(fr)
+    assert np.array_equal(oracle.color_contrast(fr, sigma_ref=16.0), np.minimum(1.0, np.sqrt(V) / 16.0))
+    # library restatement of V: uniform filters over the clamp-extended LAB planes
+    lab = oracle.rgb_to_lab(fr).reshape(fr.shape[0], fr.shape[1], 3)
+    want = np.zeros(fr.shape[:2])
+    for c in range(3):
+        m1 = ndimage.uniform_filter(lab[:, :, c], 7, mode="nearest")
+        m2 = ndimage.uniform_filter(lab[:, :, c] ** 2, 7, mode="nearest")
+        want += m2 - m1 * m1
+    assert np.allclose(V, want, rtol=0, atol=1e-9)
+
+
+def test_global_colour_term_constant_frame_and_numpy_restatement():
+    flat = np.full((28, 42, 3), 77, np.uint8)
+    assert oracle.color_contrast_global(flat).max() < 1e-12                  # below sigma_min: rounding noise stays noise
+    assert oracle.color_normalise_global(np.zeros((4, 5)), 1.0, 0.0).max() == 0.0      # no floor, no contrast: C = 0
+    fr = synth.frames(3, T=1, t0=150)[0][:84, :112]
+    V = oracle.color_variance(fr)
+    for kappa in (0.5, 1.0, 3.0):
+        want = np.minimum(1.0, np.sqrt(V) / (kappa * np.sqrt(V.mean())))
+        assert np.sqrt(V.mean()) > 0.5
+        assert np.allclose(oracle.color_contrast_global(fr, kappa=kappa), want, rtol=1e-13, atol=0)
+        assert np.allclose(oracle.color_normalise_global(V, kappa), want, rtol=1e-13, atol=0)
+    # a frame whose contrast level lies under the floor is measured against the floor
+    dim = 1e-4 * V
+    assert np.allclose(oracle.color_normalise_global(dim, 1.0, 0.5), np.minimum(1.0, np.sqrt(dim) / 0.5), rtol=1e-13, atol=0)
+
+
+def test_global_colour_term_is_invariant_to_the_contrast_scale_and_reduces_to_the_fixed_reading():
+    fr = synth.frames(2, T=1)[0][100:184, 60:172]
+    V = oracle.color_variance(fr)
+    C = oracle.color_normalise_global(V, 1.7)
+    for a in (0.01, 9.0):                                                    # V -> a^2 V: every contrast scaled by a
+        assert np.allclose(oracle.color_normalise_global(a * a * V, 1.7, 0.0), C, rtol=1e-13, atol=0)
+    kappa = 16.0 / np.sqrt(V.mean())                                         # kappa sigma_frame = sigma_ref
+    assert np.allclose(oracle.color_contrast_global(fr, kappa=kappa), oracle.color_contrast(fr, sigma_ref=16.0), rtol=1e-12, atol=0)
+
+
+def test_global_colour_term_two_valued_frame_closed_form():
+    """Left half one colour, right half another (width W): a pixel whose 7-wide window holds k columns of the other
+    colour has V = (k/7)(1 - k/7) dE^2; the frame mean of V is (8/7) dE^2 / W, so C = sqrt(k (7 - k)) / 7 /
+    (kappa sqrt(8 / (7 W))) whatever the two colours are."""
+    H, W, kappa = 20, 56, 4.0
+    maps = []
+    for ca, cb in (((200, 40, 40), (30, 160, 220)), ((90, 90, 90), (96, 90, 84))):
+        fr = np.empty((H, W, 3), np.uint8)
+        fr[:, :W // 2] = ca
+        fr[:, W // 2:] = cb
+        maps.append(oracle.color_contrast_global(fr, kappa=kappa))
+    want = np.zeros(W)
+    for d, k in ((1, 3), (2, 2), (3, 1)):
+        c = np.sqrt(k * (7 - k)) / 7 / (kappa * np.sqrt(8 / (7 * W)))
+        want[W // 2 - d] = want[W // 2 + d - 1] = c
+    assert want.max() < 1.0
+    for C in maps:
+        assert np.allclose(C, want[None, :], rtol=1e-9, atol=1e-12)
+
+
+def test_saliency_with_the_global_colour_term_is_the_blend_of_its_parts():
+    fr = synth.frames(2, T=1)[0][:112, :140]
+    p = oracle.Params(color_norm=1, color_kappa=1.3)
+    s, S = oracle.saliency(fr, p, want_map=True)
+    E = oracle.canny(oracle.gray(fr))
+    want = np.clip(0.5 * E + 0.5 * oracle.color_contrast_global(fr, kappa=1.3), 0, 1)
+    assert np.allclose(S, want, rtol=0, atol=1e-15)
+    assert np.allclose(s, want.reshape(8, 14, 10, 14).mean(axis=(1, 3)).ravel(), rtol=1e-13, atol=0)
+    assert not np.allclose(s, oracle.saliency(fr, oracle.Params()))           # and it is not the fixed reading
