@@ -45,6 +45,7 @@ extern "C" {
 #define SALICACHE_E_CAPACITY   -6   /* a tier pool is too small (rows dropped, ring == 0)  */
 #define SALICACHE_E_NOCONVERGE -7   /* edge hysteresis hit hyst_max_iters                  */
 #define SALICACHE_E_NOMEM      -8   /* scratch allocation failed at create                 */
+#define SALICACHE_E_EVICTED    -9   /* rows asked for have been overwritten in a ring pool */
 
 /* Decision code per token (Fig. 3 categories; Eq. 8 tiers). */
 #define SALICACHE_REUSE 0   /* "skipped": K/V of the previous frame's token is reused       */
@@ -191,9 +192,16 @@ SALICACHE_API int salicache_source_frames(salicache_ctx* ctx, const uint8_t* d_d
  *   int8_codes  i8  [L][2][cap_int8][HD]      int8_scale f16 [L][2][cap_int8][ng]
  *   int4_codes  u8  [L][2][cap_int4][HD/2]    int4_sz    f16 [L][2][cap_int4][ng][2]  (scale, zero)
  * The j-th token of a frame's tier list lives in row (row_offset + j) % cap when ring != 0
- * (oldest rows are overwritten: oldest-first eviction; one call must not store more than cap
- * rows in a pool, or rows of the same call overwrite each other in unspecified order), else in
- * row row_offset + j, and rows at or past cap are dropped with E_CAPACITY in the status word. */
+ * (row offsets are absolute positions; the oldest rows are overwritten: oldest-first eviction
+ * under a fixed budget; when one call stores more than cap rows in a pool, the rows that a later
+ * row of the same call lands on are skipped, so that the newest cap rows are what the pool
+ * holds), else in row row_offset + j, and rows at or past cap are dropped with E_CAPACITY in
+ * the status word.
+ *   d_fill      optional (NULL = no check): DEVICE i64 [3], the running fill salicache_select
+ *               maintains (rows ever stored per tier: FP16, INT8, INT4).  With ring != 0 it tells
+ *               salicache_unpack_kv which rows still exist: a row with row_offset + j <
+ *               fill - cap has been overwritten by a newer frame; it is not read, the output row
+ *               is zeroed, and E_EVICTED is recorded in the status word. */
 typedef struct salicache_pools {
     void* fp16_pool;
     void* int8_codes;
@@ -202,6 +210,7 @@ typedef struct salicache_pools {
     void* int4_sz;
     int64_t cap_fp16, cap_int8, cap_int4;
     int32_t ring;
+    const int64_t* d_fill;
 } salicache_pools;
 
 /*
@@ -221,12 +230,37 @@ SALICACHE_API int salicache_pack_kv(salicache_ctx* ctx, const void* d_K, const v
  * Just-in-time dequantisation (Sec. III-C) into dense f16 d_K_out, d_V_out [B][L][N_tok][HD].
  * INT8: fp16(q*s); INT4: fp16(q*s + zero) (multiply, then add); FP16 rows are bit copies;
  * PRUNE rows are zeroed when zero_fill_pruned != 0, otherwise untouched; REUSE rows are left
- * untouched (the caller resolves them through its source-frame table).
+ * untouched (the caller resolves them through its source-frame table).  With ring pools and
+ * pools->d_fill given, rows that have been overwritten are zeroed instead of read (deferred
+ * E_EVICTED).  Errors: E_NULL, E_SHAPE, E_ALIGN, E_CUDA; deferred E_CAPACITY, E_EVICTED.
  */
 SALICACHE_API int salicache_unpack_kv(salicache_ctx* ctx, const salicache_pools* pools, const int32_t* d_idx,
                         const int32_t* d_counts, const uint8_t* d_decision, const int64_t* d_row_offset, int B,
                         int zero_fill_pruned, void* d_K_out, void* d_V_out, int64_t frame_stride,
                         void* cuda_stream);
+
+/*
+ * Which stored frames a budgeted cache still holds (fixed memory budget, Sec. IV-A; ring pools with
+ * oldest-first eviction).  d_resident[b] = 1 when every row frame b stored is still in the pools at the
+ * running fill pools->d_fill (required): per tier, the frame stored nothing, or it fits the ring and
+ * row_offset >= fill - cap (linear pools: row_offset + count <= cap).  A frame's record is evicted as a
+ * whole: one overwritten tier makes it non-resident.
+ *   d_counts i32 [B][5], d_row_offset i64 [B][3] as written by salicache_select; d_resident u8 [B] written.
+ * Errors: E_NULL, E_SHAPE, E_CUDA.
+ */
+SALICACHE_API int salicache_frames_resident(salicache_ctx* ctx, const int32_t* d_counts, const int64_t* d_row_offset, int B,
+                                            const salicache_pools* pools, uint8_t* d_resident, void* cuda_stream);
+
+/*
+ * A reused token lives as long as the frame that holds its entry (Alg. 1 line 7: a pointer; a root is
+ * evicted together with every alias that points to it): d_live[b][i] = d_resident_table[d_src[b][i] -
+ * first_frame], and 0 when the source frame lies outside the table.
+ *   d_src i32 [B][N_tok] from salicache_source_frames; d_resident_table u8 [n_table] describes frames
+ *   first_frame .. first_frame + n_table - 1; d_live u8 [B][N_tok] written.
+ * Errors: E_NULL, E_SHAPE, E_CUDA.
+ */
+SALICACHE_API int salicache_tokens_live(salicache_ctx* ctx, const int32_t* d_src, int B, int first_frame,
+                                        const uint8_t* d_resident_table, int n_table, uint8_t* d_live, void* cuda_stream);
 
 /*
  * The spatial score without any allocation.  (The paper has no counterpart: this entry point

@@ -399,15 +399,37 @@ def pack_frame(K16: np.ndarray, V16: np.ndarray, idx, counts, off, pools: Pools)
         C.c_int64(pools.cap8), _p(pools.int4_codes), _p(pools.int4_sz), C.c_int64(pools.cap4)))
 
 
-def unpack_frame(n_tok: int, idx, counts, decision, off, pools: Pools, zero_fill_pruned: bool, K_out, V_out) -> int:
+def unpack_frame(n_tok: int, idx, counts, decision, off, pools: Pools, zero_fill_pruned: bool, K_out, V_out, fill=None) -> int:
+    """`fill` (running fill per tier, int64 [3]): with ring pools, rows overwritten since are zeroed and -9 returned."""
     idx, counts, off = _c(idx, np.int32), _c(counts, np.int32), _c(off, np.int64)
     decision = _c(decision, np.uint8)
     assert K_out.dtype == np.uint16 and K_out.flags.c_contiguous and V_out.flags.c_contiguous
+    fill = None if fill is None else _c(fill, np.int64)
     return int(lib().oracle_unpack_frame(
         C.c_int(pools.L), C.c_int(n_tok), C.c_int(pools.HD), C.c_int(pools.G), _p(idx), _p(counts), _p(decision),
         _p(off), C.c_int(pools.ring), _p(pools.fp16_pool), C.c_int64(pools.cap16), _p(pools.int8_codes),
         _p(pools.int8_scale), C.c_int64(pools.cap8), _p(pools.int4_codes), _p(pools.int4_sz), C.c_int64(pools.cap4),
-        C.c_int(int(zero_fill_pruned)), _p(K_out), _p(V_out)))
+        C.c_int(int(zero_fill_pruned)), _p(fill) if fill is not None else C.c_void_p(None), _p(K_out), _p(V_out)))
+
+
+def frames_resident(counts_all, off_all, caps, ring: bool, fill) -> np.ndarray:
+    """resident u8 [T]: 1 when every row frame t stored is still in the (ring) pools at running fill `fill`."""
+    c = _c(np.asarray(counts_all).reshape(-1, 5), np.int32)
+    o = _c(np.asarray(off_all).reshape(-1, 3), np.int64)
+    caps, fill = _c(caps, np.int64), _c(fill, np.int64)
+    out = np.empty(c.shape[0], np.uint8)
+    lib().oracle_frames_resident(_p(c), _p(o), C.c_int(c.shape[0]), _p(caps), C.c_int(int(ring)), _p(fill), _p(out))
+    return out
+
+
+def tokens_live(src: np.ndarray, first: int, resident: np.ndarray) -> np.ndarray:
+    """live u8 [T][n_tok]: 1 when the frame that holds the token's entry (src, reuse chains resolved) is resident;
+    resident[k] describes frame first + k."""
+    src, resident = _c(src, np.int32), _c(resident, np.uint8)
+    T, n = src.shape
+    out = np.empty((T, n), np.uint8)
+    lib().oracle_tokens_live(_p(src), C.c_int(T), C.c_int(n), C.c_int(first), _p(resident), C.c_int(resident.shape[0]), _p(out))
+    return out
 
 
 def attend(q16: np.ndarray, pools: "Pools", n_rows) -> np.ndarray:

@@ -878,11 +878,19 @@ EXPORT int oracle_pack_frame(const uint16_t* K, const uint16_t* V, int L, int n_
 /* when zero_fill_pruned; REUSE rows are left untouched (the caller resolves   */
 /* them through the source-frame table).                                       */
 /* ------------------------------------------------------------------------- */
+/* Ring pools under a budget: row r (absolute position) of a tier is still in the pool while          */
+/* fill - cap <= r, fill being the tier's running fill (rows ever stored).  With fill_or_null given,  */
+/* a row that has been overwritten since (oldest-first eviction) is not read: its output row is       */
+/* zeroed and the return value is -9.                                                                 */
+static int row_evicted(int64_t off, int64_t j, int64_t cap, int ring, const int64_t* fill_or_null, int tier) {
+    return ring && fill_or_null && off + j < fill_or_null[tier] - cap;
+}
+
 EXPORT int oracle_unpack_frame(int L, int n_tok, int HD, int G, const int32_t* idx, const int32_t* counts,
                                const uint8_t* decision, const int64_t* off, int ring, const uint16_t* fp16_pool,
                                int64_t cap16, const int8_t* int8_codes, const uint16_t* int8_scale, int64_t cap8,
                                const uint8_t* int4_codes, const uint16_t* int4_sz, int64_t cap4,
-                               int zero_fill_pruned, uint16_t* K_out, uint16_t* V_out) {
+                               int zero_fill_pruned, const int64_t* fill_or_null, uint16_t* K_out, uint16_t* V_out) {
     int status = 0;
     int ng = HD / G;
     int n16 = counts[4], n8 = counts[3], n4 = counts[2];
@@ -894,12 +902,18 @@ EXPORT int oracle_unpack_frame(int L, int n_tok, int HD, int G, const int32_t* i
             for (int j = 0; j < n16; ++j) {
                 int64_t r = pool_row(off[0], j, cap16, ring);
                 if (r < 0) { status = -1; continue; }
+                if (row_evicted(off[0], j, cap16, ring, fill_or_null, 0)) {
+                    memset(dst + (size_t)idx[0 * n_tok + j] * HD, 0, (size_t)HD * 2);
+                    status = -9;
+                    continue;
+                }
                 memcpy(dst + (size_t)idx[0 * n_tok + j] * HD, fp16_pool + (plane * cap16 + r) * HD, (size_t)HD * 2);
             }
             for (int j = 0; j < n8; ++j) {
                 int64_t r = pool_row(off[1], j, cap8, ring);
                 if (r < 0) { status = -1; continue; }
                 uint16_t* row = dst + (size_t)idx[1 * n_tok + j] * HD;
+                if (row_evicted(off[1], j, cap8, ring, fill_or_null, 1)) { memset(row, 0, (size_t)HD * 2); status = -9; continue; }
                 for (int g = 0; g < ng; ++g)
                     oracle_dequant_int8_group(int8_codes + (plane * cap8 + r) * HD + g * G, G,
                                               int8_scale[(plane * cap8 + r) * ng + g], row + g * G);
@@ -908,6 +922,7 @@ EXPORT int oracle_unpack_frame(int L, int n_tok, int HD, int G, const int32_t* i
                 int64_t r = pool_row(off[2], j, cap4, ring);
                 if (r < 0) { status = -1; continue; }
                 uint16_t* row = dst + (size_t)idx[2 * n_tok + j] * HD;
+                if (row_evicted(off[2], j, cap4, ring, fill_or_null, 2)) { memset(row, 0, (size_t)HD * 2); status = -9; continue; }
                 for (int g = 0; g < ng; ++g)
                     oracle_dequant_int4_group(int4_codes + (plane * cap4 + r) * (HD / 2) + g * (G / 2), G,
                                               int4_sz[((plane * cap4 + r) * ng + g) * 2],
@@ -1083,4 +1098,44 @@ EXPORT int64_t oracle_stored_bytes(const int64_t* counts, int64_t T, int L, int 
     int64_t payload = (int64_t)L * 2 * (n16 * HD * 2 + n8 * (HD + 2 * ng) + n4 * (HD / 2 + 4 * ng));
     int64_t meta = T * ((int64_t)n_tok + 8 + 24 + 20) + 4 * (n4 + n8 + n16);
     return payload + meta;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Which stored frames a budgeted cache still holds (the paper runs its        */
+/* baselines under a fixed memory budget, Sec. IV-A; reading for this store:   */
+/* per-tier ring pools, oldest rows overwritten first).  Frame t is resident   */
+/* in tier k when it stored no row there, or when its first row has not been   */
+/* overwritten and the frame fits the ring at all:                             */
+/*   n_tk == 0  or  (n_tk <= cap_k and off_tk >= fill_k - cap_k)               */
+/* (linear pools, ring == 0: off_tk + n_tk <= cap_k).  A frame's record is     */
+/* evicted as a whole: resident[t] = 1 only if that holds in all three tiers.  */
+/* counts [T][5] by code, off [T][3] / cap [3] / fill [3] in the order FP16,   */
+/* INT8, INT4.                                                                 */
+/* ------------------------------------------------------------------------- */
+EXPORT void oracle_frames_resident(const int32_t* counts, const int64_t* off, int T, const int64_t* cap, int ring,
+                                   const int64_t* fill, uint8_t* resident) {
+    const int code[3] = {4, 3, 2};
+    for (int t = 0; t < T; ++t) {
+        int ok = 1;
+        for (int k = 0; k < 3; ++k) {
+            int64_t n = counts[(size_t)t * 5 + code[k]], o = off[(size_t)t * 3 + k];
+            if (n == 0) continue;
+            if (ring) ok = ok && n <= cap[k] && o >= fill[k] - cap[k];
+            else ok = ok && o + n <= cap[k];
+        }
+        resident[t] = (uint8_t)ok;
+    }
+}
+
+/* A reused token lives as long as the frame that holds its entry: live[t][i] = */
+/* resident[src[t][i] - first] (0 when the source frame precedes the table),    */
+/* src being the source-frame table of oracle_source_frames: a root is evicted  */
+/* together with every alias that points to it.  Pruned tokens have no entry;   */
+/* they are reported live when their own frame is resident.                      */
+EXPORT void oracle_tokens_live(const int32_t* src, int T, int n_tok, int first, const uint8_t* resident, int n_table,
+                               uint8_t* live) {
+    for (size_t i = 0; i < (size_t)T * n_tok; ++i) {
+        int64_t k = (int64_t)src[i] - first;
+        live[i] = (k >= 0 && k < n_table) ? resident[k] : 0;
+    }
 }

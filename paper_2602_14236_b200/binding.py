@@ -13,7 +13,7 @@ from . import build as _build
 
 REUSE, PRUNE, INT4, INT8, FP16 = 0, 1, 2, 3, 4
 
-E_NULL, E_SHAPE, E_ALIGN, E_PARAM, E_CUDA, E_CAPACITY, E_NOCONVERGE, E_NOMEM = -1, -2, -3, -4, -5, -6, -7, -8
+E_NULL, E_SHAPE, E_ALIGN, E_PARAM, E_CUDA, E_CAPACITY, E_NOCONVERGE, E_NOMEM, E_EVICTED = -1, -2, -3, -4, -5, -6, -7, -8, -9
 
 
 class SalicacheError(RuntimeError):
@@ -43,6 +43,7 @@ class Pools(C.Structure):
         ("fp16_pool", C.c_void_p), ("int8_codes", C.c_void_p), ("int8_scale", C.c_void_p),
         ("int4_codes", C.c_void_p), ("int4_sz", C.c_void_p),
         ("cap_fp16", C.c_int64), ("cap_int8", C.c_int64), ("cap_int4", C.c_int64), ("ring", C.c_int32),
+        ("d_fill", C.c_void_p),
     ]
 
 
@@ -52,6 +53,7 @@ EXPORTS = [
     "salicache_pack_kv", "salicache_unpack_kv", "salicache_poll_status", "salicache_saliency_noalloc",
     "salicache_frame_redundancy", "salicache_source_frames", "salicache_diff_score", "salicache_attend",
     "salicache_select_anchored", "salicache_select_ranked", "salicache_attend_gqa", "salicache_select_anchored_batch",
+    "salicache_frames_resident", "salicache_tokens_live",
 ]
 
 _lib = None
@@ -92,6 +94,8 @@ def lib():
         _lib.salicache_attend.argtypes = [vp, vp, C.POINTER(Pools), vp, vp, vp]
         _lib.salicache_attend_gqa.argtypes = [vp, vp, i32, C.POINTER(Pools), vp, vp, vp]
         _lib.salicache_saliency_noalloc.argtypes = [C.POINTER(Params), vp, i32, vp, vp, vp]
+        _lib.salicache_frames_resident.argtypes = [vp, vp, vp, i32, C.POINTER(Pools), vp, vp]
+        _lib.salicache_tokens_live.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
     return _lib
 
 
@@ -239,6 +243,16 @@ def salicache_attend_gqa(ctx: Context, d_q, q_per_kv: int, pools: Pools, d_fill,
                                       _stream(stream)), "salicache_attend_gqa")
 
 
+def salicache_frames_resident(ctx: Context, d_counts, d_row_offset, B: int, pools: Pools, d_resident, stream=None):
+    _check(lib().salicache_frames_resident(ctx.handle, _ptr(d_counts), _ptr(d_row_offset), B, C.byref(pools), _ptr(d_resident),
+                                           _stream(stream)), "salicache_frames_resident")
+
+
+def salicache_tokens_live(ctx: Context, d_src, B: int, first_frame: int, d_resident_table, n_table: int, d_live, stream=None):
+    _check(lib().salicache_tokens_live(ctx.handle, _ptr(d_src), B, first_frame, _ptr(d_resident_table), n_table, _ptr(d_live),
+                                       _stream(stream)), "salicache_tokens_live")
+
+
 def salicache_poll_status(ctx: Context, stream=None) -> int:
     return int(lib().salicache_poll_status(ctx.handle, _stream(stream)))
 
@@ -246,7 +260,8 @@ def salicache_poll_status(ctx: Context, stream=None) -> int:
 class PoolSet:
     """Device pools as torch tensors (memory only) plus the C struct that points at them."""
 
-    def __init__(self, L: int, HD: int, cap16: int, cap8: int, cap4: int, ring: bool = False, device="cuda", G: int = 128):
+    def __init__(self, L: int, HD: int, cap16: int, cap8: int, cap4: int, ring: bool = False, device="cuda", G: int = 128,
+                 fill=None):
         import torch
         ng = HD // G
         self.L, self.HD, self.G = L, HD, G
@@ -258,7 +273,9 @@ class PoolSet:
         self.int4_codes = z((L, 2, max(cap4, 1), HD // 2), torch.uint8)
         self.int4_sz = z((L, 2, max(cap4, 1), ng, 2), torch.float16)
         self.c = Pools(self.fp16_pool.data_ptr(), self.int8_codes.data_ptr(), self.int8_scale.data_ptr(),
-                       self.int4_codes.data_ptr(), self.int4_sz.data_ptr(), cap16, cap8, cap4, int(ring))
+                       self.int4_codes.data_ptr(), self.int4_sz.data_ptr(), cap16, cap8, cap4, int(ring),
+                       None if fill is None else fill.data_ptr())
+        self.fill = fill              # keeps the tensor alive
 
     def nbytes(self) -> int:
         return sum(t.numel() * t.element_size() for t in

@@ -63,6 +63,7 @@ const char* salicache_strerror(int status) {
         case SALICACHE_E_CAPACITY: return "tier pool too small; rows were dropped";
         case SALICACHE_E_NOCONVERGE: return "edge hysteresis hit its iteration cap";
         case SALICACHE_E_NOMEM: return "scratch allocation failed";
+        case SALICACHE_E_EVICTED: return "rows asked for have been overwritten in a ring pool; zeros were returned";
         default: return "unknown status";
     }
 }
@@ -354,6 +355,21 @@ int salicache_unpack_kv(salicache_ctx* c, const salicache_pools* pools, const in
     if (!aligned16(d_K_out) || !aligned16(d_V_out)) return SALICACHE_E_ALIGN;
     return sc_unpack(c, pools, d_idx, d_counts, d_decision, d_row_offset, B, zero_fill_pruned, d_K_out, d_V_out,
                      frame_stride, (cudaStream_t)cuda_stream);
+}
+
+int salicache_frames_resident(salicache_ctx* c, const int32_t* d_counts, const int64_t* d_row_offset, int B,
+                              const salicache_pools* pools, uint8_t* d_resident, void* cuda_stream) {
+    if (!c || !d_counts || !d_row_offset || !d_resident || !pools) return SALICACHE_E_NULL;
+    if (pools->ring && !pools->d_fill) return SALICACHE_E_NULL;
+    if (pools->cap_fp16 < 0 || pools->cap_int8 < 0 || pools->cap_int4 < 0 || B < 0) return SALICACHE_E_SHAPE;
+    return sc_frames_resident(c, d_counts, d_row_offset, B, pools, d_resident, (cudaStream_t)cuda_stream);
+}
+
+int salicache_tokens_live(salicache_ctx* c, const int32_t* d_src, int B, int first_frame, const uint8_t* d_resident_table,
+                          int n_table, uint8_t* d_live, void* cuda_stream) {
+    if (!c || !d_src || !d_resident_table || !d_live) return SALICACHE_E_NULL;
+    if (B < 0 || n_table < 0 || first_frame < 0) return SALICACHE_E_SHAPE;
+    return sc_tokens_live(c, d_src, B, first_frame, d_resident_table, n_table, d_live, (cudaStream_t)cuda_stream);
 }
 
 int salicache_attend(salicache_ctx* c, const void* d_q, const salicache_pools* pools, const int64_t* d_fill, float* d_out,

@@ -73,6 +73,10 @@ int sc_sources(salicache_ctx* c, const uint8_t* d_decision, int B, int first_fra
                cudaStream_t st);
 int sc_frame_redundancy(salicache_ctx* c, const float* d_deltaP, int B, int first_has_no_prev, uint8_t* d_frame_redundant,
                         cudaStream_t st);
+int sc_frames_resident(salicache_ctx* c, const int32_t* d_counts, const int64_t* d_row_offset, int B,
+                       const salicache_pools* pools, uint8_t* d_resident, cudaStream_t st);
+int sc_tokens_live(salicache_ctx* c, const int32_t* d_src, int B, int first_frame, const uint8_t* d_table, int n_table,
+                   uint8_t* d_live, cudaStream_t st);
 // ranked.cu
 int sc_select_ranked(salicache_ctx* c, const float* d_deltaP, const float* d_s, int B, int first_has_no_prev, int pm16,
                      int pm8, int pm4, uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts, uint8_t* d_frame_redundant,

@@ -27,6 +27,7 @@ struct PoolPtrs {
     uint8_t* int4_sz;
     long long cap0, cap1, cap2;
     int ring;
+    const long long* fill;         // running fill per tier, or null
 };
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
@@ -120,9 +121,13 @@ struct Unit {
     long long cap;
 };
 
+// lim[tier] (ring pools): rows at an absolute position below it are gone: overwritten by a later row of the same
+// call when storing, by newer frames when reading back.  Such rows come back as row -2; rows past the capacity of
+// a linear pool as row -1.
 __device__ __forceinline__ Unit decode_unit(uint32_t u, const int* pre, int B, uint32_t planes,
                                             const int32_t* __restrict__ counts, const int32_t* __restrict__ idx,
-                                            const long long* __restrict__ row_offset, int n_tok, const PoolPtrs& pp) {
+                                            const long long* __restrict__ row_offset, int n_tok, const PoolPtrs& pp,
+                                            const long long* lim) {
     Unit r;
     const uint32_t q = u / planes;      // lies in [pre[b], pre[b+1]) of exactly one frame
     int lo = 0, hi = B;                 // largest b with pre[b] <= q
@@ -141,10 +146,31 @@ __device__ __forceinline__ Unit decode_unit(uint32_t u, const int* pre, int B, u
     else { r.tier = 2; j -= n16 + n8; r.cap = pp.cap2; }
     r.tok = idx[((size_t)lo * 3 + r.tier) * n_tok + j];
     long long row = row_offset[(size_t)lo * 3 + r.tier] + j;
-    if (pp.ring) row = r.cap > 0 ? row % r.cap : -1;
+    if (pp.ring) row = r.cap <= 0 ? -1 : (row < lim[r.tier] ? -2 : row % r.cap);
     else if (row >= r.cap) row = -1;
     r.row = row;
     return r;
+}
+
+// The limits above, into shared memory (3 values), behind the prefix table.
+//   storing: the call ends at absolute row end = row_offset of its last frame + that frame's count; a row
+//            below end - cap is overwritten by a later row of this call;
+//   reading: rows below fill - cap have been overwritten since (no limit when the caller gave no fill).
+__device__ __forceinline__ void build_limits(bool storing, const int32_t* __restrict__ counts,
+                                             const long long* __restrict__ row_offset, int B, const PoolPtrs& pp,
+                                             long long* lim) {
+    if (threadIdx.x < 3) {
+        const int t = threadIdx.x;
+        const int code = t == 0 ? SALICACHE_FP16 : (t == 1 ? SALICACHE_INT8 : SALICACHE_INT4);
+        const long long cap = t == 0 ? pp.cap0 : (t == 1 ? pp.cap1 : pp.cap2);
+        long long v = -0x7fffffffffffffffll;
+        if (pp.ring) {
+            if (storing) v = row_offset[(size_t)(B - 1) * 3 + t] + counts[(B - 1) * 5 + code] - cap;
+            else if (pp.fill) v = pp.fill[t] - cap;
+        }
+        lim[t] = v;
+    }
+    __syncthreads();
 }
 
 // ---- pack ---------------------------------------------------------------------------------------
@@ -300,22 +326,24 @@ k_pack(const __half* __restrict__ K, const __half* __restrict__ V, KvGeom g, con
        const int32_t* __restrict__ counts, const long long* __restrict__ row_offset, PoolPtrs pp,
        int* __restrict__ status) {
     extern __shared__ int pre[];
+    __shared__ long long lim[3];
     build_prefix(counts, g.B, pre);
+    build_limits(true, counts, row_offset, g.B, pp, lim);
     const uint32_t planes = 2u * (uint32_t)g.L;
     const uint32_t n_units = (uint32_t)pre[g.B] * planes;      // < 2^31: checked on the host
     const int lane = threadIdx.x & 31;
     const uint32_t warp0 = blockIdx.x * KV_WARPS + (threadIdx.x >> 5);
     const uint32_t wstride = gridDim.x * KV_WARPS;
     if (warp0 >= n_units) return;
-    Unit un = decode_unit(warp0, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp);
+    Unit un = decode_unit(warp0, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp, lim);
     uint4 v[ITERS];
     if (un.row >= 0) load_piece<ITERS>(v, K, V, un, 0, g, lane);
     for (uint32_t u = warp0; u < n_units; u += wstride) {
         const bool more = u + wstride < n_units;
         Unit nxt = un;
-        if (more) nxt = decode_unit(u + wstride, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp);
+        if (more) nxt = decode_unit(u + wstride, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp, lim);
         if (un.row >= 0) pack_piece<ITERS, RG>(v, un, 0, g, pp, lane);
-        else if (lane == 0) atomicMin(status, SALICACHE_E_CAPACITY);
+        else if (un.row == -1 && lane == 0) atomicMin(status, SALICACHE_E_CAPACITY);
         if (more && nxt.row >= 0) load_piece<ITERS>(v, K, V, nxt, 0, g, lane);
         un = nxt;
     }
@@ -328,21 +356,29 @@ k_unpack(__half* __restrict__ K, __half* __restrict__ V, KvGeom g, const int32_t
          const int32_t* __restrict__ counts, const long long* __restrict__ row_offset, PoolPtrs pp,
          int* __restrict__ status) {
     extern __shared__ int pre[];
+    __shared__ long long lim[3];
     build_prefix(counts, g.B, pre);
+    build_limits(false, counts, row_offset, g.B, pp, lim);
     const uint32_t planes = 2u * (uint32_t)g.L;
     const uint32_t n_units = (uint32_t)pre[g.B] * planes;      // < 2^31: checked on the host
     const int lane = threadIdx.x & 31;
     const uint32_t warp0 = blockIdx.x * KV_WARPS + (threadIdx.x >> 5);
     const uint32_t wstride = gridDim.x * KV_WARPS;
     for (uint32_t u = warp0; u < n_units; u += wstride) {
-        Unit un = decode_unit(u, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp);
-        if (un.row < 0) {
+        Unit un = decode_unit(u, pre, g.B, planes, counts, idx, row_offset, g.n_tok, pp, lim);
+        if (un.row == -1) {
             if (lane == 0) atomicMin(status, SALICACHE_E_CAPACITY);
             continue;
         }
         const int layer = un.plane >> 1, kv = un.plane & 1;
         __half* dst_h = (kv ? V : K) + (size_t)un.b * g.frame_stride + ((size_t)layer * g.n_tok + un.tok) * g.HD;
         uint4* dst = reinterpret_cast<uint4*>(dst_h) + lane;
+        if (un.row < 0) {                  // overwritten since by a newer frame: zeros, never another frame's row
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) st_stream(dst + i * 32, make_uint4(0, 0, 0, 0));
+            if (lane == 0) atomicMin(status, SALICACHE_E_EVICTED);
+            continue;
+        }
         const size_t prow = (size_t)un.plane * un.cap + un.row;
         if (un.tier == 0) {
             const uint4* src = reinterpret_cast<const uint4*>(pp.fp16_pool + prow * (size_t)g.HD * 2) + lane;
@@ -428,6 +464,7 @@ PoolPtrs make_pools(const salicache_pools* p) {
     pp.cap1 = p->cap_int8;
     pp.cap2 = p->cap_int4;
     pp.ring = p->ring;
+    pp.fill = (const long long*)p->d_fill;
     return pp;
 }
 

@@ -142,7 +142,54 @@ __global__ void k_row_offsets(const int32_t* __restrict__ counts, int B, int64_t
     fill[t] = acc;
 }
 
+// Residency of stored frames in budgeted pools: one thread per frame.
+__global__ void k_frames_resident(const int32_t* __restrict__ counts, const int64_t* __restrict__ row_offset, int B,
+                                  long long cap0, long long cap1, long long cap2, int ring, const int64_t* __restrict__ fill,
+                                  uint8_t* __restrict__ resident) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const int code[3] = {SALICACHE_FP16, SALICACHE_INT8, SALICACHE_INT4};
+    const long long cap[3] = {cap0, cap1, cap2};
+    bool ok = true;
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        const long long n = counts[(size_t)b * 5 + code[k]], o = row_offset[(size_t)b * 3 + k];
+        if (n == 0) continue;
+        if (ring) ok = ok && n <= cap[k] && o >= fill[k] - cap[k];
+        else ok = ok && o + n <= cap[k];
+    }
+    resident[b] = ok ? 1 : 0;
+}
+
+__global__ void k_tokens_live(const int32_t* __restrict__ src, long long n, int first, const uint8_t* __restrict__ table,
+                              int n_table, uint8_t* __restrict__ live) {
+    const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const long long k = (long long)src[i] - first;
+    live[i] = (k >= 0 && k < n_table) ? table[k] : 0;
+}
+
 }  // namespace
+
+int sc_frames_resident(salicache_ctx* c, const int32_t* d_counts, const int64_t* d_row_offset, int B,
+                       const salicache_pools* pools, uint8_t* d_resident, cudaStream_t st) {
+    if (B == 0) return SALICACHE_OK;
+    k_frames_resident<<<(B + 127) / 128, 128, 0, st>>>(d_counts, d_row_offset, B, pools->cap_fp16, pools->cap_int8,
+                                                       pools->cap_int4, pools->ring, pools->d_fill, d_resident);
+    c->launches++;
+    SC_CHECK(cudaGetLastError());
+    return SALICACHE_OK;
+}
+
+int sc_tokens_live(salicache_ctx* c, const int32_t* d_src, int B, int first_frame, const uint8_t* d_table, int n_table,
+                   uint8_t* d_live, cudaStream_t st) {
+    const long long n = (long long)B * c->n_tok;
+    if (n == 0) return SALICACHE_OK;
+    k_tokens_live<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(d_src, n, first_frame, d_table, n_table, d_live);
+    c->launches++;
+    SC_CHECK(cudaGetLastError());
+    return SALICACHE_OK;
+}
 
 int sc_frame_redundancy(salicache_ctx* c, const float* d_deltaP, int B, int first_has_no_prev, uint8_t* d_frame_redundant,
                         cudaStream_t st) {
