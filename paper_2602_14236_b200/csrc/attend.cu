@@ -966,7 +966,7 @@ k_attend_int8_gqa(const __half* __restrict__ q, AtPools pp, const long long* __r
 
 // ---- FP16 rows, grouped queries: the rows need no expansion, so a tile is 16 loads of 16 bytes per lane, two
 // byte permutes per value operand and 16 matrix instructions for up to 4 queries.  One query per key/value
-// head keeps the scalar kernel above (k_attend_partial), which already runs close to the memory bandwidth.
+// head is the group of one: it runs this kernel too, close to the memory bandwidth.
 struct G16Tile {
     uint4 ka[4], kb[4];            // keys of rows g8 and g8 + 8: dimensions 32 c4 .. + 31
     uint4 v[4][2];                 // values of rows c4, c4 + 4, c4 + 8, c4 + 12: dimensions 16 g8 .. + 15

@@ -36,7 +36,9 @@ def test_flow_score_matches_oracle_on_workload_1(wl1_frames, wl1_oracle_scores):
     ctx = _ctx()
     dP, s, fl = gu.gpu_scores(ctx, wl1_frames, want_flow=True)
     rdP, rs, rfl = wl1_oracle_scores
-    assert np.abs(fl - rfl).max() < 2e-5          # dense field (px): single-precision terms and window sums, double solve
+    # dense field (px): an auxiliary check beside the contract's tolerance on dP.  Single-precision terms, window sums
+    # of 225 terms and a compensated 2x2 solve leave about 5e-6 px on fields of up to 3 px; the bound is twice that.
+    assert np.abs(fl - rfl).max() < 1e-5
     gu.assert_scores_close(dP[1:], rdP[1:], "dP")
     gu.assert_scores_close(s, rs, "s")
 
