@@ -20,7 +20,6 @@ void free_scratch(salicache_ctx* c) {
         if (c->coef[l]) cudaFree(c->coef[l]);
     }
     if (c->gh_a) cudaFree(c->gh_a);
-    if (c->gh_b) cudaFree(c->gh_b);
     if (c->flow_a) cudaFree(c->flow_a);
     if (c->flow_b) cudaFree(c->flow_b);
     if (c->bits_kept) cudaFree(c->bits_kept);
@@ -120,7 +119,6 @@ int salicache_create(salicache_ctx** out, const salicache_params* p) {
         ok = ok && cudaMemset(c->coef[l], 0, cbytes) == cudaSuccess;
     }
     ok = ok && cudaMalloc(&c->gh_a, (size_t)c->chunk * 5 * P0 * sizeof(float)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->gh_b, (size_t)c->chunk * 5 * P0 * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->flow_a, (size_t)c->chunk * 2 * P0 * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->flow_b, (size_t)c->chunk * 2 * P0 * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->bits_kept, (size_t)c->chunk * p->H * words * sizeof(uint32_t)) == cudaSuccess;

@@ -37,9 +37,8 @@ struct salicache_ctx {
     // flow scratch (sized for the largest plane)
     float* pyr[3];             // [chunk+1][h_l*w_l]
     float* coef[3];            // expansion coefficients: float4 [2*chunk][h_l*w_l] + pad, then float [2*chunk][h_l*w_l] + pad
-    float* gh_a;               // [chunk][5][H*W] normal-equation terms, ping
-    float* gh_b;               //                                         pong
-    float* flow_a;             // [chunk][2][H*W] displacement carried between levels
+    float* gh_a;               // [chunk][5][H*W] normal-equation terms of the current update
+    float* flow_a;             // [chunk][H*W] (du, dv) records: the field of the level at work and of the coarser one
     float* flow_b;
     // saliency scratch
     uint32_t* bits_kept;       // [chunk][H][Ww]  NMS-kept weak or strong pixels

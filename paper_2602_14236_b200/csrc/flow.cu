@@ -7,10 +7,10 @@
 // positions are exact; the patch reduction is double.  The effect on dP stays more than an order of
 // magnitude below the 1e-4 relative tolerance on every workload.
 //
-// One displacement update = window sums of (G, h) + a 2x2 solve.  k_flow_update does that on a 56x28
-// (or 28x28) tile with separable sums (columns from registers, rows from shared memory) and, fused
-// behind the solve, the (G, h) of the NEXT update at the same pixels (which needs no halo), or the patch
-// scores after the last update.
+// One displacement update = the terms (G, h) of every pixel at the current field (k_flow_terms, one pixel
+// per thread) + window sums and a 2x2 solve (k_flow_update, on a 56x28 or 28x28 tile with separable sums:
+// columns from registers, rows from shared memory), which leaves the new field or, after the last update,
+// the patch scores.
 #include <math.h>
 
 #include "common.cuh"
@@ -221,10 +221,10 @@ __device__ __forceinline__ float det2(float a, float b, float c, float d) {
     return f + e;
 }
 
-// ---- (G, h) of the first update of a level.  Prior: zero at the coarsest level, else the coarser
-// level's field carried over as d = 2 * bilinear(d_coarse) at ((x+1/2)/2 - 1/2, (y+1/2)/2 - 1/2), clamped to the
-// coarse image.  For a fine coordinate x that position is x/2 - 1/4: left tap (x-1) >> 1 with weight 3/4 of the
-// right tap for even x and 1/4 for odd x; at x = 0 and at the last fine pixel the clamp puts it on the tap itself.
+// ---- prior of a level from the coarser level's field: d = 2 * bilinear(d_coarse) at
+// ((x+1/2)/2 - 1/2, (y+1/2)/2 - 1/2), clamped to the coarse image.  For a fine coordinate x that position is
+// x/2 - 1/4: left tap (x-1) >> 1 with weight 3/4 on the right tap for even x and 1/4 for odd x; at x = 0 and at
+// the last fine pixel the clamp puts it on the tap itself.
 __device__ __forceinline__ void coarse_tap(int x, int nc, int& i0, int& i1, float& f) {
     i0 = (x - 1) >> 1;
     f = (x & 1) ? 0.25f : 0.75f;
@@ -233,31 +233,56 @@ __device__ __forceinline__ void coarse_tap(int x, int nc, int& i0, int& i1, floa
     if (i1 > nc - 1) { i1 = nc - 1; f = 0.0f; }      // x = 2 nc - 1: position nc - 3/4, clamped to nc - 1
 }
 
+// One thread per coarse pixel: its 2x2 block of fine pixels, written as two 16-byte stores.
 __global__ void __launch_bounds__(256)
-k_flow_gh(const float4* __restrict__ q1, const float* __restrict__ r1, const float4* __restrict__ q2,
-          const float* __restrict__ r2, int h, int w, unsigned w_inv, const float* __restrict__ d_coarse, size_t flow_stride,
-          float* __restrict__ gh, size_t gh_stride, int n_pairs) {
+k_flow_prior(const float2* __restrict__ d_coarse, int hc, int wc, unsigned wc_inv, size_t d_stride, float2* __restrict__ d_fine,
+             int n_pairs) {
+    const int Pc = hc * wc;
+    const int f = blockIdx.y, r = blockIdx.x * blockDim.x + threadIdx.x;        // grid: (coarse pixels, pairs)
+    if (r >= Pc || f >= n_pairs) return;
+    const int yc = (int)__umulhi((unsigned)r, wc_inv), xc = r - yc * wc;       // wc_inv = ceil(2^32 / wc): exact here
+    const float2* src = d_coarse + (size_t)f * d_stride;
+    float2* dst = d_fine + (size_t)f * d_stride;
+    const int w = 2 * wc;
+    int xi0[2], xi1[2], yi0[2], yi1[2];
+    float fx[2], fy[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        coarse_tap(2 * xc + k, wc, xi0[k], xi1[k], fx[k]);
+        coarse_tap(2 * yc + k, hc, yi0[k], yi1[k], fy[k]);
+    }
+#pragma unroll
+    for (int a = 0; a < 2; ++a) {
+        float2 o[2];
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+            const float2 p00 = __ldg(src + yi0[a] * wc + xi0[b]), p01 = __ldg(src + yi0[a] * wc + xi1[b]);
+            const float2 p10 = __ldg(src + yi1[a] * wc + xi0[b]), p11 = __ldg(src + yi1[a] * wc + xi1[b]);
+            const float gx = 1.0f - fx[b], gy = 1.0f - fy[a];
+            o[b].x = 2.0f * lerp2(p00.x, p01.x, p10.x, p11.x, gx, fx[b], gy, fy[a]);
+            o[b].y = 2.0f * lerp2(p00.y, p01.y, p10.y, p11.y, gx, fx[b], gy, fy[a]);
+        }
+        *reinterpret_cast<float4*>(dst + (2 * yc + a) * w + 2 * xc) = make_float4(o[0].x, o[0].y, o[1].x, o[1].y);
+    }
+}
+
+// ---- (G, h) of the next update from the current field d (zero when there is none: the first update of the
+// coarsest level).  One pixel per thread: the kernel has no shared state and runs at full occupancy, which hides
+// the latency of its gathers; fused behind the solve of the update kernel it ran at a quarter of the warps and
+// took longer than the two kernels apart.
+__global__ void __launch_bounds__(256)
+k_flow_terms(const float4* __restrict__ q1, const float* __restrict__ r1, const float4* __restrict__ q2,
+             const float* __restrict__ r2, int h, int w, unsigned w_inv, const float2* __restrict__ d, size_t d_stride,
+             float* __restrict__ gh, size_t gh_stride, int n_pairs) {
     const int P = h * w;
     const int f = blockIdx.y, r = blockIdx.x * blockDim.x + threadIdx.x;        // grid: (pixels of the level, pairs)
     if (r >= P || f >= n_pairs) return;
     const int y = (int)__umulhi((unsigned)r, w_inv), x = r - y * w;             // w_inv = ceil(2^32 / w): exact for r < 2^32 / w
     const CoefView c1{q1 + (size_t)f * P, r1 + (size_t)f * P}, c2{q2 + (size_t)f * P, r2 + (size_t)f * P};
-    float du = 0.0f, dv = 0.0f;
-    if (d_coarse) {
-        const int hc = h >> 1, wc = w >> 1;
-        int x0, x1, y0, y1;
-        float fx, fy;
-        coarse_tap(x, wc, x0, x1, fx);
-        coarse_tap(y, hc, y0, y1, fy);
-        const float* cu = d_coarse + (size_t)f * flow_stride;
-        const float* cv = cu + hc * wc;
-        const int i00 = y0 * wc + x0, i01 = y0 * wc + x1, i10 = y1 * wc + x0, i11 = y1 * wc + x1;
-        const float gx = 1.0f - fx, gy = 1.0f - fy;
-        du = 2.0f * lerp2(__ldg(cu + i00), __ldg(cu + i01), __ldg(cu + i10), __ldg(cu + i11), gx, fx, gy, fy);
-        dv = 2.0f * lerp2(__ldg(cv + i00), __ldg(cv + i01), __ldg(cv + i10), __ldg(cv + i11), gx, fx, gy, fy);
-    }
+    float2 dd = make_float2(0.0f, 0.0f);
+    if (d) dd = __ldg(d + (size_t)f * d_stride + r);
     float t[5];
-    normal_terms(c1, c2, w, r, (float)-x, (float)(w - 1 - x), (float)-y, (float)(h - 1 - y), du, dv, t);
+    normal_terms(c1, c2, w, r, (float)-x, (float)(w - 1 - x), (float)-y, (float)(h - 1 - y), dd.x, dd.y, t);
     float* o = gh + (size_t)f * gh_stride + r;
 #pragma unroll
     for (int c = 0; c < 5; ++c) o[c * P] = t[c];
@@ -269,14 +294,14 @@ k_flow_gh(const float4* __restrict__ q1, const float* __restrict__ r1, const flo
 //            suffix sum of one block plus a prefix sum of the next (no subtraction) -> shared memory
 //   phase 2  one thread per (row, run of RUN columns): 15-column sums of the row sums the same way,
 //            2x2 solve -> d in shared memory
-//   phase 3  one thread per pixel: the (G, h) of the NEXT update at d (no halo needed), and / or d itself,
-//            and / or the patch scores after the last update
+//   phase 3  one thread per pixel: d itself (for k_flow_terms and for the next finer level), and / or the
+//            patch scores after the last update
 // The window covers the in-image part only: terms outside the image count as zero.
 constexpr int TH = 28;             // tile height = 2 patches
 constexpr int BR = 7;              // window radius (window 15)
 constexpr int BLK = 2 * BR;        // rows per block of the suffix / prefix scheme
 constexpr int UPD_THREADS = 224;
-constexpr int EMIT_NEXT = 1, EMIT_D = 2, EMIT_DP = 4, EMIT_D64 = 8;
+constexpr int EMIT_D = 2, EMIT_DP = 4, EMIT_D64 = 8;
 
 template <int TW>
 struct UpdGeom {
@@ -293,10 +318,8 @@ struct UpdGeom {
 
 template <int TW, int FLAGS>
 __global__ void __launch_bounds__(UPD_THREADS, 4)
-k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, float eps, const float4* __restrict__ q1,
-              const float* __restrict__ r1, const float4* __restrict__ q2, const float* __restrict__ r2,
-              float* __restrict__ gh_out, float* __restrict__ d_out, double* __restrict__ d_out64, size_t flow_stride,
-              float* __restrict__ dP, PlaneGeom g) {
+k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, float eps, float2* __restrict__ d_out,
+              size_t d_stride, double* __restrict__ d_out64, size_t flow_stride, float* __restrict__ dP, PlaneGeom g) {
     using G = UpdGeom<TW>;
     constexpr int RUN = G::RUN, EW = G::EW, S = G::S, NQ = G::NQ, DPITCH = G::DPITCH;
     extern __shared__ __align__(16) float upd_smem[];
@@ -393,32 +416,18 @@ k_flow_update(const float* __restrict__ gh_in, size_t gh_stride, int h, int w, f
     constexpr int PER = (TH * TW + UPD_THREADS - 1) / UPD_THREADS, RSTEP = UPD_THREADS / TW;
     const int ox = t % TW, oyb = t / TW;
     const int x = x0 + ox;
-    const CoefView c1{q1 + (size_t)f * P, r1 + (size_t)f * P}, c2{q2 + (size_t)f * P, r2 + (size_t)f * P};
     double acc_up = 0.0, acc_lo = 0.0;                 // upper / lower patch of the tile
-    const float xlo = (float)-x, xhi = (float)(w - 1 - x);
-    float ylo = (float)-(y0 + oyb), yhi = (float)(h - 1 - y0 - oyb);
     int p = (y0 + oyb) * w + x;
 #pragma unroll
-    for (int j = 0; j < PER; ++j, p += RSTEP * w, ylo -= (float)RSTEP, yhi -= (float)RSTEP) {
+    for (int j = 0; j < PER; ++j, p += RSTEP * w) {
         const int oy = oyb + j * RSTEP;
         if ((TH * TW) % UPD_THREADS != 0 && oy >= TH) break;
         const float2 d = dsm[oy][ox];
-        if (FLAGS & EMIT_D) {
-            float* o = d_out + (size_t)f * flow_stride;
-            o[p] = d.x;
-            o[P + p] = d.y;
-        }
+        if (FLAGS & EMIT_D) d_out[(size_t)f * d_stride + p] = d;
         if (FLAGS & EMIT_D64) {
             double* o = d_out64 + (size_t)f * flow_stride;
             o[p] = (double)d.x;
             o[P + p] = (double)d.y;
-        }
-        if (FLAGS & EMIT_NEXT) {
-            float tm[5];
-            normal_terms(c1, c2, w, p, xlo, xhi, ylo, yhi, d.x, d.y, tm);
-            float* o = gh_out + (size_t)f * gh_stride + p;
-#pragma unroll
-            for (int c = 0; c < 5; ++c) o[c * P] = tm[c];
         }
         if (FLAGS & EMIT_DP) {
             const double m = (double)d.x * (double)d.x + (double)d.y * (double)d.y;
@@ -459,26 +468,24 @@ static_assert((2 * UPD_THREADS + 2 * 56) * sizeof(double) <= 5 * TH * UpdGeom<28
 template <int TW>
 int init_update() {
 #define SC_UPD(F) SC_CHECK(cudaFuncSetAttribute(k_flow_update<TW, F>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)upd_smem_bytes<TW>()));
-    SC_UPD(EMIT_NEXT) SC_UPD(EMIT_D) SC_UPD(EMIT_DP) SC_UPD(EMIT_DP | EMIT_D64)
+    SC_UPD(EMIT_D) SC_UPD(EMIT_DP) SC_UPD(EMIT_DP | EMIT_D64)
 #undef SC_UPD
     return SALICACHE_OK;
 }
 
 struct UpdArgs {
     const float* gin; size_t gstride; int h, w; float eps;
-    const float4 *q1; const float* r1; const float4* q2; const float* r2;
-    float* gout; float* dout; double* dout64; size_t fstride; float* dP;
+    float2* dout; size_t dstride; double* dout64; size_t fstride; float* dP;
 };
 
 template <int TW>
 void launch_update(dim3 grid, cudaStream_t st, int flags, const UpdArgs& a, const PlaneGeom& g) {
 #define SC_UPD(F)                                                                                                   \
     case F:                                                                                                         \
-        k_flow_update<TW, F><<<grid, UPD_THREADS, upd_smem_bytes<TW>(), st>>>(a.gin, a.gstride, a.h, a.w, a.eps, a.q1, a.r1, \
-                                                                               a.q2, a.r2, a.gout, a.dout, a.dout64, a.fstride, a.dP, g); \
+        k_flow_update<TW, F><<<grid, UPD_THREADS, upd_smem_bytes<TW>(), st>>>(a.gin, a.gstride, a.h, a.w, a.eps, a.dout, a.dstride, \
+                                                                               a.dout64, a.fstride, a.dP, g);     \
         break;
     switch (flags) {
-        SC_UPD(EMIT_NEXT)
         SC_UPD(EMIT_D)
         SC_UPD(EMIT_DP)
         SC_UPD(EMIT_DP | EMIT_D64)
@@ -592,51 +599,48 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
             k_poly_exp<<<gp, 256, 0, st>>>(c->pyr[l], hs[l], ws[l], nf, pw, cq[l], cr[l]);
         }
         c->launches += 5;
-        // Coarse to fine: first terms, then the updates, each launch over all pairs of the pass.  (Sub-batches sized
-        // for the L2 cache were measured and are slower: the kernels are bound by issue slots and load latency, not
-        // by DRAM, and small launches add ramp-up and tail time.)
-        const size_t fstride = 2 * P0;
-        float* d_lvl[2] = {c->flow_a, c->flow_b};
-        const float* coarse = nullptr;
+        // Coarse to fine.  Per level: the prior from the coarser level's field, then `iters` times (terms of every
+        // pixel from the current field; window sums + solve -> the new field), each launch over all pairs of the
+        // pass.  (Sub-batches sized for the L2 cache were measured and are slower: the kernels are bound by issue
+        // slots and load latency, not by DRAM, and small launches add ramp-up and tail time.)
+        const size_t fstride = 2 * P0, dstride = P0;      // caller's double field; float2 fields of the scratch
+        float2* d_lvl[2] = {reinterpret_cast<float2*>(c->flow_a), reinterpret_cast<float2*>(c->flow_b)};
         for (int l = 2; l >= 0; --l) {
             const size_t Pl = (size_t)hs[l] * ws[l];
             const size_t gstride = 5 * Pl;
-            float* dl = d_lvl[l & 1];
+            float2* dl = d_lvl[l & 1];
             const int tw = ws[l] % 56 == 0 ? 56 : 28;
             const size_t second = sequence ? Pl : (size_t)nb * Pl;      // the pair's second frame, in pixels
-            const int sub = nb;
-            for (int z0 = 0; z0 < nb; z0 += sub) {
-                const int nz = nb - z0 < sub ? nb - z0 : sub;
-                const float4* q1 = cq[l] + (size_t)z0 * Pl;
-                const float* r1 = cr[l] + (size_t)z0 * Pl;
-                float* gin = c->gh_a;
-                float* gout = c->gh_b;
-                k_flow_gh<<<dim3(blocks_for((long long)Pl, 256), nz), 256, 0, st>>>(
-                    q1, r1, q1 + second, r1 + second, hs[l], ws[l], (unsigned)((0x100000000ull + ws[l] - 1) / ws[l]), coarse ? coarse + (size_t)z0 * fstride : nullptr, fstride,
-                    gin, gstride, nz);
+            const float4* q1 = cq[l];
+            const float* r1 = cr[l];
+            const unsigned w_inv = (unsigned)((0x100000000ull + ws[l] - 1) / ws[l]);
+            if (l < 2) {
+                const int hc = hs[l + 1], wc = ws[l + 1];
+                k_flow_prior<<<dim3(blocks_for((long long)hc * wc, 256), nb), 256, 0, st>>>(
+                    d_lvl[(l + 1) & 1], hc, wc, (unsigned)((0x100000000ull + wc - 1) / wc), dstride, dl, nb);
                 c->launches++;
-                dim3 grid(ws[l] / tw, hs[l] / TH, nz);
-                for (int it = 0; it < p.iters; ++it) {
-                    const bool last = it == p.iters - 1;
-                    int flags = last ? 0 : EMIT_NEXT;
-                    double* dout64 = nullptr;
-                    if (last && l > 0) flags |= EMIT_D;
-                    if (last && l == 0) {      // the field goes to the caller's buffer if there is one
-                        flags |= EMIT_DP;
-                        if (d_flow_or_null) {
-                            flags |= EMIT_D64;
-                            dout64 = d_flow_or_null + (size_t)(b0 + z0) * fstride;
-                        }
-                    }
-                    UpdArgs a{gin, gstride, hs[l], ws[l], (float)p.eps_det, q1, r1, q1 + second, r1 + second,
-                              gout, dl + (size_t)z0 * fstride, dout64, fstride, d_deltaP + (size_t)(b0 + z0) * g.n_tok};
-                    if (tw == 56) launch_update<56>(grid, st, flags, a, g);
-                    else launch_update<28>(grid, st, flags, a, g);
-                    c->launches++;
-                    float* t = gin; gin = gout; gout = t;
-                }
             }
-            coarse = dl;
+            dim3 grid(ws[l] / tw, hs[l] / TH, nb);
+            for (int it = 0; it < p.iters; ++it) {
+                const bool last = it == p.iters - 1;
+                k_flow_terms<<<dim3(blocks_for((long long)Pl, 256), nb), 256, 0, st>>>(
+                    q1, r1, q1 + second, r1 + second, hs[l], ws[l], w_inv, (l == 2 && it == 0) ? nullptr : dl, dstride, c->gh_a,
+                    gstride, nb);
+                int flags = EMIT_D;
+                double* dout64 = nullptr;
+                if (last && l == 0) {      // the field goes to the caller's buffer if there is one
+                    flags = EMIT_DP;
+                    if (d_flow_or_null) {
+                        flags |= EMIT_D64;
+                        dout64 = d_flow_or_null + (size_t)b0 * fstride;
+                    }
+                }
+                UpdArgs a{c->gh_a, gstride, hs[l], ws[l], (float)p.eps_det, dl, dstride, dout64, fstride,
+                          d_deltaP + (size_t)b0 * g.n_tok};
+                if (tw == 56) launch_update<56>(grid, st, flags, a, g);
+                else launch_update<28>(grid, st, flags, a, g);
+                c->launches += 2;
+            }
         }
     }
     SC_CHECK(cudaGetLastError());
