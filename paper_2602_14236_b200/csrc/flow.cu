@@ -223,17 +223,10 @@ __device__ __forceinline__ float det2(float a, float b, float c, float d) {
 
 // ---- prior of a level from the coarser level's field: d = 2 * bilinear(d_coarse) at
 // ((x+1/2)/2 - 1/2, (y+1/2)/2 - 1/2), clamped to the coarse image.  For a fine coordinate x that position is
-// x/2 - 1/4: left tap (x-1) >> 1 with weight 3/4 on the right tap for even x and 1/4 for odd x; at x = 0 and at
-// the last fine pixel the clamp puts it on the tap itself.
-__device__ __forceinline__ void coarse_tap(int x, int nc, int& i0, int& i1, float& f) {
-    i0 = (x - 1) >> 1;
-    f = (x & 1) ? 0.25f : 0.75f;
-    if (x == 0) { i0 = 0; f = 0.0f; }
-    i1 = i0 + 1;
-    if (i1 > nc - 1) { i1 = nc - 1; f = 0.0f; }      // x = 2 nc - 1: position nc - 3/4, clamped to nc - 1
-}
-
-// One thread per coarse pixel: its 2x2 block of fine pixels, written as two 16-byte stores.
+// x/2 - 1/4; at x = 0 and at the last fine pixel the clamp puts it on a tap itself.
+// One thread per coarse pixel: its 2x2 block of fine pixels from the 3x3 coarse neighbourhood (clamped; a tap that
+// the clamp moved carries weight zero), written as two 16-byte stores.  Fine x = 2 xc takes taps (xc - 1, xc) with
+// weight 3/4 on the right one, x = 2 xc + 1 taps (xc, xc + 1) with weight 1/4 on the right one.
 __global__ void __launch_bounds__(256)
 k_flow_prior(const float2* __restrict__ d_coarse, int hc, int wc, unsigned wc_inv, size_t d_stride, float2* __restrict__ d_fine,
              int n_pairs) {
@@ -244,20 +237,21 @@ k_flow_prior(const float2* __restrict__ d_coarse, int hc, int wc, unsigned wc_in
     const float2* src = d_coarse + (size_t)f * d_stride;
     float2* dst = d_fine + (size_t)f * d_stride;
     const int w = 2 * wc;
-    int xi0[2], xi1[2], yi0[2], yi1[2];
-    float fx[2], fy[2];
+    const int xo[3] = {xc > 0 ? -1 : 0, 0, xc < wc - 1 ? 1 : 0};
+    const int yo[3] = {yc > 0 ? -wc : 0, 0, yc < hc - 1 ? wc : 0};
+    float2 n[3][3];
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
-        coarse_tap(2 * xc + k, wc, xi0[k], xi1[k], fx[k]);
-        coarse_tap(2 * yc + k, hc, yi0[k], yi1[k], fy[k]);
-    }
+    for (int j = 0; j < 3; ++j)
+#pragma unroll
+        for (int i = 0; i < 3; ++i) n[j][i] = __ldg(src + r + yo[j] + xo[i]);
+    const float fx[2] = {xc > 0 ? 0.75f : 0.0f, xc < wc - 1 ? 0.25f : 0.0f};
+    const float fy[2] = {yc > 0 ? 0.75f : 0.0f, yc < hc - 1 ? 0.25f : 0.0f};
 #pragma unroll
     for (int a = 0; a < 2; ++a) {
         float2 o[2];
 #pragma unroll
         for (int b = 0; b < 2; ++b) {
-            const float2 p00 = __ldg(src + yi0[a] * wc + xi0[b]), p01 = __ldg(src + yi0[a] * wc + xi1[b]);
-            const float2 p10 = __ldg(src + yi1[a] * wc + xi0[b]), p11 = __ldg(src + yi1[a] * wc + xi1[b]);
+            const float2 p00 = n[a][b], p01 = n[a][b + 1], p10 = n[a + 1][b], p11 = n[a + 1][b + 1];
             const float gx = 1.0f - fx[b], gy = 1.0f - fy[a];
             o[b].x = 2.0f * lerp2(p00.x, p01.x, p10.x, p11.x, gx, fx[b], gy, fy[a]);
             o[b].y = 2.0f * lerp2(p00.y, p01.y, p10.y, p11.y, gx, fx[b], gy, fy[a]);
