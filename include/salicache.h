@@ -117,8 +117,9 @@ SALICACHE_API int64_t salicache_launch_count(const salicache_ctx* ctx);
  * d_cur == d_prev + H*W*3 (a video: pair b is frames b, b+1) is recognised and each frame is
  * expanded once.  d_flow_or_null, if given, receives the level-0 flow as double [B][2][H][W]
  * (u along x, then v); anyres contexts write only the full-resolution field.
- * Device arithmetic (Sec. III-A, Eq. 5): the polynomial expansion runs in double and its coefficients
- * are stored in single precision; the normal-equation terms, their 15x15 window sums (sums of their own
+ * Device arithmetic (Sec. III-A, Eq. 5): single precision throughout, arranged so that it holds the
+ * tolerance: the polynomial expansion takes its moments through zero-sum kernels and differences from the
+ * window centre (coefficients good to a few 1e-7 relative); the normal-equation terms, their 15x15 window sums (sums of their own
  * terms only, no running subtraction) and the 2x2 solve (compensated products) run in single precision;
  * sampling positions are exact; the patch reduction is double.  Tested bound: d_deltaP within 1e-4
  * relative (floor 1e-6) of the double-precision definition, the dense field within 2e-5 px.

@@ -1,10 +1,11 @@
 // Temporal branch (Sec. III-A, Eq. 5): gray pyramid, polynomial expansion, coarse-to-fine
 // displacement updates and the per-patch RMS flow magnitude.
 //
-// Precision: pyramid levels are exact in float; the expansion runs in double and its coefficients are
-// stored as float; the per-pixel normal-equation terms (G, h), their 15x15 window sums and the 2x2 solve
-// run in float, the sums without any subtraction and the solve with compensated products; sampling
-// positions are exact; the patch reduction is double.  The effect on dP stays more than an order of
+// Precision: everything but the patch reduction (double) runs in single precision.  Pyramid levels are exact in
+// float; the expansion takes its moments through zero-sum kernels and differences from the window centre, so
+// that its coefficients carry a relative error of a few 1e-7; the per-pixel normal-equation terms (G, h), their
+// 15x15 window sums and the 2x2 solve sum without any subtraction and solve with compensated products; sampling
+// positions are exact.  The effect on dP stays more than an order of
 // magnitude below the 1e-4 relative tolerance on every workload.
 //
 // One displacement update = the terms (G, h) of every pixel at the current field (k_flow_terms, one pixel
@@ -64,87 +65,90 @@ __global__ void k_pyr_down(const float* __restrict__ src, int h, int w, int n_fr
     dst[(size_t)f * h2 * w2 + r] = acc * (1.0f / 256.0f);
 }
 
-struct PolyW {
-    double g[5];     // normalised Gaussian applicability
-    double inv_mu2, inv_mu2sq, inv_den, mu2;
-};
-
 // ---- polynomial expansion, 5x5: r2 r3 r4 r5 r6 = (b_x, b_y, A_xx, A_yy, 2 A_xy), stored as float in the form the
 // displacement updates read: (r2, r3, r4, r5) / 2 as one 16-byte record per pixel and r6 / 4 in a plane of its own.
-// Separable, in double: a 32x32 tile grown by 2 is staged in shared memory, each grown row gets its three
-// horizontal moment sums (weights g, g*b, g*b^2), and each thread then walks down a column of 8 pixels
-// with the five rows of sums it needs in registers.
+// A 32x32 tile grown by 2 is staged in shared memory.
 constexpr int PX = 32, PY = 32, PH = 2;          // tile and halo
 constexpr int PEW = PX + 2 * PH, PEH = PY + 2 * PH;
-constexpr int PRUN = 8;                          // pixels per thread in the vertical pass
 
+// Single precision.  Every moment is taken through a kernel that sums to zero or
+// through differences from the window's centre value, so that what gets multiplied and added are local
+// differences of the image (exact in float: the levels are dyadic rationals) and never the image values
+// themselves; the coefficients then carry a relative error of a few 1e-7 instead of an absolute one of 1e-5:
+//   H1 = sum_b g(b) b f            = g1 (f[+1] - f[-1]) + 2 g2 (f[+2] - f[-2])            along a row
+//   H2 = sum_b g(b) (b^2 - mu2) f  = k1 (f[+1] + f[-1] - 2 f[0]) + k2 (f[+2] + f[-2] - 2 f[0])
+//   V1, V2 the same down a column;  S[q] = sum_a g(a) q[a] = q[0] + g1 ((q[1]-q[0]) + (q[-1]-q[0])) + g2 (...)
+//   m10 = S_rows[H1], m20 - mu2 m00 = S_rows[H2], m11 = g1 (H1[+1] - H1[-1]) + 2 g2 (H1[+2] - H1[-2]) down the rows,
+//   m01 = S_cols[V1], m02 - mu2 m00 = S_cols[V2].
+struct PolyW32 {
+    float g1, g2, k1, k2;            // g(1), g(2); g(1) (1 - mu2), g(2) (4 - mu2)
+    float s2, s3, s45, s6;           // output scalings: 1/(2 mu2), 1/(2 mu2), 1/(2 (mu4 - mu2^2)), 1/(4 mu2^2)
+};
+
+__device__ __forceinline__ float smooth5(float qm2, float qm1, float q0, float qp1, float qp2, float g1, float g2) {
+    return q0 + (g1 * ((qp1 - q0) + (qm1 - q0)) + g2 * ((qp2 - q0) + (qm2 - q0)));
+}
+
+// Block (32, 8): thread (tx, ty) owns column tx of rows ty, ty + 8, ...: every loop below has a compile-time trip
+// count and every shared-memory access is a base plus a constant.
 __global__ void __launch_bounds__(256)
-k_poly_exp(const float* __restrict__ img, int h, int w, int n_frames, PolyW pw, float4* __restrict__ cq,
-           float* __restrict__ cr) {
-    __shared__ double tile[PEH][PEW + 1];
-    __shared__ double hm[3][PEH][PX];
+k_poly_exp32(const float* __restrict__ img, int h, int w, int n_frames, PolyW32 pw, float4* __restrict__ cq,
+             float* __restrict__ cr) {
+    __shared__ float tile[PEH][PEW + 1];
+    __shared__ float H1[PEH][PX], H2[PEH][PX];
+    __shared__ float V1[PY][PEW + 1], V2[PY][PEW + 1];
+    const int tx = threadIdx.x, ty = threadIdx.y;
     const int f = blockIdx.z, x0 = blockIdx.x * PX, y0 = blockIdx.y * PY;
     const size_t P = (size_t)h * w;
     const float* s = img + (size_t)f * P;
-    for (int i = threadIdx.x; i < PEH * PEW; i += blockDim.x) {
-        const int ry = i / PEW, rx = i - ry * PEW;
-        tile[ry][rx] = (double)s[(size_t)clampi(y0 - PH + ry, 0, h - 1) * w + clampi(x0 - PH + rx, 0, w - 1)];
+    const int xa = clampi(x0 - PH + tx, 0, w - 1), xb = clampi(x0 - PH + tx + 32, 0, w - 1);
+#pragma unroll
+    for (int k = 0; k < 5; ++k) {
+        const int ry = ty + 8 * k;
+        if (ry < PEH) {
+            const float* row = s + (size_t)clampi(y0 - PH + ry, 0, h - 1) * w;
+            tile[ry][tx] = row[xa];
+            if (tx < PEW - 32) tile[ry][tx + 32] = row[xb];
+        }
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < PEH * PX; i += blockDim.x) {
-        const int ry = i / PX, ox = i - ry * PX;
-        double s0 = 0, s1 = 0, s2 = 0;
 #pragma unroll
-        for (int b = -2; b <= 2; ++b) {
-            const double v = pw.g[b + 2] * tile[ry][ox + PH + b];
-            s0 += v;
-            s1 += v * b;
-            s2 += v * (b * b);
+    for (int k = 0; k < 5; ++k) {                      // along the rows of the grown tile
+        const int ry = ty + 8 * k;
+        if (ry < PEH) {
+            const float* t = &tile[ry][tx];
+            const float c = t[2];
+            H1[ry][tx] = pw.g1 * (t[3] - t[1]) + 2.0f * pw.g2 * (t[4] - t[0]);
+            H2[ry][tx] = pw.k1 * ((t[3] - c) + (t[1] - c)) + pw.k2 * ((t[4] - c) + (t[0] - c));
         }
-        hm[0][ry][ox] = s0;
-        hm[1][ry][ox] = s1;
-        hm[2][ry][ox] = s2;
     }
+    auto down = [&](int oy, int rx) {                  // down the columns of the grown tile
+        const float c = tile[oy + 2][rx];
+        const float a1 = tile[oy + 1][rx], b1 = tile[oy + 3][rx], a2 = tile[oy][rx], b2 = tile[oy + 4][rx];
+        V1[oy][rx] = pw.g1 * (b1 - a1) + 2.0f * pw.g2 * (b2 - a2);
+        V2[oy][rx] = pw.k1 * ((b1 - c) + (a1 - c)) + pw.k2 * ((b2 - c) + (a2 - c));
+    };
+#pragma unroll
+    for (int k = 0; k < 4; ++k) down(ty + 8 * k, tx);
+    if (ty < 4) down(8 * ty + (tx >> 2), 32 + (tx & 3));          // the four columns past the 32nd: 128 items, four warps
     __syncthreads();
-    if (threadIdx.x < PX * (PY / PRUN)) {
-        const int ox = threadIdx.x % PX, oy0 = PRUN * (threadIdx.x / PX);
-        const int x = x0 + ox;
-        if (x < w) {
-            double r0[5], r1[5], r2[5];              // sliding five rows of the three sums
+    const int x = x0 + tx;
+    if (x >= w) return;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                r0[k + 1] = hm[0][oy0 + k][ox];
-                r1[k + 1] = hm[1][oy0 + k][ox];
-                r2[k + 1] = hm[2][oy0 + k][ox];
-            }
-#pragma unroll
-            for (int k = 0; k < PRUN; ++k) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) { r0[j] = r0[j + 1]; r1[j] = r1[j + 1]; r2[j] = r2[j + 1]; }
-                r0[4] = hm[0][oy0 + k + 4][ox];
-                r1[4] = hm[1][oy0 + k + 4][ox];
-                r2[4] = hm[2][oy0 + k + 4][ox];
-                double m00 = 0, m10 = 0, m01 = 0, m20 = 0, m02 = 0, m11 = 0;
-#pragma unroll
-                for (int a = -2; a <= 2; ++a) {
-                    const double ga = pw.g[a + 2];
-                    m00 += ga * r0[a + 2];
-                    m10 += ga * r1[a + 2];
-                    m20 += ga * r2[a + 2];
-                    m01 += ga * a * r0[a + 2];
-                    m11 += ga * a * r1[a + 2];
-                    m02 += ga * (a * a) * r0[a + 2];
-                }
-                const int y = y0 + oy0 + k;
-                if (y < h) {
-                    const size_t o = (size_t)f * P + (size_t)y * w + x;
-                    cq[o] = make_float4((float)(0.5 * (m10 * pw.inv_mu2)), (float)(0.5 * (m01 * pw.inv_mu2)),
-                                        (float)(0.5 * ((m20 - pw.mu2 * m00) * pw.inv_den)),
-                                        (float)(0.5 * ((m02 - pw.mu2 * m00) * pw.inv_den)));
-                    cr[o] = (float)(0.25 * (m11 * pw.inv_mu2sq));
-                }
-            }
-        }
+    for (int k = 0; k < 4; ++k) {
+        const int oy = ty + 8 * k, y = y0 + oy;
+        if (y >= h) break;
+        const float h1a = H1[oy][tx], h1b = H1[oy + 1][tx], h1c = H1[oy + 2][tx], h1d = H1[oy + 3][tx], h1e = H1[oy + 4][tx];
+        const float m10 = smooth5(h1a, h1b, h1c, h1d, h1e, pw.g1, pw.g2);
+        const float m11 = pw.g1 * (h1d - h1b) + 2.0f * pw.g2 * (h1e - h1a);
+        const float m20 = smooth5(H2[oy][tx], H2[oy + 1][tx], H2[oy + 2][tx], H2[oy + 3][tx], H2[oy + 4][tx], pw.g1, pw.g2);
+        const float* v1 = &V1[oy][tx];
+        const float* v2 = &V2[oy][tx];
+        const float m01 = smooth5(v1[0], v1[1], v1[2], v1[3], v1[4], pw.g1, pw.g2);
+        const float m02 = smooth5(v2[0], v2[1], v2[2], v2[3], v2[4], pw.g1, pw.g2);
+        const size_t o = (size_t)f * P + (size_t)y * w + x;
+        cq[o] = make_float4(m10 * pw.s2, m01 * pw.s3, m20 * pw.s45, m02 * pw.s45);
+        cr[o] = m11 * pw.s6;
     }
 }
 
@@ -550,19 +554,17 @@ int sc_diff_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
 int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, const uint8_t* d_cur, size_t frame_bytes,
                   int B, bool sequence, float* d_deltaP, double* d_flow_or_null, cudaStream_t st) {
     const salicache_params& p = c->p;
-    PolyW pw;
+    PolyW32 pw32;
     {
-        double Z = 0, mu2 = 0, mu4 = 0;
-        for (int k = -2; k <= 2; ++k) { pw.g[k + 2] = exp(-(double)(k * k) / (2.0 * p.poly_sigma * p.poly_sigma)); Z += pw.g[k + 2]; }
+        double g[5], Z = 0, mu2 = 0, mu4 = 0;
+        for (int k = -2; k <= 2; ++k) { g[k + 2] = exp(-(double)(k * k) / (2.0 * p.poly_sigma * p.poly_sigma)); Z += g[k + 2]; }
         for (int k = -2; k <= 2; ++k) {
-            pw.g[k + 2] /= Z;
-            mu2 += pw.g[k + 2] * k * k;
-            mu4 += pw.g[k + 2] * k * k * (double)(k * k);
+            g[k + 2] /= Z;
+            mu2 += g[k + 2] * k * k;
+            mu4 += g[k + 2] * k * k * (double)(k * k);
         }
-        pw.mu2 = mu2;
-        pw.inv_mu2 = 1.0 / mu2;
-        pw.inv_mu2sq = 1.0 / (mu2 * mu2);
-        pw.inv_den = 1.0 / (mu4 - mu2 * mu2);
+        pw32 = PolyW32{(float)g[3], (float)g[4], (float)(g[3] * (1.0 - mu2)), (float)(g[4] * (4.0 - mu2)),
+                       (float)(0.5 / mu2), (float)(0.5 / mu2), (float)(0.5 / (mu4 - mu2 * mu2)), (float)(0.25 / (mu2 * mu2))};
     }
     const int T = 256;
     int hs[3], ws[3];
@@ -590,7 +592,7 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
             cq[l] = reinterpret_cast<float4*>(c->coef[l]);
             cr[l] = c->coef[l] + 4 * (slots * hs[l] * ws[l] + ws[l] + 2);
             dim3 gp((ws[l] + PX - 1) / PX, (hs[l] + PY - 1) / PY, nf);
-            k_poly_exp<<<gp, 256, 0, st>>>(c->pyr[l], hs[l], ws[l], nf, pw, cq[l], cr[l]);
+            k_poly_exp32<<<gp, dim3(32, 8), 0, st>>>(c->pyr[l], hs[l], ws[l], nf, pw32, cq[l], cr[l]);
         }
         c->launches += 5;
         // Coarse to fine.  Per level: the prior from the coarser level's field, then `iters` times (terms of every
