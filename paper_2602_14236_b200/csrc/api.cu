@@ -3,6 +3,8 @@
 #include <new>
 #include <string.h>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 
 int sc_flow_init();
@@ -11,6 +13,12 @@ int sc_kv_max_batch();
 bool sc_kv_supported_hd(int HD);
 
 namespace {
+
+// A named range around the launches of one call, for timelines (costs nothing when no tool is attached).
+struct Range {
+    explicit Range(const char* name) { nvtxRangePushA(name); }
+    ~Range() { nvtxRangePop(); }
+};
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -173,6 +181,7 @@ int64_t salicache_launch_count(const salicache_ctx* c) { return c ? (int64_t)c->
 
 int salicache_flow_score(salicache_ctx* c, const uint8_t* d_prev, const uint8_t* d_cur, int B, float* d_deltaP,
                          double* d_flow_or_null, void* cuda_stream) {
+    Range range__("salicache_flow_score");
     if (!c || !d_prev || !d_cur || !d_deltaP) return SALICACHE_E_NULL;
     if (B < 0 || B > c->p.max_batch) return SALICACHE_E_SHAPE;
     if (!aligned16(d_prev) || !aligned16(d_cur) || !aligned16(d_deltaP) || !aligned16(d_flow_or_null))
@@ -210,6 +219,7 @@ int salicache_flow_score(salicache_ctx* c, const uint8_t* d_prev, const uint8_t*
 
 int salicache_diff_score(salicache_ctx* c, const uint8_t* d_prev, const uint8_t* d_cur, int B, float* d_deltaP,
                          void* cuda_stream) {
+    Range range__("salicache_diff_score");
     if (!c || !d_prev || !d_cur || !d_deltaP) return SALICACHE_E_NULL;
     if (B < 0 || B > c->p.max_batch) return SALICACHE_E_SHAPE;
     if (!aligned16(d_prev) || !aligned16(d_cur) || !aligned16(d_deltaP)) return SALICACHE_E_ALIGN;
@@ -244,6 +254,7 @@ int salicache_frame_redundancy(salicache_ctx* c, const float* d_deltaP, int B, i
 
 int salicache_saliency(salicache_ctx* c, const uint8_t* d_frames, int B, float* d_s, const uint8_t* d_skip_or_null,
                        void* cuda_stream) {
+    Range range__("salicache_saliency");
     if (!c || !d_frames || !d_s) return SALICACHE_E_NULL;
     if (B < 0 || B > c->p.max_batch) return SALICACHE_E_SHAPE;
     if (!aligned16(d_frames) || !aligned16(d_s)) return SALICACHE_E_ALIGN;
@@ -261,6 +272,7 @@ int salicache_saliency(salicache_ctx* c, const uint8_t* d_frames, int B, float* 
 int salicache_select(salicache_ctx* c, const float* d_deltaP, const float* d_s, int B, int first_has_no_prev,
                      uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts, uint8_t* d_frame_redundant,
                      int64_t* d_row_offset, int64_t* d_fill, void* cuda_stream) {
+    Range range__("salicache_select");
     if (!c || !d_s || !d_decision || !d_idx || !d_counts || !d_frame_redundant || !d_row_offset || !d_fill)
         return SALICACHE_E_NULL;
     if (B < 0 || B > c->p.max_batch) return SALICACHE_E_SHAPE;
@@ -272,6 +284,7 @@ int salicache_select_ranked(salicache_ctx* c, const float* d_deltaP, const float
                             int share_fp16_permille, int share_int8_permille, int share_int4_permille, uint8_t* d_decision,
                             int32_t* d_idx, int32_t* d_counts, uint8_t* d_frame_redundant, int64_t* d_row_offset,
                             int64_t* d_fill, void* cuda_stream) {
+    Range range__("salicache_select_ranked");
     if (!c || !d_s || !d_decision || !d_idx || !d_counts || !d_frame_redundant || !d_row_offset || !d_fill)
         return SALICACHE_E_NULL;
     if (B < 0 || B > c->p.max_batch) return SALICACHE_E_SHAPE;
@@ -286,6 +299,7 @@ int salicache_select_ranked(salicache_ctx* c, const float* d_deltaP, const float
 int salicache_select_anchored(salicache_ctx* c, const uint8_t* d_frames, const float* d_s, int B, int first_has_no_prev,
                               uint8_t* d_anchor, float* d_deltaP, uint8_t* d_decision, int32_t* d_idx, int32_t* d_counts,
                               uint8_t* d_frame_redundant, int64_t* d_row_offset, int64_t* d_fill, void* cuda_stream) {
+    Range range__("salicache_select_anchored");
     if (!c || !d_frames || !d_s || !d_anchor || !d_deltaP || !d_decision || !d_idx || !d_counts || !d_frame_redundant ||
         !d_row_offset || !d_fill)
         return SALICACHE_E_NULL;
@@ -330,6 +344,7 @@ static int check_pools(const salicache_pools* p) {
 int salicache_pack_kv(salicache_ctx* c, const void* d_K, const void* d_V, int64_t frame_stride, const int32_t* d_idx,
                       const int32_t* d_counts, const int64_t* d_row_offset, int B, const salicache_pools* pools,
                       void* cuda_stream) {
+    Range range__("salicache_pack_kv");
     if (!c || !d_K || !d_V || !d_idx || !d_counts || !d_row_offset) return SALICACHE_E_NULL;
     int rc = check_pools(pools);
     if (rc != SALICACHE_OK) return rc;
@@ -343,6 +358,7 @@ int salicache_pack_kv(salicache_ctx* c, const void* d_K, const void* d_V, int64_
 int salicache_unpack_kv(salicache_ctx* c, const salicache_pools* pools, const int32_t* d_idx, const int32_t* d_counts,
                         const uint8_t* d_decision, const int64_t* d_row_offset, int B, int zero_fill_pruned,
                         void* d_K_out, void* d_V_out, int64_t frame_stride, void* cuda_stream) {
+    Range range__("salicache_unpack_kv");
     if (!c || !d_K_out || !d_V_out || !d_idx || !d_counts || !d_row_offset) return SALICACHE_E_NULL;
     if (zero_fill_pruned && !d_decision) return SALICACHE_E_NULL;
     int rc = check_pools(pools);
@@ -372,6 +388,7 @@ int salicache_tokens_live(salicache_ctx* c, const int32_t* d_src, int B, int fir
 
 int salicache_attend(salicache_ctx* c, const void* d_q, const salicache_pools* pools, const int64_t* d_fill, float* d_out,
                      void* cuda_stream) {
+    Range range__("salicache_attend");
     if (!c || !d_q || !d_fill || !d_out) return SALICACHE_E_NULL;
     int rc = check_pools(pools);
     if (rc != SALICACHE_OK) return rc;
@@ -381,6 +398,7 @@ int salicache_attend(salicache_ctx* c, const void* d_q, const salicache_pools* p
 
 int salicache_attend_gqa(salicache_ctx* c, const void* d_q, int q_per_kv, const salicache_pools* pools, const int64_t* d_fill,
                          float* d_out, void* cuda_stream) {
+    Range range__("salicache_attend_gqa");
     if (!c || !d_q || !d_fill || !d_out) return SALICACHE_E_NULL;
     int rc = check_pools(pools);
     if (rc != SALICACHE_OK) return rc;

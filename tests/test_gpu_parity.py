@@ -456,5 +456,21 @@ def test_argument_errors_are_returned_not_raised_on_the_device():
                                  i64.data_ptr(), 1, ctypes.byref(pools.c), None) == sc.E_ALIGN
     assert lib.salicache_pack_kv(h, kv.data_ptr(), kv.data_ptr(), 100, i32.data_ptr(), i32.data_ptr(),
                                  i64.data_ptr(), 2, ctypes.byref(pools.c), None) == sc.E_SHAPE
+    # budget bookkeeping: ring pools need the running fill; counts and flags must be there
+    u8 = torch.zeros((4,), dtype=torch.uint8, device="cuda")
+    ring = sc.PoolSet(1, 4096, 4, 4, 4, ring=True)              # no fill attached
+    assert lib.salicache_frames_resident(h, i32.data_ptr(), i64.data_ptr(), 1, ctypes.byref(ring.c), u8.data_ptr(), None) == sc.E_NULL
+    assert lib.salicache_frames_resident(h, None, i64.data_ptr(), 1, ctypes.byref(pools.c), u8.data_ptr(), None) == sc.E_NULL
+    assert lib.salicache_frames_resident(h, i32.data_ptr(), i64.data_ptr(), -1, ctypes.byref(pools.c), u8.data_ptr(), None) == sc.E_SHAPE
+    assert lib.salicache_tokens_live(h, i32.data_ptr(), 1, 0, None, 1, u8.data_ptr(), None) == sc.E_NULL
+    assert lib.salicache_tokens_live(h, i32.data_ptr(), 1, -2, u8.data_ptr(), 1, u8.data_ptr(), None) == sc.E_SHAPE
+    # parameters of the frame-adaptive colour term
+    import pytest as _pt
+    for kw in (dict(color_norm=2), dict(color_norm=1, color_kappa=0.0), dict(color_norm=1, color_sigma_min=-1.0)):
+        with _pt.raises(sc.SalicacheError) as e:
+            _ctx(**kw)
+        assert e.value.status == sc.E_PARAM
+    noal = sc.salicache_default_params(L=1, color_norm=1)
+    assert lib.salicache_saliency_noalloc(ctypes.byref(noal), fr.data_ptr(), 1, dP.data_ptr(), None, None) == sc.E_PARAM
     torch.cuda.synchronize()
     assert sc.salicache_poll_status(ctx) == 0
