@@ -37,7 +37,9 @@ def test_params_struct_matches_the_header_defaults():
     assert (p.L, p.heads, p.head_dim, p.group, p.patch_reuse) == (32, 32, 128, 128, 1)
     assert abs(p.tau_t - 0.5) < 1e-7 and abs(p.theta_R - 0.9) < 1e-7
     assert (round(p.tau_high, 4), round(p.tau_med, 4), round(p.tau_low, 4)) == (0.40, 0.36, 0.25)
+    assert (p.color_norm, p.color_kappa, p.color_sigma_min) == (0, 1.0, 0.5)      # the struct's last fields: the layouts agree
     assert binding.lib().salicache_strerror(binding.E_CAPACITY).decode().startswith("tier pool")
+    assert b"overwritten" in binding.lib().salicache_strerror(binding.E_EVICTED)
 
 
 def test_host_side_argument_checks_need_no_device():
