@@ -77,6 +77,11 @@ __device__ __forceinline__ float2 sub_h2_f32(uint32_t w, float z) {
 }
 // rint(d * inv) clamped to at most 15: multiply and round to nearest even as separate operations.
 __device__ __forceinline__ int quant4(float d, float inv) { return __float2int_rn(fminf(__fmul_rn(d, inv), 15.0f)); }
+// fl(d * inv) + 1.5 * 2^23 as bits: for |product| < 2^22 the sum is the product rounded to the nearest integer (ties to
+// even), held in the low mantissa bits as a two's complement number.  Multiply and add round separately.
+__device__ __forceinline__ uint32_t rint_bits(float d, float inv) {
+    return __float_as_uint(__fadd_rn(__fmul_rn(d, inv), 12582912.0f));
+}
 // Bytes (q0 q1 q2 q3), (q4 q5 q6 q7), each 0..15 -> nibbles q0 | q1 << 4 | ... | q7 << 28.
 __device__ __forceinline__ uint32_t nibbles(uint32_t lo, uint32_t hi) {
     lo |= lo >> 4;
@@ -294,16 +299,41 @@ __device__ __forceinline__ void pack_piece(const uint4 (&v)[ITERS], const Unit& 
             reinterpret_cast<uint32_t*>(pp.int4_sz + prow * (size_t)g.ng * 4)[RG ? 0 : part * 2 * ITERS + my_group] =
                 (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(z16) << 16);
         uint32_t* dst = reinterpret_cast<uint32_t*>(pp.int4_codes + prow * (size_t)(g.HD / 2)) + part * (ITERS * 32) + lane;
+        // x >= zero, so the product is >= 0.  It exceeds 15.5 only when the stored scale was rounded down by more than
+        // 3 %, which binary16 does to subnormal scales alone (a normal one is within 2^-11 of (max - min) / 15): the
+        // upper clamp is compiled in only for rows that have such a group.
+        const bool tiny = (__half_as_ushort(s16) & 0x7fff) < 0x0400;
+        // every lane's (1/s, zero) through shared memory: one 8-byte broadcast read per iteration
+        __shared__ float2 sz_of[KV_WARPS][32];
+        float2* sz = sz_of[threadIdx.x >> 5];
+        if (!RG) {
+            __syncwarp();
+            sz[lane] = make_float2(my_inv, my_z);
+            __syncwarp();
+        }
+        if (__any_sync(0xffffffffu, tiny)) {
 #pragma unroll
-        for (int i = 0; i < ITERS; ++i) {
-            const int owner = (lane & 16) | (i << SH);
-            const float inv = RG ? my_inv : __shfl_sync(0xffffffffu, my_inv, owner);
-            const float z = RG ? my_z : __shfl_sync(0xffffffffu, my_z, owner);
-            const float2 f0 = sub_h2_f32(v[i].x, z), f1 = sub_h2_f32(v[i].y, z), f2 = sub_h2_f32(v[i].z, z), f3 = sub_h2_f32(v[i].w, z);
-            // x >= zero, so the product is >= 0; the upper clamp matters only for tiny ranges whose scale rounded down
-            int q0 = quant4(f0.x, inv), q1 = quant4(f0.y, inv), q2 = quant4(f1.x, inv), q3 = quant4(f1.y, inv);
-            int q4 = quant4(f2.x, inv), q5 = quant4(f2.y, inv), q6 = quant4(f3.x, inv), q7 = quant4(f3.y, inv);
-            st_stream(dst + i * 32, nibbles(pack_s8(q1, q0, pack_s8(q3, q2, 0)), pack_s8(q5, q4, pack_s8(q7, q6, 0))));
+            for (int i = 0; i < ITERS; ++i) {
+                const int owner = (lane & 16) | (i << SH);
+                const float2 iz = RG ? make_float2(my_inv, my_z) : sz[owner];
+                const float inv = iz.x, z = iz.y;
+                const float2 f0 = sub_h2_f32(v[i].x, z), f1 = sub_h2_f32(v[i].y, z), f2 = sub_h2_f32(v[i].z, z), f3 = sub_h2_f32(v[i].w, z);
+                int q0 = quant4(f0.x, inv), q1 = quant4(f0.y, inv), q2 = quant4(f1.x, inv), q3 = quant4(f1.y, inv);
+                int q4 = quant4(f2.x, inv), q5 = quant4(f2.y, inv), q6 = quant4(f3.x, inv), q7 = quant4(f3.y, inv);
+                st_stream(dst + i * 32, nibbles(pack_s8(q1, q0, pack_s8(q3, q2, 0)), pack_s8(q5, q4, pack_s8(q7, q6, 0))));
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) {
+                const int owner = (lane & 16) | (i << SH);
+                const float2 iz = RG ? make_float2(my_inv, my_z) : sz[owner];
+                const float inv = iz.x, z = iz.y;
+                const float2 f0 = sub_h2_f32(v[i].x, z), f1 = sub_h2_f32(v[i].y, z), f2 = sub_h2_f32(v[i].z, z), f3 = sub_h2_f32(v[i].w, z);
+                // 0 <= product < 15.5: adding 1.5 * 2^23 rounds it to nearest even and leaves the code in the low bits
+                const uint32_t a = rint_bits(f0.x, inv) + (rint_bits(f0.y, inv) << 4), b = rint_bits(f1.x, inv) + (rint_bits(f1.y, inv) << 4);
+                const uint32_t c = rint_bits(f2.x, inv) + (rint_bits(f2.y, inv) << 4), d = rint_bits(f3.x, inv) + (rint_bits(f3.y, inv) << 4);
+                st_stream(dst + i * 32, __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410));
+            }
         }
     }
 }
