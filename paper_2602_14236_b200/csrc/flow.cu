@@ -187,8 +187,8 @@ __device__ __forceinline__ void floor_fi(float v, float& f, int& i) {
 // The four taps are read at i, i+1, i+w, i+w+1 without clamping the far ones: where the position is
 // clamped to the last column or row the fraction is zero, so the far tap is multiplied by zero, and it
 // is a finite number (the next row, the next frame's plane, or the zeroed pad behind the last plane).
-__device__ __forceinline__ void normal_terms(const CoefView& c1, const CoefView& c2, int w, int p, float xlo, float xhi,
-                                             float ylo, float yhi, float du, float dv, float out[5]) {
+__device__ __forceinline__ void normal_terms(const float4 u, const float ur, const CoefView& c2, int w, int p, float xlo,
+                                             float xhi, float ylo, float yhi, float du, float dv, float out[5]) {
     const float su = fminf(fmaxf(du, xlo), xhi), sv = fminf(fmaxf(dv, ylo), yhi);
     float fdu, fdv;
     int iu, iv;
@@ -199,8 +199,6 @@ __device__ __forceinline__ void normal_terms(const CoefView& c1, const CoefView&
     const int i0 = p + iv * w + iu;
     const float4 a = __ldg(c2.q + i0), b = __ldg(c2.q + i0 + 1), c = __ldg(c2.q + i0 + w), d = __ldg(c2.q + i0 + w + 1);
     const float ra = __ldg(c2.r + i0), rb = __ldg(c2.r + i0 + 1), rc = __ldg(c2.r + i0 + w), rd = __ldg(c2.r + i0 + w + 1);
-    const float4 u = __ldg(c1.q + p);
-    const float ur = __ldg(c1.r + p);
     const float vbx = lerp2(a.x, b.x, c.x, d.x, gx, fx, gy, fy);
     const float vby = lerp2(a.y, b.y, c.y, d.y, gx, fx, gy, fy);
     const float vxx = lerp2(a.z, b.z, c.z, d.z, gx, fx, gy, fy);
@@ -265,25 +263,65 @@ k_flow_prior(const float2* __restrict__ d_coarse, int hc, int wc, unsigned wc_in
 }
 
 // ---- (G, h) of the next update from the current field d (zero when there is none: the first update of the
-// coarsest level).  One pixel per thread: the kernel has no shared state and runs at full occupancy, which hides
-// the latency of its gathers; fused behind the solve of the update kernel it ran at a quarter of the warps and
-// took longer than the two kernels apart.
-__global__ void __launch_bounds__(256)
+// coarsest level).  One pixel per thread and no state shared between threads, so the kernel runs at full occupancy,
+// which hides the latency of its gathers; fused behind the solve of the update kernel it ran at a quarter of the
+// warps and took longer than the two kernels apart.  What streams from DRAM (the pixel's own record and field
+// value, 28 bytes) is fetched one block ahead by asynchronous copies into a slot of shared memory that only the
+// thread itself reads: the next block's bytes are in flight while this block's gathers wait for the L2.
+constexpr int TERMS_THREADS = 256;
+constexpr int TERMS_BLOCKS_PER_CTA = 8;
+
+__device__ __forceinline__ void async_copy16(void* dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void async_copy8(void* dst, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void async_copy4(void* dst, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+
+__global__ void __launch_bounds__(TERMS_THREADS)
 k_flow_terms(const float4* __restrict__ q1, const float* __restrict__ r1, const float4* __restrict__ q2,
              const float* __restrict__ r2, int h, int w, unsigned w_inv, const float2* __restrict__ d, size_t d_stride,
              float* __restrict__ gh, size_t gh_stride, int n_pairs) {
+    __shared__ float4 sq[2][TERMS_THREADS];
+    __shared__ float2 sd[2][TERMS_THREADS];
+    __shared__ float sr[2][TERMS_THREADS];
     const int P = h * w;
-    const int f = blockIdx.y, r = blockIdx.x * blockDim.x + threadIdx.x;        // grid: (pixels of the level, pairs)
-    if (r >= P || f >= n_pairs) return;
-    const int y = (int)__umulhi((unsigned)r, w_inv), x = r - y * w;             // w_inv = ceil(2^32 / w): exact for r < 2^32 / w
-    const CoefView c1{q1 + (size_t)f * P, r1 + (size_t)f * P}, c2{q2 + (size_t)f * P, r2 + (size_t)f * P};
-    float2 dd = make_float2(0.0f, 0.0f);
-    if (d) dd = __ldg(d + (size_t)f * d_stride + r);
-    float t[5];
-    normal_terms(c1, c2, w, r, (float)-x, (float)(w - 1 - x), (float)-y, (float)(h - 1 - y), dd.x, dd.y, t);
-    float* o = gh + (size_t)f * gh_stride + r;
+    const int f = blockIdx.y;                                   // grid: (blocks of pixels / TERMS_BLOCKS_PER_CTA, pairs)
+    if (f >= n_pairs) return;
+    const int t = threadIdx.x;
+    const int step = gridDim.x * TERMS_THREADS;
+    const float4* qf = q1 + (size_t)f * P;
+    const float* rf = r1 + (size_t)f * P;
+    const float2* df = d ? d + (size_t)f * d_stride : nullptr;
+    const CoefView c2{q2 + (size_t)f * P, r2 + (size_t)f * P};
+    auto fetch = [&](int r, int slot) {
+        if (r < P) {
+            async_copy16(&sq[slot][t], qf + r);
+            async_copy4(&sr[slot][t], rf + r);
+            if (df) async_copy8(&sd[slot][t], df + r);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    int r = blockIdx.x * TERMS_THREADS + t;
+    fetch(r, 0);
+    for (int n = 0; r < P; r += step, ++n) {
+        fetch(r + step, (n + 1) & 1);
+        asm volatile("cp.async.wait_group 1;" ::: "memory");       // this block's copies have landed, the next block's fly
+        const int slot = n & 1;
+        const float4 u = sq[slot][t];
+        const float ur = sr[slot][t];
+        const float2 dd = df ? sd[slot][t] : make_float2(0.0f, 0.0f);
+        const int y = (int)__umulhi((unsigned)r, w_inv), x = r - y * w;         // w_inv = ceil(2^32 / w): exact for r < 2^32 / w
+        float o5[5];
+        normal_terms(u, ur, c2, w, r, (float)-x, (float)(w - 1 - x), (float)-y, (float)(h - 1 - y), dd.x, dd.y, o5);
+        float* o = gh + (size_t)f * gh_stride + r;
 #pragma unroll
-    for (int c = 0; c < 5; ++c) o[c * P] = t[c];
+        for (int c = 0; c < 5; ++c) o[c * P] = o5[c];
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
 // ---- one displacement update on a tile of TW x 28 pixels (TW / 14 x 2 patches).
@@ -619,7 +657,7 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
             dim3 grid(ws[l] / tw, hs[l] / TH, nb);
             for (int it = 0; it < p.iters; ++it) {
                 const bool last = it == p.iters - 1;
-                k_flow_terms<<<dim3(blocks_for((long long)Pl, 256), nb), 256, 0, st>>>(
+                k_flow_terms<<<dim3(blocks_for((long long)Pl, TERMS_THREADS * TERMS_BLOCKS_PER_CTA), nb), TERMS_THREADS, 0, st>>>(
                     q1, r1, q1 + second, r1 + second, hs[l], ws[l], w_inv, (l == 2 && it == 0) ? nullptr : dl, dstride, c->gh_a,
                     gstride, nb);
                 int flags = EMIT_D;

@@ -228,6 +228,7 @@ constexpr int SE = ST + 2 * SR;   // 34
 constexpr int SLP = SE + 2;       // row pitch of the planes (even: 16-byte loads of column pairs)
 constexpr int CRUN = 4;
 constexpr int CNQ = 2 * SR + CRUN;   // 10 values feed 4 windows
+constexpr int CROWS = 256 / SE;     // rows of the grown tile converted per sweep of the 256 threads (7)
 constexpr int SRAW = 8;           // 16-byte chunks staged per row: 34 pixels = 102 bytes starting up to 15 bytes into a chunk
 
 // w[k] = q[k] + ... + q[k+6], k = 0..3
@@ -283,18 +284,26 @@ k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom 
     }
     __syncthreads();
     {
+        // thread -> column rx of rows r0, r0 + 7, ...: the column's clamp and byte offset are taken once
         const double L0 = sm.shift[0], a0 = sm.shift[1], b0 = sm.shift[2];
-        for (int i = threadIdx.x; i < SE * SE; i += blockDim.x) {
-            const int ry = i / SE, rx = i - ry * SE;
+        const int rx = threadIdx.x % SE, r0 = threadIdx.x / SE;
+        if (r0 < CROWS) {
             const int x = clampi(x0 - SR + rx, 0, w - 1);
-            const uint8_t* p = reinterpret_cast<const uint8_t*>(&sm.raw[ry][0]) + (3 * x - byte0);
-            double L, a, b;
-            rgb_to_lab(sm.lut, p[0], p[1], p[2], L, a, b);
-            L -= L0; a -= a0; b -= b0;
-            sm.plane[0][ry][rx] = L;
-            sm.plane[1][ry][rx] = a;
-            sm.plane[2][ry][rx] = b;
-            sm.plane[3][ry][rx] = L * L + a * a + b * b;
+            const uint8_t* col = reinterpret_cast<const uint8_t*>(&sm.raw[0][0]) + (3 * x - byte0);
+#pragma unroll
+            for (int k = 0; k < (SE + CROWS - 1) / CROWS; ++k) {
+                const int ry = r0 + CROWS * k;
+                if (ry < SE) {
+                    const uint8_t* p = col + ry * (int)(SRAW * sizeof(uint4));
+                    double L, a, b;
+                    rgb_to_lab(sm.lut, p[0], p[1], p[2], L, a, b);
+                    L -= L0; a -= a0; b -= b0;
+                    sm.plane[0][ry][rx] = L;
+                    sm.plane[1][ry][rx] = a;
+                    sm.plane[2][ry][rx] = b;
+                    sm.plane[3][ry][rx] = L * L + a * a + b * b;
+                }
+            }
         }
     }
     __syncthreads();
@@ -343,11 +352,11 @@ k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom 
             const int oy = oy0 + k, y = y0 + oy;
             const double V = fmax(S2[k] * inv_n - M[k] * (inv_n * inv_n), 0.0);
             if (ADAPTIVE) {
-                sqrt_v[((size_t)f * h + y) * w + x] = (float)sqrt(V);
+                sqrt_v[((size_t)f * h + y) * w + x] = sqrtf((float)V);
                 acc0 += V;
                 continue;
             }
-            double C = sqrt(V) * inv_sigma;
+            double C = (double)sqrtf((float)V) * inv_sigma;      // a rounding of 6e-8 relative: far inside the tolerance of s
             C = fmin(C, 1.0);
             uint32_t e = (bits_edge[((size_t)f * h + y) * words + (x >> 5)] >> (x & 31)) & 1u;
             double S = w_edge * (double)e + w_color * C;
