@@ -14,6 +14,8 @@
 // the patch scores.
 #include <math.h>
 
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace {
@@ -269,7 +271,7 @@ k_flow_prior(const float2* __restrict__ d_coarse, int hc, int wc, unsigned wc_in
 // value, 28 bytes) is fetched one block ahead by asynchronous copies into a slot of shared memory that only the
 // thread itself reads: the next block's bytes are in flight while this block's gathers wait for the L2.
 constexpr int TERMS_THREADS = 256;
-constexpr int TERMS_BLOCKS_PER_CTA = 8;
+constexpr int TERMS_BLOCKS_PER_CTA = 8;      // at most
 
 __device__ __forceinline__ void async_copy16(void* dst, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
@@ -655,9 +657,13 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
                 c->launches++;
             }
             dim3 grid(ws[l] / tw, hs[l] / TH, nb);
+            // blocks of pixels per CTA of the terms kernel: up to 8 (so that the copies ahead pay), fewer while the
+            // launch would otherwise leave SMs without a full set of CTAs
+            const long long terms_blocks = (long long)blocks_for((long long)Pl, TERMS_THREADS) * nb;
+            const int terms_per_cta = (int)std::max(1ll, std::min((long long)TERMS_BLOCKS_PER_CTA, terms_blocks / (16ll * c->sm_count)));
             for (int it = 0; it < p.iters; ++it) {
                 const bool last = it == p.iters - 1;
-                k_flow_terms<<<dim3(blocks_for((long long)Pl, TERMS_THREADS * TERMS_BLOCKS_PER_CTA), nb), TERMS_THREADS, 0, st>>>(
+                k_flow_terms<<<dim3(blocks_for((long long)Pl, TERMS_THREADS * terms_per_cta), nb), TERMS_THREADS, 0, st>>>(
                     q1, r1, q1 + second, r1 + second, hs[l], ws[l], w_inv, (l == 2 && it == 0) ? nullptr : dl, dstride, c->gh_a,
                     gstride, nb);
                 int flags = EMIT_D;
