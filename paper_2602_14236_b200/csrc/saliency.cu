@@ -225,7 +225,9 @@ __device__ __forceinline__ void rgb_to_lab(const double* __restrict__ lut, int R
 constexpr int ST = 28;
 constexpr int SR = 3;
 constexpr int SE = ST + 2 * SR;   // 34
-constexpr int SLP = SE + 2;       // row pitch of the planes (even: 16-byte loads of column pairs)
+constexpr int SLP = SE;           // row pitch of the planes: 17 16-byte units, odd, so the 16-byte loads that eight lanes
+                                  // issue down eight rows fall on distinct banks
+constexpr int HSP = ST + 2;       // row pitch of the row sums: 15 16-byte units, odd, for the same reason
 constexpr int CRUN = 4;
 constexpr int CNQ = 2 * SR + CRUN;   // 10 values feed 4 windows
 constexpr int CROWS = 256 / SE;     // rows of the grown tile converted per sweep of the 256 threads (7)
@@ -244,7 +246,7 @@ __device__ __forceinline__ void window4(const double q[CNQ], double w[CRUN]) {
 
 struct ColorSmem {
     double plane[4][SE][SLP];     // dL, da, db, |x|^2
-    double hs[SE][ST];            // 7-column sums of one plane
+    double hs[SE][HSP];           // 7-column sums of one plane
     double lut[256];
     uint4 raw[SE][SRAW];
     double shift[3];
@@ -309,12 +311,14 @@ k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom 
     __syncthreads();
     const double inv_n = 1.0 / (double)((2 * SR + 1) * (2 * SR + 1));
     double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;   // the four patches of the tile
-    const bool owner = threadIdx.x < ST * (ST / CRUN);          // phase 3: (column, run of 4 rows)
-    const int ox = threadIdx.x % ST, oy0 = CRUN * (threadIdx.x / ST);
+    // phase 3: (column, run of 4 rows); a warp holds the 28 columns of one run of rows (its last four lanes idle), so
+    // that its 8-byte loads are consecutive
+    const int ox = threadIdx.x & 31, oy0 = CRUN * (threadIdx.x >> 5);
+    const bool owner = ox < ST && oy0 < ST;
     double M[CRUN] = {0.0, 0.0, 0.0, 0.0}, S2[CRUN] = {0.0, 0.0, 0.0, 0.0};
     for (int c = 0; c < 4; ++c) {                               // one plane's row sums in shared memory at a time
         for (int i = threadIdx.x; i < SE * (ST / CRUN); i += blockDim.x) {
-            const int run = i % (ST / CRUN), ry = i / (ST / CRUN);
+            const int ry = i % SE, run = i / SE;                // lanes run down the rows: conflict-free 16-byte accesses
             const int cx = CRUN * run;                          // windows cx .. cx+3 read columns cx .. cx+9 of the grown tile
             const double2* src = reinterpret_cast<const double2*>(&sm.plane[c][ry][cx]);
             double q[CNQ];
