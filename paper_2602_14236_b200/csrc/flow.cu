@@ -48,23 +48,46 @@ __global__ void k_gray(const uint8_t* __restrict__ frames, size_t frame_bytes, i
 
 // ---- half-scale level: 5x5 binomial [1 4 6 4 1]/16 sampled at (2y, 2x), clamp-to-edge.  Level values are
 // dyadic rationals with at most 24 significant bits, so float holds them exactly.
-__global__ void k_pyr_down(const float* __restrict__ src, int h, int w, int n_frames, float* __restrict__ dst) {
-    int h2 = h / 2, w2 = w / 2;
-    const int f = blockIdx.y, r = blockIdx.x * blockDim.x + threadIdx.x;        // grid: (pixels of a level, frames)
-    if (r >= h2 * w2 || f >= n_frames) return;
-    int y = r / w2, x = r % w2;
+// One thread per 2x2 block of outputs: its 7x7 source neighbourhood is read once, five-tap sums along the rows
+// first, then down the columns (the sums are exact, so their order does not matter).
+__global__ void __launch_bounds__(256)
+k_pyr_down(const float* __restrict__ src, int h, int w, int n_frames, float* __restrict__ dst) {
+    const int h2 = h / 2, w2 = w / 2;
+    const int bw = (w2 + 1) / 2, bh = (h2 + 1) / 2;
+    const int f = blockIdx.y, r = blockIdx.x * blockDim.x + threadIdx.x;        // grid: (2x2 blocks of a level, frames)
+    if (r >= bh * bw || f >= n_frames) return;
+    const int by = r / bw, bx = r - by * bw;
+    const int oy = 2 * by, ox = 2 * bx;
     const float* s = src + (size_t)f * h * w;
-    const float k[5] = {1.f, 4.f, 6.f, 4.f, 1.f};
-    float acc = 0.f;
+    int cx[7];
 #pragma unroll
-    for (int a = -2; a <= 2; ++a) {
-        const float* row = s + (size_t)clampi(2 * y + a, 0, h - 1) * w;
-        float ra = 0.f;
+    for (int b = 0; b < 7; ++b) cx[b] = clampi(2 * ox - 2 + b, 0, w - 1);
+    float hs[7][2];                                 // row sums of source rows 2 oy - 2 .. 2 oy + 4 for the two output columns
 #pragma unroll
-        for (int b = -2; b <= 2; ++b) ra += k[b + 2] * row[clampi(2 * x + b, 0, w - 1)];
-        acc += k[a + 2] * ra;
+    for (int a = 0; a < 7; ++a) {
+        const float* row = s + (size_t)clampi(2 * oy - 2 + a, 0, h - 1) * w;
+        float v[7];
+#pragma unroll
+        for (int b = 0; b < 7; ++b) v[b] = row[cx[b]];
+        hs[a][0] = (v[0] + v[4]) + 4.f * (v[1] + v[3]) + 6.f * v[2];
+        hs[a][1] = (v[2] + v[6]) + 4.f * (v[3] + v[5]) + 6.f * v[4];
     }
-    dst[(size_t)f * h2 * w2 + r] = acc * (1.0f / 256.0f);
+    float* d = dst + (size_t)f * h2 * w2;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        if (oy + j >= h2) break;
+        float o[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+            o[i] = ((hs[2 * j][i] + hs[2 * j + 4][i]) + 4.f * (hs[2 * j + 1][i] + hs[2 * j + 3][i]) + 6.f * hs[2 * j + 2][i]) * (1.0f / 256.0f);
+        float* q = d + (size_t)(oy + j) * w2 + ox;
+        if ((w2 & 1) == 0) {                        // even rows: the pair is inside and 8-byte aligned
+            *reinterpret_cast<float2*>(q) = make_float2(o[0], o[1]);
+        } else {
+            q[0] = o[0];
+            if (ox + 1 < w2) q[1] = o[1];
+        }
+    }
 }
 
 // ---- polynomial expansion, 5x5: r2 r3 r4 r5 r6 = (b_x, b_y, A_xx, A_yy, 2 A_xy), stored as float in the form the
@@ -623,8 +646,8 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
             c->launches++;
         }
         for (int l = 1; l < 3; ++l)
-            k_pyr_down<<<dim3(blocks_for((long long)hs[l] * ws[l], T), nf), T, 0, st>>>(c->pyr[l - 1], hs[l - 1], ws[l - 1], nf,
-                                                                                        c->pyr[l]);
+            k_pyr_down<<<dim3(blocks_for((long long)((hs[l] + 1) / 2) * ((ws[l] + 1) / 2), T), nf), T, 0, st>>>(
+                c->pyr[l - 1], hs[l - 1], ws[l - 1], nf, c->pyr[l]);
         const size_t slots = (size_t)2 * c->chunk;
         float4* cq[3];
         float* cr[3];
