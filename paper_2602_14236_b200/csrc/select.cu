@@ -128,18 +128,52 @@ __global__ void k_sources(const uint8_t* __restrict__ decision, int n_tok, int B
     carry[i] = cur;
 }
 
-// Pool row offsets: exclusive scan over the frames of the batch, continuing from the running fill.
-__global__ void k_row_offsets(const int32_t* __restrict__ counts, int B, int64_t* __restrict__ row_offset,
-                              int64_t* __restrict__ fill) {
-    int t = threadIdx.x;
-    if (t >= 3) return;
-    const int code = t == 0 ? SALICACHE_FP16 : (t == 1 ? SALICACHE_INT8 : SALICACHE_INT4);
-    int64_t acc = fill[t];
-    for (int b = 0; b < B; ++b) {
-        row_offset[(size_t)b * 3 + t] = acc;
-        acc += counts[(size_t)b * 5 + code];
+// Pool row offsets: exclusive scan over the frames of the batch, continuing from the running fill.  One CTA:
+// a frame per thread, its three tier counts scanned together (warp scans, then the warps' totals), 1024 frames per
+// sweep.  Sums within a sweep stay in 32 bits (a frame has fewer than 2^13 tokens: the edge planes of a frame must
+// fit shared memory, which bounds its pixels); the running fill is 64-bit.
+constexpr int OFF_THREADS = 1024;
+__global__ void __launch_bounds__(OFF_THREADS)
+k_row_offsets(const int32_t* __restrict__ counts, int B, int64_t* __restrict__ row_offset, int64_t* __restrict__ fill) {
+    __shared__ int wtot[OFF_THREADS / 32][3];
+    const int t = threadIdx.x, lane = t & 31, wp = t >> 5;
+    const int code[3] = {SALICACHE_FP16, SALICACHE_INT8, SALICACHE_INT4};
+    int64_t carry[3] = {fill[0], fill[1], fill[2]};
+    for (int base = 0; base < B; base += OFF_THREADS) {
+        const int b = base + t;
+        int v[3] = {0, 0, 0}, incl[3];
+#pragma unroll
+        for (int k = 0; k < 3; ++k) {
+            if (b < B) v[k] = counts[(size_t)b * 5 + code[k]];
+            incl[k] = v[k];
+        }
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+#pragma unroll
+            for (int k = 0; k < 3; ++k) {
+                const int up = __shfl_up_sync(0xffffffffu, incl[k], o);
+                if (lane >= o) incl[k] += up;
+            }
+        }
+        if (lane == 31) { wtot[wp][0] = incl[0]; wtot[wp][1] = incl[1]; wtot[wp][2] = incl[2]; }
+        __syncthreads();
+        int below[3] = {0, 0, 0}, total[3] = {0, 0, 0};
+        for (int w = 0; w < OFF_THREADS / 32; ++w) {
+#pragma unroll
+            for (int k = 0; k < 3; ++k) {
+                const int x = wtot[w][k];
+                if (w < wp) below[k] += x;
+                total[k] += x;
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 3; ++k) {
+            if (b < B) row_offset[(size_t)b * 3 + k] = carry[k] + (int64_t)(below[k] + incl[k] - v[k]);
+            carry[k] += total[k];
+        }
+        __syncthreads();
     }
-    fill[t] = acc;
+    if (t < 3) fill[t] = carry[t];
 }
 
 // Residency of stored frames in budgeted pools: one thread per frame.
@@ -218,7 +252,7 @@ int sc_select(salicache_ctx* c, const float* d_deltaP, const float* d_s, int B, 
     k_select<<<B, SEL_THREADS, 0, st>>>(d_deltaP, d_s, c->n_tok, first_has_no_prev, p.patch_reuse, p.tau_t, p.theta_R,
                                         p.tau_high, p.tau_med, p.tau_low, d_decision, d_idx, d_counts,
                                         d_frame_redundant);
-    k_row_offsets<<<1, 32, 0, st>>>(d_counts, B, d_row_offset, d_fill);
+    k_row_offsets<<<1, OFF_THREADS, 0, st>>>(d_counts, B, d_row_offset, d_fill);
     c->launches += 2;
     SC_CHECK(cudaGetLastError());
     return SALICACHE_OK;

@@ -173,6 +173,23 @@ def test_select_is_bit_exact_given_the_same_scores(wl1_oracle_scores, background
     assert counts[0, 0] == 0                          # the first frame never reuses
 
 
+def test_row_offsets_of_a_batch_longer_than_one_sweep_of_the_scan():
+    # 2500 frames: the device scans 1024 frames per sweep, so this batch takes three, the last one ragged
+    ctx = _ctx(max_batch=2500, **synth.thresholds("four"))
+    rng = np.random.default_rng(31)
+    T = 2500
+    dP = rng.uniform(0.0, 2.0 * ctx.params.tau_t, size=(T, 576)).astype(np.float32)
+    s = rng.uniform(0.0, 1.0, size=(T, 576)).astype(np.float32)
+    dP[700:720] = 0.0                                # a run of redundant frames: zero counts inside the scan
+    fill0 = (3, (1 << 33) + 1, 11)                   # a running fill beyond 32 bits
+    out = gu.gpu_select(ctx, dP, s, fill0=fill0)
+    dec, idx, counts, red, off = gu.oracle_select_all(dP, s, gu.oracle_params(ctx.params))
+    assert np.array_equal(out["counts"].cpu().numpy(), counts)
+    assert np.array_equal(out["row_offset"].cpu().numpy(), off + np.array(fill0, np.int64))
+    assert np.array_equal(out["fill"].cpu().numpy(), counts[:, [4, 3, 2]].sum(axis=0) + np.array(fill0, np.int64))
+    assert red[700:720].all() and counts[:, 2:].sum() > 0
+
+
 def test_pipeline_decisions_match_oracle_up_to_near_threshold_tokens(wl1_frames, wl1_oracle_scores):
     ctx = _ctx(**synth.thresholds("four"))
     dP, s = gu.gpu_scores(ctx, wl1_frames)
