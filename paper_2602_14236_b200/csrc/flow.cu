@@ -248,45 +248,6 @@ __device__ __forceinline__ float det2(float a, float b, float c, float d) {
     return f + e;
 }
 
-// ---- prior of a level from the coarser level's field: d = 2 * bilinear(d_coarse) at
-// ((x+1/2)/2 - 1/2, (y+1/2)/2 - 1/2), clamped to the coarse image.  For a fine coordinate x that position is
-// x/2 - 1/4; at x = 0 and at the last fine pixel the clamp puts it on a tap itself.
-// One thread per coarse pixel: its 2x2 block of fine pixels from the 3x3 coarse neighbourhood (clamped; a tap that
-// the clamp moved carries weight zero), written as two 16-byte stores.  Fine x = 2 xc takes taps (xc - 1, xc) with
-// weight 3/4 on the right one, x = 2 xc + 1 taps (xc, xc + 1) with weight 1/4 on the right one.
-__global__ void __launch_bounds__(256)
-k_flow_prior(const float2* __restrict__ d_coarse, int hc, int wc, unsigned wc_inv, size_t d_stride, float2* __restrict__ d_fine,
-             int n_pairs) {
-    const int Pc = hc * wc;
-    const int f = blockIdx.y, r = blockIdx.x * blockDim.x + threadIdx.x;        // grid: (coarse pixels, pairs)
-    if (r >= Pc || f >= n_pairs) return;
-    const int yc = (int)__umulhi((unsigned)r, wc_inv), xc = r - yc * wc;       // wc_inv = ceil(2^32 / wc): exact here
-    const float2* src = d_coarse + (size_t)f * d_stride;
-    float2* dst = d_fine + (size_t)f * d_stride;
-    const int w = 2 * wc;
-    const int xo[3] = {xc > 0 ? -1 : 0, 0, xc < wc - 1 ? 1 : 0};
-    const int yo[3] = {yc > 0 ? -wc : 0, 0, yc < hc - 1 ? wc : 0};
-    float2 n[3][3];
-#pragma unroll
-    for (int j = 0; j < 3; ++j)
-#pragma unroll
-        for (int i = 0; i < 3; ++i) n[j][i] = __ldg(src + r + yo[j] + xo[i]);
-    const float fx[2] = {xc > 0 ? 0.75f : 0.0f, xc < wc - 1 ? 0.25f : 0.0f};
-    const float fy[2] = {yc > 0 ? 0.75f : 0.0f, yc < hc - 1 ? 0.25f : 0.0f};
-#pragma unroll
-    for (int a = 0; a < 2; ++a) {
-        float2 o[2];
-#pragma unroll
-        for (int b = 0; b < 2; ++b) {
-            const float2 p00 = n[a][b], p01 = n[a][b + 1], p10 = n[a + 1][b], p11 = n[a + 1][b + 1];
-            const float gx = 1.0f - fx[b], gy = 1.0f - fy[a];
-            o[b].x = 2.0f * lerp2(p00.x, p01.x, p10.x, p11.x, gx, fx[b], gy, fy[a]);
-            o[b].y = 2.0f * lerp2(p00.y, p01.y, p10.y, p11.y, gx, fx[b], gy, fy[a]);
-        }
-        *reinterpret_cast<float4*>(dst + (2 * yc + a) * w + 2 * xc) = make_float4(o[0].x, o[0].y, o[1].x, o[1].y);
-    }
-}
-
 // ---- (G, h) of the next update from the current field d (zero when there is none: the first update of the
 // coarsest level).  One pixel per thread and no state shared between threads, so the kernel runs at full occupancy,
 // which hides the latency of its gathers; fused behind the solve of the update kernel it ran at a quarter of the
@@ -306,6 +267,12 @@ __device__ __forceinline__ void async_copy4(void* dst, const void* src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
 }
 
+// PRIOR: `d` is the COARSER level's field (h/2 x w/2) and the pixel's value is the prior of the level,
+//   d = 2 * bilinear(d_coarse) at ((x+1/2)/2 - 1/2, (y+1/2)/2 - 1/2), clamped to the coarse image:
+// for a fine coordinate x that position is x/2 - 1/4, and at x = 0 and at the last fine pixel the clamp puts it on a
+// tap itself.  It is formed here from its four taps (they come from the L2: every coarse value serves a dozen fine
+// pixels), so that the first update of a level neither writes nor reads a prior field.
+template <bool PRIOR>
 __global__ void __launch_bounds__(TERMS_THREADS)
 k_flow_terms(const float4* __restrict__ q1, const float* __restrict__ r1, const float4* __restrict__ q2,
              const float* __restrict__ r2, int h, int w, unsigned w_inv, const float2* __restrict__ d, size_t d_stride,
@@ -326,7 +293,7 @@ k_flow_terms(const float4* __restrict__ q1, const float* __restrict__ r1, const 
         if (r < P) {
             async_copy16(&sq[slot][t], qf + r);
             async_copy4(&sr[slot][t], rf + r);
-            if (df) async_copy8(&sd[slot][t], df + r);
+            if (!PRIOR && df) async_copy8(&sd[slot][t], df + r);
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
@@ -338,8 +305,25 @@ k_flow_terms(const float4* __restrict__ q1, const float* __restrict__ r1, const 
         const int slot = n & 1;
         const float4 u = sq[slot][t];
         const float ur = sr[slot][t];
-        const float2 dd = df ? sd[slot][t] : make_float2(0.0f, 0.0f);
         const int y = (int)__umulhi((unsigned)r, w_inv), x = r - y * w;         // w_inv = ceil(2^32 / w): exact for r < 2^32 / w
+        float2 dd = make_float2(0.0f, 0.0f);
+        if (PRIOR) {
+            // fine x = 2 xc takes taps (xc - 1, xc) with weight 3/4 on the right one, x = 2 xc + 1 taps (xc, xc + 1)
+            // with weight 1/4 on the right one; a tap that the clamp moved carries weight zero.  Rows alike.
+            const int wc = w >> 1, hc = h >> 1, xc = x >> 1, yc = y >> 1;
+            const bool xo = x & 1, yo = y & 1;
+            const bool xin = xo ? xc < wc - 1 : xc > 0, yin = yo ? yc < hc - 1 : yc > 0;
+            const int c0 = xc - ((!xo && xin) ? 1 : 0), c1 = xc + ((xo && xin) ? 1 : 0);
+            const int r0 = yc - ((!yo && yin) ? 1 : 0), r1c = yc + ((yo && yin) ? 1 : 0);
+            const float fx = xin ? (xo ? 0.25f : 0.75f) : 0.0f, fy = yin ? (yo ? 0.25f : 0.75f) : 0.0f;
+            const float2 p00 = __ldg(df + r0 * wc + c0), p01 = __ldg(df + r0 * wc + c1);
+            const float2 p10 = __ldg(df + r1c * wc + c0), p11 = __ldg(df + r1c * wc + c1);
+            const float gx = 1.0f - fx, gy = 1.0f - fy;
+            dd.x = 2.0f * lerp2(p00.x, p01.x, p10.x, p11.x, gx, fx, gy, fy);
+            dd.y = 2.0f * lerp2(p00.y, p01.y, p10.y, p11.y, gx, fx, gy, fy);
+        } else if (df) {
+            dd = sd[slot][t];
+        }
         float o5[5];
         normal_terms(u, ur, c2, w, r, (float)-x, (float)(w - 1 - x), (float)-y, (float)(h - 1 - y), dd.x, dd.y, o5);
         float* o = gh + (size_t)f * gh_stride + r;
@@ -658,9 +642,8 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
             k_poly_exp32<<<gp, dim3(32, 8), 0, st>>>(c->pyr[l], hs[l], ws[l], nf, pw32, cq[l], cr[l]);
         }
         c->launches += 5;
-        // Coarse to fine.  Per level: the prior from the coarser level's field, then `iters` times (terms of every
-        // pixel from the current field; window sums + solve -> the new field), each launch over all pairs of the
-        // pass.  (Sub-batches sized for the L2 cache were measured and are slower: the kernels are bound by issue
+        // Coarse to fine.  Per level `iters` times (terms of every pixel from the current field, the first time from the
+        // coarser level's field; window sums + solve -> the new field), each launch over all pairs of the pass.  (Sub-batches sized for the L2 cache were measured and are slower: the kernels are bound by issue
         // slots and load latency, not by DRAM, and small launches add ramp-up and tail time.)
         const size_t fstride = 2 * P0, dstride = P0;      // caller's double field; float2 fields of the scratch
         float2* d_lvl[2] = {reinterpret_cast<float2*>(c->flow_a), reinterpret_cast<float2*>(c->flow_b)};
@@ -673,12 +656,6 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
             const float4* q1 = cq[l];
             const float* r1 = cr[l];
             const unsigned w_inv = (unsigned)((0x100000000ull + ws[l] - 1) / ws[l]);
-            if (l < 2) {
-                const int hc = hs[l + 1], wc = ws[l + 1];
-                k_flow_prior<<<dim3(blocks_for((long long)hc * wc, 256), nb), 256, 0, st>>>(
-                    d_lvl[(l + 1) & 1], hc, wc, (unsigned)((0x100000000ull + wc - 1) / wc), dstride, dl, nb);
-                c->launches++;
-            }
             dim3 grid(ws[l] / tw, hs[l] / TH, nb);
             // blocks of pixels per CTA of the terms kernel: up to 8 (so that the copies ahead pay), fewer while the
             // launch would otherwise leave SMs without a full set of CTAs
@@ -686,9 +663,15 @@ int sc_flow_score(salicache_ctx* c, const PlaneGeom& g, const uint8_t* d_prev, c
             const int terms_per_cta = (int)std::max(1ll, std::min((long long)TERMS_BLOCKS_PER_CTA, terms_blocks / (16ll * c->sm_count)));
             for (int it = 0; it < p.iters; ++it) {
                 const bool last = it == p.iters - 1;
-                k_flow_terms<<<dim3(blocks_for((long long)Pl, TERMS_THREADS * terms_per_cta), nb), TERMS_THREADS, 0, st>>>(
-                    q1, r1, q1 + second, r1 + second, hs[l], ws[l], w_inv, (l == 2 && it == 0) ? nullptr : dl, dstride, c->gh_a,
-                    gstride, nb);
+                // the first update of a finer level starts from the coarser level's field, transferred inside the kernel
+                const dim3 tgrid(blocks_for((long long)Pl, TERMS_THREADS * terms_per_cta), nb);
+                if (it == 0 && l < 2)
+                    k_flow_terms<true><<<tgrid, TERMS_THREADS, 0, st>>>(q1, r1, q1 + second, r1 + second, hs[l], ws[l], w_inv,
+                                                                        d_lvl[(l + 1) & 1], dstride, c->gh_a, gstride, nb);
+                else
+                    k_flow_terms<false><<<tgrid, TERMS_THREADS, 0, st>>>(q1, r1, q1 + second, r1 + second, hs[l], ws[l], w_inv,
+                                                                         (l == 2 && it == 0) ? nullptr : dl, dstride, c->gh_a,
+                                                                         gstride, nb);
                 int flags = EMIT_D;
                 double* dout64 = nullptr;
                 if (last && l == 0) {      // the field goes to the caller's buffer if there is one
