@@ -144,8 +144,9 @@ SALICACHE_API int salicache_diff_score(salicache_ctx* ctx, const uint8_t* d_prev
  * d_frames: B frames.  d_skip_or_null: DEVICE u8 [B] or NULL; frames with a non-zero entry are not
  * scored and their rows of d_s are left untouched (Alg. 1 skips the spatial branch of a temporally
  * redundant frame: pass the flags of salicache_frame_redundancy).  Edge hysteresis runs to its
- * fixed point on the device; if it needs more than hyst_max_iters sweeps the status word records
- * E_NOCONVERGE (see salicache_poll_status).
+ * fixed point on the device in rounds (in a round every strip of rows is swept until it is stable, at
+ * most 64 times, then the whole frame votes); if it needs more than hyst_max_iters rounds the status
+ * word records E_NOCONVERGE (see salicache_poll_status).
  */
 SALICACHE_API int salicache_saliency(salicache_ctx* ctx, const uint8_t* d_frames, int B, float* d_s,
                                      const uint8_t* d_skip_or_null, void* cuda_stream);

@@ -132,45 +132,57 @@ k_canny_classify(const uint8_t* __restrict__ frames, size_t frame_bytes, int h, 
 }
 
 // ---- hysteresis to the fixed point: one CTA per frame, both bit planes in shared memory.
-// E starts as the strong plane and grows through 8-neighbours restricted to the kept plane.
-// Every word is owned by one thread (updates are monotone, so stale neighbour reads only delay).
+// E starts as the strong plane and grows through 8-neighbours restricted to the kept plane; the closure is unique, so
+// the order of the updates does not matter.  Every warp owns a strip of rows and sweeps it until nothing in it
+// changes (at most HYST_INNER sweeps, synchronised inside the warp only), reading its neighbours' border rows as they
+// stand (updates are monotone, so a stale read only delays); a round ends with a CTA-wide vote, and the fixed
+// point is reached when a whole round changed nothing.  `max_iters` bounds the rounds.
+constexpr int HYST_INNER = 64;
 __global__ void __launch_bounds__(1024)
 k_hysteresis(const uint32_t* __restrict__ bits_kept, uint32_t* __restrict__ bits_edge, int h, int words, int max_iters,
              int* __restrict__ status, const uint8_t* __restrict__ skip) {
     extern __shared__ uint32_t sh[];
-    uint32_t* K = sh;                      // [h][words]
-    uint32_t* E = sh + (size_t)h * words;  // [h][words]
+    uint32_t* K = sh;                               // [h][words]
+    volatile uint32_t* E = sh + (size_t)h * words;  // [h][words]
     const int f = blockIdx.x, n = h * words;
     if (skip && skip[f]) return;
     const uint32_t* gk = bits_kept + (size_t)f * n;
     uint32_t* ge = bits_edge + (size_t)f * n;
     for (int i = threadIdx.x; i < n; i += blockDim.x) { K[i] = gk[i]; E[i] = ge[i]; }
     __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const int rows_per = (h + n_warps - 1) / n_warps;
+    const int ya = min(h, warp * rows_per), yb = min(h, ya + rows_per);
     int it = 0;
     for (;;) {
         int changed = 0;
-        for (int i = threadIdx.x; i < n; i += blockDim.x) {
-            uint32_t k = K[i], e = E[i];
-            if (k == e) continue;
-            int y = i / words, wx = i % words;
-            uint32_t acc = 0;
+        for (int inner = 0; inner < HYST_INNER; ++inner) {
+            int ch = 0;
+            for (int i = ya * words + lane; i < yb * words; i += 32) {
+                const uint32_t k = K[i], e = E[i];
+                if (k == e) continue;
+                const int y = i / words, wx = i - y * words;
+                uint32_t acc = 0;
 #pragma unroll
-            for (int dy = -1; dy <= 1; ++dy) {
-                int yy = y + dy;
-                if (yy < 0 || yy >= h) continue;
-                const uint32_t* row = E + yy * words;
-                uint32_t v = row[wx];
-                uint32_t l = wx > 0 ? row[wx - 1] : 0u;
-                uint32_t r = wx + 1 < words ? row[wx + 1] : 0u;
-                acc |= v | (v << 1) | (v >> 1) | (l >> 31) | (r << 31);
+                for (int dy = -1; dy <= 1; ++dy) {
+                    const int yy = y + dy;
+                    if (yy < 0 || yy >= h) continue;
+                    const volatile uint32_t* row = E + yy * words;
+                    const uint32_t v = row[wx];
+                    const uint32_t l = wx > 0 ? row[wx - 1] : 0u;
+                    const uint32_t r = wx + 1 < words ? row[wx + 1] : 0u;
+                    acc |= v | (v << 1) | (v >> 1) | (l >> 31) | (r << 31);
+                }
+                uint32_t ne = (e | acc) & k;
+                for (;;) {   // run along the row inside the word
+                    const uint32_t g = (ne | (ne << 1) | (ne >> 1)) & k;
+                    if (g == ne) break;
+                    ne = g;
+                }
+                if (ne != e) { E[i] = ne; ch = 1; }
             }
-            uint32_t ne = (e | acc) & k;
-            for (;;) {   // run along the row inside the word
-                uint32_t g = (ne | (ne << 1) | (ne >> 1)) & k;
-                if (g == ne) break;
-                ne = g;
-            }
-            if (ne != e) { E[i] = ne; changed = 1; }
+            if (!__any_sync(0xffffffffu, ch)) break;
+            changed = 1;
         }
         if (!__syncthreads_or(changed)) break;
         if (++it >= max_iters) {
