@@ -228,7 +228,8 @@ __device__ __forceinline__ void rgb_to_lab(const double* __restrict__ lut, int R
 //   stage    the tile's bytes by 16-byte loads and the sRGB table into shared memory; warp 0 converts the
 //            tile's first pixel (the shift)
 //   convert  LAB of the 34x34 grown tile, minus the shift, and |x|^2 -> shared memory
-//   then per plane (its row sums alone occupy shared memory, which keeps four CTAs on an SM):
+//   then two planes at a time (the second plane's row sums lie over the staging area, dead by then, which keeps
+//   four CTAs on an SM):
 //   phase 2  one thread per (row, run of 4 columns): 7-column sums
 //   phase 3  one thread per (column, run of 4 rows): 7-row sums
 //   last     C, blend with the edge bit, patch partial sums
@@ -256,11 +257,17 @@ __device__ __forceinline__ void window4(const double q[CNQ], double w[CRUN]) {
     w[3] = mid + p9;
 }
 
-struct ColorSmem {
-    double plane[4][SE][SLP];     // dL, da, db, |x|^2
-    double hs[SE][HSP];           // 7-column sums of one plane
+struct ColorStage {               // what the LAB stage reads; dead once the planes are filled
     double lut[256];
     uint4 raw[SE][SRAW];
+};
+struct ColorSmem {
+    double plane[4][SE][SLP];     // dL, da, db, |x|^2
+    double hs0[SE][HSP];          // 7-column sums of two planes at a time; the second set lies over the staging area
+    union {
+        ColorStage st;
+        double hs1[SE][HSP];
+    } u;
     double shift[3];
     double psum[8][4];
 };
@@ -283,12 +290,12 @@ k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom 
     const int row_bytes = 3 * w;
     const int xa = x0 >= SR ? x0 - SR : 0;
     const int byte0 = (3 * xa) & ~15;
-    sm.lut[threadIdx.x] = __ldg(lut + threadIdx.x);
+    sm.u.st.lut[threadIdx.x] = __ldg(lut + threadIdx.x);
     for (int i = threadIdx.x; i < SE * SRAW; i += blockDim.x) {
         const int ry = i / SRAW, ch = i - ry * SRAW;
         const int y = clampi(y0 - SR + ry, 0, h - 1);
         const int off = byte0 + 16 * ch;
-        if (off < row_bytes) sm.raw[ry][ch] = __ldg(reinterpret_cast<const uint4*>(fr + (size_t)y * row_bytes + off));
+        if (off < row_bytes) sm.u.st.raw[ry][ch] = __ldg(reinterpret_cast<const uint4*>(fr + (size_t)y * row_bytes + off));
     }
     if (threadIdx.x >= 224) {          // the last warp: the shift, straight from global memory
         const uint8_t* p = fr + ((size_t)y0 * w + x0) * 3;
@@ -303,14 +310,14 @@ k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom 
         const int rx = threadIdx.x % SE, r0 = threadIdx.x / SE;
         if (r0 < CROWS) {
             const int x = clampi(x0 - SR + rx, 0, w - 1);
-            const uint8_t* col = reinterpret_cast<const uint8_t*>(&sm.raw[0][0]) + (3 * x - byte0);
+            const uint8_t* col = reinterpret_cast<const uint8_t*>(&sm.u.st.raw[0][0]) + (3 * x - byte0);
 #pragma unroll
             for (int k = 0; k < (SE + CROWS - 1) / CROWS; ++k) {
                 const int ry = r0 + CROWS * k;
                 if (ry < SE) {
                     const uint8_t* p = col + ry * (int)(SRAW * sizeof(uint4));
                     double L, a, b;
-                    rgb_to_lab(sm.lut, p[0], p[1], p[2], L, a, b);
+                    rgb_to_lab(sm.u.st.lut, p[0], p[1], p[2], L, a, b);
                     L -= L0; a -= a0; b -= b0;
                     sm.plane[0][ry][rx] = L;
                     sm.plane[1][ry][rx] = a;
@@ -328,35 +335,41 @@ k_color_patch(const uint8_t* __restrict__ frames, size_t frame_bytes, PlaneGeom 
     const int ox = threadIdx.x & 31, oy0 = CRUN * (threadIdx.x >> 5);
     const bool owner = ox < ST && oy0 < ST;
     double M[CRUN] = {0.0, 0.0, 0.0, 0.0}, S2[CRUN] = {0.0, 0.0, 0.0, 0.0};
-    for (int c = 0; c < 4; ++c) {                               // one plane's row sums in shared memory at a time
-        for (int i = threadIdx.x; i < SE * (ST / CRUN); i += blockDim.x) {
-            const int ry = i % SE, run = i / SE;                // lanes run down the rows: conflict-free 16-byte accesses
+    for (int cp = 0; cp < 2; ++cp) {                            // two planes' row sums in shared memory at a time
+        if (threadIdx.x < SE * (ST / CRUN)) {
+            const int ry = threadIdx.x % SE, run = threadIdx.x / SE;   // lanes run down the rows: conflict-free 16-byte accesses
             const int cx = CRUN * run;                          // windows cx .. cx+3 read columns cx .. cx+9 of the grown tile
-            const double2* src = reinterpret_cast<const double2*>(&sm.plane[c][ry][cx]);
-            double q[CNQ];
 #pragma unroll
-            for (int k = 0; k < CNQ / 2; ++k) {
-                double2 v = src[k];
-                q[2 * k] = v.x;
-                q[2 * k + 1] = v.y;
+            for (int pl = 0; pl < 2; ++pl) {
+                const double2* src = reinterpret_cast<const double2*>(&sm.plane[2 * cp + pl][ry][cx]);
+                double q[CNQ];
+#pragma unroll
+                for (int k = 0; k < CNQ / 2; ++k) {
+                    double2 v = src[k];
+                    q[2 * k] = v.x;
+                    q[2 * k + 1] = v.y;
+                }
+                double w1[CRUN];
+                window4(q, w1);
+                double2* dst = reinterpret_cast<double2*>(pl ? &sm.u.hs1[ry][cx] : &sm.hs0[ry][cx]);
+                dst[0] = make_double2(w1[0], w1[1]);
+                dst[1] = make_double2(w1[2], w1[3]);
             }
-            double w1[CRUN];
-            window4(q, w1);
-            double2* dst = reinterpret_cast<double2*>(&sm.hs[ry][cx]);
-            dst[0] = make_double2(w1[0], w1[1]);
-            dst[1] = make_double2(w1[2], w1[3]);
         }
         __syncthreads();
         if (owner) {
-            double q[CNQ];
 #pragma unroll
-            for (int k = 0; k < CNQ; ++k) q[k] = sm.hs[oy0 + k][ox];
-            double w1[CRUN];
-            window4(q, w1);
+            for (int pl = 0; pl < 2; ++pl) {
+                double q[CNQ];
 #pragma unroll
-            for (int k = 0; k < CRUN; ++k) {
-                if (c < 3) M[k] += w1[k] * w1[k];
-                else S2[k] = w1[k];
+                for (int k = 0; k < CNQ; ++k) q[k] = pl ? sm.u.hs1[oy0 + k][ox] : sm.hs0[oy0 + k][ox];
+                double w1[CRUN];
+                window4(q, w1);
+#pragma unroll
+                for (int k = 0; k < CRUN; ++k) {
+                    if (2 * cp + pl < 3) M[k] += w1[k] * w1[k];
+                    else S2[k] = w1[k];
+                }
             }
         }
         __syncthreads();
