@@ -114,8 +114,9 @@ __device__ __forceinline__ float smooth5(float qm2, float qm1, float q0, float q
     return q0 + (g1 * ((qp1 - q0) + (qm1 - q0)) + g2 * ((qp2 - q0) + (qm2 - q0)));
 }
 
-// Block (32, 8): thread (tx, ty) owns column tx of rows ty, ty + 8, ...: every loop below has a compile-time trip
-// count and every shared-memory access is a base plus a constant.
+// Block (32, 8): thread (tx, ty) owns column tx of rows 4 ty .. 4 ty + 3 (of rows ty, ty + 8, ... while staging and in
+// the row pass): every loop below has a compile-time trip count, every shared-memory access is a base plus a constant,
+// and the five-tap windows of a thread's four rows share their loads.
 __global__ void __launch_bounds__(256)
 k_poly_exp32(const float* __restrict__ img, int h, int w, int n_frames, PolyW32 pw, float4* __restrict__ cq,
              float* __restrict__ cr) {
@@ -154,14 +155,14 @@ k_poly_exp32(const float* __restrict__ img, int h, int w, int n_frames, PolyW32 
         V2[oy][rx] = pw.k1 * ((b1 - c) + (a1 - c)) + pw.k2 * ((b2 - c) + (a2 - c));
     };
 #pragma unroll
-    for (int k = 0; k < 4; ++k) down(ty + 8 * k, tx);
+    for (int k = 0; k < 4; ++k) down(4 * ty + k, tx);              // four consecutive rows: their taps overlap
     if (ty < 4) down(8 * ty + (tx >> 2), 32 + (tx & 3));          // the four columns past the 32nd: 128 items, four warps
     __syncthreads();
     const int x = x0 + tx;
     if (x >= w) return;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-        const int oy = ty + 8 * k, y = y0 + oy;
+        const int oy = 4 * ty + k, y = y0 + oy;                       // the rows of the column pass above: the windows overlap
         if (y >= h) break;
         const float h1a = H1[oy][tx], h1b = H1[oy + 1][tx], h1c = H1[oy + 2][tx], h1d = H1[oy + 3][tx], h1e = H1[oy + 4][tx];
         const float m10 = smooth5(h1a, h1b, h1c, h1d, h1e, pw.g1, pw.g2);
