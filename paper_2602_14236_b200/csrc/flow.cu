@@ -62,13 +62,21 @@ k_pyr_down(const float* __restrict__ src, int h, int w, int n_frames, float* __r
     int cx[7];
 #pragma unroll
     for (int b = 0; b < 7; ++b) cx[b] = clampi(2 * ox - 2 + b, 0, w - 1);
+    const bool inner = ox >= 1 && 2 * ox + 4 <= w - 1 && (w & 3) == 0;      // rows are then 16-byte aligned as well
     float hs[7][2];                                 // row sums of source rows 2 oy - 2 .. 2 oy + 4 for the two output columns
 #pragma unroll
     for (int a = 0; a < 7; ++a) {
         const float* row = s + (size_t)clampi(2 * oy - 2 + a, 0, h - 1) * w;
         float v[7];
+        if (inner) {                                // columns 4 bx - 2 .. 4 bx + 4 unclamped: 8 + 16 + 4 aligned bytes
+            const float2 a2 = *reinterpret_cast<const float2*>(row + 2 * ox - 2);
+            const float4 a4 = *reinterpret_cast<const float4*>(row + 2 * ox);
+            v[0] = a2.x; v[1] = a2.y; v[2] = a4.x; v[3] = a4.y; v[4] = a4.z; v[5] = a4.w;
+            v[6] = row[2 * ox + 4];
+        } else {
 #pragma unroll
-        for (int b = 0; b < 7; ++b) v[b] = row[cx[b]];
+            for (int b = 0; b < 7; ++b) v[b] = row[cx[b]];
+        }
         hs[a][0] = (v[0] + v[4]) + 4.f * (v[1] + v[3]) + 6.f * v[2];
         hs[a][1] = (v[2] + v[6]) + 4.f * (v[3] + v[5]) + 6.f * v[4];
     }
