@@ -38,6 +38,7 @@ constexpr int CT = 32;
 constexpr int CG = CT + 8;   // gray tile
 constexpr int CB = CT + 4;   // blur tile
 constexpr int CM = CT + 2;   // magnitude tile
+constexpr int MAG_ROWS = 5, MAG_GROUPS = (CM + MAG_ROWS - 1) / MAG_ROWS;   // rows of the magnitude tile per thread; 7 groups
 constexpr int CRAW = 9;      // 16-byte chunks staged per row: 40 pixels = 120 bytes starting up to 12 bytes into a chunk
 
 __global__ void __launch_bounds__(256)
@@ -84,49 +85,62 @@ k_canny_classify(const uint8_t* __restrict__ frames, size_t frame_bytes, int h, 
         sb[ry][rx] = (uint8_t)((acc + 128) >> 8);
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < CM * CM; i += blockDim.x) {
-        int ry = i / CM, rx = i % CM;
-        int y = y0 - 1 + ry, x = x0 - 1 + rx;
-        int m = 0;
-        if (y >= 0 && y < h && x >= 0 && x < w) {
-            int by = ry + 1, bx = rx + 1;   // position in the blur tile
-            int gx = (sb[by - 1][bx + 1] + 2 * sb[by][bx + 1] + sb[by + 1][bx + 1]) -
-                     (sb[by - 1][bx - 1] + 2 * sb[by][bx - 1] + sb[by + 1][bx - 1]);
-            int gy = (sb[by + 1][bx - 1] + 2 * sb[by + 1][bx] + sb[by + 1][bx + 1]) -
-                     (sb[by - 1][bx - 1] + 2 * sb[by - 1][bx] + sb[by - 1][bx + 1]);
-            m = gx * gx + gy * gy;
+    // magnitude and direction sector of the tile grown by 1: thread -> column rx of five consecutive rows (their 3x3
+    // neighbourhoods share rows), the sector in the four bits above the magnitude (at most 2 * 1020^2 < 2^21)
+    if (threadIdx.x < CM * MAG_GROUPS) {
+        const int rx = threadIdx.x % CM, r0 = MAG_ROWS * (threadIdx.x / CM);
+        const int x = x0 - 1 + rx;
+        const bool xin = x >= 0 && x < w;
+#pragma unroll
+        for (int k = 0; k < MAG_ROWS; ++k) {
+            const int ry = r0 + k;
+            if (ry >= CM) break;
+            const int y = y0 - 1 + ry;
+            uint32_t mv = 0;
+            if (xin && y >= 0 && y < h) {
+                const int by = ry + 1, bx = rx + 1;   // position in the blur tile
+                const int gx = (sb[by - 1][bx + 1] + 2 * sb[by][bx + 1] + sb[by + 1][bx + 1]) -
+                               (sb[by - 1][bx - 1] + 2 * sb[by][bx - 1] + sb[by + 1][bx - 1]);
+                const int gy = (sb[by + 1][bx - 1] + 2 * sb[by + 1][bx] + sb[by + 1][bx + 1]) -
+                               (sb[by - 1][bx - 1] + 2 * sb[by - 1][bx] + sb[by - 1][bx + 1]);
+                const int ax = abs(gx), ay = abs(gy);
+                // sector: 0 along the row, 1 down the column, 2 the diagonal (-1,-1)/(+1,+1), 3 the other one
+                uint32_t sec;
+                if (32768 * ay <= 13573 * ax) sec = 0;
+                else if (32768 * ax <= 13573 * ay) sec = 1;
+                else sec = ((gx > 0) == (gy > 0)) ? 2 : 3;
+                mv = (uint32_t)(gx * gx + gy * gy) | (sec << 28);
+            }
+            smag[ry][rx] = (int)mv;
         }
-        smag[ry][rx] = m;
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < CT * CT; i += blockDim.x) {
-        int oy = i / CT, ox = i % CT;     // a warp covers one row of the tile
-        int y = y0 + oy, x = x0 + ox;
-        int cls = 0;
-        if (y < h && x < w) {
-            int by = oy + 2, bx = ox + 2;
-            int gx = (sb[by - 1][bx + 1] + 2 * sb[by][bx + 1] + sb[by + 1][bx + 1]) -
-                     (sb[by - 1][bx - 1] + 2 * sb[by][bx - 1] + sb[by + 1][bx - 1]);
-            int gy = (sb[by + 1][bx - 1] + 2 * sb[by + 1][bx] + sb[by + 1][bx + 1]) -
-                     (sb[by - 1][bx - 1] + 2 * sb[by - 1][bx] + sb[by - 1][bx + 1]);
-            int my = oy + 1, mx = ox + 1;
-            int mm = smag[my][mx];
-            int ax = abs(gx), ay = abs(gy);
-            int mneg, mpos;
-            if (32768 * ay <= 13573 * ax) { mneg = smag[my][mx - 1]; mpos = smag[my][mx + 1]; }
-            else if (32768 * ax <= 13573 * ay) { mneg = smag[my - 1][mx]; mpos = smag[my + 1][mx]; }
-            else if ((gx > 0) == (gy > 0)) { mneg = smag[my - 1][mx - 1]; mpos = smag[my + 1][mx + 1]; }
-            else { mneg = smag[my - 1][mx + 1]; mpos = smag[my + 1][mx - 1]; }
-            bool keep = (mm > mneg) && (mm >= mpos);
-            if (keep && mm >= hi2) cls = 2;
-            else if (keep && mm >= lo2) cls = 1;
-        }
-        uint32_t kept = __ballot_sync(0xffffffffu, cls > 0);
-        uint32_t strong = __ballot_sync(0xffffffffu, cls == 2);
-        if ((threadIdx.x & 31) == 0 && y < h) {
-            size_t o = ((size_t)f * h + y) * words + blockIdx.x;
-            bits_kept[o] = kept;
-            bits_strong[o] = strong;
+    // a warp covers one row of the tile (the ballots), a thread four consecutive rows
+    {
+        const int ox = threadIdx.x & 31, x = x0 + ox;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int oy = 4 * (threadIdx.x >> 5) + k, y = y0 + oy;
+            int cls = 0;
+            if (y < h && x < w) {
+                const int my = oy + 1, mx = ox + 1;
+                const uint32_t mc = (uint32_t)smag[my][mx];
+                const int mm = (int)(mc & 0x0fffffffu);
+                const uint32_t sec = mc >> 28;
+                const int dy = sec != 0 ? 1 : 0;
+                const int dx = (sec == 0 || sec == 2) ? 1 : (sec == 3 ? -1 : 0);
+                const int mneg = smag[my - dy][mx - dx] & 0x0fffffff, mpos = smag[my + dy][mx + dx] & 0x0fffffff;
+                const bool keep = (mm > mneg) && (mm >= mpos);
+                if (keep && mm >= hi2) cls = 2;
+                else if (keep && mm >= lo2) cls = 1;
+            }
+            const uint32_t kept = __ballot_sync(0xffffffffu, cls > 0);
+            const uint32_t strong = __ballot_sync(0xffffffffu, cls == 2);
+            if (ox == 0 && y < h) {
+                const size_t o = ((size_t)f * h + y) * words + blockIdx.x;
+                bits_kept[o] = kept;
+                bits_strong[o] = strong;
+            }
         }
     }
 }
