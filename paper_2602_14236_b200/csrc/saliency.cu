@@ -38,6 +38,8 @@ constexpr int CT = 32;
 constexpr int CG = CT + 8;   // gray tile
 constexpr int CB = CT + 4;   // blur tile
 constexpr int CM = CT + 2;   // magnitude tile
+constexpr int GRAY_ROWS = 7, GRAY_GROUPS = (CG + GRAY_ROWS - 1) / GRAY_ROWS;   // 6 groups of 40 columns: 240 threads
+constexpr int BLUR_ROWS = 6, BLUR_GROUPS = (CG + BLUR_ROWS - 1) / BLUR_ROWS;   // 7 groups of 36 columns: 252 threads
 constexpr int MAG_ROWS = 5, MAG_GROUPS = (CM + MAG_ROWS - 1) / MAG_ROWS;   // rows of the magnitude tile per thread; 7 groups
 constexpr int CRAW = 9;      // 16-byte chunks staged per row: 40 pixels = 120 bytes starting up to 12 bytes into a chunk
 
@@ -63,26 +65,59 @@ k_canny_classify(const uint8_t* __restrict__ frames, size_t frame_bytes, int h, 
         if (off < row_bytes) sraw[ry][ch] = __ldg(reinterpret_cast<const uint4*>(fr + (size_t)y * row_bytes + off));
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < CG * CG; i += blockDim.x) {
-        const int ry = i / CG, rx = i - ry * CG;
+    // gray: thread -> column rx of seven rows (the column's clamp and byte offset once)
+    if (threadIdx.x < CG * GRAY_GROUPS) {
+        const int rx = threadIdx.x % CG, r0 = GRAY_ROWS * (threadIdx.x / CG);
         const int x = clampi(x0 - 4 + rx, 0, w - 1);
-        const uint8_t* p = reinterpret_cast<const uint8_t*>(&sraw[ry][0]) + (3 * x - byte0);
-        sg[ry][rx] = (uint8_t)((77 * p[0] + 150 * p[1] + 29 * p[2] + 128) >> 8);
+        const uint8_t* col = reinterpret_cast<const uint8_t*>(&sraw[0][0]) + (3 * x - byte0);
+#pragma unroll
+        for (int k = 0; k < GRAY_ROWS; ++k) {
+            const int ry = r0 + k;
+            if (ry >= CG) break;
+            const uint8_t* p = col + ry * (int)(CRAW * sizeof(uint4));
+            sg[ry][rx] = (uint8_t)((77 * p[0] + 150 * p[1] + 29 * p[2] + 128) >> 8);
+        }
     }
     __syncthreads();
-    // blur at the clamped position, so that the Sobel taps read Bl(clamp(y), clamp(x)): column map first
-    for (int i = threadIdx.x; i < CG * CB; i += blockDim.x) {
-        const int gy = i / CB, rx = i - gy * CB;
+    // blur at the clamped position, so that the Sobel taps read Bl(clamp(y), clamp(x)): column map first;
+    // thread -> column rx of six rows
+    if (threadIdx.x < CB * BLUR_GROUPS) {
+        const int rx = threadIdx.x % CB, r0 = BLUR_ROWS * (threadIdx.x / CB);
         const int gx0 = clampi(x0 - 2 + rx, 0, w - 1) - (x0 - 4);
-        const uint8_t* g = &sg[gy][gx0];
-        sh[gy][rx] = (uint16_t)(g[-2] + 4 * g[-1] + 6 * g[0] + 4 * g[1] + g[2]);
+#pragma unroll
+        for (int k = 0; k < BLUR_ROWS; ++k) {
+            const int gy = r0 + k;
+            if (gy >= CG) break;
+            const uint8_t* g = &sg[gy][gx0];
+            sh[gy][rx] = (uint16_t)(g[-2] + 4 * g[-1] + 6 * g[0] + 4 * g[1] + g[2]);
+        }
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < CB * CB; i += blockDim.x) {
-        const int ry = i / CB, rx = i - ry * CB;
-        const int gy0 = clampi(y0 - 2 + ry, 0, h - 1) - (y0 - 4);
-        const int acc = sh[gy0 - 2][rx] + 4 * sh[gy0 - 1][rx] + 6 * sh[gy0][rx] + 4 * sh[gy0 + 1][rx] + sh[gy0 + 2][rx];
-        sb[ry][rx] = (uint8_t)((acc + 128) >> 8);
+    // down the columns: thread -> column rx of six consecutive rows; away from the image's top and bottom their
+    // five-tap windows are rows r0 .. r0 + 9 of the row sums, each read once
+    if (threadIdx.x < CB * BLUR_GROUPS) {
+        const int rx = threadIdx.x % CB, r0 = BLUR_ROWS * (threadIdx.x / CB);
+        if (y0 >= 2 && y0 + CT + 1 <= h - 1) {               // no row of the blur tile is clamped: gy0 = ry + 2
+            int v[BLUR_ROWS + 4];
+#pragma unroll
+            for (int k = 0; k < BLUR_ROWS + 4; ++k) v[k] = sh[r0 + k < CG ? r0 + k : CG - 1][rx];
+#pragma unroll
+            for (int k = 0; k < BLUR_ROWS; ++k) {
+                const int ry = r0 + k;
+                if (ry >= CB) break;
+                const int acc = v[k] + 4 * v[k + 1] + 6 * v[k + 2] + 4 * v[k + 3] + v[k + 4];
+                sb[ry][rx] = (uint8_t)((acc + 128) >> 8);
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < BLUR_ROWS; ++k) {
+                const int ry = r0 + k;
+                if (ry >= CB) break;
+                const int gy0 = clampi(y0 - 2 + ry, 0, h - 1) - (y0 - 4);
+                const int acc = sh[gy0 - 2][rx] + 4 * sh[gy0 - 1][rx] + 6 * sh[gy0][rx] + 4 * sh[gy0 + 1][rx] + sh[gy0 + 2][rx];
+                sb[ry][rx] = (uint8_t)((acc + 128) >> 8);
+            }
+        }
     }
     __syncthreads();
     // magnitude and direction sector of the tile grown by 1: thread -> column rx of five consecutive rows (their 3x3
